@@ -1,0 +1,228 @@
+/*
+ * lpc.h -- C ABI of the B200 (sm_100a) implementation of the per-iteration path of LPC-SVRG and
+ * ALPC-SVRG (arXiv 1901.08924, "Exploring Fast and Communication-Efficient Algorithms in
+ * Large-scale Distributed Networks").
+ *
+ * The library solves  min_x P(x) = (1/n) sum_a loss(<X_a,x>, y_a) + lambda_l1*||x||_1  (Eq. 1) with
+ * N data-parallel workers simulated on one GPU as contiguous row partitions of X.  What the
+ * workers would transmit is produced bit for bit (b-bit codes plus one float per message) and
+ * counted, never sent.
+ *
+ * Conventions
+ *  - Every function returns an int status: LPC_OK or a negative LPC_ERR_* value.  Nothing throws
+ *    or aborts.  lpc_last_error() gives a text for the last failure of a context.
+ *  - Unless a parameter says "host", array arguments are DEVICE pointers owned by the caller.
+ *    The library never frees or reallocates them.  They must be 16-byte aligned, fp32 data must
+ *    be finite.  X is row-major, contiguous, leading dimension d, and d must be a multiple of 4.
+ *  - Work is enqueued on the cudaStream_t given to lpc_init (passed as void*); calls return
+ *    without waiting unless they hand back a host scalar (said per call).  Device-side problems
+ *    (non-finite input, a bounded wait that ran out) are recorded in the context and reported by
+ *    the next lpc_sync_status().
+ *  - A context may be used by one host thread at a time.
+ *
+ * Packed message layout (part of the ABI).  Coordinate j of a vector of length len has the
+ * b-bit code  c_j = k_j + 2^(b-1)  where k_j in [-2^(b-1), 2^(b-1)-1] is its index in the codebook
+ * dom(delta,b) of Section 2.2 (b = 1: c_j in {0,1} for the two points -T,+T; b = 32: the IEEE bits
+ * of the number).  Codes form a little-endian bit stream: c_j occupies stream bits [j*b,(j+1)*b),
+ * stream bit p is bit p%32 of 32-bit word p/32; unused tail bits are zero.  A message is that
+ * stream plus the float delta: 32 + b*len bits (Section 3.2).  In memory, worker i's stream for
+ * segment s starts at word  i*stride_words + word_offset[s], both multiples of 4 words
+ * (lpc_packed_layout); delta is stored at delta[i*nseg + s].
+ */
+#ifndef LPC_H_
+#define LPC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct lpc_ctx lpc_ctx;
+
+/* status codes */
+#define LPC_OK 0
+#define LPC_ERR_INVALID_ARG (-1)
+#define LPC_ERR_UNSUPPORTED (-2)
+#define LPC_ERR_NONFINITE (-3) /* a NaN or Inf reached the quantizer */
+#define LPC_ERR_CUDA (-4)
+#define LPC_ERR_TIMEOUT (-5) /* a bounded device-side wait ran out */
+
+/* loss of the linear model, f_a(x) = loss(<X_a,x>, y_a) (Section 5.1: regression and logistic models) */
+#define LPC_LOGISTIC 0      /* log(1 + exp(-y m)), y in {-1,+1} */
+#define LPC_LEAST_SQUARES 1 /* (m - y)^2 / 2 */
+
+/* clip rule: the threshold T of Eq. 2, delta = T / (2^(b-1) - 1) */
+#define LPC_CLIP_NONE 0   /* T = ||u||_inf                    (Eq. 2 with lambda = 1, unbiased) */
+#define LPC_CLIP_LAMBDA 1 /* T = clip_value * ||u||_inf       (Eq. 2, clip_value = lambda in (0,1]) */
+#define LPC_CLIP_STD 2    /* T = min(clip_value * std(u), ||u||_inf)  (the [-c sigma, c sigma] region of Section 3.1) */
+
+/* buffers of a context that lpc_get_buffer / lpc_set_buffer can copy (device to device) */
+#define LPC_BUF_X 0        /* fp32[d]   current iterate x_t (ALPC: x_{k+1} of the last step) */
+#define LPC_BUF_XTILDE 1   /* fp32[d]   snapshot */
+#define LPC_BUF_MU 2       /* fp32[d]   grad f(snapshot) */
+#define LPC_BUF_MARGINS 3  /* fp32[n]   <X_a, snapshot> */
+#define LPC_BUF_Y 4        /* fp32[d]   ALPC y_k */
+#define LPC_BUF_Z 5        /* fp32[d]   ALPC z_k */
+#define LPC_BUF_YSUM 6     /* fp32[d]   ALPC running sum of y over the epoch */
+#define LPC_BUF_CODES 7    /* u32[N*stride_words] packed messages of the last step */
+#define LPC_BUF_DELTA 8    /* fp32[N]   their scales */
+#define LPC_BUF_CLIPPED 9  /* u32[N]    d_lambda^i: coordinates outside the codebook's hull (Lemma 2) */
+#define LPC_BUF_BATCH_IDX 10 /* i64[(N+1)*B] sampled rows of the last step; the last B are ALPC's shared batch J */
+#define LPC_BUF_COEF 11    /* fp32[(N+1)*B] l'(m(x)) - l'(m(snapshot)) of those rows */
+#define LPC_BUF_U 12       /* fp32[N*d] the unquantized worker differences u^i (only while the tap is on) */
+#define LPC_BUF_V 13       /* fp32[d]   v of the last step (only while the tap is on) */
+#define LPC_BUF_VHAT 14    /* fp32[d]   ALPC full-precision estimator of the last step */
+
+/* options for lpc_set_option */
+#define LPC_OPT_SAMPLE_GLOBAL 0 /* 0 (default): worker i samples its own block of n/N rows; 1: all n rows (the paper's shared-storage setting, Section 2.1) */
+#define LPC_OPT_TAP_U 1         /* 1: inner steps also store u^i and v for inspection (slower) */
+#define LPC_OPT_CLUSTER_SIZE 2  /* thread-block cluster size per worker for the fused step: 0 = automatic, else 1, 2, 4 or 8 */
+#define LPC_OPT_USE_GRAPH 3     /* 1 (default): lpc_inner_steps replays a CUDA graph; 0: plain launches */
+
+/*
+ * Creates a context for problem (1).  Section 1 "Contribution" (Eq. 1), Section 2.1 (N workers),
+ * Algorithm 1's inputs.
+ *   X        n x d, row-major (may be NULL with n = 0 for a quantizer-only context; then only
+ *            lpc_quantize_pack, lpc_unpack_average_prox and the sizing helpers may be called and d is
+ *            ignored)
+ *   y        n labels / targets
+ *   n        rows; must be a multiple of N.  Worker i owns rows [i*n/N, (i+1)*n/N).
+ *   d        features, multiple of 4, at most 16384
+ *   N        simulated workers, 1..1024;  B minibatch size per worker, 1..64
+ *   b        bits per coordinate: 1..16 or 32 (32 = full precision, the codes are the floats)
+ *   seed     key of every random stream (minibatches, shared batch J, stochastic rounding)
+ *   stream   cudaStream_t (NULL = default stream)
+ * The iterate starts at zero.  Scratch memory is allocated here and freed by lpc_destroy.
+ */
+int lpc_init(lpc_ctx** out, const float* X, const float* y, int64_t n, int32_t d, int loss,
+             float lambda_l1, int32_t N, int32_t B, int32_t b, int clip_mode, float clip_value,
+             uint64_t seed, void* stream);
+int lpc_destroy(lpc_ctx* ctx);
+int lpc_set_option(lpc_ctx* ctx, int option, int64_t value);
+const char* lpc_last_error(const lpc_ctx* ctx);
+
+/* Waits for the stream and returns the first device-side error recorded since the last call
+ * (LPC_ERR_NONFINITE, LPC_ERR_TIMEOUT, LPC_ERR_CUDA) or LPC_OK.  Host-synchronous. */
+int lpc_sync_status(lpc_ctx* ctx);
+
+/* Copies a context buffer (LPC_BUF_*) to / from caller memory on the stream; `bytes` must not
+ * exceed the buffer's size.  Setting XTILDE, MU and MARGINS together replaces the snapshot state;
+ * the counter-based random streams carry no state, so copying X (or Y, Z, YSUM), XTILDE, MU and
+ * MARGINS and re-using the same iteration numbers resumes a run exactly. */
+int lpc_get_buffer(lpc_ctx* ctx, int which, void* dst, size_t bytes);
+int lpc_set_buffer(lpc_ctx* ctx, int which, const void* src, size_t bytes);
+int lpc_set_iterate(lpc_ctx* ctx, const float* x); /* same as lpc_set_buffer(LPC_BUF_X) with d floats */
+int lpc_get_iterate(lpc_ctx* ctx, float* x_out);
+
+/*
+ * Communication step 1 (Algorithm 1 step 4, Algorithm 2 step 3): makes the current iterate the
+ * snapshot and computes mu = grad f(snapshot) = (1/n) sum_a l'(<X_a,x~>,y_a) X_a in ONE pass over X,
+ * keeping the margins <X_a,x~> for the inner steps.  Counts 32*d*N*(N-1) step-1 bits.
+ *   mu_out      nullable, receives mu (d floats)
+ *   f_snapshot  nullable HOST pointer, receives f(snapshot); when given, the call waits for the
+ *               stream.
+ */
+int lpc_snapshot_full_grad(lpc_ctx* ctx, float* mu_out, double* f_snapshot);
+
+/*
+ * One inner iteration of Algorithm 1 (steps 6-10) for all N workers, scheme (a) (Eq. 3):
+ * worker i samples B rows (with replacement), forms u^i = (1/B) sum_a [grad f_a(x) - grad f_a(x~)],
+ * quantizes it with its own delta (Eq. 2) and packs it; then all messages are decoded, averaged,
+ * mu is added and x <- prox_{eta h}(x - eta v).  u^i is never written to memory unless the tap is on.
+ *   k  global iteration number s*m + t; it keys the random streams.
+ * Counts (32 + b*d)*N*(N-1) step-2 bits (Table 1, broadcast).
+ */
+int lpc_inner_step(lpc_ctx* ctx, float eta, uint64_t k);
+/* `count` consecutive inner steps k0, k0+1, ... replayed from a captured CUDA graph. */
+int lpc_inner_steps(lpc_ctx* ctx, float eta, uint64_t k0, int64_t count);
+
+/*
+ * Packed layout of a (segmented) vector: word_offsets_out[s] (nseg+1 host entries, nullable) is
+ * where segment s starts inside a worker's stream, *stride_words_out the distance between
+ * workers' streams, both in 32-bit words and multiples of 4.  seg_offsets: host, nseg+1 element
+ * offsets with seg_offsets[0] = 0 and seg_offsets[nseg] = len, or NULL for one segment.
+ */
+int lpc_packed_layout(int64_t len, int32_t b, const int64_t* seg_offsets, int32_t nseg,
+                      int64_t* word_offsets_out, int64_t* stride_words_out);
+int lpc_packed_words(int64_t len, int32_t b, int64_t* words_out); /* ceil(len*b/32) */
+
+/*
+ * Quantization step (Algorithm 1 step 7; Section 2.2, Eq. 2) of N worker vectors, optionally
+ * per tensor segment (each segment gets its own delta, as in layer-wise use), then packing.
+ *   U          N x len fp32, row stride ld (elements, multiple of 4)
+ *   U_sub      nullable, same shape: when given the quantized vector is U - U_sub (the SVRG
+ *              difference of a current and a snapshot gradient), formed on the fly
+ *   seg_offsets, nseg   as in lpc_packed_layout (host)
+ *   k          iteration number keying the rounding stream
+ *   codes_out  N * stride_words words, stride from lpc_packed_layout
+ *   delta_out  N * nseg floats
+ *   clipped_out nullable, N * nseg counts of coordinates outside the hull
+ * Vectors longer than L2 are read twice (once for ||u||_inf and the variance, once to quantize).
+ * N, b and the clip rule come from the context.
+ */
+int lpc_quantize_pack(lpc_ctx* ctx, const float* U, const float* U_sub, int64_t len, int64_t ld,
+                      const int64_t* seg_offsets, int32_t nseg, uint64_t k, uint32_t* codes_out,
+                      float* delta_out, uint32_t* clipped_out);
+
+/*
+ * Communication step 2 under scheme (a) and Algorithm 1 steps 9-10: decode every worker's message
+ * with its own delta, average (Eq. 3), v = u~ + mu, x <- soft-threshold(x - eta v, eta*lambda_l1)
+ * (the proximal operator of Section 2.3 for h = lambda_l1*||.||_1).
+ *   mu nullable (= 0);  x_inout len floats, updated in place;  v_out nullable, receives v.
+ */
+int lpc_unpack_average_prox(lpc_ctx* ctx, const uint32_t* codes, const float* delta, int64_t len,
+                            const int64_t* seg_offsets, int32_t nseg, const float* mu,
+                            float* x_inout, float eta, float lambda_l1, float* v_out);
+
+/*
+ * ALPC-SVRG (Algorithms 2 and 3).  lpc_alpc_begin sets y_0 = z_0 = x and clears the y sum.
+ * lpc_alpc_double_sample_step is steps 5-13 of Algorithm 2 for iteration k:
+ *   x = tau1*z + tau2*x~ + (1-tau1-tau2)*y;  v from quantized worker differences at x (as in
+ *   Algorithm 1);  v^ = (1/B) sum_{j in J}[grad f_j(x) - grad f_j(x~)] + mu on ONE shared batch J drawn
+ *   from all n rows, in full precision, nothing transmitted ("double sampling");
+ *   y <- soft(x - inv4L*v, inv4L*lambda_l1);  z <- soft(z - alpha*v^, alpha*lambda_l1);  ysum += y.
+ * lpc_alpc_end_epoch(m) is Algorithm 3 step 5: x~ candidate = ysum/m becomes the current iterate
+ * (call lpc_snapshot_full_grad next) and ysum is cleared; y and z carry over.
+ */
+int lpc_alpc_begin(lpc_ctx* ctx);
+int lpc_alpc_double_sample_step(lpc_ctx* ctx, float tau1, float tau2, float alpha, float inv4L, uint64_t k);
+int lpc_alpc_double_sample_steps(lpc_ctx* ctx, float tau1, float tau2, float alpha, float inv4L,
+                                 uint64_t k0, int64_t count);
+int lpc_alpc_end_epoch(lpc_ctx* ctx, int64_t m);
+
+/* P(x) = f(x) + lambda_l1*||x||_1 (Eq. 1) in one pass over X.  x nullable (= current iterate);
+ * P_out is a HOST pointer; the call waits for the stream. */
+int lpc_objective(lpc_ctx* ctx, const float* x, double* P_out);
+
+/* Bits that the simulated workers would have transmitted so far (host counters): step 1 =
+ * 32*d*N*(N-1) per snapshot, step 2 = (32+b*len)*N*(N-1) per inner step or quantize call (Table 1). */
+int lpc_comm_bits(const lpc_ctx* ctx, uint64_t* step1_bits, uint64_t* step2_bits);
+
+/*
+ * The whole LPC-SVRG job from HOST buffers, for callers without device memory of their own:
+ * copies X and y to the device, runs S epochs of m inner steps of Algorithm 1 from x_host_inout,
+ * copies the final snapshot back and returns P at it.  All pointers are host pointers
+ * (pinned memory makes the copies faster).  Host-synchronous.
+ */
+int lpc_svrg_run_host(const float* X_host, const float* y_host, int64_t n, int32_t d, int loss,
+                      float lambda_l1, int32_t N, int32_t B, int32_t b, int clip_mode, float clip_value,
+                      uint64_t seed, int32_t S, int64_t m, float eta, float* x_host_inout,
+                      double* objective_out, uint64_t* step2_bits_out);
+
+/*
+ * Inspection aid: writes `count` consecutive 4-word blocks, starting at block `block0`, of the
+ * counter-based random stream (tag, worker, k) keyed by `seed` to out (device, 4*count words).
+ * The streams are Philox4x32-10 (Salmon et al., SC'11) with counter (block, k_lo, worker | tag<<24,
+ * k_hi) and key (seed_lo, seed_hi); tag 0 = stochastic rounding (Section 2.2 rule 1; coordinate j
+ * uses 16-bit lane j%8 of block j/8), 1 = worker minibatches (Algorithm 1 step 6; slot a uses word 0
+ * of block a), 2 = the shared batch J (Algorithm 2 step 11).
+ */
+int lpc_debug_stream_blocks(uint64_t seed, uint32_t tag, uint32_t worker, uint64_t k, uint32_t block0,
+                            int64_t count, uint32_t* out, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LPC_H_ */

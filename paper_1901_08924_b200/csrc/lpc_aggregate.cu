@@ -1,0 +1,185 @@
+// Communication step 2 under scheme (a) (Eq. 3) fused with Algorithm 1 steps 9-10: every worker's
+// packed message is decoded with its own delta, the decoded vectors are averaged, the snapshot
+// gradient is added and the proximal (soft-threshold) step is applied, in one pass.  The same
+// kernel, in its second mode, applies Algorithm 2's y- and z-updates instead.
+//
+// A thread owns 8 consecutive coordinates per sweep: per worker it loads the 8*b bits that hold
+// their codes (b whole bytes, naturally aligned when b is 1, 2, 4, 8 or 16), and accumulates
+// delta_i * index in worker order, every operation a separate fp32 round-to-nearest operation.
+#include "lpc_device.cuh"
+#include "lpc_kernels.h"
+
+namespace lpc {
+namespace {
+
+constexpr int AT = 256;
+constexpr int AGROUP = AT * 8;
+constexpr int AITER = TILE / AGROUP;
+
+__device__ __forceinline__ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+__device__ __forceinline__ void load8f(const float* __restrict__ p, int64_t j, int64_t len, bool vec, float* v) {
+  if (vec && j + 8 <= len) {
+    const float4 a = *reinterpret_cast<const float4*>(p + j);
+    const float4 c = *reinterpret_cast<const float4*>(p + j + 4);
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = c.x; v[5] = c.y; v[6] = c.z; v[7] = c.w;
+  } else {
+#pragma unroll
+    for (int e = 0; e < 8; ++e) v[e] = (j + e < len) ? p[j + e] : 0.f;
+  }
+}
+__device__ __forceinline__ void store8f(float* __restrict__ p, int64_t j, int64_t len, bool vec, const float* v) {
+  if (vec && j + 8 <= len) {
+    *reinterpret_cast<float4*>(p + j) = make_float4(v[0], v[1], v[2], v[3]);
+    *reinterpret_cast<float4*>(p + j + 4) = make_float4(v[4], v[5], v[6], v[7]);
+  } else {
+#pragma unroll
+    for (int e = 0; e < 8; ++e)
+      if (j + e < len) p[j + e] = v[e];
+  }
+}
+
+// The 8*b bits of coordinate group j/8 of one worker's segment stream, as (lo, hi).
+template <int BITS>
+__device__ __forceinline__ void load_chunk(const uint32_t* __restrict__ w, int64_t g, int b, int64_t pad_words,
+                                           uint64_t& lo, uint64_t& hi) {
+  hi = 0;
+  if (BITS == 8) {
+    const uint2 t = *reinterpret_cast<const uint2*>(w + g * 2);
+    lo = (uint64_t)t.x | ((uint64_t)t.y << 32);
+  } else if (BITS == 4) {
+    lo = w[g];
+  } else if (BITS == 2) {
+    lo = reinterpret_cast<const uint16_t*>(w)[g];
+  } else if (BITS == 1) {
+    lo = reinterpret_cast<const uint8_t*>(w)[g];
+  } else {
+    const uint8_t* bytes = reinterpret_cast<const uint8_t*>(w);
+    const int64_t b0 = g * b, limit = pad_words * 4;
+    lo = 0;
+    for (int i = 0; i < b; ++i) {
+      const uint64_t v = (b0 + i < limit) ? bytes[b0 + i] : 0;
+      if (i < 8) lo |= v << (8 * i); else hi |= v << (8 * (i - 8));
+    }
+  }
+}
+
+__device__ __forceinline__ uint32_t extract(uint64_t lo, uint64_t hi, int pos, int b) {
+  uint64_t v;
+  if (pos < 64) {
+    v = lo >> pos;
+    if (pos + b > 64) v |= hi << (64 - pos);
+  } else {
+    v = hi >> (pos - 64);
+  }
+  return (uint32_t)v & ((1u << b) - 1u);
+}
+
+template <int BITS>  // 1, 2, 4, 8: fixed width; 0: b in 1..16 from the arguments; 32: floats
+__global__ void __launch_bounds__(AT) unpack_average_prox_kernel(AggArgs a) {
+  const int tile = blockIdx.x;
+  const int seg = a.tile_seg ? a.tile_seg[tile] : 0;
+  const SegInfo s = a.segs[seg];
+  const int64_t tstart = (int64_t)(tile - s.tile_first) * TILE;
+  const int tid = threadIdx.x;
+  const int b = (BITS == 0) ? a.b : BITS;
+
+  extern __shared__ float sdelta[];
+  for (int i = tid; i < a.N; i += AT) sdelta[i] = a.delta[(int64_t)i * a.nseg + seg];
+  __syncthreads();
+
+  const float invN = __fdiv_rn(1.0f, (float)a.N);
+  float* xs = a.x + s.off;
+  const float* mus = a.mu ? a.mu + s.off : nullptr;
+  float* vs = a.v_out ? a.v_out + s.off : nullptr;
+  const bool vec = aligned16(xs) && (!mus || aligned16(mus)) && (!vs || aligned16(vs)) &&
+                   (a.mode == 0 || (aligned16(a.y + s.off) && aligned16(a.z + s.off) && aligned16(a.ysum + s.off) &&
+                                    aligned16(a.vhat + s.off)));
+
+#pragma unroll 1
+  for (int it = 0; it < AITER; ++it) {
+    const int64_t j = tstart + (int64_t)it * AGROUP + tid * 8;
+    if (j >= s.len) break;
+    float acc[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+    const uint32_t* w = a.codes + s.word_off;
+    if constexpr (BITS == 32) {
+#pragma unroll 2
+      for (int i = 0; i < a.N; ++i) {
+        const uint32_t* wi = w + (int64_t)i * a.stride_words;
+        const float di = sdelta[i];
+        float val[8];
+        load8f(reinterpret_cast<const float*>(wi), j, s.len, true, val);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[e] = add_rn(acc[e], mul_rn(di, val[e]));
+      }
+    } else {
+#pragma unroll 4
+      for (int i = 0; i < a.N; ++i) {
+        uint64_t lo, hi;
+        load_chunk<BITS>(w + (int64_t)i * a.stride_words, j >> 3, b, s.pad_words, lo, hi);
+        const float di = sdelta[i];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          uint32_t code;
+          if constexpr (BITS == 0) code = extract(lo, hi, e * b, b);
+          else code = (uint32_t)(lo >> (e * BITS)) & ((1u << BITS) - 1u);
+          acc[e] = add_rn(acc[e], mul_rn(di, index_as_float(code, b)));
+        }
+      }
+    }
+    float xv[8], mv[8], vv[8];
+    load8f(xs, j, s.len, vec, xv);
+    if (mus) {
+      load8f(mus, j, s.len, vec, mv);
+    } else {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) mv[e] = 0.f;
+    }
+#pragma unroll
+    for (int e = 0; e < 8; ++e) vv[e] = add_rn(mul_rn(acc[e], invN), mv[e]);
+    if (vs) store8f(vs, j, s.len, vec, vv);
+    if (a.mode == 0) {
+      const float kappa = mul_rn(a.eta, a.lambda_l1);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) xv[e] = soft_threshold(__fsub_rn(xv[e], mul_rn(a.eta, vv[e])), kappa);
+      store8f(xs, j, s.len, vec, xv);
+    } else {
+      float zv[8], hv[8], sv[8], yv[8];
+      load8f(a.z + s.off, j, s.len, vec, zv);
+      load8f(a.vhat + s.off, j, s.len, vec, hv);
+      load8f(a.ysum + s.off, j, s.len, vec, sv);
+      const float ky = mul_rn(a.inv4L, a.lambda_l1), kz = mul_rn(a.alpha, a.lambda_l1);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        yv[e] = soft_threshold(__fsub_rn(xv[e], mul_rn(a.inv4L, vv[e])), ky);
+        zv[e] = soft_threshold(__fsub_rn(zv[e], mul_rn(a.alpha, hv[e])), kz);
+        sv[e] = add_rn(sv[e], yv[e]);
+      }
+      store8f(a.y + s.off, j, s.len, vec, yv);
+      store8f(a.z + s.off, j, s.len, vec, zv);
+      store8f(a.ysum + s.off, j, s.len, vec, sv);
+    }
+  }
+  if (a.k_counter && blockIdx.x == 0 && tid == 0) *a.k_counter += 1;
+}
+
+}  // namespace
+
+cudaError_t launch_unpack_average_prox(const AggArgs& a, cudaStream_t st) {
+  if (a.ntiles <= 0) return cudaSuccess;
+  const dim3 grid((unsigned)a.ntiles), block(AT);
+  const size_t sh = (size_t)a.N * sizeof(float);
+  switch (a.b) {
+    case 1: unpack_average_prox_kernel<1><<<grid, block, sh, st>>>(a); break;
+    case 2: unpack_average_prox_kernel<2><<<grid, block, sh, st>>>(a); break;
+    case 4: unpack_average_prox_kernel<4><<<grid, block, sh, st>>>(a); break;
+    case 8: unpack_average_prox_kernel<8><<<grid, block, sh, st>>>(a); break;
+    case 32: unpack_average_prox_kernel<32><<<grid, block, sh, st>>>(a); break;
+    default: unpack_average_prox_kernel<0><<<grid, block, sh, st>>>(a); break;
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace lpc

@@ -1,0 +1,258 @@
+// Device-side building blocks shared by the kernels of the library: the counter-based random
+// streams, the fixed-order fp32 reductions, the per-coordinate quantizer and small PTX wrappers.
+//
+// Arithmetic contract.  The packed codes are a deterministic function of the input floats, so every
+// fp32 operation on the way to a code is an explicit round-to-nearest intrinsic (__fmul_rn, __fadd_rn,
+// __fdiv_rn) that the compiler can neither contract into an FMA nor reorder.  The files are also
+// compiled with -fmad=false.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "lpc_status.h"
+
+namespace lpc {
+
+// ---- stream tags ---------------------------------------------------------------------------------
+constexpr uint32_t TAG_ROUND = 0;
+constexpr uint32_t TAG_BATCH = 1;
+constexpr uint32_t TAG_BATCH_J = 2;
+
+// Philox4x32-10 (Salmon et al., SC'11).  Ten rounds; each round multiplies counter words 0 and 2 by
+// two fixed constants, xors the high halves with the other two words and the key, and the key
+// advances by two Weyl increments between rounds.
+struct U4 { uint32_t x, y, z, w; };
+
+__device__ __forceinline__ U4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                            uint32_t k0, uint32_t k1) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+    c0 = hi1 ^ c1 ^ k0;
+    c1 = lo1;
+    c2 = hi0 ^ c3 ^ k1;
+    c3 = lo0;
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+  return U4{c0, c1, c2, c3};
+}
+
+// Block `block` of stream (tag, worker, k): counter = (block, k_lo, worker | tag<<24, k_hi), key = seed.
+__device__ __forceinline__ U4 stream_block(uint64_t seed, uint32_t tag, uint32_t worker, uint64_t k,
+                                           uint32_t block) {
+  return philox4x32_10(block, (uint32_t)k, (worker & 0xFFFFFFu) | (tag << 24), (uint32_t)(k >> 32),
+                       (uint32_t)seed, (uint32_t)(seed >> 32));
+}
+
+// ---- fixed-order (balanced binary tree over the coordinate index) fp32 sums ------------------------
+__device__ __forceinline__ float add_rn(float a, float b) { return __fadd_rn(a, b); }
+__device__ __forceinline__ float mul_rn(float a, float b) { return __fmul_rn(a, b); }
+
+__device__ __forceinline__ float tree8(const float* v) {
+  return add_rn(add_rn(add_rn(v[0], v[1]), add_rn(v[2], v[3])), add_rn(add_rn(v[4], v[5]), add_rn(v[6], v[7])));
+}
+__device__ __forceinline__ float tree4(float a, float b, float c, float d) {
+  return add_rn(add_rn(a, b), add_rn(c, d));
+}
+
+// All 32 lanes end with the tree sum of the 32 lane values (lane order = leaf order).
+__device__ __forceinline__ float warp_tree_sum(float v) {
+#pragma unroll
+  for (int m = 1; m < 32; m <<= 1) v = add_rn(v, __shfl_xor_sync(0xFFFFFFFFu, v, m));
+  return v;
+}
+__device__ __forceinline__ uint32_t warp_max_u32(uint32_t v) { return __reduce_max_sync(0xFFFFFFFFu, v); }
+
+// Tree sum of `count` floats (count a power of two, <= 1024) stored in order in shared memory,
+// evaluated by one thread.  Small counts only (cross-warp / cross-CTA partials).
+__device__ __forceinline__ float smem_tree_sum(const float* v, int count) {
+  // iterative pairwise reduction with a small stack, same association as the recursive definition
+  float stack[12];
+  int top = 0;
+  for (int i = 0; i < count; ++i) {
+    float cur = v[i];
+    int idx = i;
+    while (idx & 1) {  // completed a right child: combine with the waiting left sibling
+      cur = add_rn(stack[--top], cur);
+      idx >>= 1;
+    }
+    stack[top++] = cur;
+  }
+  return stack[0];
+}
+
+// ---- scale (Eq. 2) -----------------------------------------------------------------------------------
+struct Scale {
+  float delta;   // transmitted float: codebook spacing (b=1: T; b=32: 1)
+  float rdelta;  // 1/delta (0 when degenerate)
+  float T;       // clip threshold
+  float lower;   // lower end of the hull: -(T+delta)  (b=1: -T)
+  uint32_t flags;  // bit0 degenerate (send zeros), bit1 non-finite input
+};
+
+constexpr int CLIP_NONE = 0, CLIP_LAMBDA = 1, CLIP_STD = 2;
+
+// max_bits = max over coordinates of the bit pattern of |u| (monotone in |u|; NaN/Inf >= 0x7F800000).
+__device__ __forceinline__ Scale make_scale(uint32_t max_bits, float S1, float S2, int64_t len, int b,
+                                            int clip_mode, float clip_value) {
+  Scale sc;
+  if (max_bits >= 0x7F800000u) {
+    sc.delta = __int_as_float(0x7FC00000);
+    sc.rdelta = 0.f; sc.T = 0.f; sc.lower = 0.f; sc.flags = 3u;
+    return sc;
+  }
+  const float M = __uint_as_float(max_bits);
+  float T = M;
+  if (clip_mode == CLIP_LAMBDA) {
+    T = mul_rn(clip_value, M);
+  } else if (clip_mode == CLIP_STD) {
+    const double mean = __ddiv_rn((double)S1, (double)len);
+    double var = __dsub_rn(__ddiv_rn((double)S2, (double)len), __dmul_rn(mean, mean));
+    if (var < 0.0) var = 0.0;
+    double t = __dmul_rn((double)clip_value, __dsqrt_rn(var));
+    if (t > (double)M) t = (double)M;
+    T = __double2float_rn(t);
+  }
+  sc.T = T;
+  if (b == 32) {
+    sc.delta = 1.f; sc.rdelta = 1.f; sc.lower = -T; sc.flags = 0u;
+    return sc;
+  }
+  const float Lv = (float)((1 << (b - 1)) - 1);
+  const float delta = (b == 1) ? T : __fdiv_rn(T, Lv);
+  const float rdelta = __fdiv_rn(1.0f, delta);
+  if (M == 0.f || T == 0.f || delta == 0.f || isinf(rdelta) || isnan(rdelta)) {
+    sc.delta = 0.f; sc.rdelta = 0.f; sc.lower = 0.f; sc.flags = 1u;
+    return sc;
+  }
+  sc.delta = delta;
+  sc.rdelta = rdelta;
+  sc.lower = (b == 1) ? -T : -add_rn(T, delta);
+  sc.flags = 0u;
+  return sc;
+}
+
+// ---- quantizer of Section 2.2 for one coordinate -----------------------------------------------------
+// Returns the stored code c = k + 2^(b-1) (b=1: the bit).  r16 is the coordinate's 16-bit random lane.
+template <int B_>
+__device__ __forceinline__ uint32_t quantize_code(float u, float rdelta, uint32_t r16) {
+  if (B_ == 1) {
+    float s = mul_rn(u, rdelta);
+    s = fminf(fmaxf(s, -1.f), 1.f);
+    const float f = mul_rn(add_rn(s, 1.f), 0.5f);
+    return (add_rn((float)r16, 0.5f) < mul_rn(f, 65536.f)) ? 1u : 0u;
+  }
+  constexpr float lo = -(float)(1 << (B_ - 1));
+  constexpr float hi = (float)((1 << (B_ - 1)) - 1);
+  float s = mul_rn(u, rdelta);
+  s = fminf(fmaxf(s, lo), hi);  // projection onto the hull (rule 2)
+  const float fl = floorf(s);
+  const float f = __fsub_rn(s, fl);  // exact
+  const int up = (add_rn((float)r16, 0.5f) < mul_rn(f, 65536.f)) ? 1 : 0;  // rule 1
+  return (uint32_t)((int)fl + up + (1 << (B_ - 1)));
+}
+
+// Runtime-b version (b in 1..16) for the generic paths.
+__device__ __forceinline__ uint32_t quantize_code_rt(float u, float rdelta, uint32_t r16, int b) {
+  if (b == 1) return quantize_code<1>(u, rdelta, r16);
+  const float lo = -(float)(1 << (b - 1));
+  const float hi = (float)((1 << (b - 1)) - 1);
+  float s = mul_rn(u, rdelta);
+  s = fminf(fmaxf(s, lo), hi);
+  const float fl = floorf(s);
+  const float f = __fsub_rn(s, fl);
+  const int up = (add_rn((float)r16, 0.5f) < mul_rn(f, 65536.f)) ? 1 : 0;
+  return (uint32_t)((int)fl + up + (1 << (b - 1)));
+}
+
+// Exact float value of the signed codebook index of a stored code (code < 2^16).
+__device__ __forceinline__ float index_as_float(uint32_t code, int b) {
+  // 0x4B000000 is 2^23: or-ing a small integer into its mantissa and subtracting 2^23 converts exactly.
+  const float biased = __uint_as_float(0x4B000000u | code);
+  if (b == 1) return __fsub_rn(mul_rn(__fsub_rn(biased, 8388608.f), 2.f), 1.f);
+  return __fsub_rn(biased, 8388608.f + (float)(1 << (b - 1)));
+}
+
+__device__ __forceinline__ float soft_threshold(float w, float kappa) {
+  const float a = fmaxf(__fsub_rn(fabsf(w), kappa), 0.f);
+  return copysignf(a, w);
+}
+
+// The eight 16-bit lanes of a Philox block: lane e of coordinate group = bits of word e/2, low half first.
+__device__ __forceinline__ uint32_t lane16(const U4& r, int e) {
+  const uint32_t w = (e < 2) ? r.x : (e < 4) ? r.y : (e < 6) ? r.z : r.w;
+  return (e & 1) ? (w >> 16) : (w & 0xFFFFu);
+}
+
+// ---- mbarrier / bulk-copy (TMA) wrappers ---------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_fence_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+// Bounded wait: returns false when the phase did not complete within about two seconds.
+__device__ __forceinline__ uint64_t global_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint64_t limit_ns = 2000000000ull) {
+  const uint32_t addr = smem_u32(bar);
+  uint64_t t0 = 0;
+  for (uint32_t it = 0;; ++it) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(addr), "r"(parity)
+        : "memory");
+    if (ok) return true;
+    if ((it & 255u) == 255u) {
+      const uint64_t now = global_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > limit_ns) return false;
+    }
+  }
+}
+// One-dimensional bulk copy global -> this CTA's shared memory, completion counted on `bar`.
+// dst, src 16-byte aligned, bytes a multiple of 16.
+__device__ __forceinline__ void bulk_load(void* dst_smem, const void* src_gmem, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   smem_u32(dst_smem)),
+               "l"(src_gmem), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+
+__device__ __forceinline__ int64_t next_pow2_i64(int64_t n) {
+  int64_t p = 1;
+  while (p < n) p <<= 1;
+  return p;
+}
+
+// ---- losses ----------------------------------------------------------------------------------------------
+constexpr int LOSS_LOGISTIC = 0, LOSS_LEAST_SQUARES = 1;
+
+__device__ __forceinline__ float loss_deriv(int loss, float m, float y) {
+  if (loss == LOSS_LEAST_SQUARES) return __fsub_rn(m, y);
+  const double t = __dmul_rn((double)y, (double)m);
+  return __double2float_rn(__ddiv_rn(-(double)y, __dadd_rn(1.0, exp(t))));
+}
+__device__ __forceinline__ double loss_value(int loss, float m, float y) {
+  if (loss == LOSS_LEAST_SQUARES) {
+    const double r = (double)m - (double)y;
+    return 0.5 * r * r;
+  }
+  const double t = (double)y * (double)m;
+  return (t > 0.0) ? log1p(exp(-t)) : (-t + log1p(exp(t)));
+}
+
+}  // namespace lpc

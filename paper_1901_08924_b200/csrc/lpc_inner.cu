@@ -1,0 +1,460 @@
+// The fused worker side of one inner iteration (Algorithm 1 steps 6-7, Algorithm 2 steps 7-8 and 11):
+// minibatch sampling, the SVRG difference u^i, the scale of Eq. 2, the stochastic quantizer and bit
+// packing in one kernel.  u^i lives in registers from the moment it is formed until its codes are
+// stored; it is never written to memory (unless the inspection tap is on).
+//
+// Design: one thread-block cluster per worker.  The CS CTAs of a cluster split the coordinate range
+// [0, P) (P = d rounded up to a power of two) into contiguous slices of SL = P/CS coordinates.  A CTA
+// pulls its slice of the B sampled rows into shared memory with bulk copies (TMA) signalled on one
+// mbarrier, computes the slice's part of every margin <X_a, x>, and exchanges the parts through
+// distributed shared memory; after one cluster barrier every CTA knows the B margins and forms the
+// coefficients l'(m_a(x)) - l'(m_a(x~)) (the snapshot margins are cached).  u is then accumulated from
+// the rows still resident in shared memory, its max / sum / sum of squares are exchanged the same
+// way, and after a second cluster barrier every CTA derives the same scale and quantizes its slice.
+// In ALPC-SVRG one more cluster handles the shared batch J and stores v^ = u_J + mu in full
+// precision.  No load with cluster multicast is used; each CTA fetches its own slice.
+#include <cooperative_groups.h>
+
+#include "lpc_device.cuh"
+#include "lpc_inner.h"
+
+namespace cg = cooperative_groups;
+
+namespace lpc {
+namespace {
+
+constexpr int IT = 256;           // threads per CTA
+constexpr int IGROUP = IT * 8;    // coordinates per pass
+constexpr int MAXP = 4;           // passes per CTA: SL <= 8192
+constexpr int MAXB = 64;          // minibatch rows
+constexpr int MAXCS = 8;
+
+struct Smem {
+  uint64_t bar;
+  int64_t idx[MAXB];
+  float yv[MAXB];
+  float msnap[MAXB];
+  float coef[MAXB];
+  float wpart[MAXB * MAXP * 8];   // per-row warp partials of the margin products
+  float mpart[MAXB * MAXCS];      // per-row slice partials of every CTA of the cluster (written by peers)
+  float s1part[MAXCS], s2part[MAXCS];
+  uint32_t maxpart[MAXCS];
+  float ws1[MAXP * 8], ws2[MAXP * 8];
+  uint32_t wmax[8];
+  uint32_t wclip[8];
+  Scale scale;
+  int load_ok;
+  __align__(16) uint8_t stage[IT * 16];
+};
+
+template <int BITS>  // 1, 2, 4, 8: fixed-width packing; 0: b from the arguments (1..16 or 32)
+__global__ void __launch_bounds__(IT) inner_kernel(InnerArgs a) {
+  cg::cluster_group cluster = cg::this_cluster();
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  Smem& sm = *reinterpret_cast<Smem*>(smem_raw);
+  float* rows = reinterpret_cast<float*>(smem_raw + ((sizeof(Smem) + 15) & ~(size_t)15));  // B x SL
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int rank = (int)cluster.block_rank();
+  const int CS = a.CS, SL = a.SL, B = a.B, d = a.d;
+  const int worker = blockIdx.y;
+  const bool is_J = (worker == a.N);
+  const uint64_t k = a.k_base + (a.k_dev ? *a.k_dev : 0ull);
+  const int b = BITS ? BITS : a.b;
+  const int passes = (SL + IGROUP - 1) / IGROUP;
+  const int c0 = rank * SL;                         // first coordinate of this CTA's slice
+  const int width = max(0, min(SL, d - c0));        // coordinates of the slice that exist
+
+  // ---- sampling (Algorithm 1 step 6): slot a uses word 0 of block a of the batch stream -----------------
+  if (tid < B) {
+    int64_t lo, span;
+    uint32_t tag, wk;
+    if (is_J) { lo = 0; span = a.n; tag = TAG_BATCH_J; wk = 0; }
+    else if (a.sample_global) { lo = 0; span = a.n; tag = TAG_BATCH; wk = (uint32_t)worker; }
+    else { span = a.n / a.N; lo = (int64_t)worker * span; tag = TAG_BATCH; wk = (uint32_t)worker; }
+    const U4 r = stream_block(a.seed, tag, wk, k, (uint32_t)tid);
+    const int64_t row = lo + (int64_t)(((uint64_t)r.x * (uint64_t)span) >> 32);
+    sm.idx[tid] = row;
+    sm.yv[tid] = a.y[row];
+    sm.msnap[tid] = a.margins[row];
+  }
+  if (tid == 0) {
+    mbar_init(&sm.bar, 1);
+    mbar_fence_init();
+  }
+  // Every CTA of the cluster announces that it is running; peers wait for this before their first
+  // store into this CTA's shared memory.
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  __syncthreads();
+  if (tid == 0 && width > 0) {
+    const uint32_t bytes = (uint32_t)width * 4u;
+    mbar_expect_tx(&sm.bar, bytes * (uint32_t)B);
+    for (int r = 0; r < B; ++r) bulk_load(rows + (size_t)r * SL, a.X + sm.idx[r] * (int64_t)d + c0, bytes, &sm.bar);
+  }
+
+  // ---- this thread's coordinates and the iterate at them ---------------------------------------------------
+  float xr[MAXP][8];
+#pragma unroll
+  for (int p = 0; p < MAXP; ++p) {
+    const int off = p * IGROUP + tid * 8;  // offset inside the slice
+#pragma unroll
+    for (int e = 0; e < 8; ++e) xr[p][e] = 0.f;
+    if (p < passes && off < width) {  // width is a multiple of 4
+      const float4 v0 = *reinterpret_cast<const float4*>(a.x + c0 + off);
+      xr[p][0] = v0.x; xr[p][1] = v0.y; xr[p][2] = v0.z; xr[p][3] = v0.w;
+      if (off + 4 < width) {
+        const float4 v1 = *reinterpret_cast<const float4*>(a.x + c0 + off + 4);
+        xr[p][4] = v1.x; xr[p][5] = v1.y; xr[p][6] = v1.z; xr[p][7] = v1.w;
+      }
+    }
+  }
+
+  bool ok = true;
+  if (width > 0) ok = mbar_wait(&sm.bar, 0);
+  if (!ok) {
+    atomicOr(a.dev_status, DEV_TIMEOUT);
+    ok = mbar_wait(&sm.bar, 0);  // one more bounded chance for the copies in flight before going on
+  }
+
+  // A row value of the slice (zero outside the existing columns).
+  auto row8 = [&](int r, int off, float* v) {
+#pragma unroll
+    for (int e = 0; e < 8; ++e) v[e] = 0.f;
+    if (off < width) {
+      const float4 v0 = *reinterpret_cast<const float4*>(rows + (size_t)r * SL + off);
+      v[0] = v0.x; v[1] = v0.y; v[2] = v0.z; v[3] = v0.w;
+      if (off + 4 < width) {
+        const float4 v1 = *reinterpret_cast<const float4*>(rows + (size_t)r * SL + off + 4);
+        v[4] = v1.x; v[5] = v1.y; v[6] = v1.z; v[7] = v1.w;
+      }
+    }
+  };
+
+  // ---- margins <X_a, x>: balanced tree over the column index ---------------------------------------------------
+  for (int r = 0; r < B; ++r) {
+#pragma unroll
+    for (int p = 0; p < MAXP; ++p) {
+      if (p < passes) {
+        float v[8], pr[8];
+        row8(r, p * IGROUP + tid * 8, v);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) pr[e] = mul_rn(v[e], xr[p][e]);
+        const float s = warp_tree_sum(tree8(pr));
+        if (lane == 0) sm.wpart[(r * MAXP + p) * 8 + warp] = s;
+      }
+    }
+  }
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");  // all peers have started
+  __syncthreads();
+  if (tid < B) {
+    int np = 1;
+    while (np < passes) np <<= 1;
+    float part;
+    if (np == 1) {
+      part = smem_tree_sum(&sm.wpart[tid * MAXP * 8], 8);
+    } else {
+      float tmp[MAXP];
+      for (int p = 0; p < np; ++p) tmp[p] = (p < passes) ? smem_tree_sum(&sm.wpart[(tid * MAXP + p) * 8], 8) : 0.f;
+      part = (np == 2) ? add_rn(tmp[0], tmp[1]) : tree4(tmp[0], tmp[1], tmp[2], tmp[3]);
+    }
+    for (int q = 0; q < CS; ++q) {
+      float* peer = cluster.map_shared_rank(sm.mpart, q);
+      peer[tid * MAXCS + rank] = part;
+    }
+  }
+  cluster.sync();
+  if (tid < B) {
+    const float m = smem_tree_sum(&sm.mpart[tid * MAXCS], CS);
+    const float g_cur = loss_deriv(a.loss, m, sm.yv[tid]);
+    const float g_snap = loss_deriv(a.loss, sm.msnap[tid], sm.yv[tid]);
+    const float c = __fsub_rn(g_cur, g_snap);
+    sm.coef[tid] = c;
+    if (rank == 0) {
+      if (a.idx_tap) a.idx_tap[(int64_t)worker * B + tid] = sm.idx[tid];
+      if (a.coef_tap) a.coef_tap[(int64_t)worker * B + tid] = c;
+    }
+  }
+  __syncthreads();
+
+  // ---- u = (1/B) sum_a c_a X_a, summed in batch order (Algorithm 1 step 6) ------------------------------------
+  const float invB = __fdiv_rn(1.0f, (float)B);
+  float u[MAXP][8];
+#pragma unroll
+  for (int p = 0; p < MAXP; ++p) {
+#pragma unroll
+    for (int e = 0; e < 8; ++e) u[p][e] = 0.f;
+    if (p < passes) {
+      for (int r = 0; r < B; ++r) {
+        float v[8];
+        row8(r, p * IGROUP + tid * 8, v);
+        const float c = sm.coef[r];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) u[p][e] = add_rn(u[p][e], mul_rn(c, v[e]));
+      }
+#pragma unroll
+      for (int e = 0; e < 8; ++e) u[p][e] = mul_rn(u[p][e], invB);
+    }
+  }
+
+  if (is_J) {  // double sampling: v^ = u_J + mu in full precision, nothing quantized
+#pragma unroll
+    for (int p = 0; p < MAXP; ++p) {
+      const int off = p * IGROUP + tid * 8;
+      if (p < passes) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e)
+          if (off + e < width) a.vhat[c0 + off + e] = add_rn(u[p][e], a.mu[c0 + off + e]);
+      }
+    }
+    return;  // the whole cluster leaves together: no further cluster barrier on this path
+  }
+  if (a.u_tap) {
+#pragma unroll
+    for (int p = 0; p < MAXP; ++p) {
+      const int off = p * IGROUP + tid * 8;
+      if (p < passes) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e)
+          if (off + e < width) a.u_tap[(int64_t)worker * d + c0 + off + e] = u[p][e];
+      }
+    }
+  }
+
+  // ---- scale (Eq. 2): max |u| and, for the c*std rule, tree sums of u and u^2 ----------------------------------
+  uint32_t mx = 0;
+#pragma unroll
+  for (int p = 0; p < MAXP; ++p) {
+    if (p < passes) {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) mx = max(mx, __float_as_uint(fabsf(u[p][e])));
+      if (a.clip_mode == CLIP_STD) {
+        float sq[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) sq[e] = mul_rn(u[p][e], u[p][e]);
+        const float s1 = warp_tree_sum(tree8(u[p]));
+        const float s2 = warp_tree_sum(tree8(sq));
+        if (lane == 0) { sm.ws1[p * 8 + warp] = s1; sm.ws2[p * 8 + warp] = s2; }
+      }
+    }
+  }
+  mx = warp_max_u32(mx);
+  if (lane == 0) sm.wmax[warp] = mx;
+  __syncthreads();
+  if (tid == 0) {
+    uint32_t m = 0;
+    for (int w = 0; w < 8; ++w) m = max(m, sm.wmax[w]);
+    float s1 = 0.f, s2 = 0.f;
+    if (a.clip_mode == CLIP_STD) {
+      int np = 1;
+      while (np < passes) np <<= 1;
+      for (int i = passes * 8; i < np * 8; ++i) { sm.ws1[i] = 0.f; sm.ws2[i] = 0.f; }
+      s1 = smem_tree_sum(sm.ws1, np * 8);
+      s2 = smem_tree_sum(sm.ws2, np * 8);
+    }
+    for (int q = 0; q < CS; ++q) {
+      cluster.map_shared_rank(sm.maxpart, q)[rank] = m;
+      cluster.map_shared_rank(sm.s1part, q)[rank] = s1;
+      cluster.map_shared_rank(sm.s2part, q)[rank] = s2;
+    }
+  }
+  cluster.sync();
+  if (tid == 0) {
+    uint32_t m = 0;
+    for (int q = 0; q < CS; ++q) m = max(m, sm.maxpart[q]);
+    float S1 = 0.f, S2 = 0.f;
+    if (a.clip_mode == CLIP_STD) { S1 = smem_tree_sum(sm.s1part, CS); S2 = smem_tree_sum(sm.s2part, CS); }
+    sm.scale = make_scale(m, S1, S2, d, b, a.clip_mode, a.clip_value);
+    if (rank == 0) {
+      a.delta[worker] = sm.scale.delta;
+      if (sm.scale.flags & 2u) atomicOr(a.dev_status, DEV_NONFINITE);
+    }
+  }
+  __syncthreads();
+  const Scale sc = sm.scale;
+  const bool degenerate = (sc.flags & 1u) != 0;
+  const uint32_t zero_code = (b == 1) ? 0u : (1u << (b - 1));
+  uint32_t* out = a.codes + (int64_t)worker * a.stride_words;
+
+  // ---- quantize (Section 2.2) and pack ---------------------------------------------------------------------------
+  uint32_t nclip = 0;
+#pragma unroll
+  for (int p = 0; p < MAXP; ++p) {
+    if (p >= passes) break;
+    const int off = p * IGROUP + tid * 8;
+    const int c = c0 + off;  // global coordinate, multiple of 8
+    const bool mine = off < SL;
+    if (b == 32) {
+      if (mine) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          float v = u[p][e];
+          if (a.clip_mode != CLIP_NONE && c + e < d) {
+            if (v > sc.T) { v = sc.T; ++nclip; }
+            if (v < -sc.T) { v = -sc.T; ++nclip; }
+          }
+          if (c + e < a.pad_words) out[c + e] = (c + e < d) ? __float_as_uint(v) : 0u;
+        }
+      }
+      continue;
+    }
+    uint64_t lo = 0, hi = 0;
+    if (mine && c < d) {
+      U4 r = U4{0, 0, 0, 0};
+      if (!degenerate) r = stream_block(a.seed, TAG_ROUND, (uint32_t)worker, k, (uint32_t)(c >> 3));
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        if (c + e < d) {
+          uint32_t code = zero_code;
+          if (!degenerate) {
+            code = BITS ? quantize_code<BITS ? BITS : 2>(u[p][e], sc.rdelta, lane16(r, e))
+                        : quantize_code_rt(u[p][e], sc.rdelta, lane16(r, e), b);
+            nclip += (u[p][e] > sc.T || u[p][e] < sc.lower) ? 1u : 0u;
+          }
+          const int pos = e * b;
+          if (pos < 64) {
+            lo |= (uint64_t)code << pos;
+            if (pos + b > 64) hi |= (uint64_t)code >> (64 - pos);
+          } else {
+            hi |= (uint64_t)code << (pos - 64);
+          }
+        }
+      }
+    }
+    if (BITS == 8) {
+      const int64_t w = (int64_t)(c >> 3) * 2;
+      if (mine && w < a.pad_words) *reinterpret_cast<uint2*>(out + w) = make_uint2((uint32_t)lo, (uint32_t)(lo >> 32));
+    } else if (BITS == 4) {
+      const int64_t w = c >> 3;
+      if (mine && w < a.pad_words) out[w] = (uint32_t)lo;
+    } else if (BITS == 2) {
+      const uint32_t own = (uint32_t)lo;
+      const uint32_t next = __shfl_down_sync(0xFFFFFFFFu, own, 1);
+      const int64_t w = c >> 4;
+      if (mine && (lane & 1) == 0 && w < a.pad_words) out[w] = own | (next << 16);
+    } else if (BITS == 1) {
+      const uint32_t own = (uint32_t)lo;
+      const uint32_t n1 = __shfl_down_sync(0xFFFFFFFFu, own, 1);
+      const uint32_t n2 = __shfl_down_sync(0xFFFFFFFFu, own, 2);
+      const uint32_t n3 = __shfl_down_sync(0xFFFFFFFFu, own, 3);
+      const int64_t w = c >> 5;
+      if (mine && (lane & 3) == 0 && w < a.pad_words) out[w] = own | (n1 << 8) | (n2 << 16) | (n3 << 24);
+    } else {
+      if (p > 0) __syncthreads();
+      for (int i = 0; i < b; ++i)
+        sm.stage[tid * b + i] = (uint8_t)((i < 8) ? (lo >> (8 * i)) : (hi >> (8 * (i - 8))));
+      __syncthreads();
+      const int span = min(IGROUP, SL - p * IGROUP);           // coordinates of this pass (multiple of 32)
+      const int64_t w0 = (int64_t)((c0 + p * IGROUP) >> 5) * b;  // exact: the pass starts on a multiple of 32
+      const uint32_t* st = reinterpret_cast<const uint32_t*>(sm.stage);
+      for (int w = tid; w < (span / 32) * b; w += IT)
+        if (w0 + w < a.pad_words) out[w0 + w] = st[w];
+    }
+  }
+  nclip = __reduce_add_sync(0xFFFFFFFFu, nclip);
+  if (lane == 0) sm.wclip[warp] = nclip;
+  __syncthreads();
+  if (tid == 0) {
+    uint32_t t = 0;
+    for (int w = 0; w < 8; ++w) t += sm.wclip[w];
+    a.clipped_part[worker * MAXCS + rank] = t;
+  }
+}
+
+template <int BITS>
+cudaError_t launch_t(const InnerArgs& a, size_t smem, cudaStream_t st) {
+  cudaError_t e = cudaFuncSetAttribute(inner_kernel<BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)a.CS, (unsigned)(a.N + (a.has_J ? 1 : 0)), 1);
+  cfg.blockDim = dim3(IT, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = (unsigned)a.CS;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, inner_kernel<BITS>, a);
+}
+
+__global__ void clipped_sum_kernel(const uint32_t* __restrict__ part, int N, uint32_t* __restrict__ out) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < N) {
+    uint32_t t = 0;
+    for (int q = 0; q < MAXCS; ++q) t += part[i * MAXCS + q];
+    out[i] = t;
+  }
+}
+
+// x = tau1*z + tau2*x~ + (1 - tau1 - tau2)*y  (Algorithm 2 step 6), evaluated as ((tau1*z)+(tau2*x~))+(tau3*y).
+__global__ void coupling_kernel(const float* __restrict__ z, const float* __restrict__ xt, const float* __restrict__ y,
+                                float tau1, float tau2, int d, float* __restrict__ x) {
+  const float tau3 = __fsub_rn(__fsub_rn(1.0f, tau1), tau2);
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j < d) x[j] = add_rn(add_rn(mul_rn(tau1, z[j]), mul_rn(tau2, xt[j])), mul_rn(tau3, y[j]));
+}
+
+// x~ candidate = ysum / m (Algorithm 3 step 5) becomes the iterate; ysum is cleared.
+__global__ void mean_y_kernel(float* __restrict__ ysum, float inv_m, int d, float* __restrict__ x) {
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j < d) {
+    x[j] = mul_rn(ysum[j], inv_m);
+    ysum[j] = 0.f;
+  }
+}
+
+}  // namespace
+
+int inner_max_b() { return MAXB; }
+int inner_clipped_stride() { return MAXCS; }
+
+// Picks the cluster size and slice width.  Returns false when d is too large for the fused kernel.
+bool inner_plan(int d, int B, int want_cs, int max_smem, int* CS_out, int* SL_out, size_t* smem_out) {
+  int P = 1;
+  while (P < d) P <<= 1;
+  if (P < 32) P = 32;
+  for (int cs = 1; cs <= MAXCS; cs <<= 1) {
+    if (want_cs > 0 && cs != want_cs) continue;
+    const int SL = P / cs;
+    if (SL < 32) break;
+    if (SL > IGROUP * MAXP) continue;
+    const size_t smem = ((sizeof(Smem) + 15) & ~(size_t)15) + (size_t)B * SL * 4;
+    if (smem > (size_t)max_smem) continue;
+    // automatic choice: the first (smallest) cluster whose slice is covered in one pass
+    if (want_cs > 0 || SL <= IGROUP || cs == MAXCS) {
+      *CS_out = cs; *SL_out = SL; *smem_out = smem;
+      return true;
+    }
+  }
+  return false;
+}
+
+cudaError_t launch_inner(const InnerArgs& a, size_t smem, cudaStream_t st) {
+  switch (a.b) {
+    case 1: return launch_t<1>(a, smem, st);
+    case 2: return launch_t<2>(a, smem, st);
+    case 4: return launch_t<4>(a, smem, st);
+    case 8: return launch_t<8>(a, smem, st);
+    default: return launch_t<0>(a, smem, st);
+  }
+}
+
+cudaError_t launch_clipped_sum(const uint32_t* part, int N, uint32_t* out, cudaStream_t st) {
+  clipped_sum_kernel<<<(N + 127) / 128, 128, 0, st>>>(part, N, out);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_coupling(const float* z, const float* xt, const float* y, float tau1, float tau2, int d, float* x,
+                            cudaStream_t st) {
+  coupling_kernel<<<(d + 255) / 256, 256, 0, st>>>(z, xt, y, tau1, tau2, d, x);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_mean_y(float* ysum, float inv_m, int d, float* x, cudaStream_t st) {
+  mean_y_kernel<<<(d + 255) / 256, 256, 0, st>>>(ysum, inv_m, d, x);
+  return cudaGetLastError();
+}
+
+}  // namespace lpc

@@ -1,0 +1,48 @@
+// Launch interface of the fused worker kernel and the small ALPC helper kernels.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace lpc {
+
+struct InnerArgs {
+  const float* X;
+  const float* y;
+  int64_t n;
+  int d;
+  int loss;
+  int N, B, b;
+  int clip_mode;
+  float clip_value;
+  uint64_t seed;
+  int sample_global;
+  uint64_t k_base;         // iteration number = k_base + *k_dev (k_dev nullable)
+  const uint64_t* k_dev;
+  const float* x;          // point where the minibatch gradients are taken (d)
+  const float* margins;    // cached <X_a, snapshot> (n)
+  const float* mu;         // snapshot gradient, read by the J cluster only
+  int has_J;               // 1: an extra cluster (index N) handles ALPC's shared batch J
+  float* vhat;             // d, written by the J cluster
+  uint32_t* codes;         // N * stride_words
+  int64_t stride_words;
+  int64_t pad_words;       // words of one worker's stream including zero padding (multiple of 4)
+  float* delta;            // N
+  uint32_t* clipped_part;  // N * inner_clipped_stride()
+  int64_t* idx_tap;        // (N+1) * B, nullable
+  float* coef_tap;         // (N+1) * B, nullable
+  float* u_tap;            // N * d, nullable
+  unsigned int* dev_status;
+  int CS;                  // CTAs per cluster
+  int SL;                  // coordinates per CTA slice
+};
+
+int inner_max_b();
+int inner_clipped_stride();
+bool inner_plan(int d, int B, int want_cs, int max_smem, int* CS_out, int* SL_out, size_t* smem_out);
+cudaError_t launch_inner(const InnerArgs& a, size_t smem, cudaStream_t st);
+cudaError_t launch_clipped_sum(const uint32_t* part, int N, uint32_t* out, cudaStream_t st);
+cudaError_t launch_coupling(const float* z, const float* xt, const float* y, float tau1, float tau2, int d, float* x,
+                            cudaStream_t st);
+cudaError_t launch_mean_y(float* ysum, float inv_m, int d, float* x, cudaStream_t st);
+
+}  // namespace lpc

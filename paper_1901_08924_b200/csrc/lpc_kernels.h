@@ -1,0 +1,91 @@
+// Internal launch interface between the C ABI (lpc_api.cu) and the kernel files.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace lpc {
+
+constexpr int TILE = 8192;  // coordinates per CTA tile of the standalone quantizer / aggregator kernels
+
+// One tensor segment of a (segmented) vector.
+struct SegInfo {
+  int64_t off;         // first element in the vector
+  int64_t len;         // elements
+  int64_t word_off;    // first word of its packed stream inside a worker's stream (multiple of 4)
+  int64_t pad_words;   // words reserved for it (multiple of 4)
+  uint32_t block_base; // first Philox block of its rounding stream
+  int32_t tile_first;  // first tile index
+  int32_t tile_count;
+  int32_t pad_;
+};
+
+struct ScaleRec {  // result of the scale rule for one (worker, segment)
+  float delta, rdelta, T, lower;
+  uint32_t flags, pad0, pad1, pad2;
+};
+
+struct QuantArgs {
+  const float* U;
+  const float* U_sub;  // nullable
+  int64_t ld;
+  int N;
+  int b;
+  int clip_mode;
+  float clip_value;
+  uint64_t seed;
+  uint64_t k;
+  const SegInfo* segs;     // device, nseg entries
+  const int32_t* tile_seg; // device, ntiles entries
+  int nseg;
+  int ntiles;
+  // scratch
+  uint32_t* pmax;  // N * ntiles
+  float* ps1;      // N * ntiles
+  float* ps2;      // N * ntiles
+  ScaleRec* scales;  // N * nseg
+  // outputs
+  uint32_t* codes;
+  int64_t stride_words;
+  float* delta_out;       // N * nseg
+  uint32_t* clipped_out;  // N * nseg (nullable -> internal scratch is passed instead)
+  unsigned int* dev_status;
+};
+
+cudaError_t launch_quantize_pack(const QuantArgs& a, cudaStream_t st);
+
+struct AggArgs {
+  const uint32_t* codes;
+  int64_t stride_words;
+  const float* delta;  // N * nseg
+  int N;
+  int b;
+  const SegInfo* segs;
+  const int32_t* tile_seg;
+  int nseg;
+  int ntiles;
+  const float* mu;  // nullable
+  float* x;         // in/out
+  float eta;
+  float lambda_l1;
+  float* v_out;     // nullable
+  uint64_t* k_counter;  // nullable: incremented by one when the kernel finishes (graph replay)
+  // mode 1 (Algorithm 2, steps 12-13): x is read only (the coupled point x_{k+1}) and instead of the
+  // proximal step on x the kernel updates  y = soft(x - inv4L*v, inv4L*lambda_l1),
+  // z = soft(z - alpha*vhat, alpha*lambda_l1),  ysum += y.
+  int mode;
+  float* y;
+  float* z;
+  float* ysum;
+  const float* vhat;
+  float alpha;
+  float inv4L;
+};
+
+cudaError_t launch_unpack_average_prox(const AggArgs& a, cudaStream_t st);
+
+}  // namespace lpc
+
+namespace lpc {
+cudaError_t launch_stream_blocks(uint64_t seed, uint32_t tag, uint32_t worker, uint64_t k, uint32_t block0,
+                                 int64_t count, uint32_t* out, cudaStream_t st);
+}  // namespace lpc

@@ -1,0 +1,322 @@
+// Quantization step of Algorithm 1 (step 7) for stand-alone worker vectors: the scale of Eq. 2
+// (a reduction pass), then the stochastic quantizer Q_(delta,b) of Section 2.2 and bit packing
+// (a second pass).  Vectors may be split into tensor segments that each get their own scale.
+//
+// Layout of the work: a CTA owns one tile of TILE consecutive coordinates of one segment of one
+// worker; a thread owns groups of 8 consecutive coordinates (two 128-bit loads, one Philox block,
+// 8*b packed bits).  All sums follow the balanced binary tree over the coordinate index, so the
+// scale -- and with it every code -- does not depend on the tiling.
+#include "lpc_device.cuh"
+#include "lpc_kernels.h"
+
+namespace lpc {
+namespace {
+
+constexpr int QT = 256;                   // threads per CTA
+constexpr int QGROUP = QT * 8;            // coordinates per CTA sweep
+constexpr int QITER = TILE / QGROUP;      // sweeps per tile
+static_assert(QITER * QGROUP == TILE, "tile must be a whole number of sweeps");
+
+// Eight consecutive values u[j..j+8) of (p - q), zero beyond len.  `vec` says 16-byte loads are legal.
+__device__ __forceinline__ void load8(const float* __restrict__ p, const float* __restrict__ q, int64_t j,
+                                      int64_t len, bool vec, float* v) {
+  if (vec && j + 8 <= len) {
+    const float4 a = *reinterpret_cast<const float4*>(p + j);
+    const float4 c = *reinterpret_cast<const float4*>(p + j + 4);
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = c.x; v[5] = c.y; v[6] = c.z; v[7] = c.w;
+    if (q) {
+      const float4 e = *reinterpret_cast<const float4*>(q + j);
+      const float4 f = *reinterpret_cast<const float4*>(q + j + 4);
+      v[0] = __fsub_rn(v[0], e.x); v[1] = __fsub_rn(v[1], e.y); v[2] = __fsub_rn(v[2], e.z); v[3] = __fsub_rn(v[3], e.w);
+      v[4] = __fsub_rn(v[4], f.x); v[5] = __fsub_rn(v[5], f.y); v[6] = __fsub_rn(v[6], f.z); v[7] = __fsub_rn(v[7], f.w);
+    }
+  } else {
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const int64_t i = j + e;
+      v[e] = (i < len) ? (q ? __fsub_rn(p[i], q[i]) : p[i]) : 0.f;
+    }
+  }
+}
+
+__device__ __forceinline__ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// ---- pass 1: per-tile partial (max |u| as bit pattern, tree sums of u and u^2) ---------------------------
+template <bool NEED_SUMS>
+__global__ void __launch_bounds__(QT) stats_kernel(QuantArgs a) {
+  const int tile = blockIdx.x, worker = blockIdx.y;
+  const int seg = a.tile_seg ? a.tile_seg[tile] : 0;
+  const SegInfo s = a.segs[seg];
+  const int64_t tstart = (int64_t)(tile - s.tile_first) * TILE;
+  const float* p = a.U + (int64_t)worker * a.ld + s.off;
+  const float* q = a.U_sub ? a.U_sub + (int64_t)worker * a.ld + s.off : nullptr;
+  const bool vec = aligned16(p) && (!q || aligned16(q));
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+  __shared__ float sh1[QITER * 8], sh2[QITER * 8];
+  __shared__ uint32_t shm[8];
+
+  uint32_t mx = 0;
+#pragma unroll
+  for (int it = 0; it < QITER; ++it) {
+    const int64_t j = tstart + (int64_t)it * QGROUP + tid * 8;
+    float v[8];
+    if (j < s.len) {
+      load8(p, q, j, s.len, vec, v);
+    } else {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) v[e] = 0.f;
+    }
+#pragma unroll
+    for (int e = 0; e < 8; ++e) mx = max(mx, __float_as_uint(fabsf(v[e])));
+    if (NEED_SUMS) {
+      float sq[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) sq[e] = mul_rn(v[e], v[e]);
+      const float s1 = warp_tree_sum(tree8(v));
+      const float s2 = warp_tree_sum(tree8(sq));
+      if (lane == 0) { sh1[it * 8 + warp] = s1; sh2[it * 8 + warp] = s2; }
+    }
+  }
+  mx = warp_max_u32(mx);
+  if (lane == 0) shm[warp] = mx;
+  __syncthreads();
+  if (tid == 0) {
+    uint32_t m = 0;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) m = max(m, shm[w]);
+    const int64_t o = (int64_t)worker * a.ntiles + tile;
+    a.pmax[o] = m;
+    if (NEED_SUMS) {
+      a.ps1[o] = smem_tree_sum(sh1, QITER * 8);
+      a.ps2[o] = smem_tree_sum(sh2, QITER * 8);
+    }
+  }
+}
+
+// Tree sum over `count` tile partials by one CTA of QT threads (leaf order = tile order).
+__device__ float block_tree_sum(const float* __restrict__ v, int count, float* sh8) {
+  int64_t P = 1;
+  while (P < count) P <<= 1;
+  const int chunk = (P >= QT) ? (int)(P / QT) : 1;
+  const int lo = threadIdx.x * chunk;
+  float stack[32];
+  int top = 0;
+  for (int i = 0; i < chunk; ++i) {
+    float cur = (lo + i < count) ? v[lo + i] : 0.f;
+    int idx = i;
+    while (idx & 1) { cur = add_rn(stack[--top], cur); idx >>= 1; }
+    stack[top++] = cur;
+  }
+  const float w = warp_tree_sum(stack[0]);
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) sh8[threadIdx.x >> 5] = w;
+  __syncthreads();
+  return tree8(sh8);
+}
+
+// ---- between the passes: one CTA per (segment, worker) finishes the reductions and applies Eq. 2 -------
+__global__ void __launch_bounds__(QT) finish_kernel(QuantArgs a) {
+  const int seg = blockIdx.x, worker = blockIdx.y;
+  const SegInfo s = a.segs[seg];
+  const int64_t base = (int64_t)worker * a.ntiles + s.tile_first;
+  __shared__ float sh8[8];
+  __shared__ uint32_t shm[8];
+  uint32_t mx = 0;
+  for (int t = threadIdx.x; t < s.tile_count; t += QT) mx = max(mx, a.pmax[base + t]);
+  mx = warp_max_u32(mx);
+  if ((threadIdx.x & 31) == 0) shm[threadIdx.x >> 5] = mx;
+  float S1 = 0.f, S2 = 0.f;
+  if (a.clip_mode == CLIP_STD) {
+    S1 = block_tree_sum(a.ps1 + base, s.tile_count, sh8);
+    S2 = block_tree_sum(a.ps2 + base, s.tile_count, sh8);
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    uint32_t m = 0;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) m = max(m, shm[w]);
+    const Scale sc = make_scale(m, S1, S2, s.len, a.b, a.clip_mode, a.clip_value);
+    const int64_t o = (int64_t)worker * a.nseg + seg;
+    ScaleRec r;
+    r.delta = sc.delta; r.rdelta = sc.rdelta; r.T = sc.T; r.lower = sc.lower; r.flags = sc.flags;
+    r.pad0 = r.pad1 = r.pad2 = 0;
+    a.scales[o] = r;
+    a.delta_out[o] = sc.delta;
+    a.clipped_out[o] = 0;
+    if (sc.flags & 2u) atomicOr(a.dev_status, DEV_NONFINITE);
+  }
+}
+
+// ---- pass 2: quantize and pack -----------------------------------------------------------------------------
+// BITS = 1, 2, 4, 8: register/shuffle packing with direct coalesced stores.
+// BITS = 0: any b in 1..16 read from the arguments; each thread's 8*b bits are b whole bytes, staged
+//           through shared memory and written out as words.
+template <int BITS>
+__global__ void __launch_bounds__(QT) quantize_kernel(QuantArgs a) {
+  const int tile = blockIdx.x, worker = blockIdx.y;
+  const int seg = a.tile_seg ? a.tile_seg[tile] : 0;
+  const SegInfo s = a.segs[seg];
+  const int64_t tstart = (int64_t)(tile - s.tile_first) * TILE;
+  const float* p = a.U + (int64_t)worker * a.ld + s.off;
+  const float* q = a.U_sub ? a.U_sub + (int64_t)worker * a.ld + s.off : nullptr;
+  const bool vec = aligned16(p) && (!q || aligned16(q));
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int b = BITS ? BITS : a.b;
+  const ScaleRec sc = a.scales[(int64_t)worker * a.nseg + seg];
+  const bool degenerate = (sc.flags & 1u) != 0;
+  const uint32_t zero_code = (b == 1) ? 0u : (1u << (b - 1));
+  uint32_t* out = a.codes + (int64_t)worker * a.stride_words + s.word_off;
+
+  __shared__ __align__(16) uint8_t stage[BITS == 0 ? QT * 16 : 16];
+
+  uint32_t nclip = 0;
+#pragma unroll
+  for (int it = 0; it < QITER; ++it) {
+    const int64_t sweep0 = tstart + (int64_t)it * QGROUP;  // first coordinate of this sweep (segment-local)
+    const int64_t j = sweep0 + tid * 8;
+    uint64_t lo = 0, hi = 0;  // this thread's 8*b bits
+    if (j < s.len) {
+      float v[8];
+      load8(p, q, j, s.len, vec, v);
+      U4 r = U4{0, 0, 0, 0};
+      if (!degenerate) r = stream_block(a.seed, TAG_ROUND, (uint32_t)worker, a.k, s.block_base + (uint32_t)(j >> 3));
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        if (j + e < s.len) {
+          uint32_t code = zero_code;
+          if (!degenerate) {
+            code = BITS ? quantize_code<BITS ? BITS : 2>(v[e], sc.rdelta, lane16(r, e))
+                        : quantize_code_rt(v[e], sc.rdelta, lane16(r, e), b);
+            nclip += (v[e] > sc.T || v[e] < sc.lower) ? 1u : 0u;
+          }
+          const int pos = e * b;
+          if (pos < 64) {
+            lo |= (uint64_t)code << pos;
+            if (pos + b > 64) hi |= (uint64_t)code >> (64 - pos);
+          } else {
+            hi |= (uint64_t)code << (pos - 64);
+          }
+        }
+      }
+    }
+    // ---- store
+    if (BITS == 8) {
+      const int64_t w = (j >> 3) * 2;
+      if (w < s.pad_words) *reinterpret_cast<uint2*>(out + w) = make_uint2((uint32_t)lo, (uint32_t)(lo >> 32));
+    } else if (BITS == 4) {
+      const int64_t w = j >> 3;
+      if (w < s.pad_words) out[w] = (uint32_t)lo;
+    } else if (BITS == 2) {
+      const uint32_t mine = (uint32_t)lo;  // 16 bits
+      const uint32_t next = __shfl_down_sync(0xFFFFFFFFu, mine, 1);
+      const int64_t w = j >> 4;
+      if ((lane & 1) == 0 && w < s.pad_words) out[w] = mine | (next << 16);
+    } else if (BITS == 1) {
+      const uint32_t mine = (uint32_t)lo;  // 8 bits
+      const uint32_t n1 = __shfl_down_sync(0xFFFFFFFFu, mine, 1);
+      const uint32_t n2 = __shfl_down_sync(0xFFFFFFFFu, mine, 2);
+      const uint32_t n3 = __shfl_down_sync(0xFFFFFFFFu, mine, 3);
+      const int64_t w = j >> 5;
+      if ((lane & 3) == 0 && w < s.pad_words) out[w] = mine | (n1 << 8) | (n2 << 16) | (n3 << 24);
+    } else {
+      // generic: b bytes per thread at byte tid*b of the sweep's 256*b-byte block
+      if (it > 0) __syncthreads();
+      for (int i = 0; i < b; ++i)
+        stage[tid * b + i] = (uint8_t)((i < 8) ? (lo >> (8 * i)) : (hi >> (8 * (i - 8))));
+      __syncthreads();
+      const int64_t w0 = (sweep0 >> 5) * b;  // sweep0 is a multiple of 2048, so this is exact
+      const uint32_t* st = reinterpret_cast<const uint32_t*>(stage);
+      for (int w = tid; w < (QGROUP / 32) * b; w += QT)
+        if (w0 + w < s.pad_words) out[w0 + w] = st[w];
+    }
+  }
+  nclip = __reduce_add_sync(0xFFFFFFFFu, nclip);
+  if (lane == 0 && nclip) atomicAdd(&a.clipped_out[(int64_t)worker * a.nseg + seg], nclip);
+}
+
+// b = 32: the message is the vector itself (clamped to [-T, T] when a clip rule is set).
+__global__ void __launch_bounds__(QT) bypass_kernel(QuantArgs a) {
+  const int tile = blockIdx.x, worker = blockIdx.y;
+  const int seg = a.tile_seg ? a.tile_seg[tile] : 0;
+  const SegInfo s = a.segs[seg];
+  const int64_t tstart = (int64_t)(tile - s.tile_first) * TILE;
+  const float* p = a.U + (int64_t)worker * a.ld + s.off;
+  const float* q = a.U_sub ? a.U_sub + (int64_t)worker * a.ld + s.off : nullptr;
+  const bool vec = aligned16(p) && (!q || aligned16(q));
+  const int tid = threadIdx.x, lane = tid & 31;
+  const ScaleRec sc = a.scales[(int64_t)worker * a.nseg + seg];
+  uint32_t* out = a.codes + (int64_t)worker * a.stride_words + s.word_off;
+  uint32_t nclip = 0;
+#pragma unroll
+  for (int it = 0; it < QITER; ++it) {
+    const int64_t j = tstart + (int64_t)it * QGROUP + tid * 8;
+    if (j >= s.pad_words) continue;
+    float v[8];
+    if (j < s.len) {
+      load8(p, q, j, s.len, vec, v);
+    } else {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) v[e] = 0.f;
+    }
+    if (a.clip_mode != CLIP_NONE) {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        if (j + e < s.len) {
+          if (v[e] > sc.T) { v[e] = sc.T; ++nclip; }
+          if (v[e] < -sc.T) { v[e] = -sc.T; ++nclip; }
+        }
+      }
+    }
+#pragma unroll
+    for (int e = 0; e < 8; ++e)
+      if (j + e < s.pad_words) out[j + e] = (j + e < s.len) ? __float_as_uint(v[e]) : 0u;
+  }
+  nclip = __reduce_add_sync(0xFFFFFFFFu, nclip);
+  if (lane == 0 && nclip) atomicAdd(&a.clipped_out[(int64_t)worker * a.nseg + seg], nclip);
+}
+
+}  // namespace
+
+cudaError_t launch_quantize_pack(const QuantArgs& a, cudaStream_t st) {
+  if (a.N <= 0 || a.nseg <= 0) return cudaSuccess;
+  const dim3 grid((unsigned)(a.ntiles > 0 ? a.ntiles : 1), (unsigned)a.N), block(QT);
+  if (a.ntiles > 0) {
+    if (a.clip_mode == CLIP_STD)
+      stats_kernel<true><<<grid, block, 0, st>>>(a);
+    else
+      stats_kernel<false><<<grid, block, 0, st>>>(a);
+  }
+  finish_kernel<<<dim3((unsigned)a.nseg, (unsigned)a.N), block, 0, st>>>(a);  // also covers empty segments
+  if (a.ntiles <= 0) return cudaGetLastError();
+  switch (a.b) {
+    case 1: quantize_kernel<1><<<grid, block, 0, st>>>(a); break;
+    case 2: quantize_kernel<2><<<grid, block, 0, st>>>(a); break;
+    case 4: quantize_kernel<4><<<grid, block, 0, st>>>(a); break;
+    case 8: quantize_kernel<8><<<grid, block, 0, st>>>(a); break;
+    case 32: bypass_kernel<<<grid, block, 0, st>>>(a); break;
+    default: quantize_kernel<0><<<grid, block, 0, st>>>(a); break;
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace lpc
+
+namespace lpc {
+namespace {
+__global__ void stream_blocks_kernel(uint64_t seed, uint32_t tag, uint32_t worker, uint64_t k, uint32_t block0,
+                                     int64_t count, uint32_t* __restrict__ out) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < count) {
+    const U4 r = stream_block(seed, tag, worker, k, block0 + (uint32_t)i);
+    out[4 * i + 0] = r.x; out[4 * i + 1] = r.y; out[4 * i + 2] = r.z; out[4 * i + 3] = r.w;
+  }
+}
+}  // namespace
+
+cudaError_t launch_stream_blocks(uint64_t seed, uint32_t tag, uint32_t worker, uint64_t k, uint32_t block0,
+                                 int64_t count, uint32_t* out, cudaStream_t st) {
+  stream_blocks_kernel<<<(unsigned)((count + 255) / 256), 256, 0, st>>>(seed, tag, worker, k, block0, count, out);
+  return cudaGetLastError();
+}
+}  // namespace lpc
