@@ -80,6 +80,16 @@ typedef struct lpc_ctx lpc_ctx;
 #define LPC_OPT_TAP_U 1         /* 1: inner steps also store u^i and v for inspection (slower) */
 #define LPC_OPT_CLUSTER_SIZE 2  /* thread-block cluster size per worker for the fused step: 0 = automatic, else 1, 2, 4 or 8 */
 #define LPC_OPT_USE_GRAPH 3     /* 1 (default): lpc_inner_steps replays a CUDA graph; 0: plain launches */
+#define LPC_OPT_PROFILE 4       /* 1: record CUDA events around every kernel launch (graph replay is off meanwhile) */
+
+/* kernel classes reported by lpc_get_profile */
+#define LPC_KERNEL_SNAPSHOT 0    /* the pass over X of lpc_snapshot_full_grad / lpc_objective */
+#define LPC_KERNEL_WORKER 1      /* fused sampling + SVRG difference + scale + quantize + pack */
+#define LPC_KERNEL_AGGREGATE 2   /* unpack + average + proximal step (or ALPC y/z updates) */
+#define LPC_KERNEL_QUANT_STATS 3 /* first pass of lpc_quantize_pack (max, sums) */
+#define LPC_KERNEL_QUANT_PACK 4  /* second pass of lpc_quantize_pack (quantize + pack) */
+#define LPC_KERNEL_OTHER 5       /* small helper kernels */
+#define LPC_KERNEL_KINDS 6
 
 /*
  * Creates a context for problem (1).  Section 1 "Contribution" (Eq. 1), Section 2.1 (N workers),
@@ -195,6 +205,11 @@ int lpc_alpc_end_epoch(lpc_ctx* ctx, int64_t m);
 /* P(x) = f(x) + lambda_l1*||x||_1 (Eq. 1) in one pass over X.  x nullable (= current iterate);
  * P_out is a HOST pointer; the call waits for the stream. */
 int lpc_objective(lpc_ctx* ctx, const float* x, double* P_out);
+
+/* Per-kernel device time measured with CUDA events on the context's stream while LPC_OPT_PROFILE is
+ * on: ms_out[kind] total milliseconds, launches_out[kind] launches (both HOST arrays of
+ * LPC_KERNEL_KINDS entries, nullable).  reset != 0 clears the totals.  Host-synchronous. */
+int lpc_get_profile(lpc_ctx* ctx, double* ms_out, int64_t* launches_out, int32_t reset);
 
 /* Bits that the simulated workers would have transmitted so far (host counters): step 1 =
  * 32*d*N*(N-1) per snapshot, step 2 = (32+b*len)*N*(N-1) per inner step or quantize call (Table 1). */

@@ -90,7 +90,15 @@ struct lpc_ctx {
   size_t q_scale_cap = 0;
   // graph replay
   cudaGraphExec_t graph = nullptr;
+  cudaStream_t cap_stream = nullptr;  // used only to capture the graph
   GraphKey graph_key;
+  // per-kernel timing (LPC_OPT_PROFILE): event pairs recorded around launches, resolved on demand
+  int profile = 0;
+  std::vector<cudaEvent_t> ev_pool;   // 2 events per timed launch
+  std::vector<int> ev_kind;
+  size_t ev_used = 0;                 // timed launches recorded and not yet resolved
+  double prof_ms[LPC_KERNEL_KINDS] = {0};
+  int64_t prof_n[LPC_KERNEL_KINDS] = {0};
   // accounting
   uint64_t step1_bits = 0, step2_bits = 0;
   int sm_count = 148, max_smem = 227 * 1024;
@@ -214,6 +222,57 @@ int dalloc(lpc_ctx* c, T** p, size_t count) {
 
 bool has_model(const lpc_ctx* c) { return c->X != nullptr; }
 
+// ---- per-kernel timing ------------------------------------------------------------------------------
+int prof_resolve(lpc_ctx* c) {
+  if (c->ev_used == 0) return LPC_OK;
+  CU(c, cudaStreamSynchronize(c->stream));
+  for (size_t i = 0; i < c->ev_used; ++i) {
+    float ms = 0.f;
+    CU(c, cudaEventElapsedTime(&ms, c->ev_pool[2 * i], c->ev_pool[2 * i + 1]));
+    c->prof_ms[c->ev_kind[i]] += (double)ms;
+    c->prof_n[c->ev_kind[i]] += 1;
+  }
+  c->ev_used = 0;
+  return LPC_OK;
+}
+
+struct ProfScope {  // records an event before and after one launch when profiling is on
+  lpc_ctx* c;
+  cudaEvent_t stop = nullptr;
+  ProfScope(lpc_ctx* ctx, int kind) : c(ctx) {
+    if (!c->profile) return;
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(c->stream, &cs) != cudaSuccess || cs != cudaStreamCaptureStatusNone) return;
+    if (c->ev_used >= 32768) prof_resolve(c);
+    if (c->ev_pool.size() < 2 * (c->ev_used + 1)) {
+      cudaEvent_t a = nullptr, b = nullptr;
+      if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) return;
+      c->ev_pool.push_back(a);
+      c->ev_pool.push_back(b);
+      c->ev_kind.push_back(kind);
+    }
+    c->ev_kind[c->ev_used] = kind;
+    cudaEventRecord(c->ev_pool[2 * c->ev_used], c->stream);
+    stop = c->ev_pool[2 * c->ev_used + 1];
+    c->ev_used += 1;
+  }
+  ~ProfScope() {
+    if (stop) cudaEventRecord(stop, c->stream);
+  }
+};
+
+void prof_hook(void* user, int kind, int begin) {
+  // used by launch functions that issue several kernels: begin = 1 opens a scope, 0 closes it
+  static thread_local ProfScope* open = nullptr;
+  lpc_ctx* c = static_cast<lpc_ctx*>(user);
+  if (begin) {
+    open = new ProfScope(c, kind);
+  } else if (open) {
+    delete open;
+    open = nullptr;
+  }
+}
+
 InnerArgs inner_args(lpc_ctx* c, uint64_t k_base, const uint64_t* k_dev, int has_J) {
   InnerArgs a;
   a.X = c->X; a.y = c->y; a.n = c->n; a.d = c->d; a.loss = c->loss;
@@ -249,23 +308,23 @@ int replan_inner(lpc_ctx* c) {
 // One LPC inner step enqueued on the stream (Algorithm 1 steps 6-10).
 int enqueue_lpc_step(lpc_ctx* c, float eta, uint64_t k_base, const uint64_t* k_dev, uint64_t* k_counter) {
   InnerArgs ia = inner_args(c, k_base, k_dev, 0);
-  CU(c, launch_inner(ia, c->innerSmem, c->stream));
+  { ProfScope ps_(c, LPC_KERNEL_WORKER); CU(c, launch_inner(ia, c->innerSmem, c->stream)); }
   AggArgs ag = agg_args(c, c->inner_seg, c->codes, c->delta, c->mu, c->x, eta, c->lambda_l1, c->tap_u ? c->v_tap : nullptr);
   ag.k_counter = k_counter;
-  CU(c, launch_unpack_average_prox(ag, c->stream));
+  { ProfScope ps_(c, LPC_KERNEL_AGGREGATE); CU(c, launch_unpack_average_prox(ag, c->stream)); }
   return LPC_OK;
 }
 
 // One ALPC step enqueued on the stream (Algorithm 2 steps 6-13).
 int enqueue_alpc_step(lpc_ctx* c, float tau1, float tau2, float alpha, float inv4L, uint64_t k_base,
                       const uint64_t* k_dev, uint64_t* k_counter) {
-  CU(c, launch_coupling(c->zv, c->xt, c->yv, tau1, tau2, c->d, c->x, c->stream));
+  { ProfScope ps_(c, LPC_KERNEL_OTHER); CU(c, launch_coupling(c->zv, c->xt, c->yv, tau1, tau2, c->d, c->x, c->stream)); }
   InnerArgs ia = inner_args(c, k_base, k_dev, 1);
-  CU(c, launch_inner(ia, c->innerSmem, c->stream));
+  { ProfScope ps_(c, LPC_KERNEL_WORKER); CU(c, launch_inner(ia, c->innerSmem, c->stream)); }
   AggArgs ag = agg_args(c, c->inner_seg, c->codes, c->delta, c->mu, c->x, 0.f, c->lambda_l1, c->tap_u ? c->v_tap : nullptr);
   ag.k_counter = k_counter;
   ag.mode = 1; ag.y = c->yv; ag.z = c->zv; ag.ysum = c->ysum; ag.vhat = c->vhat; ag.alpha = alpha; ag.inv4L = inv4L;
-  CU(c, launch_unpack_average_prox(ag, c->stream));
+  { ProfScope ps_(c, LPC_KERNEL_AGGREGATE); CU(c, launch_unpack_average_prox(ag, c->stream)); }
   return LPC_OK;
 }
 
@@ -278,17 +337,23 @@ int run_steps(lpc_ctx* c, int kind, const float* p, uint64_t k0, int64_t count) 
     return kind == 0 ? enqueue_lpc_step(c, p[0], kb, kd, kc) : enqueue_alpc_step(c, p[0], p[1], p[2], p[3], kb, kd, kc);
   };
   int64_t done = 0;
-  if (c->use_graph && count >= GRAPH_STEPS) {
+  if (c->use_graph && !c->profile && count >= GRAPH_STEPS) {
     GraphKey key;
     key.kind = kind; key.steps = GRAPH_STEPS; key.tap = c->tap_u; key.cs = c->CS; key.sample_global = c->sample_global;
     for (int i = 0; i < 4; ++i) key.p[i] = p[i];
     if (!c->graph || !(c->graph_key == key)) {
       if (c->graph) { cudaGraphExecDestroy(c->graph); c->graph = nullptr; }
       cudaGraph_t g = nullptr;
-      CU(c, cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal));
+      // Capture on a stream of our own: the caller's stream may be the legacy default stream, which
+      // cannot be captured.  Nothing runs during capture; the graph is launched on the caller's stream.
+      if (!c->cap_stream) CU(c, cudaStreamCreateWithFlags(&c->cap_stream, cudaStreamNonBlocking));
+      cudaStream_t user = c->stream;
+      CU(c, cudaStreamBeginCapture(c->cap_stream, cudaStreamCaptureModeThreadLocal));
+      c->stream = c->cap_stream;
       int rc = LPC_OK;
       for (int i = 0; i < GRAPH_STEPS && rc == LPC_OK; ++i) rc = one(0, c->k_dev, c->k_dev);
-      cudaError_t e = cudaStreamEndCapture(c->stream, &g);
+      c->stream = user;
+      cudaError_t e = cudaStreamEndCapture(c->cap_stream, &g);
       if (rc != LPC_OK) { if (g) cudaGraphDestroy(g); return rc; }
       CU(c, e);
       e = cudaGraphInstantiate(&c->graph, g, 0);
@@ -341,7 +406,7 @@ int snapshot_pass(lpc_ctx* c, const float* point, bool grad, float* margins_out)
   a.partial_f = c->partial_f;
   a.dev_status = c->dev_status;
   const int grid = (int)std::min<int64_t>(c->snapGrid, std::max<int64_t>(a.ntiles, 1));
-  CU(c, launch_snapshot(a, grid, c->snapSmem, c->stream));
+  { ProfScope ps_(c, LPC_KERNEL_SNAPSHOT); CU(c, launch_snapshot(a, grid, c->snapSmem, c->stream)); }
   CU(c, launch_snapshot_reduce(a.partial_mu, c->partial_f, grid, c->dpad, c->d, c->n, c->mu, nullptr, &c->f_dev[0], c->stream));
   return LPC_OK;
 }
@@ -432,6 +497,8 @@ int lpc_destroy(lpc_ctx* c) {
   if (!c) return LPC_OK;
   cudaStreamSynchronize(c->stream);
   if (c->graph) cudaGraphExecDestroy(c->graph);
+  if (c->cap_stream) cudaStreamDestroy(c->cap_stream);
+  for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
   void* ptrs[] = {c->x, c->xt, c->mu, c->margins, c->yv, c->zv, c->ysum, c->vhat, c->v_tap, c->u_tap, c->codes,
                   c->delta, c->clipped_part, c->clipped, c->idx_tap, c->coef_tap, c->k_dev, c->dev_status, c->f_dev,
                   c->partial_mu, c->partial_f, c->q_pmax, c->q_ps1, c->q_ps2, c->q_scales, c->q_clip};
@@ -462,6 +529,10 @@ int lpc_set_option(lpc_ctx* c, int option, int64_t value) {
       }
       return LPC_OK;
     case LPC_OPT_USE_GRAPH: c->use_graph = value ? 1 : 0; return LPC_OK;
+    case LPC_OPT_PROFILE:
+      TRY(prof_resolve(c));
+      c->profile = value ? 1 : 0;
+      return LPC_OK;
     default: return fail(c, LPC_ERR_INVALID_ARG, "unknown option");
   }
 }
@@ -583,6 +654,17 @@ int lpc_objective(lpc_ctx* c, const float* x, double* P_out) {
   return LPC_OK;
 }
 
+int lpc_get_profile(lpc_ctx* c, double* ms_out, int64_t* launches_out, int32_t reset) {
+  if (!c) return LPC_ERR_INVALID_ARG;
+  TRY(prof_resolve(c));
+  for (int i = 0; i < LPC_KERNEL_KINDS; ++i) {
+    if (ms_out) ms_out[i] = c->prof_ms[i];
+    if (launches_out) launches_out[i] = c->prof_n[i];
+    if (reset) { c->prof_ms[i] = 0.0; c->prof_n[i] = 0; }
+  }
+  return LPC_OK;
+}
+
 int lpc_comm_bits(const lpc_ctx* c, uint64_t* step1_bits, uint64_t* step2_bits) {
   if (!c) return LPC_ERR_INVALID_ARG;
   if (step1_bits) *step1_bits = c->step1_bits;
@@ -619,7 +701,7 @@ int lpc_quantize_pack(lpc_ctx* c, const float* U, const float* U_sub, int64_t le
   a.pmax = c->q_pmax; a.ps1 = c->q_ps1; a.ps2 = c->q_ps2; a.scales = c->q_scales;
   a.codes = codes_out; a.stride_words = p.stride_words; a.delta_out = delta_out;
   a.clipped_out = clipped_out ? clipped_out : c->q_clip; a.dev_status = c->dev_status;
-  CU(c, launch_quantize_pack(a, c->stream));
+  CU(c, launch_quantize_pack(a, c->stream, c->profile ? prof_hook : nullptr, c));
   c->step2_bits += p.msg_bits * (uint64_t)c->N * (uint64_t)(c->N - 1);
   return LPC_OK;
 }
@@ -631,7 +713,7 @@ int lpc_unpack_average_prox(lpc_ctx* c, const uint32_t* codes, const float* delt
   if (!aligned16(codes)) return fail(c, LPC_ERR_INVALID_ARG, "codes must be 16-byte aligned");
   TRY(make_plan(c, c->seg, len, c->b, seg_offsets, nseg));
   AggArgs a = agg_args(c, c->seg, codes, delta, mu, x_inout, eta, lambda_l1, v_out);
-  CU(c, launch_unpack_average_prox(a, c->stream));
+  { ProfScope ps_(c, LPC_KERNEL_AGGREGATE); CU(c, launch_unpack_average_prox(a, c->stream)); }
   return LPC_OK;
 }
 

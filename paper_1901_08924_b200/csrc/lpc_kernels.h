@@ -51,7 +51,9 @@ struct QuantArgs {
   unsigned int* dev_status;
 };
 
-cudaError_t launch_quantize_pack(const QuantArgs& a, cudaStream_t st);
+// hook(user, kind, begin) is called around each kernel of the sequence (kind = LPC_KERNEL_* of lpc.h) when non-null.
+typedef void (*LaunchHook)(void* user, int kind, int begin);
+cudaError_t launch_quantize_pack(const QuantArgs& a, cudaStream_t st, LaunchHook hook = nullptr, void* user = nullptr);
 
 struct AggArgs {
   const uint32_t* codes;

@@ -278,17 +278,26 @@ __global__ void __launch_bounds__(QT) bypass_kernel(QuantArgs a) {
 
 }  // namespace
 
-cudaError_t launch_quantize_pack(const QuantArgs& a, cudaStream_t st) {
+cudaError_t launch_quantize_pack(const QuantArgs& a, cudaStream_t st, LaunchHook hook, void* user) {
   if (a.N <= 0 || a.nseg <= 0) return cudaSuccess;
   const dim3 grid((unsigned)(a.ntiles > 0 ? a.ntiles : 1), (unsigned)a.N), block(QT);
   if (a.ntiles > 0) {
+    if (hook) hook(user, 3 /* LPC_KERNEL_QUANT_STATS */, 1);
     if (a.clip_mode == CLIP_STD)
       stats_kernel<true><<<grid, block, 0, st>>>(a);
     else
       stats_kernel<false><<<grid, block, 0, st>>>(a);
+    if (hook) hook(user, 3, 0);
   }
+  if (hook) hook(user, 5 /* LPC_KERNEL_OTHER */, 1);
   finish_kernel<<<dim3((unsigned)a.nseg, (unsigned)a.N), block, 0, st>>>(a);  // also covers empty segments
+  if (hook) hook(user, 5, 0);
   if (a.ntiles <= 0) return cudaGetLastError();
+  struct Close {  // closes the timing scope of the second pass on every return path
+    LaunchHook h; void* u;
+    ~Close() { if (h) h(u, 4, 0); }
+  } close_{hook, user};
+  if (hook) hook(user, 4 /* LPC_KERNEL_QUANT_PACK */, 1);
   switch (a.b) {
     case 1: quantize_kernel<1><<<grid, block, 0, st>>>(a); break;
     case 2: quantize_kernel<2><<<grid, block, 0, st>>>(a); break;

@@ -122,7 +122,7 @@ def test_inner_step_chain_of_custody(loss, cfg):
 @pytest.mark.parametrize("cs", [1, 2, 4, 8])
 @pytest.mark.parametrize("clip", [(orc.CLIP_NONE, 1.0), (orc.CLIP_LAMBDA, 0.9), (orc.CLIP_STD, 2.0)])
 def test_inner_step_cluster_sizes_and_clip_rules(cs, clip):
-    P, ctx = _setup(128, 4096, "least_squares", N=3, B=4, b=4, clip=clip)
+    P, ctx = _setup(128, 4096, "least_squares", N=4, B=4, b=4, clip=clip)
     ctx.set_option(lpc.OPT_TAP_U, 1)
     ctx.set_option(lpc.OPT_CLUSTER_SIZE, cs)
     rng = np.random.default_rng(cs)
