@@ -1,0 +1,437 @@
+#!/usr/bin/env python
+"""Benchmark of the LPC-SVRG hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+One "step" is one LPC-SVRG epoch of the least-squares + L1 workload (131,072 x 4,096, 16 workers,
+minibatch 8, 4 bits, clip 3 std): the snapshot full-gradient pass over X followed by m = n/(8N) =
+1,024 fused inner iterations.  The headline value is inner iterations per second over all GPUs
+(each GPU runs an independent replica: the method's communication is counted, never sent).
+The JSON line also carries the roofline of the dominant kernel, per-kernel device times, the
+stand-alone quantize+aggregate bandwidths, the end-to-end number from host buffers and the CPU
+oracle's throughput on the same workload.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "svrg_inner_iters_per_sec"
+UNIT = "inner-iters/s"
+
+WORKLOADS = {
+    # name: n, d, loss, lambda_l1, N, B, b, clip c (std rule), sparsity of w*, label noise
+    "lpc_svrg_ls_131072x4096_N16_B8_b4": dict(n=131072, d=4096, loss="least_squares", lam=1e-4, N=16, B=8, b=4, c=3.0,
+                                              sparsity=0.05, noise=0.01),
+    # the main workload with 1/8 of the rows (X = 268 MB, still larger than L2): for profiler captures
+    "lpc_svrg_ls_16384x4096_N16_B8_b4": dict(n=16384, d=4096, loss="least_squares", lam=1e-4, N=16, B=8, b=4, c=3.0,
+                                             sparsity=0.05, noise=0.01),
+    "lpc_svrg_logistic_4000x1000_N4_B1_b2": dict(n=4000, d=1000, loss="logistic", lam=1e-4, N=4, B=1, b=2, c=2.5,
+                                                 sparsity=0.10, noise=0.1, m=1000, eta=0.1),
+}
+DEFAULT_WORKLOAD = "lpc_svrg_ls_131072x4096_N16_B8_b4"
+
+
+def read_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.path = index, None, None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.index)], stdout=open(self.path, "w"),
+                                         stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        rows = []
+        try:
+            for line in open(self.path):
+                p = [t.strip() for t in line.split(",")]
+                if len(p) >= 7 and p[0].replace(".", "").isdigit():
+                    rows.append(p)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if rows:
+            out["sm_mhz"] = statistics.median(float(r[0]) for r in rows)
+            out["sm_max_mhz"] = max(float(r[1]) for r in rows)
+            names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+            out["reasons"] = [nm for i, nm in enumerate(names) if any(r[3 + i].lower().startswith("active") for r in rows)]
+            out["samples"] = len(rows)
+        return out
+
+
+def visible_index(local_rank):
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        parts = [p for p in vis.split(",") if p]
+        if local_rank < len(parts) and parts[local_rank].isdigit():
+            return int(parts[local_rank])
+    return local_rank
+
+
+def make_problem(w, seed, device):
+    import torch
+    from paper_1901_08924_b200 import synth
+    X, y, _ = synth.linear_problem(w["n"], w["d"], loss=w["loss"], sparsity=w["sparsity"], noise=w["noise"], seed=seed,
+                                   device=device)
+    m = w.get("m", w["n"] // (w["B"] * w["N"]))
+    if "eta" in w:
+        eta = w["eta"]
+    else:  # eta = 1/(6 L) with L = c_loss * max_a ||X_a||^2 (c_loss = 1 least squares, 1/4 logistic)
+        L = float((X.double() ** 2).sum(dim=1).max().item()) * (1.0 if w["loss"] == "least_squares" else 0.25)
+        eta = 1.0 / (6.0 * L)
+    return X, y, m, float(eta)
+
+
+def loss_code(w):
+    from paper_1901_08924_b200 import lpc
+    return lpc.LEAST_SQUARES if w["loss"] == "least_squares" else lpc.LOGISTIC
+
+
+def bytes_per_launch(w, m):
+    """Algorithmic bytes one launch of each kernel class must move."""
+    n, d, N, B, b = w["n"], w["d"], w["N"], w["B"], w["b"]
+    W = (d * b + 31) // 32
+    return {
+        "snapshot": n * d * 4 + n * 4 + n * 4 + d * 4,                       # X once, y, margins written, x~
+        "worker": N * B * d * 4 + N * B * 8 + d * 4 + N * (W * 4 + 4),       # rows once, y + cached margin, x, codes out
+        "aggregate": N * (W * 4 + 4) + 3 * d * 4,                            # codes in, mu, x in, x out
+    }
+
+
+def run_ours(args):
+    import torch
+    from paper_1901_08924_b200 import dist_util, lpc, synth
+
+    size, rank, local = dist_util.world()
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist_util.init("nccl")
+    w = WORKLOADS[args.workload]
+    X, y, m, eta = make_problem(w, seed=rank, device=dev)
+    n, d, N, B, b = w["n"], w["d"], w["N"], w["B"], w["b"]
+    ctx = lpc.Context(X, y, loss_code(w), w["lam"], N, B, b, lpc.CLIP_STD, w["c"], seed=rank)
+
+    def epoch(s):
+        ctx.snapshot_full_grad()
+        ctx.inner_steps(eta, s * m, m)
+
+    s_next = 0
+    for _ in range(max(args.warmup, 3)):
+        epoch(s_next)
+        s_next += 1
+    ctx.sync_status()
+    sampler = ClockSampler(visible_index(local))
+    sampler.start()
+    time.sleep(0.3)
+    st = torch.cuda.current_stream(dev)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2 * args.steps + 1)]
+    dist_util.barrier()
+    torch.cuda.synchronize(dev)
+    t_wall = time.perf_counter()
+    ev[0].record(st)
+    for i in range(args.steps):
+        ctx.snapshot_full_grad()
+        ev[2 * i + 1].record(st)
+        ctx.inner_steps(eta, s_next * m, m)
+        ev[2 * i + 2].record(st)
+        s_next += 1
+    torch.cuda.synchronize(dev)
+    dist_util.barrier()
+    t_wall = time.perf_counter() - t_wall
+    ms_local = ev[0].elapsed_time(ev[-1])
+    snap_ms = sum(ev[2 * i].elapsed_time(ev[2 * i + 1]) for i in range(args.steps)) / args.steps
+    inner_ms = sum(ev[2 * i + 1].elapsed_time(ev[2 * i + 2]) for i in range(args.steps)) / args.steps
+    # keep the GPU busy a little longer so that the clock samples cover load, then stop sampling
+    clocks = sampler.stop()
+    ctx.sync_status()
+    value, ms = dist_util.whole_job_throughput(args.steps * m, ms_local, dev)
+    P_end = ctx.objective()
+
+    # ---- per-kernel device time: the same steps again with an event pair around every launch -------------------
+    ctx.set_option(lpc.OPT_PROFILE, 1)
+    prof_steps = min(args.steps, 2)
+    for _ in range(prof_steps):
+        epoch(s_next)
+        s_next += 1
+    prof = ctx.get_profile()
+    ctx.set_option(lpc.OPT_PROFILE, 0)
+    peak, peak_kind = read_peak()
+    bpl = bytes_per_launch(w, m)
+    bpl["inner_loop"] = m * (bpl["worker"] + bpl["aggregate"])  # one persistent launch runs all m steps
+    kernels = {}
+    for name in ("snapshot", "inner_loop", "worker", "aggregate"):
+        tot_ms, cnt = prof[name]
+        if cnt:
+            us = tot_ms / cnt * 1e3
+            kernels[name] = {"launches_per_step": cnt // prof_steps, "avg_us": round(us, 3),
+                             "share_of_step": round(tot_ms / prof_steps / (snap_ms + inner_ms), 4),
+                             "bytes_per_launch": bpl[name], "gbs": round(bpl[name] / us * 1e-3, 1),
+                             "frac": round(bpl[name] / us * 1e-3 / peak, 4)}
+    dominant = max(kernels, key=lambda k: kernels[k]["avg_us"] * kernels[k]["launches_per_step"]) if kernels else None
+    # Launch duration of the dominant kernel inside the timed region: the events recorded after the snapshot
+    # pass and after the inner loop bracket exactly one persistent launch (or, on the per-step path, m
+    # worker+aggregate pairs whose time is split by the two kernels' event-timed ratio).
+    roofline = None
+    if dominant:
+        kd = kernels[dominant]
+        if dominant == "snapshot":
+            dur_us = snap_ms * 1e3
+        elif dominant == "inner_loop":
+            dur_us = inner_ms * 1e3
+        else:
+            pair = kernels["worker"]["avg_us"] + kernels["aggregate"]["avg_us"]
+            dur_us = inner_ms * 1e3 / m * kd["avg_us"] / pair
+        ach = kd["bytes_per_launch"] / dur_us * 1e-3
+        roofline = {"bound": "hbm", "kernel": dominant, "achieved": round(ach, 1), "peak": peak, "unit": "GB/s",
+                    "frac": round(ach / peak, 4), "traffic": None, "peak_source": f"of {peak_kind}",
+                    "launch_us": round(dur_us, 3),
+                    "note": "latency-bound: an inner step moves %.2f MB behind a strict step-to-step dependency; "
+                            "see kernels{} and quantize_aggregate{} for the bandwidth-bound kernels"
+                            % ((bpl["worker"] + bpl["aggregate"]) / 1e6)}
+    launches_per_epoch = 2 + sum(kernels[k]["launches_per_step"] for k in kernels if k != "snapshot")
+
+    out = {
+        "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": size, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": round(ms / args.steps, 4), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": args.workload, "step": "1 epoch = snapshot full gradient + %d inner iterations" % m,
+                   "n": n, "d": d, "N": N, "B": B, "b": b, "clip": "%.1f*std" % w["c"], "eta": eta,
+                   "l2": "inputs larger than L2 (X is %.2f GB, rows sampled at random)" % (n * d * 4 / 1e9),
+                   "parallelism": "replicas only" if size > 1 else "1 GPU"},
+        "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
+                   "samples": clocks["samples"]},
+        "gpu_launches": args.steps * launches_per_epoch,
+        "snapshot_ms": round(snap_ms, 4), "inner_loop_ms": round(inner_ms, 4),
+        "inner_step_us": round(inner_ms * 1e3 / m, 3), "wall_s": round(t_wall, 4), "objective_end": P_end,
+        "roofline": roofline, "kernels": kernels,
+        "launch_plan": {"loop_cluster_size": ctx.query(lpc.INFO_LOOP_CLUSTER_SIZE),
+                        "loop_launches": ctx.query(lpc.INFO_LOOP_LAUNCHES),
+                        "step_cluster_size": ctx.query(lpc.INFO_STEP_CLUSTER_SIZE),
+                        "snapshot_rows_per_tile": ctx.query(lpc.INFO_SNAPSHOT_ROWS_PER_TILE),
+                        "snapshot_stages": ctx.query(lpc.INFO_SNAPSHOT_STAGES)},
+    }
+    if rank == 0 and size == 1 and not args.quick:
+        out["quantize_aggregate"] = quantize_aggregate_bench(dev, peak)
+        out["e2e"] = e2e_bench(w, X, y, m, eta, dev)
+        out["cpu_baseline"] = cpu_baseline(w, X, y, m, eta)
+    elif rank == 0:
+        out["e2e"] = None
+    ctx.close()
+    dist_util.barrier()
+    if rank == 0:
+        print(json.dumps(out))
+    dist_util.shutdown()
+
+
+def _time_calls(fn, dev, reps):
+    import torch
+    st = torch.cuda.current_stream(dev)
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for _ in range(3):
+        fn()
+    torch.cuda.synchronize(dev)
+    a.record(st)
+    for _ in range(reps):
+        fn()
+    b.record(st)
+    torch.cuda.synchronize(dev)
+    return a.elapsed_time(b) / reps
+
+
+def quantize_aggregate_bench(dev, peak):
+    """Stand-alone quantize+pack and unpack+average+prox at sizes where one call is bandwidth-bound."""
+    import torch
+    from paper_1901_08924_b200 import lpc, synth
+    res = {}
+    # sweep point: 8 workers x 2^26 coordinates (2.1 GB of gradients), Gaussian, b = 4, clip 2 std
+    N, length, b = 8, 1 << 26, 4
+    U = synth.gradient_vectors(N, length, "gauss", seed=1, device=dev)
+    q = lpc.Context(None, None, lpc.LOGISTIC, 0.0, N, 1, b, lpc.CLIP_STD, 2.0, 0)
+    _, stride = lpc.packed_layout(length, b)
+    codes = torch.empty((N, stride), dtype=torch.int32, device=dev)
+    delta = torch.empty((N, 1), dtype=torch.float32, device=dev)
+    clipped = torch.empty((N, 1), dtype=torch.int32, device=dev)
+    x = torch.zeros(length, device=dev)
+    it = [0]
+
+    def quant():
+        it[0] += 1
+        q.quantize_pack(U, it[0], codes_out=codes, delta_out=delta, clipped_out=clipped)
+
+    def agg():
+        q.unpack_average_prox(codes, delta, length, x, 1.0, 1e-3)
+
+    tq, ta = _time_calls(quant, dev, 5), _time_calls(agg, dev, 10)
+    q.sync_status()
+    bq, ba = N * length * (8 + b / 8), length * (N * b / 8 + 12)
+    res["sweep_N8_len2^26_b4"] = {
+        "quantize_pack": {"ms": round(tq, 4), "bytes": bq, "gbs": round(bq / tq * 1e-6, 1), "frac": round(bq / tq * 1e-6 / peak, 4),
+                          "note": "two passes: 4 B stats read + 4 B quantize read + b/8 B written per element"},
+        "unpack_average_prox": {"ms": round(ta, 4), "bytes": ba, "gbs": round(ba / ta * 1e-6, 1), "frac": round(ba / ta * 1e-6 / peak, 4)},
+        "combined_gbs": round((bq + ba) / (tq + ta) * 1e-6, 1)}
+    q.close()
+    del U, codes, x
+    # layer-wise DNN-shaped aggregation: 62 tensors, 11.7M parameters, 16 workers, b = 4, clip 2.5 std per tensor
+    N, b = 16, 4
+    cur, snap, mu, offs = synth.dnn_gradients(N, seed=2, device=dev)
+    total = offs[-1]
+    q = lpc.Context(None, None, lpc.LOGISTIC, 0.0, N, 1, b, lpc.CLIP_STD, 2.5, 0)
+    _, stride = lpc.packed_layout(total, b, offs)
+    codes = torch.empty((N, stride), dtype=torch.int32, device=dev)
+    delta = torch.empty((N, len(offs) - 1), dtype=torch.float32, device=dev)
+    clipped = torch.empty((N, len(offs) - 1), dtype=torch.int32, device=dev)
+    x = torch.zeros(total, device=dev)
+
+    def quant2():
+        it[0] += 1
+        q.quantize_pack(cur, it[0], U_sub=snap, seg_offsets=offs, codes_out=codes, delta_out=delta, clipped_out=clipped)
+
+    def agg2():
+        q.unpack_average_prox(codes, delta, total, x, 0.1, 0.0, mu=mu, seg_offsets=offs)
+
+    tq, ta = _time_calls(quant2, dev, 10), _time_calls(agg2, dev, 20)
+    q.sync_status()
+    bq, ba = N * total * (16 + b / 8), total * (N * b / 8 + 12)
+    res["dnn_62_tensors_N16_b4"] = {
+        "quantize_pack": {"ms": round(tq, 4), "bytes": bq, "gbs": round(bq / tq * 1e-6, 1), "frac": round(bq / tq * 1e-6 / peak, 4),
+                          "note": "u = cur - snap formed on the fly: 2 x 8 B read + b/8 B written per element"},
+        "unpack_average_prox": {"ms": round(ta, 4), "bytes": ba, "gbs": round(ba / ta * 1e-6, 1), "frac": round(ba / ta * 1e-6 / peak, 4)},
+        "combined_gbs": round((bq + ba) / (tq + ta) * 1e-6, 1)}
+    q.close()
+    return res
+
+
+def e2e_bench(w, X, y, m, eta, dev):
+    """The whole job of the workload (5 epochs) through the host-buffer entry point: X, y copied in, x copied out."""
+    import torch
+    from paper_1901_08924_b200 import lpc
+    S = 5
+    Xh = torch.empty(X.shape, dtype=torch.float32, pin_memory=True)
+    yh = torch.empty(y.shape, dtype=torch.float32, pin_memory=True)
+    Xh.copy_(X)
+    yh.copy_(y)
+    x0 = torch.zeros(w["d"], dtype=torch.float32).pin_memory()
+    torch.cuda.synchronize(dev)
+    best = None
+    for rep in range(2):  # first call warms the context up
+        t0 = time.perf_counter()
+        xh, P, bits = lpc.svrg_run_host(Xh, yh, loss_code(w), w["lam"], w["N"], w["B"], w["b"], lpc.CLIP_STD, w["c"], 0, S, m,
+                                        eta, x0)
+        dt = time.perf_counter() - t0
+        best = dt if best is None else min(best, dt)
+    h2d = Xh.numel() * 4 + yh.numel() * 4 + w["d"] * 4
+    return {"value": round(S * m / best, 1), "unit": UNIT, "h2d_bytes_per_step": h2d // S, "d2h_bytes_per_step": (w["d"] * 4 + 8) // S,
+            "job": "%d epochs via lpc_svrg_run_host from pinned host buffers, wall clock incl. allocation and copies" % S,
+            "seconds": round(best, 4), "objective": P}
+
+
+def oracle_epoch_sample(w, Xh, yh, m, eta, rows, steps, seed=0):
+    """Times the oracle on a slice of one epoch: the full-gradient pass over `rows` rows and `steps` inner steps."""
+    import numpy as np
+    import oracle as orc
+    code = orc.LEAST_SQUARES if w["loss"] == "least_squares" else orc.LOGISTIC
+    P = orc.Problem(Xh, yh, code, w["lam"], w["N"], w["B"], w["b"], orc.CLIP_STD, w["c"], seed)
+    x = np.zeros(w["d"], np.float32)
+    t0 = time.perf_counter()
+    mu, _, _ = orc.full_grad(Xh[:rows], yh[:rows], code, x)
+    t_snap = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    xs = x.copy()
+    for k in range(steps):
+        x = orc.lpc_inner_step(P, k, eta, x, xs, mu)
+    t_inner = time.perf_counter() - t0
+    return t_snap, t_inner
+
+
+def cpu_baseline(w, X, y, m, eta):
+    Xh, yh = X.cpu().numpy(), y.cpu().numpy()
+    rows, steps = w["n"] // 2, min(m, 512)  # about 10-15 s of single-core work on the main workload
+    t_snap, t_inner = oracle_epoch_sample(w, Xh, yh, m, eta, rows, steps)
+    epoch_s = t_snap * (w["n"] / rows) + t_inner * (m / steps)
+    return {"value": round(m / epoch_s, 2), "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": "full-gradient pass over %d of %d rows (%.1f s) and %d of %d inner steps (%.1f s), scaled to one epoch"
+                      % (rows, w["n"], t_snap, steps, m, t_inner)}
+
+
+def run_reference(args):
+    """The CPU oracle, as it stands, on the same workload and metric (rank 0 only)."""
+    import torch
+    from paper_1901_08924_b200 import dist_util
+    size, rank, _ = dist_util.world()
+    if rank != 0:
+        return
+    w = WORKLOADS[args.workload]
+    X, y, m, eta = make_problem(w, seed=0, device="cpu")
+    Xh, yh = X.numpy(), y.numpy()
+    rows, steps = w["n"] // 32, max(1, m // 32)  # one step = 1/32 of an epoch
+    times = []
+    for i in range(max(args.warmup, 0) + args.steps):
+        t_snap, t_inner = oracle_epoch_sample(w, Xh, yh, m, eta, rows, steps, seed=i)
+        times.append(t_snap + t_inner)
+    times = times[max(args.warmup, 0):]
+    total = sum(times)
+    value = args.steps * steps / total
+    sample = "per step: full-gradient pass over %d of %d rows and %d of %d inner steps (1/32 epoch)" % (rows, w["n"], steps, m)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": size, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": round(total / args.steps * 1e3, 3), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": args.workload, "n": w["n"], "d": w["d"], "N": w["N"], "B": w["B"], "b": w["b"]},
+        "cpu_baseline": {"value": round(value, 3), "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": round(value, 3), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
+    ap.add_argument("--quick", action="store_true", help="skip the e2e, CPU-baseline and stand-alone kernel legs")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -82,6 +82,8 @@ typedef struct lpc_ctx lpc_ctx;
 #define LPC_OPT_USE_GRAPH 3     /* 1 (default): lpc_inner_steps replays a CUDA graph; 0: plain launches */
 #define LPC_OPT_PROFILE 4       /* 1: record CUDA events around every kernel launch (graph replay is off meanwhile) */
 
+#define LPC_OPT_PERSISTENT 5    /* 1 (default): lpc_inner_steps runs the whole loop in one cooperative launch when it fits */
+
 /* kernel classes reported by lpc_get_profile */
 #define LPC_KERNEL_SNAPSHOT 0    /* the pass over X of lpc_snapshot_full_grad / lpc_objective */
 #define LPC_KERNEL_WORKER 1      /* fused sampling + SVRG difference + scale + quantize + pack */
@@ -89,7 +91,8 @@ typedef struct lpc_ctx lpc_ctx;
 #define LPC_KERNEL_QUANT_STATS 3 /* first pass of lpc_quantize_pack (max, sums) */
 #define LPC_KERNEL_QUANT_PACK 4  /* second pass of lpc_quantize_pack (quantize + pack) */
 #define LPC_KERNEL_OTHER 5       /* small helper kernels */
-#define LPC_KERNEL_KINDS 6
+#define LPC_KERNEL_INNER_LOOP 6  /* the persistent kernel that runs all steps of one lpc_inner_steps call */
+#define LPC_KERNEL_KINDS 7
 
 /*
  * Creates a context for problem (1).  Section 1 "Contribution" (Eq. 1), Section 2.1 (N workers),
@@ -205,6 +208,14 @@ int lpc_alpc_end_epoch(lpc_ctx* ctx, int64_t m);
 /* P(x) = f(x) + lambda_l1*||x||_1 (Eq. 1) in one pass over X.  x nullable (= current iterate);
  * P_out is a HOST pointer; the call waits for the stream. */
 int lpc_objective(lpc_ctx* ctx, const float* x, double* P_out);
+
+/* Launch-plan facts of a context (host scalars): what = LPC_INFO_*. */
+#define LPC_INFO_STEP_CLUSTER_SIZE 0       /* CTAs per worker cluster of the per-step kernel (0: d too large) */
+#define LPC_INFO_LOOP_CLUSTER_SIZE 1       /* CTAs per worker cluster of the one-launch inner loop (0: not available) */
+#define LPC_INFO_LOOP_LAUNCHES 2           /* lpc_inner_steps calls served by the one-launch inner loop so far */
+#define LPC_INFO_SNAPSHOT_ROWS_PER_TILE 3  /* rows per shared-memory stage of the snapshot pass */
+#define LPC_INFO_SNAPSHOT_STAGES 4         /* shared-memory stages of the snapshot pass */
+int lpc_query(const lpc_ctx* ctx, int what, int64_t* out);
 
 /* Per-kernel device time measured with CUDA events on the context's stream while LPC_OPT_PROFILE is
  * on: ms_out[kind] total milliseconds, launches_out[kind] launches (both HOST arrays of

@@ -58,7 +58,7 @@ struct lpc_ctx {
   uint64_t seed = 0;
   cudaStream_t stream = nullptr;
   // options
-  int sample_global = 0, tap_u = 0, want_cs = 0, use_graph = 1;
+  int sample_global = 0, tap_u = 0, want_cs = 0, use_graph = 1, use_persist = 1;
   // device state of the linear-model path
   float *x = nullptr, *xt = nullptr, *mu = nullptr, *margins = nullptr;
   float *yv = nullptr, *zv = nullptr, *ysum = nullptr, *vhat = nullptr, *v_tap = nullptr, *u_tap = nullptr;
@@ -80,6 +80,12 @@ struct lpc_ctx {
   int CS = 1, SL = 0;
   size_t innerSmem = 0;
   SegPlan inner_seg;  // one segment of length d for the aggregator
+  // persistent inner loop
+  bool persist_ok = false;
+  int pCS = 1, pSL = 0;
+  size_t persistSmem = 0;
+  unsigned int* flags = nullptr;  // 256 step counters + 1 abort word
+  int64_t persist_launches = 0;
   // stand-alone quantizer
   SegPlan seg;
   uint32_t* q_pmax = nullptr;
@@ -302,6 +308,8 @@ int replan_inner(lpc_ctx* c) {
   int cs = 1, sl = 0;
   c->inner_ok = inner_plan(c->d, c->B, c->want_cs, c->max_smem, &cs, &sl, &smem);
   if (c->inner_ok) { c->CS = cs; c->SL = sl; c->innerSmem = smem; }
+  c->persist_ok = persist_plan(c->d, c->N, c->B, c->b, c->want_cs, c->max_smem, &cs, &sl, &smem);
+  if (c->persist_ok) { c->pCS = cs; c->pSL = sl; c->persistSmem = smem; }
   return LPC_OK;
 }
 
@@ -337,7 +345,25 @@ int run_steps(lpc_ctx* c, int kind, const float* p, uint64_t k0, int64_t count) 
     return kind == 0 ? enqueue_lpc_step(c, p[0], kb, kd, kc) : enqueue_alpc_step(c, p[0], p[1], p[2], p[3], kb, kd, kc);
   };
   int64_t done = 0;
-  if (c->use_graph && !c->profile && count >= GRAPH_STEPS) {
+  if (kind == 0 && c->use_persist && c->persist_ok && count >= 2 && count <= 0x7FFFFFFF) {
+    // the whole loop in one cooperative launch; on a launch refusal fall through to the per-step kernels
+    PersistArgs pa;
+    pa.in = inner_args(c, k0, nullptr, 0);
+    pa.in.CS = c->pCS; pa.in.SL = c->pSL;
+    pa.count = (int)count; pa.eta = p[0]; pa.lambda_l1 = c->lambda_l1;
+    pa.flags = c->flags; pa.abort_flag = c->flags + 256; pa.x_out = c->x; pa.v_tap = c->tap_u ? c->v_tap : nullptr;
+    CU(c, cudaMemsetAsync(c->flags, 0, 257 * sizeof(unsigned int), c->stream));
+    cudaError_t e;
+    { ProfScope ps_(c, LPC_KERNEL_INNER_LOOP); e = launch_persist(pa, c->persistSmem, c->stream); }
+    if (e == cudaSuccess) {
+      done = count;
+      c->persist_launches += 1;
+    } else {
+      cudaGetLastError();  // clear the refusal and use the per-step path
+      c->persist_ok = false;
+    }
+  }
+  if (done < count && c->use_graph && !c->profile && count >= GRAPH_STEPS) {
     GraphKey key;
     key.kind = kind; key.steps = GRAPH_STEPS; key.tap = c->tap_u; key.cs = c->CS; key.sample_global = c->sample_global;
     for (int i = 0; i < 4; ++i) key.p[i] = p[i];
@@ -476,11 +502,13 @@ int lpc_init(lpc_ctx** out, const float* X, const float* y, int64_t n, int32_t d
     A(dalloc(c, &c->x, dd)); A(dalloc(c, &c->xt, dd)); A(dalloc(c, &c->mu, dd)); A(dalloc(c, &c->margins, (size_t)n));
     A(dalloc(c, &c->yv, dd)); A(dalloc(c, &c->zv, dd)); A(dalloc(c, &c->ysum, dd)); A(dalloc(c, &c->vhat, dd));
     A(dalloc(c, &c->v_tap, dd));
-    A(dalloc(c, &c->delta, (size_t)N)); A(dalloc(c, &c->clipped, (size_t)N));
+    A(dalloc(c, &c->delta, 2 * (size_t)N));  // two halves: the persistent loop alternates between them
+    A(dalloc(c, &c->clipped, (size_t)N));
     A(dalloc(c, &c->clipped_part, (size_t)N * inner_clipped_stride()));
+    A(dalloc(c, &c->flags, 257));
     A(dalloc(c, &c->idx_tap, (size_t)(N + 1) * B)); A(dalloc(c, &c->coef_tap, (size_t)(N + 1) * B));
     if (rc == LPC_OK) rc = make_plan(c, c->inner_seg, d, b, nullptr, 1);
-    if (rc == LPC_OK) A(dalloc(c, &c->codes, (size_t)N * (size_t)c->inner_seg.stride_words));
+    if (rc == LPC_OK) A(dalloc(c, &c->codes, 2 * (size_t)N * (size_t)c->inner_seg.stride_words));
     c->dpad = snapshot_dpad(d);
     snapshot_plan(d, c->max_smem, &c->snapR, &c->snapStages, &c->snapSmem);
     c->snapGrid = c->sm_count;
@@ -501,7 +529,7 @@ int lpc_destroy(lpc_ctx* c) {
   for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
   void* ptrs[] = {c->x, c->xt, c->mu, c->margins, c->yv, c->zv, c->ysum, c->vhat, c->v_tap, c->u_tap, c->codes,
                   c->delta, c->clipped_part, c->clipped, c->idx_tap, c->coef_tap, c->k_dev, c->dev_status, c->f_dev,
-                  c->partial_mu, c->partial_f, c->q_pmax, c->q_ps1, c->q_ps2, c->q_scales, c->q_clip};
+                  c->partial_mu, c->partial_f, c->flags, c->q_pmax, c->q_ps1, c->q_ps2, c->q_scales, c->q_clip};
   for (void* p : ptrs)
     if (p) cudaFree(p);
   free_plan(c->inner_seg);
@@ -529,6 +557,7 @@ int lpc_set_option(lpc_ctx* c, int option, int64_t value) {
       }
       return LPC_OK;
     case LPC_OPT_USE_GRAPH: c->use_graph = value ? 1 : 0; return LPC_OK;
+    case LPC_OPT_PERSISTENT: c->use_persist = value ? 1 : 0; return LPC_OK;
     case LPC_OPT_PROFILE:
       TRY(prof_resolve(c));
       c->profile = value ? 1 : 0;
@@ -652,6 +681,18 @@ int lpc_objective(lpc_ctx* c, const float* x, double* P_out) {
   CU(c, cudaStreamSynchronize(c->stream));
   *P_out = h[0] + (double)c->lambda_l1 * h[1];
   return LPC_OK;
+}
+
+int lpc_query(const lpc_ctx* c, int what, int64_t* out) {
+  if (!c || !out) return LPC_ERR_INVALID_ARG;
+  switch (what) {
+    case LPC_INFO_STEP_CLUSTER_SIZE: *out = c->inner_ok ? c->CS : 0; return LPC_OK;
+    case LPC_INFO_LOOP_CLUSTER_SIZE: *out = c->persist_ok ? c->pCS : 0; return LPC_OK;
+    case LPC_INFO_LOOP_LAUNCHES: *out = c->persist_launches; return LPC_OK;
+    case LPC_INFO_SNAPSHOT_ROWS_PER_TILE: *out = c->snapR; return LPC_OK;
+    case LPC_INFO_SNAPSHOT_STAGES: *out = c->snapStages; return LPC_OK;
+    default: return LPC_ERR_INVALID_ARG;
+  }
 }
 
 int lpc_get_profile(lpc_ctx* c, double* ms_out, int64_t* launches_out, int32_t reset) {

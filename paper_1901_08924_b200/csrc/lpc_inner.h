@@ -36,6 +36,20 @@ struct InnerArgs {
   int SL;                  // coordinates per CTA slice
 };
 
+// Arguments of the persistent inner loop (lpc_persist.cu): `count` steps k_base, k_base+1, ... in one launch.
+struct PersistArgs {
+  InnerArgs in;              // in.x = iterate at entry, in.k_dev unused, in.has_J = 0
+  int count;
+  float eta;
+  float lambda_l1;
+  unsigned int* flags;       // N * CS step counters, zero at launch
+  unsigned int* abort_flag;  // zero at launch; set when a bounded wait ran out
+  float* x_out;              // iterate after `count` steps (may alias in.x)
+  float* v_tap;              // nullable: v of the last step
+};
+bool persist_plan(int d, int N, int B, int b, int want_cs, int max_smem, int* CS_out, int* SL_out, size_t* smem_out);
+cudaError_t launch_persist(const PersistArgs& pa, size_t smem, cudaStream_t st);
+
 int inner_max_b();
 int inner_clipped_stride();
 bool inner_plan(int d, int B, int want_cs, int max_smem, int* CS_out, int* SL_out, size_t* smem_out);

@@ -1,0 +1,588 @@
+// The whole inner loop of Algorithm 1 (steps 5-11) in ONE cooperative launch.
+//
+// An inner iteration moves only N*B rows of X, so it is bound by latency, not bandwidth: the chain
+// "all workers' codes of step t -> x_{t+1} -> margins -> u -> scale -> codes of step t+1" is strictly
+// serial.  Launching kernels per step pays a launch + drain for every link of that chain.  Here the
+// grid stays resident for `count` steps (one cluster per worker, one CTA per SM, launched
+// cooperatively so that co-residency is guaranteed) and the only grid-wide dependency per step is a
+// flag wait:
+//   - every CTA keeps its slice of x and of mu in REGISTERS across steps;
+//   - the rows of step t+1 do not depend on step t (sampling is counter-based), so they are sampled
+//     and fetched by bulk copies (TMA) into the other half of a double buffer while step t computes;
+//   - when a CTA has stored the codes of its slice it raises its flag (release); at the top of the next
+//     step every CTA waits until all N*CS flags show the step (acquire), decodes all workers' codes for
+//     ITS slice with L1-bypassing loads, averages, adds mu and applies the proximal step in registers.
+// Every wait is bounded; when one runs out the CTA records LPC_ERR_TIMEOUT in the status word, raises a
+// global abort flag that makes every other wait return at once, and the loop finishes without hanging
+// (all CTAs still execute the same cluster barriers).
+//
+// The arithmetic (sampling, margins as balanced-tree sums, u summed in batch order, Eq. 2, the
+// quantizer, Eq. 3, the proximal step) is operation for operation that of the per-step kernels.
+#include <cooperative_groups.h>
+
+#include "lpc_device.cuh"
+#include "lpc_inner.h"
+
+namespace cg = cooperative_groups;
+
+namespace lpc {
+namespace {
+
+constexpr int PT = 256;
+constexpr int PGROUP = PT * 8;
+constexpr int PMAXP = 2;   // passes per CTA: SL <= 4096
+constexpr int PMAXB = 64;
+constexpr int PMAXCS = 8;
+constexpr int PMAXFLAGS = 256;
+
+struct PSmem {
+  uint64_t bar[2];
+  int64_t idx[2][PMAXB];
+  float yv[2][PMAXB];
+  float msnap[2][PMAXB];
+  float coef[PMAXB];
+  float wpart[PMAXB * PMAXP * 8];
+  float mpart[PMAXB * PMAXCS];
+  float s1part[PMAXCS], s2part[PMAXCS];
+  uint32_t maxpart[PMAXCS];
+  float ws1[PMAXP * 8], ws2[PMAXP * 8];
+  uint32_t wmax[8];
+  uint32_t wclip[8];
+  float sdelta[PMAXFLAGS];
+  Scale scale;
+  int abort;
+  __align__(16) uint8_t stage[PT * 16];
+};
+
+__device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int* p) {
+  unsigned int v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_release_u32(unsigned int* p, unsigned int v) {
+  asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
+// The 8*b bits of coordinate group g of a stream, loaded around L1 (other SMs wrote them this launch).
+template <int BITS>
+__device__ __forceinline__ void load_chunk_cg(const uint32_t* w, int64_t g, int b, int64_t pad_words, uint64_t& lo,
+                                              uint64_t& hi) {
+  hi = 0;
+  if (BITS == 8) {
+    const uint2 t = __ldcg(reinterpret_cast<const uint2*>(w + g * 2));
+    lo = (uint64_t)t.x | ((uint64_t)t.y << 32);
+  } else if (BITS == 4) {
+    lo = __ldcg(w + g);
+  } else if (BITS == 2) {
+    lo = __ldcg(reinterpret_cast<const unsigned short*>(w) + g);
+  } else if (BITS == 1) {
+    lo = __ldcg(reinterpret_cast<const unsigned char*>(w) + g);
+  } else {
+    const unsigned char* bytes = reinterpret_cast<const unsigned char*>(w);
+    const int64_t b0 = g * b, limit = pad_words * 4;
+    lo = 0;
+    for (int i = 0; i < b; ++i) {
+      const uint64_t v = (b0 + i < limit) ? __ldcg(bytes + b0 + i) : 0;
+      if (i < 8) lo |= v << (8 * i); else hi |= v << (8 * (i - 8));
+    }
+  }
+}
+
+__device__ __forceinline__ uint32_t extract_bits(uint64_t lo, uint64_t hi, int pos, int b) {
+  uint64_t v;
+  if (pos < 64) {
+    v = lo >> pos;
+    if (pos + b > 64) v |= hi << (64 - pos);
+  } else {
+    v = hi >> (pos - 64);
+  }
+  return (uint32_t)v & ((1u << b) - 1u);
+}
+
+template <int BITS>  // 1, 2, 4, 8 fixed width; 0: b from the arguments (1..16 or 32)
+__global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
+  const InnerArgs& a = pa.in;
+  cg::cluster_group cluster = cg::this_cluster();
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  PSmem& sm = *reinterpret_cast<PSmem*>(smem_raw);
+  const int CS = a.CS, SL = a.SL, B = a.B, d = a.d, N = a.N;
+  float* rows = reinterpret_cast<float*>(smem_raw + ((sizeof(PSmem) + 15) & ~(size_t)15));  // 2 x B x SL
+  const size_t buf_floats = (size_t)B * SL;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int rank = (int)cluster.block_rank();
+  const int worker = blockIdx.y;
+  const int b = BITS ? BITS : a.b;
+  const int passes = (SL + PGROUP - 1) / PGROUP;
+  const int c0 = rank * SL;
+  const int width = max(0, min(SL, d - c0));
+  const int nflags = N * CS;
+  const float invN = __fdiv_rn(1.0f, (float)N);
+  const float invB = __fdiv_rn(1.0f, (float)B);
+  const float kappa = mul_rn(pa.eta, pa.lambda_l1);
+  const uint32_t zero_code = (b == 1) ? 0u : (1u << (b - 1));
+  // Codes and scales are double-buffered by step parity: a fast CTA may already store step t+1 while a
+  // slow one still decodes step t.  The parity is chosen so that the last step lands in buffer 0.
+  const int64_t codes_buf = (int64_t)N * a.stride_words;
+
+  if (tid == 0) {
+    mbar_init(&sm.bar[0], 1);
+    mbar_init(&sm.bar[1], 1);
+    mbar_fence_init();
+    sm.abort = 0;
+  }
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  __syncthreads();
+
+  // Samples the minibatch of step t and starts fetching this CTA's slice of its rows into buffer t&1.
+  auto prefetch = [&](int t) {
+    const int s = t & 1;
+    if (tid == 0 && width > 0) mbar_expect_tx(&sm.bar[s], (uint32_t)width * 4u * (uint32_t)B);
+    if (tid < B) {
+      int64_t lo, span;
+      if (a.sample_global) { lo = 0; span = a.n; }
+      else { span = a.n / N; lo = (int64_t)worker * span; }
+      const U4 r = stream_block(a.seed, TAG_BATCH, (uint32_t)worker, a.k_base + (uint64_t)t, (uint32_t)tid);
+      const int64_t row = lo + (int64_t)(((uint64_t)r.x * (uint64_t)span) >> 32);
+      if (width > 0) bulk_load(rows + s * buf_floats + (size_t)tid * SL, a.X + row * (int64_t)d + c0, (uint32_t)width * 4u, &sm.bar[s]);
+      sm.idx[s][tid] = row;
+      sm.yv[s][tid] = a.y[row];
+      sm.msnap[s][tid] = a.margins[row];
+    }
+  };
+
+  // this thread's slice of the iterate and of the snapshot gradient stay in registers for the whole loop
+  float xr[PMAXP][8], mur[PMAXP][8];
+#pragma unroll
+  for (int p = 0; p < PMAXP; ++p) {
+    const int off = p * PGROUP + tid * 8;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const bool in = (p < passes) && (off + e < width);
+      xr[p][e] = in ? a.x[c0 + off + e] : 0.f;
+      mur[p][e] = in ? a.mu[c0 + off + e] : 0.f;
+    }
+  }
+  if (pa.count > 0) prefetch(0);
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+
+  auto row8 = [&](const float* base, int r, int off, float* v) {
+#pragma unroll
+    for (int e = 0; e < 8; ++e) v[e] = 0.f;
+    if (off < width) {
+      const float4 v0 = *reinterpret_cast<const float4*>(base + (size_t)r * SL + off);
+      v[0] = v0.x; v[1] = v0.y; v[2] = v0.z; v[3] = v0.w;
+      if (off + 4 < width) {
+        const float4 v1 = *reinterpret_cast<const float4*>(base + (size_t)r * SL + off + 4);
+        v[4] = v1.x; v[5] = v1.y; v[6] = v1.z; v[7] = v1.w;
+      }
+    }
+  };
+
+  // Waits until every CTA of the grid has published step `target`; then applies that step's update to xr.
+  auto apply_update = [&](unsigned int target) {
+    if (tid < nflags) {
+      const unsigned int* f = pa.flags + tid;
+      uint64_t t0 = 0;
+      for (uint32_t it = 0;; ++it) {
+        if (ld_acquire_u32(f) >= target) break;
+        if ((it & 63u) == 63u) {
+          if (ld_acquire_u32(pa.abort_flag) != 0u) { sm.abort = 1; break; }
+          const uint64_t now = global_ns();
+          if (t0 == 0) t0 = now;
+          else if (now - t0 > 2000000000ull) {
+            atomicOr(a.dev_status, DEV_TIMEOUT);
+            st_release_u32(pa.abort_flag, 1u);
+            sm.abort = 1;
+            break;
+          }
+        }
+      }
+    }
+    __syncthreads();
+    const int rpar = (pa.count - (int)target) & 1;  // buffer that holds step target-1
+    const uint32_t* codes_in = a.codes + rpar * codes_buf;
+    if (tid < N) sm.sdelta[tid] = __ldcg(a.delta + rpar * N + tid);
+    __syncthreads();
+#pragma unroll
+    for (int p = 0; p < PMAXP; ++p) {
+      if (p >= passes) break;
+      const int off = p * PGROUP + tid * 8;
+      if (off >= SL) continue;
+      const int c = c0 + off;
+      float acc[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+      if (c < d) {
+        if (b == 32) {
+          for (int i = 0; i < N; ++i) {
+            const uint32_t* wi = codes_in + (int64_t)i * a.stride_words;
+            const float di = sm.sdelta[i];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              const float val = (c + e < d) ? __uint_as_float(__ldcg(wi + c + e)) : 0.f;
+              acc[e] = add_rn(acc[e], mul_rn(di, val));
+            }
+          }
+        } else {
+#pragma unroll 4
+          for (int i = 0; i < N; ++i) {
+            uint64_t lo, hi;
+            load_chunk_cg<BITS>(codes_in + (int64_t)i * a.stride_words, c >> 3, b, a.pad_words, lo, hi);
+            const float di = sm.sdelta[i];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              uint32_t code;
+              if constexpr (BITS == 0) code = extract_bits(lo, hi, e * b, b);
+              else code = (uint32_t)(lo >> (e * BITS)) & ((1u << BITS) - 1u);
+              acc[e] = add_rn(acc[e], mul_rn(di, index_as_float(code, b)));
+            }
+          }
+        }
+      }
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        if (c + e < d) {
+          const float v = add_rn(mul_rn(acc[e], invN), mur[p][e]);
+          xr[p][e] = soft_threshold(__fsub_rn(xr[p][e], mul_rn(pa.eta, v)), kappa);
+          if (pa.v_tap && worker == 0) pa.v_tap[c + e] = v;
+        }
+      }
+    }
+  };
+
+  for (int t = 0; t < pa.count; ++t) {
+    const int s = t & 1;
+    const uint64_t k = a.k_base + (uint64_t)t;
+    const float* buf = rows + s * buf_floats;
+    const int wpar = (pa.count - 1 - t) & 1;
+    uint32_t* out = a.codes + wpar * codes_buf + (int64_t)worker * a.stride_words;
+    if (t + 1 < pa.count) prefetch(t + 1);
+
+    // rounding bits of this step: they depend on the counters only, so they are drawn before the data arrives
+    U4 rnd[PMAXP];
+#pragma unroll
+    for (int p = 0; p < PMAXP; ++p)
+      rnd[p] = stream_block(a.seed, TAG_ROUND, (uint32_t)worker, k, (uint32_t)((c0 + p * PGROUP + tid * 8) >> 3));
+
+    if (t > 0) apply_update((unsigned int)t);  // x_t = prox(x_{t-1} - eta v_{t-1})
+
+    bool ok = true;
+    if (width > 0) ok = mbar_wait(&sm.bar[s], (uint32_t)((t >> 1) & 1));
+    if (!ok) {
+      atomicOr(a.dev_status, DEV_TIMEOUT);
+      mbar_wait(&sm.bar[s], (uint32_t)((t >> 1) & 1));
+    }
+
+    // margins <X_a, x_t>
+    for (int r = 0; r < B; ++r) {
+#pragma unroll
+      for (int p = 0; p < PMAXP; ++p) {
+        if (p < passes) {
+          float v[8], pr[8];
+          row8(buf, r, p * PGROUP + tid * 8, v);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) pr[e] = mul_rn(v[e], xr[p][e]);
+          const float sv = warp_tree_sum(tree8(pr));
+          if (lane == 0) sm.wpart[(r * PMAXP + p) * 8 + warp] = sv;
+        }
+      }
+    }
+    __syncthreads();
+    if (tid < B) {
+      float part = smem_tree_sum(&sm.wpart[tid * PMAXP * 8], 8);
+      if (passes == 2) part = add_rn(part, smem_tree_sum(&sm.wpart[(tid * PMAXP + 1) * 8], 8));
+      for (int q = 0; q < CS; ++q) cluster.map_shared_rank(sm.mpart, q)[tid * PMAXCS + rank] = part;
+    }
+    cluster.sync();
+    if (tid < B) {
+      const float m = smem_tree_sum(&sm.mpart[tid * PMAXCS], CS);
+      const float yy = sm.yv[s][tid];
+      const float c = __fsub_rn(loss_deriv(a.loss, m, yy), loss_deriv(a.loss, sm.msnap[s][tid], yy));
+      sm.coef[tid] = c;
+      if (rank == 0 && t == pa.count - 1) {
+        if (a.idx_tap) a.idx_tap[(int64_t)worker * B + tid] = sm.idx[s][tid];
+        if (a.coef_tap) a.coef_tap[(int64_t)worker * B + tid] = c;
+      }
+    }
+    __syncthreads();
+
+    // u = (1/B) sum_a c_a X_a in batch order
+    float u[PMAXP][8];
+#pragma unroll
+    for (int p = 0; p < PMAXP; ++p) {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) u[p][e] = 0.f;
+      if (p < passes) {
+        for (int r = 0; r < B; ++r) {
+          float v[8];
+          row8(buf, r, p * PGROUP + tid * 8, v);
+          const float c = sm.coef[r];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) u[p][e] = add_rn(u[p][e], mul_rn(c, v[e]));
+        }
+#pragma unroll
+        for (int e = 0; e < 8; ++e) u[p][e] = mul_rn(u[p][e], invB);
+      }
+    }
+    if (a.u_tap && t == pa.count - 1) {
+#pragma unroll
+      for (int p = 0; p < PMAXP; ++p) {
+        const int off = p * PGROUP + tid * 8;
+        if (p < passes) {
+#pragma unroll
+          for (int e = 0; e < 8; ++e)
+            if (off + e < width) a.u_tap[(int64_t)worker * d + c0 + off + e] = u[p][e];
+        }
+      }
+    }
+
+    // scale (Eq. 2)
+    uint32_t mx = 0;
+#pragma unroll
+    for (int p = 0; p < PMAXP; ++p) {
+      if (p < passes) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) mx = max(mx, __float_as_uint(fabsf(u[p][e])));
+        if (a.clip_mode == CLIP_STD) {
+          float sq[8];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) sq[e] = mul_rn(u[p][e], u[p][e]);
+          const float s1 = warp_tree_sum(tree8(u[p]));
+          const float s2 = warp_tree_sum(tree8(sq));
+          if (lane == 0) { sm.ws1[p * 8 + warp] = s1; sm.ws2[p * 8 + warp] = s2; }
+        }
+      }
+    }
+    mx = warp_max_u32(mx);
+    if (lane == 0) sm.wmax[warp] = mx;
+    __syncthreads();
+    if (tid == 0) {
+      uint32_t m = 0;
+      for (int w = 0; w < 8; ++w) m = max(m, sm.wmax[w]);
+      float s1 = 0.f, s2 = 0.f;
+      if (a.clip_mode == CLIP_STD) {
+        s1 = smem_tree_sum(sm.ws1, 8);
+        s2 = smem_tree_sum(sm.ws2, 8);
+        if (passes == 2) { s1 = add_rn(s1, smem_tree_sum(sm.ws1 + 8, 8)); s2 = add_rn(s2, smem_tree_sum(sm.ws2 + 8, 8)); }
+      }
+      for (int q = 0; q < CS; ++q) {
+        cluster.map_shared_rank(sm.maxpart, q)[rank] = m;
+        cluster.map_shared_rank(sm.s1part, q)[rank] = s1;
+        cluster.map_shared_rank(sm.s2part, q)[rank] = s2;
+      }
+    }
+    cluster.sync();
+    if (tid == 0) {
+      uint32_t m = 0;
+      for (int q = 0; q < CS; ++q) m = max(m, sm.maxpart[q]);
+      float S1 = 0.f, S2 = 0.f;
+      if (a.clip_mode == CLIP_STD) { S1 = smem_tree_sum(sm.s1part, CS); S2 = smem_tree_sum(sm.s2part, CS); }
+      sm.scale = make_scale(m, S1, S2, d, b, a.clip_mode, a.clip_value);
+      if (rank == 0) {
+        a.delta[wpar * N + worker] = sm.scale.delta;
+        if (sm.scale.flags & 2u) atomicOr(a.dev_status, DEV_NONFINITE);
+      }
+    }
+    __syncthreads();
+    const Scale sc = sm.scale;
+    const bool degenerate = (sc.flags & 1u) != 0;
+
+    // quantize (Section 2.2) and pack
+    uint32_t nclip = 0;
+#pragma unroll
+    for (int p = 0; p < PMAXP; ++p) {
+      if (p >= passes) break;
+      const int off = p * PGROUP + tid * 8;
+      const int c = c0 + off;
+      const bool mine = off < SL;
+      if (b == 32) {
+        if (mine) {
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            float v = u[p][e];
+            if (a.clip_mode != CLIP_NONE && c + e < d) {
+              if (v > sc.T) { v = sc.T; ++nclip; }
+              if (v < -sc.T) { v = -sc.T; ++nclip; }
+            }
+            if (c + e < a.pad_words) out[c + e] = (c + e < d) ? __float_as_uint(v) : 0u;
+          }
+        }
+        continue;
+      }
+      uint64_t lo = 0, hi = 0;
+      if (mine && c < d) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          if (c + e < d) {
+            uint32_t code = zero_code;
+            if (!degenerate) {
+              code = BITS ? quantize_code<BITS ? BITS : 2>(u[p][e], sc.rdelta, lane16(rnd[p], e))
+                          : quantize_code_rt(u[p][e], sc.rdelta, lane16(rnd[p], e), b);
+              nclip += (u[p][e] > sc.T || u[p][e] < sc.lower) ? 1u : 0u;
+            }
+            const int pos = e * b;
+            if (pos < 64) {
+              lo |= (uint64_t)code << pos;
+              if (pos + b > 64) hi |= (uint64_t)code >> (64 - pos);
+            } else {
+              hi |= (uint64_t)code << (pos - 64);
+            }
+          }
+        }
+      }
+      if (BITS == 8) {
+        const int64_t w = (int64_t)(c >> 3) * 2;
+        if (mine && w < a.pad_words) *reinterpret_cast<uint2*>(out + w) = make_uint2((uint32_t)lo, (uint32_t)(lo >> 32));
+      } else if (BITS == 4) {
+        const int64_t w = c >> 3;
+        if (mine && w < a.pad_words) out[w] = (uint32_t)lo;
+      } else if (BITS == 2) {
+        const uint32_t own = (uint32_t)lo;
+        const uint32_t next = __shfl_down_sync(0xFFFFFFFFu, own, 1);
+        const int64_t w = c >> 4;
+        if (mine && (lane & 1) == 0 && w < a.pad_words) out[w] = own | (next << 16);
+      } else if (BITS == 1) {
+        const uint32_t own = (uint32_t)lo;
+        const uint32_t n1 = __shfl_down_sync(0xFFFFFFFFu, own, 1);
+        const uint32_t n2 = __shfl_down_sync(0xFFFFFFFFu, own, 2);
+        const uint32_t n3 = __shfl_down_sync(0xFFFFFFFFu, own, 3);
+        const int64_t w = c >> 5;
+        if (mine && (lane & 3) == 0 && w < a.pad_words) out[w] = own | (n1 << 8) | (n2 << 16) | (n3 << 24);
+      } else {
+        if (p > 0) __syncthreads();
+        for (int i = 0; i < b; ++i)
+          sm.stage[tid * b + i] = (uint8_t)((i < 8) ? (lo >> (8 * i)) : (hi >> (8 * (i - 8))));
+        __syncthreads();
+        const int span = min(PGROUP, SL - p * PGROUP);
+        const int64_t w0 = (int64_t)((c0 + p * PGROUP) >> 5) * b;
+        const uint32_t* st = reinterpret_cast<const uint32_t*>(sm.stage);
+        for (int w = tid; w < (span / 32) * b; w += PT)
+          if (w0 + w < a.pad_words) out[w0 + w] = st[w];
+      }
+    }
+    nclip = __reduce_add_sync(0xFFFFFFFFu, nclip);
+    if (lane == 0) sm.wclip[warp] = nclip;
+    __syncthreads();  // every thread of this CTA has stored its codes
+    if (tid == 0) {
+      uint32_t tc = 0;
+      for (int w = 0; w < 8; ++w) tc += sm.wclip[w];
+      a.clipped_part[worker * PMAXCS + rank] = tc;
+      __threadfence();
+      st_release_u32(pa.flags + worker * CS + rank, (unsigned int)(t + 1));  // publish step t
+    }
+  }
+
+  // the last step's update, then the slice of the final iterate goes back to memory (worker 0's cluster)
+  if (pa.count > 0) apply_update((unsigned int)pa.count);
+  if (worker == 0) {
+#pragma unroll
+    for (int p = 0; p < PMAXP; ++p) {
+      const int off = p * PGROUP + tid * 8;
+      if (p < passes) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e)
+          if (off + e < width) pa.x_out[c0 + off + e] = xr[p][e];
+      }
+    }
+  }
+  cluster.sync();  // no CTA leaves while a peer could still address its shared memory
+}
+
+template <int BITS>
+cudaError_t launch_p(const PersistArgs& pa, size_t smem, cudaStream_t st) {
+  cudaError_t e = cudaFuncSetAttribute(persist_kernel<BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)pa.in.CS, (unsigned)pa.in.N, 1);
+  cfg.blockDim = dim3(PT, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = (unsigned)pa.in.CS;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeCooperative;  // all CTAs co-resident or the launch fails
+  attr[1].val.cooperative = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
+  return cudaLaunchKernelEx(&cfg, persist_kernel<BITS>, pa);
+}
+
+}  // namespace
+
+namespace {
+template <int BITS>
+int max_clusters_t(int cs, size_t smem) {
+  if (cudaFuncSetAttribute(persist_kernel<BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+    cudaGetLastError();
+    return 0;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)cs, 1, 1);
+  cfg.blockDim = dim3(PT, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = (unsigned)cs;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, persist_kernel<BITS>, &cfg) != cudaSuccess) {
+    cudaGetLastError();
+    return 0;
+  }
+  return n;
+}
+int max_clusters(int b, int cs, size_t smem) {
+  switch (b) {
+    case 1: return max_clusters_t<1>(cs, smem);
+    case 2: return max_clusters_t<2>(cs, smem);
+    case 4: return max_clusters_t<4>(cs, smem);
+    case 8: return max_clusters_t<8>(cs, smem);
+    default: return max_clusters_t<0>(cs, smem);
+  }
+}
+}  // namespace
+
+// Cluster size / slice for the persistent loop: all N clusters must be co-resident (the occupancy query
+// says how many clusters of a given size the device can hold) and the double-buffered row slices must fit
+// in shared memory.  Among the sizes that fit, the largest cluster whose slices still keep a CTA busy wins:
+// more CTAs per worker shorten every serial phase of a step.
+bool persist_plan(int d, int N, int B, int b, int want_cs, int max_smem, int* CS_out, int* SL_out, size_t* smem_out) {
+  int P = 1;
+  while (P < d) P <<= 1;
+  if (P < 32) P = 32;
+  if (B > PMAXB) return false;
+  bool found = false;
+  for (int cs = 1; cs <= PMAXCS; cs <<= 1) {
+    if (want_cs > 0 && cs != want_cs) continue;
+    const int SL = P / cs;
+    if (SL < 32) break;
+    if (SL > PGROUP * PMAXP) continue;
+    if (N * cs > PMAXFLAGS) break;
+    const size_t smem = ((sizeof(PSmem) + 15) & ~(size_t)15) + 2 * (size_t)B * SL * 4;
+    if (smem > (size_t)max_smem) continue;
+    if (max_clusters(b, cs, smem) < N) continue;
+    *CS_out = cs; *SL_out = SL; *smem_out = smem;
+    found = true;
+    if (want_cs > 0) break;
+    if (SL <= 512) break;  // slices below 512 coordinates leave most of a CTA idle
+  }
+  return found;
+}
+
+cudaError_t launch_persist(const PersistArgs& pa, size_t smem, cudaStream_t st) {
+  switch (pa.in.b) {
+    case 1: return launch_p<1>(pa, smem, st);
+    case 2: return launch_p<2>(pa, smem, st);
+    case 4: return launch_p<4>(pa, smem, st);
+    case 8: return launch_p<8>(pa, smem, st);
+    default: return launch_p<0>(pa, smem, st);
+  }
+}
+
+}  // namespace lpc

@@ -17,8 +17,9 @@ LOGISTIC, LEAST_SQUARES = 0, 1
 CLIP_NONE, CLIP_LAMBDA, CLIP_STD = 0, 1, 2
 (BUF_X, BUF_XTILDE, BUF_MU, BUF_MARGINS, BUF_Y, BUF_Z, BUF_YSUM, BUF_CODES, BUF_DELTA, BUF_CLIPPED, BUF_BATCH_IDX,
  BUF_COEF, BUF_U, BUF_V, BUF_VHAT) = range(15)
-OPT_SAMPLE_GLOBAL, OPT_TAP_U, OPT_CLUSTER_SIZE, OPT_USE_GRAPH, OPT_PROFILE = 0, 1, 2, 3, 4
-KERNEL_NAMES = ["snapshot", "worker", "aggregate", "quant_stats", "quant_pack", "other"]
+OPT_SAMPLE_GLOBAL, OPT_TAP_U, OPT_CLUSTER_SIZE, OPT_USE_GRAPH, OPT_PROFILE, OPT_PERSISTENT = 0, 1, 2, 3, 4, 5
+INFO_STEP_CLUSTER_SIZE, INFO_LOOP_CLUSTER_SIZE, INFO_LOOP_LAUNCHES, INFO_SNAPSHOT_ROWS_PER_TILE, INFO_SNAPSHOT_STAGES = range(5)
+KERNEL_NAMES = ["snapshot", "worker", "aggregate", "quant_stats", "quant_pack", "other", "inner_loop"]
 
 # every symbol that include/lpc.h declares: (name, restype, argtypes)
 _vp, _i64, _i32, _u64, _f32, _int = C.c_void_p, C.c_int64, C.c_int32, C.c_uint64, C.c_float, C.c_int
@@ -47,6 +48,7 @@ SYMBOLS = [
     ("lpc_objective", _int, [_vp, _vp, _f64p]),
     ("lpc_comm_bits", _int, [_vp, _u64p, _u64p]),
     ("lpc_get_profile", _int, [_vp, _f64p, _i64p, _i32]),
+    ("lpc_query", _int, [_vp, _int, _i64p]),
     ("lpc_svrg_run_host", _int, [_vp, _vp, _i64, _i32, _int, _f32, _i32, _i32, _i32, _int, _f32, _u64, _i32, _i64,
                                  _f32, _vp, _f64p, _u64p]),
     ("lpc_debug_stream_blocks", _int, [_u64, C.c_uint32, C.c_uint32, _u64, C.c_uint32, _i64, _vp, _vp]),
@@ -232,6 +234,11 @@ class Context:
         P = C.c_double(0)
         self._ck(lib().lpc_objective(self._h, _ptr(x), C.byref(P)))
         return P.value
+
+    def query(self, what):
+        out = C.c_int64(0)
+        self._ck(lib().lpc_query(self._h, what, C.byref(out)))
+        return out.value
 
     def get_profile(self, reset=True):
         """Returns {kernel name: (total ms, launches)} measured since profiling was switched on / last reset."""

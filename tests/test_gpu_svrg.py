@@ -249,6 +249,43 @@ def test_graph_replay_equals_plain_launches_and_resume():
     ctx2.close()
 
 
+@pytest.mark.parametrize("cfg", [
+    dict(n=64, d=8, N=4, B=1, b=2), dict(n=256, d=1000, N=4, B=1, b=2), dict(n=256, d=1000, N=4, B=3, b=3),
+    dict(n=128, d=4096, N=16, B=8, b=4), dict(n=64, d=8192, N=4, B=16, b=8), dict(n=64, d=5000, N=2, B=4, b=1),
+    dict(n=64, d=3000, N=2, B=4, b=32), dict(n=64, d=12288, N=2, B=2, b=5), dict(n=256, d=2048, N=32, B=2, b=4),
+])
+@pytest.mark.parametrize("mode", ["persistent", "graph"])
+def test_multi_step_paths_equal_single_launches(cfg, mode):
+    # the one-launch persistent loop and the graph replay must give the bits of one-step-at-a-time launches
+    c = dict(cfg)
+    P, ctx = _setup(c.pop("n"), c.pop("d"), "logistic", **c)
+    ref = lpc.Context(ctx.X, ctx.y, P.loss, P.lambda_l1, P.N, P.B, P.b, P.clip_mode, P.clip_value, P.seed)
+    x0 = (np.random.default_rng(9).standard_normal(P.d) * 0.1).astype(np.float32)
+    count = 131 if mode == "graph" else 7
+    for cx in (ctx, ref):
+        cx.set_option(lpc.OPT_TAP_U, 1)
+        cx.set_iterate(torch.from_numpy(x0).to(DEV))
+        cx.snapshot_full_grad()
+        cx.inner_step(0.05, 0)
+    if mode == "graph":
+        ctx.set_option(lpc.OPT_PERSISTENT, 0)
+    ctx.inner_steps(0.05, 1, count)
+    for k in range(1, 1 + count):
+        ref.inner_step(0.05, k)
+    ctx.sync_status()
+    ref.sync_status()
+    for w in (lpc.BUF_X, lpc.BUF_CODES, lpc.BUF_DELTA, lpc.BUF_CLIPPED, lpc.BUF_BATCH_IDX, lpc.BUF_COEF, lpc.BUF_U, lpc.BUF_V):
+        got, want = ctx.get_buffer(w), ref.get_buffer(w)
+        if w in (lpc.BUF_BATCH_IDX, lpc.BUF_COEF):
+            got, want = got[: P.N], want[: P.N]
+        assert _same(got, want), w
+    assert ctx.comm_bits() == ref.comm_bits()
+    assert ctx.query(lpc.INFO_LOOP_LAUNCHES) == (1 if mode == "persistent" else 0)  # the intended path really ran
+    assert ref.query(lpc.INFO_LOOP_LAUNCHES) == 0
+    ctx.close()
+    ref.close()
+
+
 @pytest.mark.parametrize("loss", ["least_squares", "logistic"])
 @pytest.mark.parametrize("cfg", [dict(n=128, d=1000, N=4, B=2, b=2), dict(n=128, d=8192, N=4, B=16, b=8),
                                  dict(n=64, d=4096, N=2, B=4, b=4)])
