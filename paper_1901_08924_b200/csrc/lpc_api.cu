@@ -84,7 +84,7 @@ struct lpc_ctx {
   bool persist_ok = false;
   int pCS = 1, pSL = 0;
   size_t persistSmem = 0;
-  unsigned int* flags = nullptr;  // 256 step counters + 1 abort word
+  unsigned long long* flags = nullptr;  // 2 x 256 publication words, 128 bytes apart, + 1 abort word
   int64_t persist_launches = 0;
   // stand-alone quantizer
   SegPlan seg;
@@ -351,8 +351,8 @@ int run_steps(lpc_ctx* c, int kind, const float* p, uint64_t k0, int64_t count) 
     pa.in = inner_args(c, k0, nullptr, 0);
     pa.in.CS = c->pCS; pa.in.SL = c->pSL;
     pa.count = (int)count; pa.eta = p[0]; pa.lambda_l1 = c->lambda_l1;
-    pa.flags = c->flags; pa.abort_flag = c->flags + 256; pa.x_out = c->x; pa.v_tap = c->tap_u ? c->v_tap : nullptr;
-    CU(c, cudaMemsetAsync(c->flags, 0, 257 * sizeof(unsigned int), c->stream));
+    pa.pub = c->flags; pa.abort_flag = reinterpret_cast<unsigned int*>(c->flags + 512 * 16); pa.x_out = c->x; pa.v_tap = c->tap_u ? c->v_tap : nullptr;
+    CU(c, cudaMemsetAsync(c->flags, 0, (512 * 16 + 1) * sizeof(unsigned long long), c->stream));
     cudaError_t e;
     { ProfScope ps_(c, LPC_KERNEL_INNER_LOOP); e = launch_persist(pa, c->persistSmem, c->stream); }
     if (e == cudaSuccess) {
@@ -505,7 +505,7 @@ int lpc_init(lpc_ctx** out, const float* X, const float* y, int64_t n, int32_t d
     A(dalloc(c, &c->delta, 2 * (size_t)N));  // two halves: the persistent loop alternates between them
     A(dalloc(c, &c->clipped, (size_t)N));
     A(dalloc(c, &c->clipped_part, (size_t)N * inner_clipped_stride()));
-    A(dalloc(c, &c->flags, 257));
+    A(dalloc(c, &c->flags, 512 * 16 + 1));
     A(dalloc(c, &c->idx_tap, (size_t)(N + 1) * B)); A(dalloc(c, &c->coef_tap, (size_t)(N + 1) * B));
     if (rc == LPC_OK) rc = make_plan(c, c->inner_seg, d, b, nullptr, 1);
     if (rc == LPC_OK) A(dalloc(c, &c->codes, 2 * (size_t)N * (size_t)c->inner_seg.stride_words));

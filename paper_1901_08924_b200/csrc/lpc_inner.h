@@ -42,7 +42,7 @@ struct PersistArgs {
   int count;
   float eta;
   float lambda_l1;
-  unsigned int* flags;       // N * CS step counters, zero at launch
+  unsigned long long* pub;   // 2 x 256 publication words (step count | delta << 32), 128 bytes apart, zero at launch
   unsigned int* abort_flag;  // zero at launch; set when a bounded wait ran out
   float* x_out;              // iterate after `count` steps (may alias in.x)
   float* v_tap;              // nullable: v of the last step

@@ -5,16 +5,25 @@
 // serial.  Launching kernels per step pays a launch + drain for every link of that chain.  Here the
 // grid stays resident for `count` steps (one cluster per worker, one CTA per SM, launched
 // cooperatively so that co-residency is guaranteed) and the only grid-wide dependency per step is a
-// flag wait:
+// wait on publication words:
 //   - every CTA keeps its slice of x and of mu in REGISTERS across steps;
 //   - the rows of step t+1 do not depend on step t (sampling is counter-based), so they are sampled
 //     and fetched by bulk copies (TMA) into the other half of a double buffer while step t computes;
-//   - when a CTA has stored the codes of its slice it raises its flag (release); at the top of the next
-//     step every CTA waits until all N*CS flags show the step (acquire), decodes all workers' codes for
-//     ITS slice with L1-bypassing loads, averages, adds mu and applies the proximal step in registers.
-// Every wait is bounded; when one runs out the CTA records LPC_ERR_TIMEOUT in the status word, raises a
-// global abort flag that makes every other wait return at once, and the loop finishes without hanging
-// (all CTAs still execute the same cluster barriers).
+//     labels and cached snapshot margins of those rows travel in registers of the thread that owns the
+//     minibatch slot;
+//   - when a CTA has stored the codes of its slice it publishes (step, delta) in one 64-bit release
+//     store to a word with a cache line of its own; at the top of the next step thread i of every CTA
+//     waits for the word of worker i's CTA of the same rank (acquire), then the CTA decodes all workers'
+//     codes for ITS slice with L1-bypassing loads, averages, adds mu and applies the proximal step in
+//     registers.  Codes and publication words are double-buffered by step parity, because a fast CTA may
+//     store step t+1 while a slow one still decodes step t.
+// Every wait is bounded; when one runs out the CTA records a timeout in the status word, raises a global
+// abort flag that makes every other wait return at once, and the loop finishes without hanging (all CTAs
+// still execute the same cluster barriers).
+//
+// The loop body is re-fetched from the instruction cache hierarchy every step, so its size shows up in the
+// step latency: the number of 2048-coordinate passes per CTA is a template parameter (no dead second pass)
+// and loops are unrolled only as far as instruction-level parallelism needs.
 //
 // The arithmetic (sampling, margins as balanced-tree sums, u summed in batch order, Eq. 2, the
 // quantizer, Eq. 3, the proximal step) is operation for operation that of the per-step kernels.
@@ -34,12 +43,10 @@ constexpr int PMAXP = 2;   // passes per CTA: SL <= 4096
 constexpr int PMAXB = 64;
 constexpr int PMAXCS = 8;
 constexpr int PMAXFLAGS = 256;
+constexpr int PUB_STRIDE = 16;  // publication words sit 128 bytes apart: one cache line each
 
 struct PSmem {
   uint64_t bar[2];
-  int64_t idx[2][PMAXB];
-  float yv[2][PMAXB];
-  float msnap[2][PMAXB];
   float coef[PMAXB];
   float wpart[PMAXB * PMAXP * 8];
   float mpart[PMAXB * PMAXCS];
@@ -50,10 +57,17 @@ struct PSmem {
   uint32_t wclip[8];
   float sdelta[PMAXFLAGS];
   Scale scale;
-  int abort;
   __align__(16) uint8_t stage[PT * 16];
 };
 
+__device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p) {
+  unsigned long long v;
+  asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_release_u64(unsigned long long* p, unsigned long long v) {
+  asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
 __device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int* p) {
   unsigned int v;
   asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
@@ -99,7 +113,21 @@ __device__ __forceinline__ uint32_t extract_bits(uint64_t lo, uint64_t hi, int p
   return (uint32_t)v & ((1u << b) - 1u);
 }
 
-template <int BITS>  // 1, 2, 4, 8 fixed width; 0: b from the arguments (1..16 or 32)
+// Phase timestamps of one CTA for latency studies; compiled in only with -DLPC_TRACE.
+#ifdef LPC_TRACE
+__device__ unsigned long long g_trace[64 * 16];
+#define LPC_TRACE_MARK(i)                                                                   \
+  do {                                                                                      \
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0 && t >= 8 && t < 72)         \
+      g_trace[(t - 8) * 16 + (i)] = global_ns();                                            \
+  } while (0)
+#else
+#define LPC_TRACE_MARK(i) do { } while (0)
+#endif
+
+// BITS: 1, 2, 4, 8 fixed width; 0: b from the arguments (1..16 or 32).
+// NP: passes of 2048 coordinates that a CTA makes over its slice (1 or 2).
+template <int BITS, int NP>
 __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
   const InnerArgs& a = pa.in;
   cg::cluster_group cluster = cg::this_cluster();
@@ -113,28 +141,27 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
   const int rank = (int)cluster.block_rank();
   const int worker = blockIdx.y;
   const int b = BITS ? BITS : a.b;
-  const int passes = (SL + PGROUP - 1) / PGROUP;
   const int c0 = rank * SL;
   const int width = max(0, min(SL, d - c0));
-  const int nflags = N * CS;
   const float invN = __fdiv_rn(1.0f, (float)N);
   const float invB = __fdiv_rn(1.0f, (float)B);
   const float kappa = mul_rn(pa.eta, pa.lambda_l1);
   const uint32_t zero_code = (b == 1) ? 0u : (1u << (b - 1));
-  // Codes and scales are double-buffered by step parity: a fast CTA may already store step t+1 while a
-  // slow one still decodes step t.  The parity is chosen so that the last step lands in buffer 0.
-  const int64_t codes_buf = (int64_t)N * a.stride_words;
+  const int64_t codes_buf = (int64_t)N * a.stride_words;  // one parity half of the code buffer
 
   if (tid == 0) {
     mbar_init(&sm.bar[0], 1);
     mbar_init(&sm.bar[1], 1);
     mbar_fence_init();
-    sm.abort = 0;
   }
   asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   __syncthreads();
 
-  // Samples the minibatch of step t and starts fetching this CTA's slice of its rows into buffer t&1.
+  // Thread a < B owns minibatch slot a.  prefetch(t) samples step t's row for the slot, starts the bulk copy
+  // of this CTA's slice of it into buffer t&1 and loads its label and cached snapshot margin into registers
+  // (a step ahead, so these loads never stall the step that issues them).
+  int64_t row_next = 0, row_cur = 0;
+  float y_next = 0.f, y_cur = 0.f, ms_next = 0.f, ms_cur = 0.f;
   auto prefetch = [&](int t) {
     const int s = t & 1;
     if (tid == 0 && width > 0) mbar_expect_tx(&sm.bar[s], (uint32_t)width * 4u * (uint32_t)B);
@@ -145,20 +172,20 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
       const U4 r = stream_block(a.seed, TAG_BATCH, (uint32_t)worker, a.k_base + (uint64_t)t, (uint32_t)tid);
       const int64_t row = lo + (int64_t)(((uint64_t)r.x * (uint64_t)span) >> 32);
       if (width > 0) bulk_load(rows + s * buf_floats + (size_t)tid * SL, a.X + row * (int64_t)d + c0, (uint32_t)width * 4u, &sm.bar[s]);
-      sm.idx[s][tid] = row;
-      sm.yv[s][tid] = a.y[row];
-      sm.msnap[s][tid] = a.margins[row];
+      row_next = row;
+      y_next = a.y[row];
+      ms_next = a.margins[row];
     }
   };
 
   // this thread's slice of the iterate and of the snapshot gradient stay in registers for the whole loop
-  float xr[PMAXP][8], mur[PMAXP][8];
+  float xr[NP][8], mur[NP][8];
 #pragma unroll
-  for (int p = 0; p < PMAXP; ++p) {
+  for (int p = 0; p < NP; ++p) {
     const int off = p * PGROUP + tid * 8;
 #pragma unroll
     for (int e = 0; e < 8; ++e) {
-      const bool in = (p < passes) && (off + e < width);
+      const bool in = off + e < width;
       xr[p][e] = in ? a.x[c0 + off + e] : 0.f;
       mur[p][e] = in ? a.mu[c0 + off + e] : 0.f;
     }
@@ -179,64 +206,67 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
     }
   };
 
-  // Waits until every CTA of the grid has published step `target`; then applies that step's update to xr.
+  // Waits until step target-1 has been published by the CTAs that wrote this slice's codes (those of the same
+  // rank in every worker's cluster), then applies that step's update to xr:
+  //   x <- prox_{eta h}(x - eta (mean_i delta_i k_i + mu)).
   auto apply_update = [&](unsigned int target) {
-    if (tid < nflags) {
-      const unsigned int* f = pa.flags + tid;
+    const int rpar = (pa.count - (int)target) & 1;  // parity half that holds step target-1
+    const unsigned long long* words = pa.pub + (size_t)rpar * PMAXFLAGS * PUB_STRIDE;
+    if (tid < N) {  // thread i watches worker i; N <= 256 = threads of the CTA
+      const unsigned long long* f = words + (size_t)(tid * CS + rank) * PUB_STRIDE;
+      unsigned long long w = 0;
       uint64_t t0 = 0;
       for (uint32_t it = 0;; ++it) {
-        if (ld_acquire_u32(f) >= target) break;
+        w = ld_acquire_u64(f);
+        if ((unsigned int)w >= target) break;
         if ((it & 63u) == 63u) {
-          if (ld_acquire_u32(pa.abort_flag) != 0u) { sm.abort = 1; break; }
+          if (ld_acquire_u32(pa.abort_flag) != 0u) break;
           const uint64_t now = global_ns();
           if (t0 == 0) t0 = now;
           else if (now - t0 > 2000000000ull) {
             atomicOr(a.dev_status, DEV_TIMEOUT);
             st_release_u32(pa.abort_flag, 1u);
-            sm.abort = 1;
             break;
           }
         }
       }
+      sm.sdelta[tid] = __uint_as_float((unsigned int)(w >> 32));
     }
     __syncthreads();
-    const int rpar = (pa.count - (int)target) & 1;  // buffer that holds step target-1
+#ifdef LPC_TRACE
+    { const int t = (int)target; LPC_TRACE_MARK(3); }
+#endif
     const uint32_t* codes_in = a.codes + rpar * codes_buf;
-    if (tid < N) sm.sdelta[tid] = __ldcg(a.delta + rpar * N + tid);
-    __syncthreads();
 #pragma unroll
-    for (int p = 0; p < PMAXP; ++p) {
-      if (p >= passes) break;
+    for (int p = 0; p < NP; ++p) {
       const int off = p * PGROUP + tid * 8;
-      if (off >= SL) continue;
       const int c = c0 + off;
+      if (off >= SL || c >= d) continue;
       float acc[8];
 #pragma unroll
       for (int e = 0; e < 8; ++e) acc[e] = 0.f;
-      if (c < d) {
-        if (b == 32) {
-          for (int i = 0; i < N; ++i) {
-            const uint32_t* wi = codes_in + (int64_t)i * a.stride_words;
-            const float di = sm.sdelta[i];
+      if (b == 32) {
+        for (int i = 0; i < N; ++i) {
+          const float di = sm.sdelta[i];
+          const uint32_t* wi = codes_in + (int64_t)i * a.stride_words;
 #pragma unroll
-            for (int e = 0; e < 8; ++e) {
-              const float val = (c + e < d) ? __uint_as_float(__ldcg(wi + c + e)) : 0.f;
-              acc[e] = add_rn(acc[e], mul_rn(di, val));
-            }
+          for (int e = 0; e < 8; ++e) {
+            const float val = (c + e < d) ? __uint_as_float(__ldcg(wi + c + e)) : 0.f;
+            acc[e] = add_rn(acc[e], mul_rn(di, val));
           }
-        } else {
+        }
+      } else {
 #pragma unroll 4
-          for (int i = 0; i < N; ++i) {
-            uint64_t lo, hi;
-            load_chunk_cg<BITS>(codes_in + (int64_t)i * a.stride_words, c >> 3, b, a.pad_words, lo, hi);
-            const float di = sm.sdelta[i];
+        for (int i = 0; i < N; ++i) {
+          const float di = sm.sdelta[i];
+          uint64_t lo, hi;
+          load_chunk_cg<BITS>(codes_in + (int64_t)i * a.stride_words, c >> 3, b, a.pad_words, lo, hi);
 #pragma unroll
-            for (int e = 0; e < 8; ++e) {
-              uint32_t code;
-              if constexpr (BITS == 0) code = extract_bits(lo, hi, e * b, b);
-              else code = (uint32_t)(lo >> (e * BITS)) & ((1u << BITS) - 1u);
-              acc[e] = add_rn(acc[e], mul_rn(di, index_as_float(code, b)));
-            }
+          for (int e = 0; e < 8; ++e) {
+            uint32_t code;
+            if constexpr (BITS == 0) code = extract_bits(lo, hi, e * b, b);
+            else code = (uint32_t)(lo >> (e * BITS)) & ((1u << BITS) - 1u);
+            acc[e] = add_rn(acc[e], mul_rn(di, index_as_float(code, b)));
           }
         }
       }
@@ -251,21 +281,27 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
     }
   };
 
+#pragma unroll 1
   for (int t = 0; t < pa.count; ++t) {
     const int s = t & 1;
     const uint64_t k = a.k_base + (uint64_t)t;
     const float* buf = rows + s * buf_floats;
-    const int wpar = (pa.count - 1 - t) & 1;
+    const int wpar = (pa.count - 1 - t) & 1;  // the last step lands in parity half 0
     uint32_t* out = a.codes + wpar * codes_buf + (int64_t)worker * a.stride_words;
+    LPC_TRACE_MARK(0);
+    row_cur = row_next; y_cur = y_next; ms_cur = ms_next;
     if (t + 1 < pa.count) prefetch(t + 1);
+    LPC_TRACE_MARK(1);
 
     // rounding bits of this step: they depend on the counters only, so they are drawn before the data arrives
-    U4 rnd[PMAXP];
+    U4 rnd[NP];
 #pragma unroll
-    for (int p = 0; p < PMAXP; ++p)
+    for (int p = 0; p < NP; ++p)
       rnd[p] = stream_block(a.seed, TAG_ROUND, (uint32_t)worker, k, (uint32_t)((c0 + p * PGROUP + tid * 8) >> 3));
 
+    LPC_TRACE_MARK(2);
     if (t > 0) apply_update((unsigned int)t);  // x_t = prox(x_{t-1} - eta v_{t-1})
+    LPC_TRACE_MARK(4);
 
     bool ok = true;
     if (width > 0) ok = mbar_wait(&sm.bar[s], (uint32_t)((t >> 1) & 1));
@@ -273,90 +309,121 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
       atomicOr(a.dev_status, DEV_TIMEOUT);
       mbar_wait(&sm.bar[s], (uint32_t)((t >> 1) & 1));
     }
+    LPC_TRACE_MARK(5);
 
-    // margins <X_a, x_t>
-    for (int r = 0; r < B; ++r) {
+    // margins <X_a, x_t>: four rows at a time so that their shuffle chains overlap
+#pragma unroll 1
+    for (int r0 = 0; r0 < B; r0 += 4) {
+      float sv[4][NP];
 #pragma unroll
-      for (int p = 0; p < PMAXP; ++p) {
-        if (p < passes) {
+      for (int j = 0; j < 4; ++j) {
+#pragma unroll
+        for (int p = 0; p < NP; ++p) {
           float v[8], pr[8];
-          row8(buf, r, p * PGROUP + tid * 8, v);
+          row8(buf, min(r0 + j, B - 1), p * PGROUP + tid * 8, v);
 #pragma unroll
           for (int e = 0; e < 8; ++e) pr[e] = mul_rn(v[e], xr[p][e]);
-          const float sv = warp_tree_sum(tree8(pr));
-          if (lane == 0) sm.wpart[(r * PMAXP + p) * 8 + warp] = sv;
+          sv[j][p] = tree8(pr);
+        }
+      }
+#pragma unroll
+      for (int m = 1; m < 32; m <<= 1) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+#pragma unroll
+          for (int p = 0; p < NP; ++p) sv[j][p] = add_rn(sv[j][p], __shfl_xor_sync(0xFFFFFFFFu, sv[j][p], m));
+        }
+      }
+      if (lane == 0) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+#pragma unroll
+          for (int p = 0; p < NP; ++p)
+            if (r0 + j < B) sm.wpart[((r0 + j) * NP + p) * 8 + warp] = sv[j][p];
         }
       }
     }
     __syncthreads();
+    LPC_TRACE_MARK(6);
     if (tid < B) {
-      float part = smem_tree_sum(&sm.wpart[tid * PMAXP * 8], 8);
-      if (passes == 2) part = add_rn(part, smem_tree_sum(&sm.wpart[(tid * PMAXP + 1) * 8], 8));
+      float part = smem_tree_sum(&sm.wpart[tid * NP * 8], 8);
+      if (NP == 2) part = add_rn(part, smem_tree_sum(&sm.wpart[(tid * NP + 1) * 8], 8));
       for (int q = 0; q < CS; ++q) cluster.map_shared_rank(sm.mpart, q)[tid * PMAXCS + rank] = part;
     }
     cluster.sync();
+    LPC_TRACE_MARK(7);
     if (tid < B) {
       const float m = smem_tree_sum(&sm.mpart[tid * PMAXCS], CS);
-      const float yy = sm.yv[s][tid];
-      const float c = __fsub_rn(loss_deriv(a.loss, m, yy), loss_deriv(a.loss, sm.msnap[s][tid], yy));
+      const float c = __fsub_rn(loss_deriv(a.loss, m, y_cur), loss_deriv(a.loss, ms_cur, y_cur));
       sm.coef[tid] = c;
       if (rank == 0 && t == pa.count - 1) {
-        if (a.idx_tap) a.idx_tap[(int64_t)worker * B + tid] = sm.idx[s][tid];
+        if (a.idx_tap) a.idx_tap[(int64_t)worker * B + tid] = row_cur;
         if (a.coef_tap) a.coef_tap[(int64_t)worker * B + tid] = c;
       }
     }
     __syncthreads();
+    LPC_TRACE_MARK(8);
 
-    // u = (1/B) sum_a c_a X_a in batch order
-    float u[PMAXP][8];
+    // u = (1/B) sum_a c_a X_a: four rows are loaded together, the adds keep batch order
+    float u[NP][8];
 #pragma unroll
-    for (int p = 0; p < PMAXP; ++p) {
+    for (int p = 0; p < NP; ++p) {
 #pragma unroll
       for (int e = 0; e < 8; ++e) u[p][e] = 0.f;
-      if (p < passes) {
-        for (int r = 0; r < B; ++r) {
-          float v[8];
-          row8(buf, r, p * PGROUP + tid * 8, v);
-          const float c = sm.coef[r];
+#pragma unroll 1
+      for (int r0 = 0; r0 < B; r0 += 4) {
+        float v[4][8], cf[4];
 #pragma unroll
-          for (int e = 0; e < 8; ++e) u[p][e] = add_rn(u[p][e], mul_rn(c, v[e]));
+        for (int j = 0; j < 4; ++j) {
+          const int r = min(r0 + j, B - 1);
+          row8(buf, r, p * PGROUP + tid * 8, v[j]);
+          cf[j] = sm.coef[r];
         }
 #pragma unroll
-        for (int e = 0; e < 8; ++e) u[p][e] = mul_rn(u[p][e], invB);
+        for (int j = 0; j < 4; ++j) {
+          if (r0 + j < B) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) u[p][e] = add_rn(u[p][e], mul_rn(cf[j], v[j][e]));
+          }
+        }
       }
+#pragma unroll
+      for (int e = 0; e < 8; ++e) u[p][e] = mul_rn(u[p][e], invB);
     }
     if (a.u_tap && t == pa.count - 1) {
 #pragma unroll
-      for (int p = 0; p < PMAXP; ++p) {
+      for (int p = 0; p < NP; ++p) {
         const int off = p * PGROUP + tid * 8;
-        if (p < passes) {
 #pragma unroll
-          for (int e = 0; e < 8; ++e)
-            if (off + e < width) a.u_tap[(int64_t)worker * d + c0 + off + e] = u[p][e];
-        }
+        for (int e = 0; e < 8; ++e)
+          if (off + e < width) a.u_tap[(int64_t)worker * d + c0 + off + e] = u[p][e];
       }
     }
 
+    LPC_TRACE_MARK(9);
     // scale (Eq. 2)
     uint32_t mx = 0;
 #pragma unroll
-    for (int p = 0; p < PMAXP; ++p) {
-      if (p < passes) {
+    for (int p = 0; p < NP; ++p) {
 #pragma unroll
-        for (int e = 0; e < 8; ++e) mx = max(mx, __float_as_uint(fabsf(u[p][e])));
-        if (a.clip_mode == CLIP_STD) {
-          float sq[8];
+      for (int e = 0; e < 8; ++e) mx = max(mx, __float_as_uint(fabsf(u[p][e])));
+      if (a.clip_mode == CLIP_STD) {
+        float sq[8];
 #pragma unroll
-          for (int e = 0; e < 8; ++e) sq[e] = mul_rn(u[p][e], u[p][e]);
-          const float s1 = warp_tree_sum(tree8(u[p]));
-          const float s2 = warp_tree_sum(tree8(sq));
-          if (lane == 0) { sm.ws1[p * 8 + warp] = s1; sm.ws2[p * 8 + warp] = s2; }
+        for (int e = 0; e < 8; ++e) sq[e] = mul_rn(u[p][e], u[p][e]);
+        float s1 = tree8(u[p]), s2 = tree8(sq);
+#pragma unroll
+        for (int m = 1; m < 32; m <<= 1) {
+          s1 = add_rn(s1, __shfl_xor_sync(0xFFFFFFFFu, s1, m));
+          s2 = add_rn(s2, __shfl_xor_sync(0xFFFFFFFFu, s2, m));
         }
+        if (lane == 0) { sm.ws1[p * 8 + warp] = s1; sm.ws2[p * 8 + warp] = s2; }
       }
     }
     mx = warp_max_u32(mx);
     if (lane == 0) sm.wmax[warp] = mx;
     __syncthreads();
+    LPC_TRACE_MARK(10);
     if (tid == 0) {
       uint32_t m = 0;
       for (int w = 0; w < 8; ++w) m = max(m, sm.wmax[w]);
@@ -364,7 +431,7 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
       if (a.clip_mode == CLIP_STD) {
         s1 = smem_tree_sum(sm.ws1, 8);
         s2 = smem_tree_sum(sm.ws2, 8);
-        if (passes == 2) { s1 = add_rn(s1, smem_tree_sum(sm.ws1 + 8, 8)); s2 = add_rn(s2, smem_tree_sum(sm.ws2 + 8, 8)); }
+        if (NP == 2) { s1 = add_rn(s1, smem_tree_sum(sm.ws1 + 8, 8)); s2 = add_rn(s2, smem_tree_sum(sm.ws2 + 8, 8)); }
       }
       for (int q = 0; q < CS; ++q) {
         cluster.map_shared_rank(sm.maxpart, q)[rank] = m;
@@ -373,6 +440,7 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
       }
     }
     cluster.sync();
+    LPC_TRACE_MARK(11);
     if (tid == 0) {
       uint32_t m = 0;
       for (int q = 0; q < CS; ++q) m = max(m, sm.maxpart[q]);
@@ -385,14 +453,14 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
       }
     }
     __syncthreads();
+    LPC_TRACE_MARK(12);
     const Scale sc = sm.scale;
     const bool degenerate = (sc.flags & 1u) != 0;
 
     // quantize (Section 2.2) and pack
     uint32_t nclip = 0;
 #pragma unroll
-    for (int p = 0; p < PMAXP; ++p) {
-      if (p >= passes) break;
+    for (int p = 0; p < NP; ++p) {
       const int off = p * PGROUP + tid * 8;
       const int c = c0 + off;
       const bool mine = off < SL;
@@ -464,88 +532,99 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
     nclip = __reduce_add_sync(0xFFFFFFFFu, nclip);
     if (lane == 0) sm.wclip[warp] = nclip;
     __syncthreads();  // every thread of this CTA has stored its codes
+    LPC_TRACE_MARK(13);
     if (tid == 0) {
       uint32_t tc = 0;
       for (int w = 0; w < 8; ++w) tc += sm.wclip[w];
       a.clipped_part[worker * PMAXCS + rank] = tc;
-      __threadfence();
-      st_release_u32(pa.flags + worker * CS + rank, (unsigned int)(t + 1));  // publish step t
+      // publish step t: (step count, delta) in one word; the release store orders every code stored above
+      st_release_u64(pa.pub + ((size_t)wpar * PMAXFLAGS + worker * CS + rank) * PUB_STRIDE,
+                     (unsigned long long)(unsigned int)(t + 1) | ((unsigned long long)__float_as_uint(sm.scale.delta) << 32));
     }
+    LPC_TRACE_MARK(14);
   }
 
   // the last step's update, then the slice of the final iterate goes back to memory (worker 0's cluster)
   if (pa.count > 0) apply_update((unsigned int)pa.count);
   if (worker == 0) {
 #pragma unroll
-    for (int p = 0; p < PMAXP; ++p) {
+    for (int p = 0; p < NP; ++p) {
       const int off = p * PGROUP + tid * 8;
-      if (p < passes) {
 #pragma unroll
-        for (int e = 0; e < 8; ++e)
-          if (off + e < width) pa.x_out[c0 + off + e] = xr[p][e];
-      }
+      for (int e = 0; e < 8; ++e)
+        if (off + e < width) pa.x_out[c0 + off + e] = xr[p][e];
     }
   }
   cluster.sync();  // no CTA leaves while a peer could still address its shared memory
 }
 
-template <int BITS>
-cudaError_t launch_p(const PersistArgs& pa, size_t smem, cudaStream_t st) {
-  cudaError_t e = cudaFuncSetAttribute(persist_kernel<BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) return e;
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)pa.in.CS, (unsigned)pa.in.N, 1);
-  cfg.blockDim = dim3(PT, 1, 1);
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = st;
-  cudaLaunchAttribute attr[2];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = (unsigned)pa.in.CS;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  attr[1].id = cudaLaunchAttributeCooperative;  // all CTAs co-resident or the launch fails
-  attr[1].val.cooperative = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 2;
-  return cudaLaunchKernelEx(&cfg, persist_kernel<BITS>, pa);
-}
-
-}  // namespace
-
-namespace {
-template <int BITS>
-int max_clusters_t(int cs, size_t smem) {
-  if (cudaFuncSetAttribute(persist_kernel<BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
-    cudaGetLastError();
-    return 0;
-  }
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)cs, 1, 1);
-  cfg.blockDim = dim3(PT, 1, 1);
-  cfg.dynamicSmemBytes = smem;
-  cudaLaunchAttribute attr[1];
+template <int BITS, int NP>
+void fill_config(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr, int cs, int clusters, size_t smem, cudaStream_t st,
+                 bool cooperative) {
+  *cfg = cudaLaunchConfig_t{};
+  cfg->gridDim = dim3((unsigned)cs, (unsigned)clusters, 1);
+  cfg->blockDim = dim3(PT, 1, 1);
+  cfg->dynamicSmemBytes = smem;
+  cfg->stream = st;
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = (unsigned)cs;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  attr[1].id = cudaLaunchAttributeCooperative;  // all CTAs co-resident or the launch fails
+  attr[1].val.cooperative = 1;
+  cfg->attrs = attr;
+  cfg->numAttrs = cooperative ? 2 : 1;
+}
+
+template <int BITS, int NP>
+cudaError_t launch_p(const PersistArgs& pa, size_t smem, cudaStream_t st) {
+  cudaError_t e = cudaFuncSetAttribute(persist_kernel<BITS, NP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  cudaLaunchConfig_t cfg;
+  cudaLaunchAttribute attr[2];
+  fill_config<BITS, NP>(&cfg, attr, pa.in.CS, pa.in.N, smem, st, true);
+  return cudaLaunchKernelEx(&cfg, persist_kernel<BITS, NP>, pa);
+}
+
+template <int BITS, int NP>
+int max_clusters_t(int cs, size_t smem) {
+  if (cudaFuncSetAttribute(persist_kernel<BITS, NP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+    cudaGetLastError();
+    return 0;
+  }
+  cudaLaunchConfig_t cfg;
+  cudaLaunchAttribute attr[2];
+  fill_config<BITS, NP>(&cfg, attr, cs, 1, smem, nullptr, false);
   int n = 0;
-  if (cudaOccupancyMaxActiveClusters(&n, persist_kernel<BITS>, &cfg) != cudaSuccess) {
+  if (cudaOccupancyMaxActiveClusters(&n, persist_kernel<BITS, NP>, &cfg) != cudaSuccess) {
     cudaGetLastError();
     return 0;
   }
   return n;
 }
-int max_clusters(int b, int cs, size_t smem) {
+
+template <int NP>
+int max_clusters_np(int b, int cs, size_t smem) {
   switch (b) {
-    case 1: return max_clusters_t<1>(cs, smem);
-    case 2: return max_clusters_t<2>(cs, smem);
-    case 4: return max_clusters_t<4>(cs, smem);
-    case 8: return max_clusters_t<8>(cs, smem);
-    default: return max_clusters_t<0>(cs, smem);
+    case 1: return max_clusters_t<1, NP>(cs, smem);
+    case 2: return max_clusters_t<2, NP>(cs, smem);
+    case 4: return max_clusters_t<4, NP>(cs, smem);
+    case 8: return max_clusters_t<8, NP>(cs, smem);
+    default: return max_clusters_t<0, NP>(cs, smem);
   }
 }
+
+template <int NP>
+cudaError_t launch_np(const PersistArgs& pa, size_t smem, cudaStream_t st) {
+  switch (pa.in.b) {
+    case 1: return launch_p<1, NP>(pa, smem, st);
+    case 2: return launch_p<2, NP>(pa, smem, st);
+    case 4: return launch_p<4, NP>(pa, smem, st);
+    case 8: return launch_p<8, NP>(pa, smem, st);
+    default: return launch_p<0, NP>(pa, smem, st);
+  }
+}
+
 }  // namespace
 
 // Cluster size / slice for the persistent loop: all N clusters must be co-resident (the occupancy query
@@ -556,7 +635,7 @@ bool persist_plan(int d, int N, int B, int b, int want_cs, int max_smem, int* CS
   int P = 1;
   while (P < d) P <<= 1;
   if (P < 32) P = 32;
-  if (B > PMAXB) return false;
+  if (B > PMAXB || N > PMAXFLAGS) return false;
   bool found = false;
   for (int cs = 1; cs <= PMAXCS; cs <<= 1) {
     if (want_cs > 0 && cs != want_cs) continue;
@@ -566,7 +645,8 @@ bool persist_plan(int d, int N, int B, int b, int want_cs, int max_smem, int* CS
     if (N * cs > PMAXFLAGS) break;
     const size_t smem = ((sizeof(PSmem) + 15) & ~(size_t)15) + 2 * (size_t)B * SL * 4;
     if (smem > (size_t)max_smem) continue;
-    if (max_clusters(b, cs, smem) < N) continue;
+    const int fit = (SL > PGROUP) ? max_clusters_np<2>(b, cs, smem) : max_clusters_np<1>(b, cs, smem);
+    if (fit < N) continue;
     *CS_out = cs; *SL_out = SL; *smem_out = smem;
     found = true;
     if (want_cs > 0) break;
@@ -576,13 +656,13 @@ bool persist_plan(int d, int N, int B, int b, int want_cs, int max_smem, int* CS
 }
 
 cudaError_t launch_persist(const PersistArgs& pa, size_t smem, cudaStream_t st) {
-  switch (pa.in.b) {
-    case 1: return launch_p<1>(pa, smem, st);
-    case 2: return launch_p<2>(pa, smem, st);
-    case 4: return launch_p<4>(pa, smem, st);
-    case 8: return launch_p<8>(pa, smem, st);
-    default: return launch_p<0>(pa, smem, st);
-  }
+  return (pa.in.SL > PGROUP) ? launch_np<2>(pa, smem, st) : launch_np<1>(pa, smem, st);
 }
+
+#ifdef LPC_TRACE
+extern "C" int lpc_trace_read(unsigned long long* host_out) {
+  return cudaMemcpyFromSymbol(host_out, g_trace, sizeof(g_trace)) == cudaSuccess ? 0 : -4;
+}
+#endif
 
 }  // namespace lpc
