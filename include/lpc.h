@@ -238,6 +238,31 @@ int lpc_svrg_run_host(const float* X_host, const float* y_host, int64_t n, int32
                       double* objective_out, uint64_t* step2_bits_out);
 
 /*
+ * Quantize + pack for callers that must not allocate device memory.  The paper has no counterpart:
+ * this is the same operation as lpc_quantize_pack on one unsegmented vector per worker (Algorithm 1
+ * step 7), offered for code that cannot call cudaMalloc where it runs: a latency-critical loop that may
+ * not take the allocator's locks or provoke its implicit synchronisation, a plug-in living inside a
+ * host application's fixed memory budget, a process whose device memory is already fully partitioned.
+ * It needs no context.  Its working memory (tile partials, scale records) is a fixed array of about
+ * 0.8 MB inside the library image, held by every GPU that loads the library until the process exits.
+ *   U            N x len fp32, row stride ld (device)
+ *   codes_out    N * stride_words words, stride_words from lpc_packed_layout(len, b, NULL, 1) (device,
+ *                16-byte aligned);  delta_out N floats;  clipped_out N counts (all required)
+ *   stream       cudaStream_t
+ * Limits: N <= LPC_STATIC_MAX_WORKERS and N * ceil(len / 8192) <= LPC_STATIC_MAX_TILES; anything larger
+ * returns LPC_ERR_UNSUPPORTED and launches nothing.  Non-finite input yields a NaN delta.
+ * The first call on a device looks up the array's device address; make that first call outside any
+ * stream capture.  All calls share the array and it keeps the previous call's contents (what has to
+ * start from zero is cleared by the call itself), so two calls that can overlap on the GPU (different
+ * streams, several host threads) race: serialise them.  The call allocates and frees nothing.
+ */
+#define LPC_STATIC_MAX_WORKERS 64
+#define LPC_STATIC_MAX_TILES 65536
+int lpc_quantize_pack_static(const float* U, int64_t len, int64_t ld, int32_t N, int32_t b, int clip_mode,
+                             float clip_value, uint64_t seed, uint64_t k, uint32_t* codes_out, float* delta_out,
+                             uint32_t* clipped_out, void* stream);
+
+/*
  * Inspection aid: writes `count` consecutive 4-word blocks, starting at block `block0`, of the
  * counter-based random stream (tag, worker, k) keyed by `seed` to out (device, 4*count words).
  * The streams are Philox4x32-10 (Salmon et al., SC'11) with counter (block, k_lo, worker | tag<<24,

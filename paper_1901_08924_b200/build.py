@@ -14,7 +14,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "liblpcsvrg.so")
-SOURCES = ["lpc_api.cu", "lpc_quantize.cu", "lpc_aggregate.cu", "lpc_snapshot.cu", "lpc_inner.cu", "lpc_persist.cu"]
+SOURCES = ["lpc_api.cu", "lpc_quantize.cu", "lpc_aggregate.cu", "lpc_snapshot.cu", "lpc_inner.cu", "lpc_persist.cu", "lpc_noalloc.cu"]
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-fmad=false",
               "-Xcompiler", "-fPIC", "-Xptxas", "-v"]

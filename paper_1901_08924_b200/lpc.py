@@ -51,6 +51,7 @@ SYMBOLS = [
     ("lpc_query", _int, [_vp, _int, _i64p]),
     ("lpc_svrg_run_host", _int, [_vp, _vp, _i64, _i32, _int, _f32, _i32, _i32, _i32, _int, _f32, _u64, _i32, _i64,
                                  _f32, _vp, _f64p, _u64p]),
+    ("lpc_quantize_pack_static", _int, [_vp, _i64, _i64, _i32, _i32, _int, _f32, _u64, _u64, _vp, _vp, _vp, _vp]),
     ("lpc_debug_stream_blocks", _int, [_u64, C.c_uint32, C.c_uint32, _u64, C.c_uint32, _i64, _vp, _vp]),
 ]
 
@@ -274,3 +275,17 @@ def debug_stream_blocks(seed, tag, worker, k, block0, count, device=None):
     if rc != OK:
         raise LpcError(rc, "lpc_debug_stream_blocks")
     return out
+
+
+def quantize_pack_static(U, b, clip_mode, clip_value, seed, k, codes_out, delta_out, clipped_out):
+    """Quantize + pack without any device allocation inside the library (see lpc_quantize_pack_static).
+
+    The caller supplies every buffer: U (N, len) fp32, codes_out (N, stride_words) int32 with stride_words from
+    packed_layout(len, b), delta_out (N,) fp32, clipped_out (N,) int32.  Returns the status code.
+    """
+    assert U.is_cuda and U.dtype == torch.float32 and U.dim() == 2 and U.stride(1) == 1
+    N, length = U.shape
+    ld = U.stride(0) if N > 1 else max(length, 1)
+    st = torch.cuda.current_stream(U.device)
+    return lib().lpc_quantize_pack_static(_ptr(U), length, ld, N, b, clip_mode, clip_value, seed, k, _ptr(codes_out),
+                                          _ptr(delta_out), _ptr(clipped_out), C.c_void_p(st.cuda_stream))
