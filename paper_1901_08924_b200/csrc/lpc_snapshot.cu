@@ -6,8 +6,11 @@
 // Design: a persistent grid of one CTA per SM.  A CTA pulls tiles of R consecutive rows (contiguous
 // in memory) into a ring of shared-memory stages with one bulk-copy (TMA) transaction per tile,
 // tracked by an mbarrier per stage, so several tiles are in flight per SM while one is processed.
-// A tile is read from shared memory twice: once for the margins and once, scaled by l', for the
-// column sums, which stay in registers (thread t owns columns 4t..4t+3 of every 1024-column chunk).
+// Each thread copies its part of a tile (columns 4t..4t+3 of every 1024-column chunk, all R rows:
+// R*KMAX = 16 float4) from shared memory into registers ONCE; the stage is handed back to the copy
+// engine right after that.  From the registers come both the margin products and, once l' is known,
+// the column sums, which also stay in registers.  The 16 per-thread partial products are reduced
+// across the warp by recursive halving (16 shuffles instead of 16 x 5).
 // The margin of a row is the balanced-tree fp32 sum of its products in column order, so it is
 // bit-identical to the margin any other kernel of the library computes for the same row and point.
 #include "lpc_device.cuh"
@@ -21,38 +24,70 @@ constexpr int ST = 256;       // threads
 constexpr int CHUNK = ST * 4; // columns covered by one sweep of the CTA
 constexpr int MAXLEAF = 128;  // 128-column leaves of the margin tree: d <= 16384
 
+__host__ __device__ constexpr int rows_per_tile(int kmax) { return kmax >= 16 ? 1 : kmax >= 8 ? 2 : kmax >= 4 ? 4 : 8; }
+
+// Warp reduction of V values per lane by recursive halving.  At the stage with lane mask 1<<S a lane
+// keeps one half of its values and receives the partner's partial sums for that half; lanes with the bit
+// clear keep the lower half.  After log2(V) stages one value is left, and the remaining stages are plain
+// butterflies.  Partner sums are added in lane order, which is the balanced tree over the 32 lanes.
+template <int V, int S>
+struct WarpHalving {
+  static __device__ __forceinline__ void run(float* v, int lane) {
+    if constexpr (S < 5) {
+      if constexpr (V > 1) {
+        const bool up = (lane >> S) & 1;
+#pragma unroll
+        for (int i = 0; i < V / 2; ++i) {
+          const float send = up ? v[i] : v[i + V / 2];
+          const float keep = up ? v[i + V / 2] : v[i];
+          v[i] = add_rn(keep, __shfl_xor_sync(0xFFFFFFFFu, send, 1 << S));
+        }
+        WarpHalving<V / 2, S + 1>::run(v, lane);
+      } else {
+        v[0] = add_rn(v[0], __shfl_xor_sync(0xFFFFFFFFu, v[0], 1 << S));
+        WarpHalving<1, S + 1>::run(v, lane);
+      }
+    }
+  }
+};
+
 template <int KMAX, bool GRAD>
 __global__ void __launch_bounds__(ST, 1) snapshot_kernel(SnapArgs a) {
+  constexpr int R = rows_per_tile(KMAX);
+  constexpr int NV = R * KMAX;  // float4 values per thread and tile
+  constexpr int LOGV = NV == 16 ? 4 : NV == 8 ? 3 : NV == 4 ? 2 : NV == 2 ? 1 : 0;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int d = a.d;
-  const int dpad = KMAX * CHUNK;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem_raw);                       // nstage
   float* part = reinterpret_cast<float*>(smem_raw + 64);                        // R * MAXLEAF
-  float* coef = part + a.R * MAXLEAF;                                           // R (padded to 4)
-  float* xs = coef + ((a.R + 3) & ~3);                                          // dpad
-  float* stages = xs + dpad;                                                    // nstage * R * d
+  float* coef = part + R * MAXLEAF;                                             // 8
+  float* stages = coef + 8;                                                     // nstage * R * d
   __shared__ double fsh[8];
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int64_t stage_floats = (int64_t)a.R * d;
+  const int64_t stage_floats = (int64_t)R * d;
 
-  for (int c = tid; c < dpad; c += ST) xs[c] = (c < d) ? a.x[c] : 0.f;
+  // this thread's columns of the point x
+  float4 xq[KMAX];
+#pragma unroll
+  for (int k = 0; k < KMAX; ++k) {
+    const int col = k * CHUNK + tid * 4;
+    xq[k] = (col < d) ? *reinterpret_cast<const float4*>(a.x + col) : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
   if (tid == 0) {
     for (int s = 0; s < a.nstage; ++s) mbar_init(&bars[s], 1);
     mbar_fence_init();
   }
   __syncthreads();
 
-  // leaves of the margin tree
   int P = 1;
   while (P < d) P <<= 1;
-  const int nleaf = (P >= 128) ? P / 128 : 1;
+  const int nleaf = (P >= 128) ? P / 128 : 1;  // leaves of the margin tree
 
   const int64_t my_tiles = (a.ntiles > (int64_t)blockIdx.x) ? (a.ntiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
   auto issue = [&](int64_t i) {  // thread 0 only
-    const int64_t tile = (int64_t)blockIdx.x + i * gridDim.x;
-    const int64_t row0 = tile * a.R;
-    const int rows = (int)min((int64_t)a.R, a.n - row0);
+    const int64_t row0 = ((int64_t)blockIdx.x + i * gridDim.x) * R;
+    const int rows = (int)min((int64_t)R, a.n - row0);
     const uint32_t bytes = (uint32_t)((int64_t)rows * d * 4);
     const int s = (int)(i % a.nstage);
     mbar_expect_tx(&bars[s], bytes);
@@ -61,6 +96,13 @@ __global__ void __launch_bounds__(ST, 1) snapshot_kernel(SnapArgs a) {
   if (tid == 0)
     for (int64_t i = 0; i < min((int64_t)a.nstage, my_tiles); ++i) issue(i);
 
+  // lane 0 of warp r owns row r of a tile: its label is fetched one tile ahead
+  float y_next = 0.f;
+  if (lane == 0 && warp < R && my_tiles > 0) {
+    const int64_t row = (int64_t)blockIdx.x * R + warp;
+    if (row < a.n) y_next = a.y[row];
+  }
+
   float4 acc[KMAX];
 #pragma unroll
   for (int k = 0; k < KMAX; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -68,68 +110,77 @@ __global__ void __launch_bounds__(ST, 1) snapshot_kernel(SnapArgs a) {
   int64_t done = 0;  // tiles whose data has been consumed
   bool failed = false;
 
+#pragma unroll 1
   for (int64_t i = 0; i < my_tiles; ++i) {
     const int s = (int)(i % a.nstage);
     const uint32_t parity = (uint32_t)((i / a.nstage) & 1);
     const int ok = mbar_wait(&bars[s], parity) ? 1 : 0;
     if (!__syncthreads_and(ok)) { failed = true; break; }
-    const int64_t tile = (int64_t)blockIdx.x + i * gridDim.x;
-    const int64_t row0 = tile * a.R;
-    const int rows = (int)min((int64_t)a.R, a.n - row0);
+    const int64_t row0 = ((int64_t)blockIdx.x + i * gridDim.x) * R;
+    const int rows = (int)min((int64_t)R, a.n - row0);
     const float* st = stages + (int64_t)s * stage_floats;
 
-    // phase A: partial tree sums of the products, one leaf (128 columns) per warp and chunk
-    for (int r = 0; r < rows; ++r) {
-      const float* row = st + (int64_t)r * d;
+    // phase A: tile -> registers, products, per-warp leaves (128 columns each) of every row's margin tree
+    float4 xv[NV];
+    float pv[NV];
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
 #pragma unroll
       for (int k = 0; k < KMAX; ++k) {
         const int col = k * CHUNK + tid * 4;
-        float sv = 0.f;
-        if (col < d) {  // d is a multiple of 4
-          const float4 xv = *reinterpret_cast<const float4*>(row + col);
-          const float4 wv = *reinterpret_cast<const float4*>(xs + col);
-          sv = tree4(mul_rn(xv.x, wv.x), mul_rn(xv.y, wv.y), mul_rn(xv.z, wv.z), mul_rn(xv.w, wv.w));
-        }
-        if (k * CHUNK < d) sv = warp_tree_sum(sv);  // chunks past the row contribute zero leaves
-        if (lane == 0 && k * 8 + warp < nleaf) part[r * MAXLEAF + k * 8 + warp] = sv;
+        const int q = r * KMAX + k;
+        xv[q] = (col < d && r < rows) ? *reinterpret_cast<const float4*>(st + (int64_t)r * d + col)
+                                      : make_float4(0.f, 0.f, 0.f, 0.f);
+        pv[q] = tree4(mul_rn(xv[q].x, xq[k].x), mul_rn(xv[q].y, xq[k].y), mul_rn(xv[q].z, xq[k].z), mul_rn(xv[q].w, xq[k].w));
       }
     }
-    __syncthreads();
-    // phase B: warp r finishes row r's tree, applies the loss derivative
-    for (int r = warp; r < rows; r += ST / 32) {
+    WarpHalving<NV, 0>::run(pv, lane);
+    if ((lane >> LOGV) == 0) {
+      // the value left in this lane belongs to q whose bits, most significant first, are the lane's low bits
+      int q = 0;
+#pragma unroll
+      for (int sft = 0; sft < LOGV; ++sft) q |= ((lane >> sft) & 1) << (LOGV - 1 - sft);
+      const int r = q / KMAX, k = q % KMAX;
+      if (k * 8 + warp < nleaf) part[r * MAXLEAF + k * 8 + warp] = pv[0];
+    }
+    __syncthreads();  // leaves visible; every thread holds its part of the tile in registers
+    ++done;
+    if (tid == 0 && i + a.nstage < my_tiles) issue(i + a.nstage);  // the stage can be refilled already
+
+    // phase B: warp r finishes row r's tree and applies the loss derivative
+    if (warp < R) {
       float v4[4];
 #pragma unroll
-      for (int e = 0; e < 4; ++e) v4[e] = (lane * 4 + e < nleaf) ? part[r * MAXLEAF + lane * 4 + e] : 0.f;
+      for (int e = 0; e < 4; ++e) v4[e] = (lane * 4 + e < nleaf) ? part[warp * MAXLEAF + lane * 4 + e] : 0.f;
       const float m = warp_tree_sum(tree4(v4[0], v4[1], v4[2], v4[3]));
       if (lane == 0) {
-        const float yy = a.y[row0 + r];
-        if (a.margins_out) a.margins_out[row0 + r] = m;
-        coef[r] = loss_deriv(a.loss, m, yy);
-        fsum += loss_value(a.loss, m, yy);
+        float c = 0.f;
+        if (warp < rows) {
+          if (a.margins_out) a.margins_out[row0 + warp] = m;
+          c = loss_deriv(a.loss, m, y_next);
+          fsum += loss_value(a.loss, m, y_next);
+        }
+        coef[warp] = c;
+        const int64_t nrow = row0 + (int64_t)gridDim.x * R + warp;  // same slot of this CTA's next tile
+        if (i + 1 < my_tiles && nrow < a.n) y_next = a.y[nrow];
       }
     }
     if (GRAD) {
       __syncthreads();
-      // phase C: column sums  acc += l'_r * X_r
-      for (int r = 0; r < rows; ++r) {
-        const float* row = st + (int64_t)r * d;
+      // phase C: column sums  acc += l'_r * X_r, from registers
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
         const float c = coef[r];
 #pragma unroll
         for (int k = 0; k < KMAX; ++k) {
-          const int col = k * CHUNK + tid * 4;
-          if (col < d) {
-            const float4 xv = *reinterpret_cast<const float4*>(row + col);
-            acc[k].x = __fmaf_rn(c, xv.x, acc[k].x);
-            acc[k].y = __fmaf_rn(c, xv.y, acc[k].y);
-            acc[k].z = __fmaf_rn(c, xv.z, acc[k].z);
-            acc[k].w = __fmaf_rn(c, xv.w, acc[k].w);
-          }
+          const int q = r * KMAX + k;
+          acc[k].x = __fmaf_rn(c, xv[q].x, acc[k].x);
+          acc[k].y = __fmaf_rn(c, xv[q].y, acc[k].y);
+          acc[k].z = __fmaf_rn(c, xv[q].z, acc[k].z);
+          acc[k].w = __fmaf_rn(c, xv[q].w, acc[k].w);
         }
       }
     }
-    __syncthreads();  // every thread is done reading stage s
-    ++done;
-    if (tid == 0 && i + a.nstage < my_tiles) issue(i + a.nstage);
   }
 
   if (failed) {
@@ -144,12 +195,9 @@ __global__ void __launch_bounds__(ST, 1) snapshot_kernel(SnapArgs a) {
   }
 
   if (GRAD) {
-    float* out = a.partial_mu + (int64_t)blockIdx.x * dpad;
+    float* out = a.partial_mu + (int64_t)blockIdx.x * (KMAX * CHUNK);
 #pragma unroll
-    for (int k = 0; k < KMAX; ++k) {
-      const int col = k * CHUNK + tid * 4;
-      *reinterpret_cast<float4*>(out + col) = acc[k];
-    }
+    for (int k = 0; k < KMAX; ++k) *reinterpret_cast<float4*>(out + k * CHUNK + tid * 4) = acc[k];
   }
   // f partial of this CTA
 #pragma unroll
@@ -223,22 +271,14 @@ int snapshot_dpad(int d) {
 }
 
 void snapshot_plan(int d, int max_smem, int* R_out, int* nstage_out, size_t* smem_out) {
-  const int dpad = snapshot_dpad(d);
-  const size_t row_bytes = (size_t)d * 4;
-  int R = 1;
-  while (R < 8 && (size_t)(2 * R) * row_bytes <= 65536) R <<= 1;  // up to 64 KB per stage
-  for (;;) {
-    const size_t fixed = 64 + ((size_t)R * MAXLEAF + ((R + 3) & ~3) + dpad) * 4;
-    const size_t stage = (size_t)R * row_bytes;
-    int nstage = (int)(((size_t)max_smem - fixed) / stage);
-    if (nstage > 6) nstage = 6;
-    if (nstage >= 2 || R == 1) {
-      if (nstage < 1) nstage = 1;
-      *R_out = R; *nstage_out = nstage; *smem_out = fixed + (size_t)nstage * stage;
-      return;
-    }
-    R >>= 1;
-  }
+  const int kmax = snapshot_dpad(d) / CHUNK;
+  const int R = rows_per_tile(kmax);  // fixed by the register layout: R * kmax = 16 float4 per thread (8 for kmax = 1)
+  const size_t fixed = 64 + ((size_t)R * MAXLEAF + 8) * 4;
+  const size_t stage = (size_t)R * d * 4;
+  int nstage = (int)(((size_t)max_smem - fixed) / stage);
+  if (nstage > 8) nstage = 8;
+  if (nstage < 1) nstage = 1;
+  *R_out = R; *nstage_out = nstage; *smem_out = fixed + (size_t)nstage * stage;
 }
 
 cudaError_t launch_snapshot(const SnapArgs& a, int grid, size_t smem, cudaStream_t st) {
