@@ -206,9 +206,11 @@ int quantize_coord(float u, float rdelta, int b, uint32_t r16) {
   if (s < lo) s = lo;  // rule (2): outside the hull -> smallest ...
   if (s > hi) s = hi;  //                            ... or largest codebook value
   const float fl = std::floor(s);
-  const float f = s - fl;  // exact
-  // rule (1): round up with probability (x - z)/delta = f, realised on a 2^-16 grid
-  const bool up = ((float)r16 + 0.5f) < f * 65536.0f;
+  // rule (1): round up with probability (x - z)/delta = s - floor(s), realised on a 2^-16 grid.  The
+  // fraction is taken in fp64, where it is exact for every fp32 s (an fp32 subtraction would round it
+  // when s is negative), and so is the comparison.
+  const double f = (double)s - (double)fl;
+  const bool up = ((double)r16 + 0.5) < f * 65536.0;
   return (int)fl + (up ? 1 : 0);
 }
 

@@ -741,7 +741,7 @@ int lpc_quantize_pack(lpc_ctx* c, const float* U, const float* U_sub, int64_t le
   a.seed = c->seed; a.k = k; a.segs = p.d_segs; a.tile_seg = p.d_tile_seg; a.nseg = p.nseg; a.ntiles = p.ntiles;
   a.pmax = c->q_pmax; a.ps1 = c->q_ps1; a.ps2 = c->q_ps2; a.scales = c->q_scales;
   a.codes = codes_out; a.stride_words = p.stride_words; a.delta_out = delta_out;
-  a.clipped_out = clipped_out ? clipped_out : c->q_clip; a.dev_status = c->dev_status;
+  a.clipped_out = clipped_out ? clipped_out : c->q_clip; a.count_clipped = clipped_out ? 1 : 0; a.dev_status = c->dev_status;
   CU(c, launch_quantize_pack(a, c->stream, c->profile ? prof_hook : nullptr, c));
   c->step2_bits += p.msg_bits * (uint64_t)c->N * (uint64_t)(c->N - 1);
   return LPC_OK;

@@ -27,8 +27,10 @@ __device__ __forceinline__ U4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c
                                             uint32_t k0, uint32_t k1) {
 #pragma unroll
   for (int r = 0; r < 10; ++r) {
-    const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
-    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+    const uint64_t p0 = (uint64_t)0xD2511F53u * (uint64_t)c0;  // one wide multiply gives both halves
+    const uint64_t p1 = (uint64_t)0xCD9E8D57u * (uint64_t)c2;
+    const uint32_t hi0 = (uint32_t)(p0 >> 32), lo0 = (uint32_t)p0;
+    const uint32_t hi1 = (uint32_t)(p1 >> 32), lo1 = (uint32_t)p1;
     c0 = hi1 ^ c1 ^ k0;
     c1 = lo1;
     c2 = hi0 ^ c3 ^ k1;
@@ -136,42 +138,50 @@ __device__ __forceinline__ Scale make_scale(uint32_t max_bits, float S1, float S
 
 // ---- quantizer of Section 2.2 for one coordinate -----------------------------------------------------
 // Returns the stored code c = k + 2^(b-1) (b=1: the bit).  r16 is the coordinate's 16-bit random lane.
+// s = u/delta (fp32) is clamped to the hull first (rule 2), then rounded down or up with probability
+// frac(s) = s - floor(s), taken exactly (rule 1):   up  <=>  r16 + 0.5 < frac(s) * 65536.
+//
+// The decision is evaluated in fixed point, exactly and with few instructions (the quantize pass is bound
+// by instruction issue).  Z = ceil(s * 2^17) is exact (a power-of-two scaling and one conversion).  Then
+//   A := ceil(s * 65536 - 1/2) = floor(Z / 2),
+//   r16 + 1/2 < frac(s) * 65536   <=>   r16 < A - 65536 * floor(s)          (r16 is an integer),
+//   floor(s) + [r16 < A - 65536 floor(s)] = floor((A + 65535 - r16) / 65536)  (0 <= r16 <= 65535),
+// and both floors are arithmetic right shifts.
 template <int B_>
 __device__ __forceinline__ uint32_t quantize_code(float u, float rdelta, uint32_t r16) {
-  if (B_ == 1) {
+  static_assert(B_ >= 1 && B_ <= 8, "32-bit fixed point covers b <= 8");
+  if constexpr (B_ == 1) {
     float s = mul_rn(u, rdelta);
     s = fminf(fmaxf(s, -1.f), 1.f);
-    const float f = mul_rn(add_rn(s, 1.f), 0.5f);
-    return (add_rn((float)r16, 0.5f) < mul_rn(f, 65536.f)) ? 1u : 0u;
+    // position between the two code points, ((s + 1) / 2) * 65536 = (s + 1) * 32768 with s + 1 rounded to fp32
+    const int A = __float2int_ru(mul_rn(add_rn(s, 1.f), 65536.f)) >> 1;  // ceil(t - 1/2), in [0, 65536]
+    return ((int)r16 < A) ? 1u : 0u;
+  } else {
+    constexpr float lo = -(float)(1 << (B_ - 1));
+    constexpr float hi = (float)((1 << (B_ - 1)) - 1);
+    float s = mul_rn(u, rdelta);
+    s = fminf(fmaxf(s, lo), hi);  // projection onto the hull (rule 2)
+    const int A = __float2int_ru(mul_rn(s, 131072.f)) >> 1;
+    return (uint32_t)((A + (65535 + (65536 << (B_ - 1))) - (int)r16) >> 16);  // floor(s) + up + 2^(b-1)
   }
-  constexpr float lo = -(float)(1 << (B_ - 1));
-  constexpr float hi = (float)((1 << (B_ - 1)) - 1);
-  float s = mul_rn(u, rdelta);
-  s = fminf(fmaxf(s, lo), hi);  // projection onto the hull (rule 2)
-  const float fl = floorf(s);
-  const float f = __fsub_rn(s, fl);  // exact
-  const int up = (add_rn((float)r16, 0.5f) < mul_rn(f, 65536.f)) ? 1 : 0;  // rule 1
-  return (uint32_t)((int)fl + up + (1 << (B_ - 1)));
 }
 
-// Runtime-b version (b in 1..16) for the generic paths.
+// Any b in 1..16 (64-bit fixed point).
 __device__ __forceinline__ uint32_t quantize_code_rt(float u, float rdelta, uint32_t r16, int b) {
   if (b == 1) return quantize_code<1>(u, rdelta, r16);
   const float lo = -(float)(1 << (b - 1));
   const float hi = (float)((1 << (b - 1)) - 1);
   float s = mul_rn(u, rdelta);
   s = fminf(fmaxf(s, lo), hi);
-  const float fl = floorf(s);
-  const float f = __fsub_rn(s, fl);
-  const int up = (add_rn((float)r16, 0.5f) < mul_rn(f, 65536.f)) ? 1 : 0;
-  return (uint32_t)((int)fl + up + (1 << (b - 1)));
+  const long long A = __float2ll_ru(mul_rn(s, 131072.f)) >> 1;
+  return (uint32_t)((A + (65535ll + (65536ll << (b - 1))) - (long long)r16) >> 16);
 }
 
 // Exact float value of the signed codebook index of a stored code (code < 2^16).
 __device__ __forceinline__ float index_as_float(uint32_t code, int b) {
   // 0x4B000000 is 2^23: or-ing a small integer into its mantissa and subtracting 2^23 converts exactly.
   const float biased = __uint_as_float(0x4B000000u | code);
-  if (b == 1) return __fsub_rn(mul_rn(__fsub_rn(biased, 8388608.f), 2.f), 1.f);
+  if (b == 1) return code ? 1.0f : -1.0f;
   return __fsub_rn(biased, 8388608.f + (float)(1 << (b - 1)));
 }
 

@@ -47,7 +47,8 @@ struct QuantArgs {
   uint32_t* codes;
   int64_t stride_words;
   float* delta_out;       // N * nseg
-  uint32_t* clipped_out;  // N * nseg (nullable -> internal scratch is passed instead)
+  uint32_t* clipped_out;  // N * nseg, cleared by the finish kernel (never null: internal scratch when the caller gives none)
+  int count_clipped;      // 0: skip counting the coordinates outside the hull (the counts stay zero)
   unsigned int* dev_status;
 };
 

@@ -152,7 +152,7 @@ __global__ void __launch_bounds__(QT) finish_kernel(QuantArgs a) {
 // BITS = 1, 2, 4, 8: register/shuffle packing with direct coalesced stores.
 // BITS = 0: any b in 1..16 read from the arguments; each thread's 8*b bits are b whole bytes, staged
 //           through shared memory and written out as words.
-template <int BITS>
+template <int BITS, bool COUNT>
 __global__ void __launch_bounds__(QT) quantize_kernel(QuantArgs a) {
   const int tile = blockIdx.x, worker = blockIdx.y;
   const int seg = a.tile_seg ? a.tile_seg[tile] : 0;
@@ -176,26 +176,48 @@ __global__ void __launch_bounds__(QT) quantize_kernel(QuantArgs a) {
     const int64_t sweep0 = tstart + (int64_t)it * QGROUP;  // first coordinate of this sweep (segment-local)
     const int64_t j = sweep0 + tid * 8;
     uint64_t lo = 0, hi = 0;  // this thread's 8*b bits
-    if (j < s.len) {
+    const int nvalid = (j < s.len) ? (int)min((int64_t)8, s.len - j) : 0;
+    if (nvalid > 0) {
       float v[8];
       load8(p, q, j, s.len, vec, v);
-      U4 r = U4{0, 0, 0, 0};
-      if (!degenerate) r = stream_block(a.seed, TAG_ROUND, (uint32_t)worker, a.k, s.block_base + (uint32_t)(j >> 3));
+      if (!degenerate) {
+        const U4 r = stream_block(a.seed, TAG_ROUND, (uint32_t)worker, a.k, s.block_base + (uint32_t)(j >> 3));
+        if constexpr (BITS != 0) {
+          // all eight coordinates are computed without bounds tests; codes past the end are masked off below
+          uint32_t w0 = 0, w1 = 0;
 #pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        if (j + e < s.len) {
-          uint32_t code = zero_code;
-          if (!degenerate) {
-            code = BITS ? quantize_code<BITS ? BITS : 2>(v[e], sc.rdelta, lane16(r, e))
-                        : quantize_code_rt(v[e], sc.rdelta, lane16(r, e), b);
-            nclip += (v[e] > sc.T || v[e] < sc.lower) ? 1u : 0u;
+          for (int e = 0; e < 8; ++e) {
+            const uint32_t code = quantize_code<BITS ? BITS : 1>(v[e], sc.rdelta, lane16(r, e));
+            if (COUNT) nclip += (v[e] > sc.T || v[e] < sc.lower) ? 1u : 0u;  // zero padding is never counted
+            if (e * BITS < 32) w0 += code << ((e * BITS) & 31);
+            else w1 += code << ((e * BITS) & 31);
           }
+          lo = (uint64_t)w0 | ((uint64_t)w1 << 32);
+          if (nvalid < 8) lo &= (1ull << (nvalid * BITS)) - 1ull;
+        } else {
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            if (e < nvalid) {
+              const uint32_t code = quantize_code_rt(v[e], sc.rdelta, lane16(r, e), b);
+              if (COUNT) nclip += (v[e] > sc.T || v[e] < sc.lower) ? 1u : 0u;
+              const int pos = e * b;
+              if (pos < 64) {
+                lo |= (uint64_t)code << pos;
+                if (pos + b > 64) hi |= (uint64_t)code >> (64 - pos);
+              } else {
+                hi |= (uint64_t)code << (pos - 64);
+              }
+            }
+          }
+        }
+      } else {
+        for (int e = 0; e < nvalid; ++e) {
           const int pos = e * b;
           if (pos < 64) {
-            lo |= (uint64_t)code << pos;
-            if (pos + b > 64) hi |= (uint64_t)code >> (64 - pos);
+            lo |= (uint64_t)zero_code << pos;
+            if (pos + b > 64) hi |= (uint64_t)zero_code >> (64 - pos);
           } else {
-            hi |= (uint64_t)code << (pos - 64);
+            hi |= (uint64_t)zero_code << (pos - 64);
           }
         }
       }
@@ -232,7 +254,7 @@ __global__ void __launch_bounds__(QT) quantize_kernel(QuantArgs a) {
     }
   }
   nclip = __reduce_add_sync(0xFFFFFFFFu, nclip);
-  if (lane == 0 && nclip) atomicAdd(&a.clipped_out[(int64_t)worker * a.nseg + seg], nclip);
+  if (COUNT && lane == 0 && nclip) atomicAdd(&a.clipped_out[(int64_t)worker * a.nseg + seg], nclip);
 }
 
 // b = 32: the message is the vector itself (clamped to [-T, T] when a clip rule is set).
@@ -298,13 +320,24 @@ cudaError_t launch_quantize_pack(const QuantArgs& a, cudaStream_t st, LaunchHook
     ~Close() { if (h) h(u, 4, 0); }
   } close_{hook, user};
   if (hook) hook(user, 4 /* LPC_KERNEL_QUANT_PACK */, 1);
-  switch (a.b) {
-    case 1: quantize_kernel<1><<<grid, block, 0, st>>>(a); break;
-    case 2: quantize_kernel<2><<<grid, block, 0, st>>>(a); break;
-    case 4: quantize_kernel<4><<<grid, block, 0, st>>>(a); break;
-    case 8: quantize_kernel<8><<<grid, block, 0, st>>>(a); break;
-    case 32: bypass_kernel<<<grid, block, 0, st>>>(a); break;
-    default: quantize_kernel<0><<<grid, block, 0, st>>>(a); break;
+  if (a.count_clipped) {
+    switch (a.b) {
+      case 1: quantize_kernel<1, true><<<grid, block, 0, st>>>(a); break;
+      case 2: quantize_kernel<2, true><<<grid, block, 0, st>>>(a); break;
+      case 4: quantize_kernel<4, true><<<grid, block, 0, st>>>(a); break;
+      case 8: quantize_kernel<8, true><<<grid, block, 0, st>>>(a); break;
+      case 32: bypass_kernel<<<grid, block, 0, st>>>(a); break;
+      default: quantize_kernel<0, true><<<grid, block, 0, st>>>(a); break;
+    }
+  } else {
+    switch (a.b) {
+      case 1: quantize_kernel<1, false><<<grid, block, 0, st>>>(a); break;
+      case 2: quantize_kernel<2, false><<<grid, block, 0, st>>>(a); break;
+      case 4: quantize_kernel<4, false><<<grid, block, 0, st>>>(a); break;
+      case 8: quantize_kernel<8, false><<<grid, block, 0, st>>>(a); break;
+      case 32: bypass_kernel<<<grid, block, 0, st>>>(a); break;
+      default: quantize_kernel<0, false><<<grid, block, 0, st>>>(a); break;
+    }
   }
   return cudaGetLastError();
 }
