@@ -115,7 +115,7 @@ __global__ void __launch_bounds__(AT) unpack_average_prox_kernel(AggArgs a) {
         for (int e = 0; e < 8; ++e) acc[e] = add_rn(acc[e], mul_rn(di, val[e]));
       }
     } else {
-#pragma unroll 4
+#pragma unroll 8
       for (int i = 0; i < a.N; ++i) {
         uint64_t lo, hi;
         load_chunk<BITS>(w + (int64_t)i * a.stride_words, j >> 3, b, s.pad_words, lo, hi);
