@@ -146,6 +146,8 @@ def run_ours(args):
     X, y, m, eta = make_problem(w, seed=rank, device=dev)
     n, d, N, B, b = w["n"], w["d"], w["N"], w["B"], w["b"]
     ctx = lpc.Context(X, y, loss_code(w), w["lam"], N, B, b, lpc.CLIP_STD, w["c"], seed=rank)
+    if args.per_step_kernels:
+        ctx.set_option(lpc.OPT_PERSISTENT, 0)
 
     def epoch(s):
         ctx.snapshot_full_grad()
@@ -274,13 +276,13 @@ def _time_calls(fn, dev, reps):
     return a.elapsed_time(b) / reps
 
 
-def quantize_aggregate_bench(dev, peak):
+def quantize_aggregate_bench(dev, peak, log2_len=26, dnn=True):
     """Stand-alone quantize+pack and unpack+average+prox at sizes where one call is bandwidth-bound."""
     import torch
     from paper_1901_08924_b200 import lpc, synth
     res = {}
     # sweep point: 8 workers x 2^26 coordinates (2.1 GB of gradients), Gaussian, b = 4, clip 2 std
-    N, length, b = 8, 1 << 26, 4
+    N, length, b = 8, 1 << log2_len, 4
     U = synth.gradient_vectors(N, length, "gauss", seed=1, device=dev)
     q = lpc.Context(None, None, lpc.LOGISTIC, 0.0, N, 1, b, lpc.CLIP_STD, 2.0, 0)
     _, stride = lpc.packed_layout(length, b)
@@ -300,13 +302,15 @@ def quantize_aggregate_bench(dev, peak):
     tq, ta = _time_calls(quant, dev, 5), _time_calls(agg, dev, 10)
     q.sync_status()
     bq, ba = N * length * (8 + b / 8), length * (N * b / 8 + 12)
-    res["sweep_N8_len2^26_b4"] = {
+    res["sweep_N8_len2^%d_b4" % log2_len] = {
         "quantize_pack": {"ms": round(tq, 4), "bytes": bq, "gbs": round(bq / tq * 1e-6, 1), "frac": round(bq / tq * 1e-6 / peak, 4),
                           "note": "two passes: 4 B stats read + 4 B quantize read + b/8 B written per element"},
         "unpack_average_prox": {"ms": round(ta, 4), "bytes": ba, "gbs": round(ba / ta * 1e-6, 1), "frac": round(ba / ta * 1e-6 / peak, 4)},
         "combined_gbs": round((bq + ba) / (tq + ta) * 1e-6, 1)}
     q.close()
     del U, codes, x
+    if not dnn:
+        return res
     # layer-wise DNN-shaped aggregation: 62 tensors, 11.7M parameters, 16 workers, b = 4, clip 2.5 std per tensor
     N, b = 16, 4
     cur, snap, mu, offs = synth.dnn_gradients(N, seed=2, device=dev)
@@ -426,8 +430,18 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
     ap.add_argument("--quick", action="store_true", help="skip the e2e, CPU-baseline and stand-alone kernel legs")
+    ap.add_argument("--quantize-aggregate-only", type=int, default=0, metavar="LOG2LEN",
+                    help="run only the stand-alone quantize+aggregate sweep point with 8 x 2^LOG2LEN values "
+                         "(a small case for profiler captures)")
+    ap.add_argument("--per-step-kernels", action="store_true",
+                    help="run the inner loop as per-step kernels (graph replay) instead of the one-launch loop; "
+                         "for profiler captures, which cannot replay the cooperative launch")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.quantize_aggregate_only:
+        import torch
+        peak, _ = read_peak()
+        print(json.dumps(quantize_aggregate_bench(torch.device("cuda", 0), peak, args.quantize_aggregate_only, dnn=False)))
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)
