@@ -67,6 +67,41 @@ __device__ __forceinline__ float warp_tree_sum(float v) {
 }
 __device__ __forceinline__ uint32_t warp_max_u32(uint32_t v) { return __reduce_max_sync(0xFFFFFFFFu, v); }
 
+// Warp reduction of V values per lane by recursive halving.  At the stage with lane mask 1<<S a lane
+// keeps one half of its values and receives the partner's partial sums for that half; lanes with the bit
+// clear keep the lower half.  After log2(V) stages one value is left, and the remaining stages are plain
+// butterflies.  Partner sums are added in lane order, which is the balanced tree over the 32 lanes.
+template <int V, int S>
+struct WarpHalving {
+  static __device__ __forceinline__ void run(float* v, int lane) {
+    if constexpr (S < 5) {
+      if constexpr (V > 1) {
+        const bool up = (lane >> S) & 1;
+#pragma unroll
+        for (int i = 0; i < V / 2; ++i) {
+          const float send = up ? v[i] : v[i + V / 2];
+          const float keep = up ? v[i + V / 2] : v[i];
+          v[i] = add_rn(keep, __shfl_xor_sync(0xFFFFFFFFu, send, 1 << S));
+        }
+        WarpHalving<V / 2, S + 1>::run(v, lane);
+      } else {
+        v[0] = add_rn(v[0], __shfl_xor_sync(0xFFFFFFFFu, v[0], 1 << S));
+        WarpHalving<1, S + 1>::run(v, lane);
+      }
+    }
+  }
+};
+
+// Index q (0 <= q < 2^LOGV) of the value that WarpHalving leaves in a lane: its bits, most significant first,
+// are the lane's low bits.  Lanes with (lane >> LOGV) != 0 hold copies.
+template <int LOGV>
+__device__ __forceinline__ int halving_index(int lane) {
+  int q = 0;
+#pragma unroll
+  for (int s = 0; s < LOGV; ++s) q |= ((lane >> s) & 1) << (LOGV - 1 - s);
+  return q;
+}
+
 // Tree sum of `count` floats (count a power of two, <= 1024) stored in order in shared memory,
 // evaluated by one thread.  Small counts only (cross-warp / cross-CTA partials).
 __device__ __forceinline__ float smem_tree_sum(const float* v, int count) {

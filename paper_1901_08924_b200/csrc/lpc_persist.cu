@@ -77,26 +77,31 @@ __device__ __forceinline__ void st_release_u32(unsigned int* p, unsigned int v) 
   asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 
-// The 8*b bits of coordinate group g of a stream, loaded around L1 (other SMs wrote them this launch).
-template <int BITS>
-__device__ __forceinline__ void load_chunk_cg(const uint32_t* w, int64_t g, int b, int64_t pad_words, uint64_t& lo,
-                                              uint64_t& hi) {
+// The 8*b bits of coordinate group g of a stream.  CG = true: from global memory around L1 (other SMs wrote
+// them during this launch); CG = false: from a copy staged in shared memory.
+template <int BITS, bool CG>
+__device__ __forceinline__ void load_chunk(const uint32_t* w, int64_t g, int b, int64_t limit_words, uint64_t& lo,
+                                           uint64_t& hi) {
   hi = 0;
   if (BITS == 8) {
-    const uint2 t = __ldcg(reinterpret_cast<const uint2*>(w + g * 2));
+    const uint2* q = reinterpret_cast<const uint2*>(w + g * 2);
+    const uint2 t = CG ? __ldcg(q) : *q;
     lo = (uint64_t)t.x | ((uint64_t)t.y << 32);
   } else if (BITS == 4) {
-    lo = __ldcg(w + g);
+    lo = CG ? __ldcg(w + g) : w[g];
   } else if (BITS == 2) {
-    lo = __ldcg(reinterpret_cast<const unsigned short*>(w) + g);
+    const unsigned short* q = reinterpret_cast<const unsigned short*>(w) + g;
+    lo = CG ? __ldcg(q) : *q;
   } else if (BITS == 1) {
-    lo = __ldcg(reinterpret_cast<const unsigned char*>(w) + g);
+    const unsigned char* q = reinterpret_cast<const unsigned char*>(w) + g;
+    lo = CG ? __ldcg(q) : *q;
   } else {
     const unsigned char* bytes = reinterpret_cast<const unsigned char*>(w);
-    const int64_t b0 = g * b, limit = pad_words * 4;
+    const int64_t b0 = g * b, limit = limit_words * 4;
     lo = 0;
     for (int i = 0; i < b; ++i) {
-      const uint64_t v = (b0 + i < limit) ? __ldcg(bytes + b0 + i) : 0;
+      uint64_t v = 0;
+      if (b0 + i < limit) v = CG ? __ldcg(bytes + b0 + i) : bytes[b0 + i];
       if (i < 8) lo |= v << (8 * i); else hi |= v << (8 * (i - 8));
     }
   }
@@ -232,11 +237,11 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
       }
       sm.sdelta[tid] = __uint_as_float((unsigned int)(w >> 32));
     }
+    const uint32_t* codes_in = a.codes + rpar * codes_buf;
     __syncthreads();
 #ifdef LPC_TRACE
     { const int t = (int)target; LPC_TRACE_MARK(3); }
 #endif
-    const uint32_t* codes_in = a.codes + rpar * codes_buf;
 #pragma unroll
     for (int p = 0; p < NP; ++p) {
       const int off = p * PGROUP + tid * 8;
@@ -251,16 +256,18 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
           const uint32_t* wi = codes_in + (int64_t)i * a.stride_words;
 #pragma unroll
           for (int e = 0; e < 8; ++e) {
-            const float val = (c + e < d) ? __uint_as_float(__ldcg(wi + c + e)) : 0.f;
+            float val = 0.f;
+            if (c + e < d) val = __uint_as_float(__ldcg(wi + c + e));
             acc[e] = add_rn(acc[e], mul_rn(di, val));
           }
         }
       } else {
-#pragma unroll 4
+        // all workers' loads are issued before the first is used: one L2 round trip instead of several
+#pragma unroll 16
         for (int i = 0; i < N; ++i) {
           const float di = sm.sdelta[i];
           uint64_t lo, hi;
-          load_chunk_cg<BITS>(codes_in + (int64_t)i * a.stride_words, c >> 3, b, a.pad_words, lo, hi);
+          load_chunk<BITS, true>(codes_in + (int64_t)i * a.stride_words, c >> 3, b, a.pad_words, lo, hi);
 #pragma unroll
           for (int e = 0; e < 8; ++e) {
             uint32_t code;
@@ -311,36 +318,28 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
     }
     LPC_TRACE_MARK(5);
 
-    // margins <X_a, x_t>: four rows at a time so that their shuffle chains overlap
+    // margins <X_a, x_t>: eight rows at a time; their 8*NP per-thread partial sums are reduced across the
+    // warp together by recursive halving (9 or 12 shuffles instead of 5 per value)
+    constexpr int RG = 8, NVAL = RG * NP, LOGV = (NP == 2) ? 4 : 3;
 #pragma unroll 1
-    for (int r0 = 0; r0 < B; r0 += 4) {
-      float sv[4][NP];
+    for (int r0 = 0; r0 < B; r0 += RG) {
+      float sv[NVAL];
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
+      for (int j = 0; j < RG; ++j) {
 #pragma unroll
         for (int p = 0; p < NP; ++p) {
           float v[8], pr[8];
           row8(buf, min(r0 + j, B - 1), p * PGROUP + tid * 8, v);
 #pragma unroll
           for (int e = 0; e < 8; ++e) pr[e] = mul_rn(v[e], xr[p][e]);
-          sv[j][p] = tree8(pr);
+          sv[j * NP + p] = tree8(pr);
         }
       }
-#pragma unroll
-      for (int m = 1; m < 32; m <<= 1) {
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-#pragma unroll
-          for (int p = 0; p < NP; ++p) sv[j][p] = add_rn(sv[j][p], __shfl_xor_sync(0xFFFFFFFFu, sv[j][p], m));
-        }
-      }
-      if (lane == 0) {
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-#pragma unroll
-          for (int p = 0; p < NP; ++p)
-            if (r0 + j < B) sm.wpart[((r0 + j) * NP + p) * 8 + warp] = sv[j][p];
-        }
+      WarpHalving<NVAL, 0>::run(sv, lane);
+      if ((lane >> LOGV) == 0) {
+        const int q = halving_index<LOGV>(lane);
+        const int j = q / NP, p = q % NP;
+        if (r0 + j < B) sm.wpart[((r0 + j) * NP + p) * 8 + warp] = sv[0];
       }
     }
     __syncthreads();

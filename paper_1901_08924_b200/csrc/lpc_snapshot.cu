@@ -26,31 +26,6 @@ constexpr int MAXLEAF = 128;  // 128-column leaves of the margin tree: d <= 1638
 
 __host__ __device__ constexpr int rows_per_tile(int kmax) { return kmax >= 16 ? 1 : kmax >= 8 ? 2 : kmax >= 4 ? 4 : 8; }
 
-// Warp reduction of V values per lane by recursive halving.  At the stage with lane mask 1<<S a lane
-// keeps one half of its values and receives the partner's partial sums for that half; lanes with the bit
-// clear keep the lower half.  After log2(V) stages one value is left, and the remaining stages are plain
-// butterflies.  Partner sums are added in lane order, which is the balanced tree over the 32 lanes.
-template <int V, int S>
-struct WarpHalving {
-  static __device__ __forceinline__ void run(float* v, int lane) {
-    if constexpr (S < 5) {
-      if constexpr (V > 1) {
-        const bool up = (lane >> S) & 1;
-#pragma unroll
-        for (int i = 0; i < V / 2; ++i) {
-          const float send = up ? v[i] : v[i + V / 2];
-          const float keep = up ? v[i + V / 2] : v[i];
-          v[i] = add_rn(keep, __shfl_xor_sync(0xFFFFFFFFu, send, 1 << S));
-        }
-        WarpHalving<V / 2, S + 1>::run(v, lane);
-      } else {
-        v[0] = add_rn(v[0], __shfl_xor_sync(0xFFFFFFFFu, v[0], 1 << S));
-        WarpHalving<1, S + 1>::run(v, lane);
-      }
-    }
-  }
-};
-
 template <int KMAX, bool GRAD>
 __global__ void __launch_bounds__(ST, 1) snapshot_kernel(SnapArgs a) {
   constexpr int R = rows_per_tile(KMAX);
