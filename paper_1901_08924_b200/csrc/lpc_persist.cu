@@ -118,6 +118,22 @@ __device__ __forceinline__ uint32_t extract_bits(uint64_t lo, uint64_t hi, int p
   return (uint32_t)v & ((1u << b) - 1u);
 }
 
+// Bulky scalar routines that one thread (or B threads) run once per step: kept out of line so that the loop
+// body every warp walks through stays small.
+__device__ __noinline__ Scale scale_out_of_line(uint32_t max_bits, float S1, float S2, int64_t len, int b, int clip_mode,
+                                               float clip_value) {
+  return make_scale(max_bits, S1, S2, len, b, clip_mode, clip_value);
+}
+__device__ __noinline__ float coef_out_of_line(int loss, float m, float m_snap, float y) {
+  return __fsub_rn(loss_deriv(loss, m, y), loss_deriv(loss, m_snap, y));
+}
+__device__ __forceinline__ float tree_small(const float* v, int n) {  // n in {1, 2, 4, 8}
+  if (n == 1) return v[0];
+  if (n == 2) return add_rn(v[0], v[1]);
+  if (n == 4) return tree4(v[0], v[1], v[2], v[3]);
+  return tree8(v);
+}
+
 // Phase timestamps of one CTA for latency studies; compiled in only with -DLPC_TRACE.
 #ifdef LPC_TRACE
 __device__ unsigned long long g_trace[64 * 16];
@@ -165,17 +181,16 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
   // Thread a < B owns minibatch slot a.  prefetch(t) samples step t's row for the slot, starts the bulk copy
   // of this CTA's slice of it into buffer t&1 and loads its label and cached snapshot margin into registers
   // (a step ahead, so these loads never stall the step that issues them).
+  const int64_t samp_span = a.sample_global ? a.n : a.n / N;            // rows a worker samples from
+  const int64_t samp_lo = a.sample_global ? 0 : (int64_t)worker * samp_span;
   int64_t row_next = 0, row_cur = 0;
   float y_next = 0.f, y_cur = 0.f, ms_next = 0.f, ms_cur = 0.f;
   auto prefetch = [&](int t) {
     const int s = t & 1;
     if (tid == 0 && width > 0) mbar_expect_tx(&sm.bar[s], (uint32_t)width * 4u * (uint32_t)B);
     if (tid < B) {
-      int64_t lo, span;
-      if (a.sample_global) { lo = 0; span = a.n; }
-      else { span = a.n / N; lo = (int64_t)worker * span; }
       const U4 r = stream_block(a.seed, TAG_BATCH, (uint32_t)worker, a.k_base + (uint64_t)t, (uint32_t)tid);
-      const int64_t row = lo + (int64_t)(((uint64_t)r.x * (uint64_t)span) >> 32);
+      const int64_t row = samp_lo + (int64_t)(((uint64_t)r.x * (uint64_t)samp_span) >> 32);
       if (width > 0) bulk_load(rows + s * buf_floats + (size_t)tid * SL, a.X + row * (int64_t)d + c0, (uint32_t)width * 4u, &sm.bar[s]);
       row_next = row;
       y_next = a.y[row];
@@ -345,15 +360,15 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
     __syncthreads();
     LPC_TRACE_MARK(6);
     if (tid < B) {
-      float part = smem_tree_sum(&sm.wpart[tid * NP * 8], 8);
-      if (NP == 2) part = add_rn(part, smem_tree_sum(&sm.wpart[(tid * NP + 1) * 8], 8));
+      float part = tree8(&sm.wpart[tid * NP * 8]);
+      if (NP == 2) part = add_rn(part, tree8(&sm.wpart[(tid * NP + 1) * 8]));
       for (int q = 0; q < CS; ++q) cluster.map_shared_rank(sm.mpart, q)[tid * PMAXCS + rank] = part;
     }
     cluster.sync();
     LPC_TRACE_MARK(7);
     if (tid < B) {
-      const float m = smem_tree_sum(&sm.mpart[tid * PMAXCS], CS);
-      const float c = __fsub_rn(loss_deriv(a.loss, m, y_cur), loss_deriv(a.loss, ms_cur, y_cur));
+      const float m = tree_small(&sm.mpart[tid * PMAXCS], CS);
+      const float c = coef_out_of_line(a.loss, m, ms_cur, y_cur);
       sm.coef[tid] = c;
       if (rank == 0 && t == pa.count - 1) {
         if (a.idx_tap) a.idx_tap[(int64_t)worker * B + tid] = row_cur;
@@ -428,9 +443,9 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
       for (int w = 0; w < 8; ++w) m = max(m, sm.wmax[w]);
       float s1 = 0.f, s2 = 0.f;
       if (a.clip_mode == CLIP_STD) {
-        s1 = smem_tree_sum(sm.ws1, 8);
-        s2 = smem_tree_sum(sm.ws2, 8);
-        if (NP == 2) { s1 = add_rn(s1, smem_tree_sum(sm.ws1 + 8, 8)); s2 = add_rn(s2, smem_tree_sum(sm.ws2 + 8, 8)); }
+        s1 = tree8(sm.ws1);
+        s2 = tree8(sm.ws2);
+        if (NP == 2) { s1 = add_rn(s1, tree8(sm.ws1 + 8)); s2 = add_rn(s2, tree8(sm.ws2 + 8)); }
       }
       for (int q = 0; q < CS; ++q) {
         cluster.map_shared_rank(sm.maxpart, q)[rank] = m;
@@ -444,16 +459,16 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
       uint32_t m = 0;
       for (int q = 0; q < CS; ++q) m = max(m, sm.maxpart[q]);
       float S1 = 0.f, S2 = 0.f;
-      if (a.clip_mode == CLIP_STD) { S1 = smem_tree_sum(sm.s1part, CS); S2 = smem_tree_sum(sm.s2part, CS); }
-      sm.scale = make_scale(m, S1, S2, d, b, a.clip_mode, a.clip_value);
+      if (a.clip_mode == CLIP_STD) { S1 = tree_small(sm.s1part, CS); S2 = tree_small(sm.s2part, CS); }
+      sm.scale = scale_out_of_line(m, S1, S2, d, b, a.clip_mode, a.clip_value);
       if (rank == 0) {
         a.delta[wpar * N + worker] = sm.scale.delta;
         if (sm.scale.flags & 2u) atomicOr(a.dev_status, DEV_NONFINITE);
       }
     }
     __syncthreads();
-    LPC_TRACE_MARK(12);
     const Scale sc = sm.scale;
+    LPC_TRACE_MARK(12);
     const bool degenerate = (sc.flags & 1u) != 0;
 
     // quantize (Section 2.2) and pack
@@ -538,7 +553,7 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
       a.clipped_part[worker * PMAXCS + rank] = tc;
       // publish step t: (step count, delta) in one word; the release store orders every code stored above
       st_release_u64(pa.pub + ((size_t)wpar * PMAXFLAGS + worker * CS + rank) * PUB_STRIDE,
-                     (unsigned long long)(unsigned int)(t + 1) | ((unsigned long long)__float_as_uint(sm.scale.delta) << 32));
+                     (unsigned long long)(unsigned int)(t + 1) | ((unsigned long long)__float_as_uint(sc.delta) << 32));
     }
     LPC_TRACE_MARK(14);
   }
