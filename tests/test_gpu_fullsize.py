@@ -1,0 +1,148 @@
+"""Parity at the full sizes of the workloads, in the launch configuration the benchmark times.
+
+Where the oracle can do the whole job in seconds it does (least-squares epoch, layer-wise DNN
+aggregation); elsewhere it checks what it can compute one by one: scales from full passes, codes and
+updated coordinates in sampled windows, sampled margins.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle as orc
+from paper_1901_08924_b200 import lpc, synth
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _bits(a):
+    a = a.detach().cpu().numpy() if isinstance(a, torch.Tensor) else np.asarray(a)
+    return a.view(np.uint32) if a.dtype == np.float32 else a
+
+
+def test_least_squares_workload_full_epoch_bitwise():
+    # 131,072 x 4,096, N = 16, B = 8, b = 4, clip 3 std, m = 1,024: one whole epoch through the one-launch loop
+    n, d, N, B, b, m = 131072, 4096, 16, 8, 4, 1024
+    X, y, _ = synth.linear_problem(n, d, loss="least_squares", sparsity=0.05, noise=0.01, seed=0, device=DEV)
+    eta = 1.0 / (6.0 * float((X.double() ** 2).sum(dim=1).max().item()))
+    ctx = lpc.Context(X, y, lpc.LEAST_SQUARES, 1e-4, N, B, b, lpc.CLIP_STD, 3.0, 0)
+    Xh, yh = X.cpu().numpy(), y.cpu().numpy()
+    P = orc.Problem(Xh, yh, orc.LEAST_SQUARES, 1e-4, N, B, b, orc.CLIP_STD, 3.0, 0)
+    x0 = (np.random.default_rng(0).standard_normal(d) * 0.01).astype(np.float32)
+    ctx.set_iterate(torch.from_numpy(x0).to(DEV))
+    f = ctx.snapshot_full_grad(want_f=True)
+    mu_g = ctx.get_buffer(lpc.BUF_MU).cpu().numpy()
+    mu, margins, fr = orc.full_grad(Xh, yh, P.loss, x0)
+    assert (_bits(ctx.get_buffer(lpc.BUF_MARGINS)) == _bits(margins)).all()
+    assert np.linalg.norm(mu_g - mu) <= 2e-6 * np.linalg.norm(mu)
+    assert abs(f - fr) <= 1e-10 * abs(fr)
+    ctx.inner_steps(eta, 0, m)
+    ctx.sync_status()
+    assert ctx.query(lpc.INFO_LOOP_LAUNCHES) == 1
+    x = x0.copy()
+    for k in range(m):
+        x = orc.lpc_inner_step(P, k, eta, x, x0, mu_g)
+    xg = ctx.get_iterate().cpu().numpy()
+    assert (_bits(xg) == _bits(x)).all()
+    pg = ctx.objective()
+    assert abs(pg - orc.objective(Xh, yh, P.loss, x, P.lambda_l1)) <= 1e-10 * abs(pg)
+    assert ctx.comm_bits() == (32 * d * N * (N - 1), m * orc.broadcast_bits(d, b, N))
+    ctx.close()
+
+
+@pytest.mark.parametrize("b", [2, 8])
+def test_alpc_workload_full_size_steps(b):
+    # 262,144 x 8,192 logistic with ill-conditioned columns, N = 32, B = 16, clip 2 std (ALPC, double sampling)
+    n, d, N, B = 262144, 8192, 32, 16
+    X, y, _ = synth.linear_problem(n, d, loss="logistic", sparsity=0.02, noise=0.1, seed=1, col_scale_range=(0.1, 10.0),
+                                   device=DEV)
+    ctx = lpc.Context(X, y, lpc.LOGISTIC, 1e-5, N, B, b, lpc.CLIP_STD, 2.0, 5)
+    Xh, yh = X.cpu().numpy(), y.cpu().numpy()
+    P = orc.Problem(Xh, yh, orc.LOGISTIC, 1e-5, N, B, b, orc.CLIP_STD, 2.0, 5)
+    L = 0.25 * float((X * X).sum(dim=1).max().item())
+    x0 = np.zeros(d, np.float32)
+    ctx.set_iterate(torch.from_numpy(x0).to(DEV))
+    ctx.alpc_begin()
+    ctx.snapshot_full_grad()
+    ctx.sync_status()
+    rows = np.random.default_rng(2).integers(0, n, 64)
+    mg = ctx.get_buffer(lpc.BUF_MARGINS).cpu().numpy()
+    for a in rows:  # sampled margins, bit for bit
+        assert _bits(mg[a:a + 1])[0] == _bits(np.array([orc.margin(Xh[a], x0)], np.float32))[0]
+    mu = ctx.get_buffer(lpc.BUF_MU).cpu().numpy()
+    tau1, alpha, inv4L = np.float32(0.5), np.float32(1.0 / (6.0 * L * 0.5)), np.float32(1.0 / (4.0 * L))
+    yv, zv, ys = x0.copy(), x0.copy(), x0.copy()
+    steps = 6
+    for k in range(steps):
+        ctx.alpc_double_sample_step(float(tau1), 0.5, float(alpha), float(inv4L), k)
+        yv, zv, ys, t = orc.alpc_step(P, k, tau1, 0.5, alpha, inv4L, x0, mu, yv, zv, ys, taps=True)
+        ctx.sync_status()
+        idx = ctx.get_buffer(lpc.BUF_BATCH_IDX).cpu().numpy()
+        assert (idx[N] == orc.sample_batch(P.seed, orc.TAG_BATCH_J, 0, k, B, 0, n)).all()
+        for w, ref in ((lpc.BUF_Y, yv), (lpc.BUF_Z, zv), (lpc.BUF_YSUM, ys), (lpc.BUF_VHAT, t["vhat"])):
+            got = ctx.get_buffer(w).cpu().numpy()
+            assert np.linalg.norm(got - ref) <= 1e-5 * np.linalg.norm(ref) + 1e-9, (k, w)
+        # continue from the GPU's state so that one-ulp differences in exp() do not accumulate in the comparison
+        yv, zv, ys = (ctx.get_buffer(w).cpu().numpy() for w in (lpc.BUF_Y, lpc.BUF_Z, lpc.BUF_YSUM))
+    ctx.close()
+
+
+def test_sweep_full_length_sampled_windows():
+    # 8 worker vectors of 2^26 heavy-tailed values, b = 4, clip 2 std: scales from full passes, codes and updated
+    # coordinates in sampled windows
+    N, length, b, seed, k = 8, 1 << 26, 4, 11, 3
+    U = synth.gradient_vectors(N, length, "student_t3", seed=4, device=DEV)
+    q = lpc.Context(None, None, lpc.LOGISTIC, 0.0, N, 1, b, lpc.CLIP_STD, 2.0, seed)
+    codes, delta, clipped = q.quantize_pack(U, k)
+    x = torch.zeros(length, device=DEV)
+    q.unpack_average_prox(codes, delta, length, x, 1.0, 1e-3)
+    q.sync_status()
+    Uh = U.cpu().numpy()
+    sc = [orc.scale(Uh[i], b, orc.CLIP_STD, 2.0) for i in range(N)]
+    dl = delta.cpu().numpy()[:, 0]
+    assert (_bits(dl) == _bits(np.array([s["delta"] for s in sc], np.float32))).all()
+    lower = [-(np.float32(s["T"]) + np.float32(s["delta"])) for s in sc]
+    want_clip = [int(((Uh[i] > sc[i]["T"]) | (Uh[i] < lower[i])).sum()) for i in range(N)]
+    assert clipped.cpu().numpy()[:, 0].tolist() == want_clip
+    W = 2048
+    starts = [0, 8192 * 1000 + 8, (1 << 25) - 1024, length - W]
+    ch = codes.cpu().numpy().view(np.uint32)
+    xh = x.cpu().numpy()
+    for s0 in starts:
+        words = np.zeros((N, W * b // 32), np.uint32)
+        for i in range(N):
+            c = np.array([orc.quantize_coord(Uh[i, j], sc[i]["rdelta"], b, orc.rounding_bits(seed, i, k, 0, j)) + 8
+                          for j in range(s0, s0 + W)], np.uint32)
+            words[i] = orc.pack(c, b)
+        assert (ch[:, s0 * b // 32:(s0 + W) * b // 32] == words).all(), s0
+        ref = orc.unpack_average_prox(words, dl, W, b, None, np.zeros(W, np.float32), 1.0, 1e-3)
+        assert (_bits(xh[s0:s0 + W]) == _bits(ref)).all(), s0
+    q.close()
+
+
+def test_dnn_shaped_aggregation_full_bitwise():
+    # 62 tensors, 11,689,512 parameters, N = 16, b = 4, per-tensor clip 2.5 std; u = current - snapshot gradient
+    N, b, seed, k = 16, 4, 2, 9
+    cur, snap, mu, offs = synth.dnn_gradients(N, seed=3, device=DEV)
+    total, nseg = offs[-1], len(offs) - 1
+    q = lpc.Context(None, None, lpc.LOGISTIC, 0.0, N, 1, b, lpc.CLIP_STD, 2.5, seed)
+    codes, delta, clipped = q.quantize_pack(cur, k, U_sub=snap, seg_offsets=offs)
+    x = torch.zeros(total, device=DEV)
+    q.unpack_average_prox(codes, delta, total, x, -1.0, 0.0, mu=mu, seg_offsets=offs)  # x = v
+    q.sync_status()
+    u = (cur - snap).cpu().numpy()
+    woff, stride = lpc.packed_layout(total, b, offs)
+    ch, dh, clh, xh, muh = codes.cpu().numpy().view(np.uint32), delta.cpu().numpy(), clipped.cpu().numpy(), x.cpu().numpy(), mu.cpu().numpy()
+    base = 0
+    for s in range(nseg):
+        ln = offs[s + 1] - offs[s]
+        W = orc.packed_words(ln, b)
+        words = np.zeros((N, W), np.uint32)
+        for i in range(N):
+            words[i], dli, cli = orc.quantize_pack(u[i, offs[s]:offs[s + 1]], b, orc.CLIP_STD, 2.5, seed, i, k, base)
+            assert _bits(np.array([dli], np.float32))[0] == _bits(dh[i, s:s + 1])[0] and cli == clh[i, s]
+        assert (ch[:, woff[s]:woff[s] + W] == words).all(), s
+        ref = orc.unpack_average_prox(words, dh[:, s], ln, b, muh[offs[s]:offs[s + 1]], np.zeros(ln, np.float32), -1.0, 0.0)
+        assert (_bits(xh[offs[s]:offs[s + 1]]) == _bits(ref)).all(), s
+        base += (ln + 7) // 8
+    q.close()
