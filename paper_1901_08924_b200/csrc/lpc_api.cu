@@ -81,9 +81,9 @@ struct lpc_ctx {
   size_t innerSmem = 0;
   SegPlan inner_seg;  // one segment of length d for the aggregator
   // persistent inner loop
-  bool persist_ok = false;
-  int pCS = 1, pSL = 0;
-  size_t persistSmem = 0;
+  bool persist_ok = false, apersist_ok = false;  // Algorithm 1 loop / Algorithm 2 loop
+  int pCS = 1, pSL = 0, pNbuf = 2, aCS = 1, aSL = 0, aNbuf = 2;
+  size_t persistSmem = 0, apersistSmem = 0;
   unsigned long long* flags = nullptr;  // 2 x 256 publication words, 128 bytes apart, + 1 abort word
   int64_t persist_launches = 0;
   // stand-alone quantizer
@@ -308,8 +308,11 @@ int replan_inner(lpc_ctx* c) {
   int cs = 1, sl = 0;
   c->inner_ok = inner_plan(c->d, c->B, c->want_cs, c->max_smem, &cs, &sl, &smem);
   if (c->inner_ok) { c->CS = cs; c->SL = sl; c->innerSmem = smem; }
-  c->persist_ok = persist_plan(c->d, c->N, c->B, c->b, c->want_cs, c->max_smem, &cs, &sl, &smem);
-  if (c->persist_ok) { c->pCS = cs; c->pSL = sl; c->persistSmem = smem; }
+  int nbuf = 2;
+  c->persist_ok = persist_plan(c->d, c->N, c->B, c->b, 0, c->want_cs, c->max_smem, &cs, &sl, &smem, &nbuf);
+  if (c->persist_ok) { c->pCS = cs; c->pSL = sl; c->persistSmem = smem; c->pNbuf = nbuf; }
+  c->apersist_ok = persist_plan(c->d, c->N, c->B, c->b, 1, c->want_cs, c->max_smem, &cs, &sl, &smem, &nbuf);
+  if (c->apersist_ok) { c->aCS = cs; c->aSL = sl; c->apersistSmem = smem; c->aNbuf = nbuf; }
   return LPC_OK;
 }
 
@@ -345,22 +348,28 @@ int run_steps(lpc_ctx* c, int kind, const float* p, uint64_t k0, int64_t count) 
     return kind == 0 ? enqueue_lpc_step(c, p[0], kb, kd, kc) : enqueue_alpc_step(c, p[0], p[1], p[2], p[3], kb, kd, kc);
   };
   int64_t done = 0;
-  if (kind == 0 && c->use_persist && c->persist_ok && count >= 2 && count <= 0x7FFFFFFF) {
+  const bool loop_ok = (kind == 0) ? c->persist_ok : c->apersist_ok;
+  if (c->use_persist && loop_ok && count >= 2 && count <= 0x7FFFFFFF) {
     // the whole loop in one cooperative launch; on a launch refusal fall through to the per-step kernels
     PersistArgs pa;
     pa.in = inner_args(c, k0, nullptr, 0);
-    pa.in.CS = c->pCS; pa.in.SL = c->pSL;
-    pa.count = (int)count; pa.eta = p[0]; pa.lambda_l1 = c->lambda_l1;
-    pa.pub = c->flags; pa.abort_flag = reinterpret_cast<unsigned int*>(c->flags + 512 * 16); pa.x_out = c->x; pa.v_tap = c->tap_u ? c->v_tap : nullptr;
+    pa.in.CS = kind == 0 ? c->pCS : c->aCS;
+    pa.in.SL = kind == 0 ? c->pSL : c->aSL;
+    pa.nbuf = kind == 0 ? c->pNbuf : c->aNbuf;
+    pa.count = (int)count; pa.eta = kind == 0 ? p[0] : 0.f; pa.lambda_l1 = c->lambda_l1;
+    pa.pub = c->flags; pa.abort_flag = reinterpret_cast<unsigned int*>(c->flags + 512 * 16); pa.x_out = c->x;
+    pa.v_tap = c->tap_u ? c->v_tap : nullptr;
+    pa.alpc = kind; pa.tau1 = p[0]; pa.tau2 = p[1]; pa.alpha = p[2]; pa.inv4L = p[3];
+    pa.y = c->yv; pa.z = c->zv; pa.ysum = c->ysum; pa.xt = c->xt; pa.vhat = c->vhat;
     CU(c, cudaMemsetAsync(c->flags, 0, (512 * 16 + 1) * sizeof(unsigned long long), c->stream));
     cudaError_t e;
-    { ProfScope ps_(c, LPC_KERNEL_INNER_LOOP); e = launch_persist(pa, c->persistSmem, c->stream); }
+    { ProfScope ps_(c, LPC_KERNEL_INNER_LOOP); e = launch_persist(pa, kind == 0 ? c->persistSmem : c->apersistSmem, c->stream); }
     if (e == cudaSuccess) {
       done = count;
       c->persist_launches += 1;
     } else {
       cudaGetLastError();  // clear the refusal and use the per-step path
-      c->persist_ok = false;
+      if (kind == 0) c->persist_ok = false; else c->apersist_ok = false;
     }
   }
   if (done < count && c->use_graph && !c->profile && count >= GRAPH_STEPS) {
@@ -500,7 +509,7 @@ int lpc_init(lpc_ctx** out, const float* X, const float* y, int64_t n, int32_t d
   if (model && rc == LPC_OK) {
     const size_t dd = (size_t)d;
     A(dalloc(c, &c->x, dd)); A(dalloc(c, &c->xt, dd)); A(dalloc(c, &c->mu, dd)); A(dalloc(c, &c->margins, (size_t)n));
-    A(dalloc(c, &c->yv, dd)); A(dalloc(c, &c->zv, dd)); A(dalloc(c, &c->ysum, dd)); A(dalloc(c, &c->vhat, dd));
+    A(dalloc(c, &c->yv, dd)); A(dalloc(c, &c->zv, dd)); A(dalloc(c, &c->ysum, dd)); A(dalloc(c, &c->vhat, 2 * dd));  // two halves: the persistent loop alternates between them
     A(dalloc(c, &c->v_tap, dd));
     A(dalloc(c, &c->delta, 2 * (size_t)N));  // two halves: the persistent loop alternates between them
     A(dalloc(c, &c->clipped, (size_t)N));

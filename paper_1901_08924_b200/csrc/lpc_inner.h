@@ -46,8 +46,19 @@ struct PersistArgs {
   unsigned int* abort_flag;  // zero at launch; set when a bounded wait ran out
   float* x_out;              // iterate after `count` steps (may alias in.x)
   float* v_tap;              // nullable: v of the last step
+  int nbuf;                  // shared-memory row buffers: 2 (prefetch a step ahead) or 1
+  // Algorithm 2 (alpc = 1): in.x is not read; y, z, ysum are read at entry and written at exit, xt is the
+  // snapshot, vhat has two halves of d floats (step parity), x_out receives the last coupled point
+  int alpc;
+  float tau1, tau2, alpha, inv4L;
+  float* y;
+  float* z;
+  float* ysum;
+  const float* xt;
+  float* vhat;
 };
-bool persist_plan(int d, int N, int B, int b, int want_cs, int max_smem, int* CS_out, int* SL_out, size_t* smem_out);
+bool persist_plan(int d, int N, int B, int b, int alpc, int want_cs, int max_smem, int* CS_out, int* SL_out,
+                  size_t* smem_out, int* nbuf_out);
 cudaError_t launch_persist(const PersistArgs& pa, size_t smem, cudaStream_t st);
 
 int inner_max_b();

@@ -148,7 +148,8 @@ __device__ unsigned long long g_trace[64 * 16];
 
 // BITS: 1, 2, 4, 8 fixed width; 0: b from the arguments (1..16 or 32).
 // NP: passes of 2048 coordinates that a CTA makes over its slice (1 or 2).
-template <int BITS, int NP>
+// ALPC: Algorithm 2's step (coupling, double sampling on one more cluster, y/z updates) instead of Algorithm 1's.
+template <int BITS, int NP, bool ALPC>
 __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
   const InnerArgs& a = pa.in;
   cg::cluster_group cluster = cg::this_cluster();
@@ -161,6 +162,8 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int rank = (int)cluster.block_rank();
   const int worker = blockIdx.y;
+  const bool is_J = ALPC && (worker == N);  // the extra cluster that handles the shared batch J
+  const int nbuf = pa.nbuf;                  // 2: rows of the next step are fetched while this one computes
   const int b = BITS ? BITS : a.b;
   const int c0 = rank * SL;
   const int width = max(0, min(SL, d - c0));
@@ -181,15 +184,15 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
   // Thread a < B owns minibatch slot a.  prefetch(t) samples step t's row for the slot, starts the bulk copy
   // of this CTA's slice of it into buffer t&1 and loads its label and cached snapshot margin into registers
   // (a step ahead, so these loads never stall the step that issues them).
-  const int64_t samp_span = a.sample_global ? a.n : a.n / N;            // rows a worker samples from
-  const int64_t samp_lo = a.sample_global ? 0 : (int64_t)worker * samp_span;
+  const int64_t samp_span = (a.sample_global || is_J) ? a.n : a.n / N;  // rows this cluster samples from
+  const int64_t samp_lo = (a.sample_global || is_J) ? 0 : (int64_t)worker * samp_span;
   int64_t row_next = 0, row_cur = 0;
   float y_next = 0.f, y_cur = 0.f, ms_next = 0.f, ms_cur = 0.f;
   auto prefetch = [&](int t) {
-    const int s = t & 1;
+    const int s = (nbuf == 2) ? (t & 1) : 0;
     if (tid == 0 && width > 0) mbar_expect_tx(&sm.bar[s], (uint32_t)width * 4u * (uint32_t)B);
     if (tid < B) {
-      const U4 r = stream_block(a.seed, TAG_BATCH, (uint32_t)worker, a.k_base + (uint64_t)t, (uint32_t)tid);
+      const U4 r = stream_block(a.seed, is_J ? TAG_BATCH_J : TAG_BATCH, is_J ? 0u : (uint32_t)worker, a.k_base + (uint64_t)t, (uint32_t)tid);
       const int64_t row = samp_lo + (int64_t)(((uint64_t)r.x * (uint64_t)samp_span) >> 32);
       if (width > 0) bulk_load(rows + s * buf_floats + (size_t)tid * SL, a.X + row * (int64_t)d + c0, (uint32_t)width * 4u, &sm.bar[s]);
       row_next = row;
@@ -210,6 +213,24 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
       mur[p][e] = in ? a.mu[c0 + off + e] : 0.f;
     }
   }
+  // Algorithm 2 keeps y, z, the running sum of y and the snapshot in registers too; xr is then the coupled point
+  float yr[ALPC ? NP : 1][8], zr[ALPC ? NP : 1][8], sr[ALPC ? NP : 1][8], xtr[ALPC ? NP : 1][8];
+  if constexpr (ALPC) {
+#pragma unroll
+    for (int p = 0; p < NP; ++p) {
+      const int off = p * PGROUP + tid * 8;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const bool in = off + e < width;
+        yr[p][e] = in ? pa.y[c0 + off + e] : 0.f;
+        zr[p][e] = in ? pa.z[c0 + off + e] : 0.f;
+        sr[p][e] = in ? pa.ysum[c0 + off + e] : 0.f;
+        xtr[p][e] = in ? pa.xt[c0 + off + e] : 0.f;
+      }
+    }
+  }
+  const float tau3 = __fsub_rn(__fsub_rn(1.0f, pa.tau1), pa.tau2);
+  const float kappa_y = mul_rn(pa.inv4L, pa.lambda_l1), kappa_z = mul_rn(pa.alpha, pa.lambda_l1);
   if (pa.count > 0) prefetch(0);
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 
@@ -232,7 +253,7 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
   auto apply_update = [&](unsigned int target) {
     const int rpar = (pa.count - (int)target) & 1;  // parity half that holds step target-1
     const unsigned long long* words = pa.pub + (size_t)rpar * PMAXFLAGS * PUB_STRIDE;
-    if (tid < N) {  // thread i watches worker i; N <= 256 = threads of the CTA
+    if (tid < N + (ALPC ? 1 : 0)) {  // thread i watches cluster i (in Algorithm 2 one more: the J cluster)
       const unsigned long long* f = words + (size_t)(tid * CS + rank) * PUB_STRIDE;
       unsigned long long w = 0;
       uint64_t t0 = 0;
@@ -296,7 +317,14 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
       for (int e = 0; e < 8; ++e) {
         if (c + e < d) {
           const float v = add_rn(mul_rn(acc[e], invN), mur[p][e]);
-          xr[p][e] = soft_threshold(__fsub_rn(xr[p][e], mul_rn(pa.eta, v)), kappa);
+          if constexpr (ALPC) {  // steps 12-13 of Algorithm 2
+            const float vh = __ldcg(pa.vhat + rpar * d + c + e);
+            yr[p][e] = soft_threshold(__fsub_rn(xr[p][e], mul_rn(pa.inv4L, v)), kappa_y);
+            zr[p][e] = soft_threshold(__fsub_rn(zr[p][e], mul_rn(pa.alpha, vh)), kappa_z);
+            sr[p][e] = add_rn(sr[p][e], yr[p][e]);
+          } else {
+            xr[p][e] = soft_threshold(__fsub_rn(xr[p][e], mul_rn(pa.eta, v)), kappa);
+          }
           if (pa.v_tap && worker == 0) pa.v_tap[c + e] = v;
         }
       }
@@ -305,14 +333,15 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
 
 #pragma unroll 1
   for (int t = 0; t < pa.count; ++t) {
-    const int s = t & 1;
+    const int s = (nbuf == 2) ? (t & 1) : 0;
+    const uint32_t row_parity = (nbuf == 2) ? (uint32_t)((t >> 1) & 1) : (uint32_t)(t & 1);
     const uint64_t k = a.k_base + (uint64_t)t;
     const float* buf = rows + s * buf_floats;
     const int wpar = (pa.count - 1 - t) & 1;  // the last step lands in parity half 0
     uint32_t* out = a.codes + wpar * codes_buf + (int64_t)worker * a.stride_words;
     LPC_TRACE_MARK(0);
     row_cur = row_next; y_cur = y_next; ms_cur = ms_next;
-    if (t + 1 < pa.count) prefetch(t + 1);
+    if (nbuf == 2 && t + 1 < pa.count) prefetch(t + 1);
     LPC_TRACE_MARK(1);
 
     // rounding bits of this step: they depend on the counters only, so they are drawn before the data arrives
@@ -322,14 +351,21 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
       rnd[p] = stream_block(a.seed, TAG_ROUND, (uint32_t)worker, k, (uint32_t)((c0 + p * PGROUP + tid * 8) >> 3));
 
     LPC_TRACE_MARK(2);
-    if (t > 0) apply_update((unsigned int)t);  // x_t = prox(x_{t-1} - eta v_{t-1})
+    if (t > 0) apply_update((unsigned int)t);  // x_t = prox(x_{t-1} - eta v_{t-1})  (Algorithm 2: y_t, z_t)
+    if constexpr (ALPC) {  // step 6: x = tau1 z + tau2 x~ + (1 - tau1 - tau2) y
+#pragma unroll
+      for (int p = 0; p < NP; ++p)
+#pragma unroll
+        for (int e = 0; e < 8; ++e)
+          xr[p][e] = add_rn(add_rn(mul_rn(pa.tau1, zr[p][e]), mul_rn(pa.tau2, xtr[p][e])), mul_rn(tau3, yr[p][e]));
+    }
     LPC_TRACE_MARK(4);
 
     bool ok = true;
-    if (width > 0) ok = mbar_wait(&sm.bar[s], (uint32_t)((t >> 1) & 1));
+    if (width > 0) ok = mbar_wait(&sm.bar[s], row_parity);
     if (!ok) {
       atomicOr(a.dev_status, DEV_TIMEOUT);
-      mbar_wait(&sm.bar[s], (uint32_t)((t >> 1) & 1));
+      mbar_wait(&sm.bar[s], row_parity);
     }
     LPC_TRACE_MARK(5);
 
@@ -415,6 +451,21 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
     }
 
     LPC_TRACE_MARK(9);
+    if (is_J) {
+      // double sampling (Algorithm 2 step 11): v^ = u_J + mu in full precision, nothing is quantized or counted
+#pragma unroll
+      for (int p = 0; p < NP; ++p) {
+        const int off = p * PGROUP + tid * 8;
+#pragma unroll
+        for (int e = 0; e < 8; ++e)
+          if (off + e < width) pa.vhat[wpar * d + c0 + off + e] = add_rn(u[p][e], mur[p][e]);
+      }
+      __syncthreads();  // the slice of v^ is stored and nobody reads the row buffer any more
+      if (nbuf == 1 && t + 1 < pa.count) prefetch(t + 1);
+      if (tid == 0)
+        st_release_u64(pa.pub + ((size_t)wpar * PMAXFLAGS + worker * CS + rank) * PUB_STRIDE, (unsigned long long)(unsigned int)(t + 1));
+      continue;
+    }
     // scale (Eq. 2)
     uint32_t mx = 0;
 #pragma unroll
@@ -438,6 +489,7 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
     if (lane == 0) sm.wmax[warp] = mx;
     __syncthreads();
     LPC_TRACE_MARK(10);
+    if (nbuf == 1 && t + 1 < pa.count) prefetch(t + 1);  // single row buffer: it is free once u is formed
     if (tid == 0) {
       uint32_t m = 0;
       for (int w = 0; w < 8; ++w) m = max(m, sm.wmax[w]);
@@ -558,21 +610,29 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
     LPC_TRACE_MARK(14);
   }
 
-  // the last step's update, then the slice of the final iterate goes back to memory (worker 0's cluster)
+  // the last step's update, then the slices of the final state go back to memory (worker 0's cluster)
   if (pa.count > 0) apply_update((unsigned int)pa.count);
   if (worker == 0) {
 #pragma unroll
     for (int p = 0; p < NP; ++p) {
       const int off = p * PGROUP + tid * 8;
 #pragma unroll
-      for (int e = 0; e < 8; ++e)
-        if (off + e < width) pa.x_out[c0 + off + e] = xr[p][e];
+      for (int e = 0; e < 8; ++e) {
+        if (off + e < width) {
+          pa.x_out[c0 + off + e] = xr[p][e];  // Algorithm 2: the coupled point of the last step
+          if constexpr (ALPC) {
+            pa.y[c0 + off + e] = yr[p][e];
+            pa.z[c0 + off + e] = zr[p][e];
+            pa.ysum[c0 + off + e] = sr[p][e];
+          }
+        }
+      }
     }
   }
   cluster.sync();  // no CTA leaves while a peer could still address its shared memory
 }
 
-template <int BITS, int NP>
+template <int BITS, int NP, bool ALPC>
 void fill_config(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr, int cs, int clusters, size_t smem, cudaStream_t st,
                  bool cooperative) {
   *cfg = cudaLaunchConfig_t{};
@@ -590,78 +650,88 @@ void fill_config(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr, int cs, int
   cfg->numAttrs = cooperative ? 2 : 1;
 }
 
-template <int BITS, int NP>
+template <int BITS, int NP, bool ALPC>
 cudaError_t launch_p(const PersistArgs& pa, size_t smem, cudaStream_t st) {
-  cudaError_t e = cudaFuncSetAttribute(persist_kernel<BITS, NP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t e = cudaFuncSetAttribute(persist_kernel<BITS, NP, ALPC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg;
   cudaLaunchAttribute attr[2];
-  fill_config<BITS, NP>(&cfg, attr, pa.in.CS, pa.in.N, smem, st, true);
-  return cudaLaunchKernelEx(&cfg, persist_kernel<BITS, NP>, pa);
+  fill_config<BITS, NP, ALPC>(&cfg, attr, pa.in.CS, pa.in.N + (ALPC ? 1 : 0), smem, st, true);
+  return cudaLaunchKernelEx(&cfg, persist_kernel<BITS, NP, ALPC>, pa);
 }
 
-template <int BITS, int NP>
+template <int BITS, int NP, bool ALPC>
 int max_clusters_t(int cs, size_t smem) {
-  if (cudaFuncSetAttribute(persist_kernel<BITS, NP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+  if (cudaFuncSetAttribute(persist_kernel<BITS, NP, ALPC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
     cudaGetLastError();
     return 0;
   }
   cudaLaunchConfig_t cfg;
   cudaLaunchAttribute attr[2];
-  fill_config<BITS, NP>(&cfg, attr, cs, 1, smem, nullptr, false);
+  fill_config<BITS, NP, ALPC>(&cfg, attr, cs, 1, smem, nullptr, false);
   int n = 0;
-  if (cudaOccupancyMaxActiveClusters(&n, persist_kernel<BITS, NP>, &cfg) != cudaSuccess) {
+  if (cudaOccupancyMaxActiveClusters(&n, persist_kernel<BITS, NP, ALPC>, &cfg) != cudaSuccess) {
     cudaGetLastError();
     return 0;
   }
   return n;
 }
 
-template <int NP>
+template <int NP, bool ALPC>
 int max_clusters_np(int b, int cs, size_t smem) {
   switch (b) {
-    case 1: return max_clusters_t<1, NP>(cs, smem);
-    case 2: return max_clusters_t<2, NP>(cs, smem);
-    case 4: return max_clusters_t<4, NP>(cs, smem);
-    case 8: return max_clusters_t<8, NP>(cs, smem);
-    default: return max_clusters_t<0, NP>(cs, smem);
+    case 1: return max_clusters_t<1, NP, ALPC>(cs, smem);
+    case 2: return max_clusters_t<2, NP, ALPC>(cs, smem);
+    case 4: return max_clusters_t<4, NP, ALPC>(cs, smem);
+    case 8: return max_clusters_t<8, NP, ALPC>(cs, smem);
+    default: return max_clusters_t<0, NP, ALPC>(cs, smem);
   }
 }
 
-template <int NP>
+template <int NP, bool ALPC>
 cudaError_t launch_np(const PersistArgs& pa, size_t smem, cudaStream_t st) {
   switch (pa.in.b) {
-    case 1: return launch_p<1, NP>(pa, smem, st);
-    case 2: return launch_p<2, NP>(pa, smem, st);
-    case 4: return launch_p<4, NP>(pa, smem, st);
-    case 8: return launch_p<8, NP>(pa, smem, st);
-    default: return launch_p<0, NP>(pa, smem, st);
+    case 1: return launch_p<1, NP, ALPC>(pa, smem, st);
+    case 2: return launch_p<2, NP, ALPC>(pa, smem, st);
+    case 4: return launch_p<4, NP, ALPC>(pa, smem, st);
+    case 8: return launch_p<8, NP, ALPC>(pa, smem, st);
+    default: return launch_p<0, NP, ALPC>(pa, smem, st);
   }
 }
 
 }  // namespace
 
-// Cluster size / slice for the persistent loop: all N clusters must be co-resident (the occupancy query
-// says how many clusters of a given size the device can hold) and the double-buffered row slices must fit
-// in shared memory.  Among the sizes that fit, the largest cluster whose slices still keep a CTA busy wins:
-// more CTAs per worker shorten every serial phase of a step.
-bool persist_plan(int d, int N, int B, int b, int want_cs, int max_smem, int* CS_out, int* SL_out, size_t* smem_out) {
+// Cluster size, slice and row buffering for the persistent loop.  All clusters (N, plus one for the shared
+// batch J in Algorithm 2) must be co-resident -- the occupancy query says how many clusters of a given size the
+// device can hold -- and the row slices must fit in shared memory, double-buffered when possible (rows of the
+// next step are fetched while this one computes), single-buffered otherwise (they are fetched as soon as u is
+// formed).  Among the sizes that fit, the largest cluster whose slices still keep a CTA busy wins: more CTAs per
+// worker shorten every serial phase of a step.
+bool persist_plan(int d, int N, int B, int b, int alpc, int want_cs, int max_smem, int* CS_out, int* SL_out,
+                  size_t* smem_out, int* nbuf_out) {
   int P = 1;
   while (P < d) P <<= 1;
   if (P < 32) P = 32;
-  if (B > PMAXB || N > PMAXFLAGS) return false;
+  const int clusters = N + (alpc ? 1 : 0);
+  if (B > PMAXB || clusters > PMAXFLAGS) return false;
   bool found = false;
   for (int cs = 1; cs <= PMAXCS; cs <<= 1) {
     if (want_cs > 0 && cs != want_cs) continue;
     const int SL = P / cs;
     if (SL < 32) break;
     if (SL > PGROUP * PMAXP) continue;
-    if (N * cs > PMAXFLAGS) break;
-    const size_t smem = ((sizeof(PSmem) + 15) & ~(size_t)15) + 2 * (size_t)B * SL * 4;
-    if (smem > (size_t)max_smem) continue;
-    const int fit = (SL > PGROUP) ? max_clusters_np<2>(b, cs, smem) : max_clusters_np<1>(b, cs, smem);
-    if (fit < N) continue;
-    *CS_out = cs; *SL_out = SL; *smem_out = smem;
+    if (clusters * cs > PMAXFLAGS) break;
+    const size_t fixed = (sizeof(PSmem) + 15) & ~(size_t)15;
+    const size_t one = (size_t)B * SL * 4;
+    int nbuf = 2;
+    if (fixed + 2 * one > (size_t)max_smem) nbuf = 1;
+    if (fixed + nbuf * one > (size_t)max_smem) continue;
+    const size_t smem = fixed + nbuf * one;
+    int fit;
+    if (alpc) fit = (SL > PGROUP) ? max_clusters_np<2, true>(b, cs, smem) : max_clusters_np<1, true>(b, cs, smem);
+    else fit = (SL > PGROUP) ? max_clusters_np<2, false>(b, cs, smem) : max_clusters_np<1, false>(b, cs, smem);
+    if (fit < clusters) continue;
+    *CS_out = cs; *SL_out = SL; *smem_out = smem; *nbuf_out = nbuf;
     found = true;
     if (want_cs > 0) break;
     if (SL <= 512) break;  // slices below 512 coordinates leave most of a CTA idle
@@ -670,7 +740,8 @@ bool persist_plan(int d, int N, int B, int b, int want_cs, int max_smem, int* CS
 }
 
 cudaError_t launch_persist(const PersistArgs& pa, size_t smem, cudaStream_t st) {
-  return (pa.in.SL > PGROUP) ? launch_np<2>(pa, smem, st) : launch_np<1>(pa, smem, st);
+  if (pa.alpc) return (pa.in.SL > PGROUP) ? launch_np<2, true>(pa, smem, st) : launch_np<1, true>(pa, smem, st);
+  return (pa.in.SL > PGROUP) ? launch_np<2, false>(pa, smem, st) : launch_np<1, false>(pa, smem, st);
 }
 
 #ifdef LPC_TRACE

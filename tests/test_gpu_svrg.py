@@ -372,3 +372,36 @@ def test_unsupported_and_invalid_calls_are_refused():
     assert lpc.lib().lpc_snapshot_full_grad(q._h, None, None) == lpc.ERR_UNSUPPORTED
     assert lpc.lib().lpc_quantize_pack(q._h, None, None, 10, 10, None, 1, 0, None, None, None) == lpc.ERR_INVALID_ARG
     q.close()
+
+
+@pytest.mark.parametrize("cfg", [
+    dict(n=256, d=1000, N=4, B=2, b=2), dict(n=128, d=4096, N=16, B=8, b=4), dict(n=64, d=8192, N=4, B=16, b=8),
+    dict(n=64, d=5000, N=2, B=4, b=1), dict(n=64, d=3000, N=2, B=4, b=32), dict(n=96, d=12288, N=3, B=2, b=5),
+    dict(n=128, d=8192, N=32, B=16, b=2),
+])
+@pytest.mark.parametrize("loss", ["least_squares", "logistic"])
+def test_alpc_one_launch_loop_equals_single_steps(cfg, loss):
+    # Algorithm 2's steps run as one persistent launch must give the bits of one-step-at-a-time launches
+    c = dict(cfg)
+    P, ctx = _setup(c.pop("n"), c.pop("d"), loss, **c)
+    ref = lpc.Context(ctx.X, ctx.y, P.loss, P.lambda_l1, P.N, P.B, P.b, P.clip_mode, P.clip_value, P.seed)
+    x0 = (np.random.default_rng(5).standard_normal(P.d) * 0.1).astype(np.float32)
+    tau1, tau2, alpha, inv4L, count = 0.4, 0.5, 0.3, 0.2, 9
+    for cx in (ctx, ref):
+        cx.set_option(lpc.OPT_TAP_U, 1)
+        cx.set_iterate(torch.from_numpy(x0).to(DEV))
+        cx.alpc_begin()
+        cx.snapshot_full_grad()
+        cx.alpc_double_sample_step(tau1, tau2, alpha, inv4L, 0)
+    ctx.alpc_double_sample_steps(tau1, tau2, alpha, inv4L, 1, count)
+    for k in range(1, 1 + count):
+        ref.alpc_double_sample_step(tau1, tau2, alpha, inv4L, k)
+    ctx.sync_status()
+    ref.sync_status()
+    assert ctx.query(lpc.INFO_LOOP_LAUNCHES) == 1 and ref.query(lpc.INFO_LOOP_LAUNCHES) == 0
+    for w in (lpc.BUF_X, lpc.BUF_Y, lpc.BUF_Z, lpc.BUF_YSUM, lpc.BUF_VHAT, lpc.BUF_V, lpc.BUF_CODES, lpc.BUF_DELTA,
+              lpc.BUF_CLIPPED, lpc.BUF_BATCH_IDX, lpc.BUF_COEF, lpc.BUF_U):
+        assert _same(ctx.get_buffer(w), ref.get_buffer(w)), w
+    assert ctx.comm_bits() == ref.comm_bits()
+    ctx.close()
+    ref.close()
