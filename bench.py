@@ -252,6 +252,10 @@ def run_ours(args):
         out["quantize_aggregate"] = quantize_aggregate_bench(dev, peak)
         out["e2e"] = e2e_bench(w, X, y, m, eta, dev)
         out["cpu_baseline"] = cpu_baseline(w, X, y, m, eta)
+        del X, y
+        ctx.close()
+        torch.cuda.empty_cache()
+        out["alpc"] = alpc_bench(dev)
     elif rank == 0:
         out["e2e"] = None
     ctx.close()
@@ -331,7 +335,7 @@ def quantize_aggregate_bench(dev, peak, log2_len=26, dnn=True):
 
     tq, ta = _time_calls(quant2, dev, 10), _time_calls(agg2, dev, 20)
     q.sync_status()
-    bq, ba = N * total * (16 + b / 8), total * (N * b / 8 + 12)
+    bq, ba = N * total * (16 + b / 8), total * (N * b / 8 + 16)  # aggregate: codes + mu + x read + x write
     res["dnn_62_tensors_N16_b4"] = {
         "quantize_pack": {"ms": round(tq, 4), "bytes": bq, "gbs": round(bq / tq * 1e-6, 1), "frac": round(bq / tq * 1e-6 / peak, 4),
                           "note": "u = cur - snap formed on the fly: 2 x 8 B read + b/8 B written per element"},
@@ -339,6 +343,45 @@ def quantize_aggregate_bench(dev, peak, log2_len=26, dnn=True):
         "combined_gbs": round((bq + ba) / (tq + ta) * 1e-6, 1)}
     q.close()
     return res
+
+
+def alpc_bench(dev):
+    """ALPC-SVRG (Algorithms 2/3) on the ill-conditioned logistic workload: 262,144 x 8,192, N = 32, B = 16,
+    clip 2 std, b in {2, 8}; one epoch = snapshot pass + m = n/(B N) = 512 double-sampling steps."""
+    import torch
+    from paper_1901_08924_b200 import lpc, synth
+    n, d, N, B = 262144, 8192, 32, 16
+    X, y, _ = synth.linear_problem(n, d, loss="logistic", sparsity=0.02, noise=0.1, seed=1, col_scale_range=(0.1, 10.0),
+                                   device=dev)
+    L = 0.25 * float((X * X).sum(dim=1).max().item())
+    m = n // (B * N)
+    out = {"workload": "alpc_svrg_logistic_262144x8192_N32_B16", "m": m}
+    for b in (2, 8):
+        ctx = lpc.Context(X, y, lpc.LOGISTIC, 1e-5, N, B, b, lpc.CLIP_STD, 2.0, 0)
+        ctx.alpc_begin()
+        st = torch.cuda.current_stream(dev)
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        times = []
+        for s in range(5):  # Algorithm 3: tau1 = 2/(s+4), alpha = 1/(6 L tau1), tau2 = 1/2
+            tau1 = 2.0 / (s + 4)
+            ev[0].record(st)
+            ctx.snapshot_full_grad()
+            ev[1].record(st)
+            ctx.alpc_double_sample_steps(tau1, 0.5, 1.0 / (6.0 * L * tau1), 1.0 / (4.0 * L), s * m, m)
+            ctx.alpc_end_epoch(m)
+            ev[2].record(st)
+            torch.cuda.synchronize(dev)
+            times.append((ev[0].elapsed_time(ev[1]), ev[1].elapsed_time(ev[2])))
+        ctx.sync_status()
+        snap = statistics.median(t[0] for t in times[2:])
+        loop = statistics.median(t[1] for t in times[2:])
+        out["b%d" % b] = {"iters_per_s": round(m / ((snap + loop) * 1e-3), 1), "step_us": round(loop * 1e3 / m, 3),
+                          "snapshot_ms": round(snap, 4), "snapshot_gbs": round(n * d * 4 / snap * 1e-6, 1),
+                          "loop_cluster_size": ctx.query(lpc.INFO_ALPC_LOOP_CLUSTER_SIZE),
+                          "loop_row_buffers": ctx.query(lpc.INFO_ALPC_LOOP_ROW_BUFFERS),
+                          "one_launch_loops": ctx.query(lpc.INFO_LOOP_LAUNCHES), "objective": ctx.objective()}
+        ctx.close()
+    return out
 
 
 def e2e_bench(w, X, y, m, eta, dev):
@@ -385,7 +428,7 @@ def oracle_epoch_sample(w, Xh, yh, m, eta, rows, steps, seed=0):
 
 def cpu_baseline(w, X, y, m, eta):
     Xh, yh = X.cpu().numpy(), y.cpu().numpy()
-    rows, steps = w["n"] // 2, min(m, 512)  # about 10-15 s of single-core work on the main workload
+    rows, steps = w["n"], m  # one whole epoch: about 10 s of single-core work on the main workload
     t_snap, t_inner = oracle_epoch_sample(w, Xh, yh, m, eta, rows, steps)
     epoch_s = t_snap * (w["n"] / rows) + t_inner * (m / steps)
     return {"value": round(m / epoch_s, 2), "unit": UNIT, "cores": 1, "kind": "oracle",

@@ -215,6 +215,9 @@ int lpc_objective(lpc_ctx* ctx, const float* x, double* P_out);
 #define LPC_INFO_LOOP_LAUNCHES 2           /* lpc_inner_steps calls served by the one-launch inner loop so far */
 #define LPC_INFO_SNAPSHOT_ROWS_PER_TILE 3  /* rows per shared-memory stage of the snapshot pass */
 #define LPC_INFO_SNAPSHOT_STAGES 4         /* shared-memory stages of the snapshot pass */
+#define LPC_INFO_ALPC_LOOP_CLUSTER_SIZE 5  /* as LOOP_CLUSTER_SIZE, for the one-launch loop of Algorithm 2 */
+#define LPC_INFO_LOOP_ROW_BUFFERS 6        /* sampled-row buffers per CTA of the one-launch loop (1 or 2; 0: not available) */
+#define LPC_INFO_ALPC_LOOP_ROW_BUFFERS 7   /* the same for the loop of Algorithm 2 */
 int lpc_query(const lpc_ctx* ctx, int what, int64_t* out);
 
 /* Per-kernel device time measured with CUDA events on the context's stream while LPC_OPT_PROFILE is

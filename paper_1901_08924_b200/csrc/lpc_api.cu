@@ -697,6 +697,9 @@ int lpc_query(const lpc_ctx* c, int what, int64_t* out) {
   switch (what) {
     case LPC_INFO_STEP_CLUSTER_SIZE: *out = c->inner_ok ? c->CS : 0; return LPC_OK;
     case LPC_INFO_LOOP_CLUSTER_SIZE: *out = c->persist_ok ? c->pCS : 0; return LPC_OK;
+    case LPC_INFO_ALPC_LOOP_CLUSTER_SIZE: *out = c->apersist_ok ? c->aCS : 0; return LPC_OK;
+    case LPC_INFO_LOOP_ROW_BUFFERS: *out = c->persist_ok ? c->pNbuf : 0; return LPC_OK;
+    case LPC_INFO_ALPC_LOOP_ROW_BUFFERS: *out = c->apersist_ok ? c->aNbuf : 0; return LPC_OK;
     case LPC_INFO_LOOP_LAUNCHES: *out = c->persist_launches; return LPC_OK;
     case LPC_INFO_SNAPSHOT_ROWS_PER_TILE: *out = c->snapR; return LPC_OK;
     case LPC_INFO_SNAPSHOT_STAGES: *out = c->snapStages; return LPC_OK;
