@@ -120,13 +120,15 @@ __global__ void __launch_bounds__(AT) unpack_average_prox_kernel(AggArgs a) {
         uint64_t lo, hi;
         load_chunk<BITS>(w + (int64_t)i * a.stride_words, j >> 3, b, s.pad_words, lo, hi);
         const float di = sdelta[i];
+        float kf[8];
+        if constexpr (BITS == 0) {
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          uint32_t code;
-          if constexpr (BITS == 0) code = extract(lo, hi, e * b, b);
-          else code = (uint32_t)(lo >> (e * BITS)) & ((1u << BITS) - 1u);
-          acc[e] = add_rn(acc[e], mul_rn(di, index_as_float(code, b)));
+          for (int e = 0; e < 8; ++e) kf[e] = index_as_float(extract(lo, hi, e * b, b), b);
+        } else {
+          decode8<(BITS == 0 || BITS == 32) ? 1 : BITS>(lo, kf);
         }
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[e] = add_rn(acc[e], mul_rn(di, kf[e]));
       }
     }
     float xv[8], mv[8], vv[8];

@@ -84,7 +84,12 @@ struct lpc_ctx {
   bool persist_ok = false, apersist_ok = false;  // Algorithm 1 loop / Algorithm 2 loop
   int pCS = 1, pSL = 0, pNbuf = 2, aCS = 1, aSL = 0, aNbuf = 2;
   size_t persistSmem = 0, apersistSmem = 0;
-  unsigned long long* flags = nullptr;  // 2 x 256 publication words, 128 bytes apart, + 1 abort word
+  // exchange buffers of the one-launch loops: tagged 64-bit words (payload | tag << 32), two step-parity halves
+  unsigned long long* flags = nullptr;    // scale words: 2 x 256, 128 bytes apart, + 1 abort word
+  unsigned long long* ll = nullptr;       // code words: 2 x N x dpow2/8 groups x ll_wpg
+  unsigned long long* ll_vhat = nullptr;  // second estimator of Algorithm 2: 2 x dpow2
+  int ll_wpg = 1;                         // words per group of 8 coordinates
+  uint32_t ll_tag = 0;                    // tags handed out so far; the buffers start zeroed and tag 0 is never used
   int64_t persist_launches = 0;
   // stand-alone quantizer
   SegPlan seg;
@@ -358,15 +363,26 @@ int run_steps(lpc_ctx* c, int kind, const float* p, uint64_t k0, int64_t count) 
     pa.nbuf = kind == 0 ? c->pNbuf : c->aNbuf;
     pa.count = (int)count; pa.eta = kind == 0 ? p[0] : 0.f; pa.lambda_l1 = c->lambda_l1;
     pa.pub = c->flags; pa.abort_flag = reinterpret_cast<unsigned int*>(c->flags + 512 * 16); pa.x_out = c->x;
+    pa.ll = c->ll; pa.ll_vhat = c->ll_vhat; pa.wpg = c->ll_wpg;
+    if ((uint64_t)c->ll_tag + (uint64_t)count >= 0xFFFFFFF0ull) {  // tags would wrap: start over from cleared buffers
+      int dp = 32;
+      while (dp < c->d) dp <<= 1;
+      CU(c, cudaMemsetAsync(c->flags, 0, (512 * 16 + 1) * sizeof(unsigned long long), c->stream));
+      CU(c, cudaMemsetAsync(c->ll, 0, sizeof(unsigned long long) * 2 * (size_t)c->N * (size_t)(dp / 8) * c->ll_wpg, c->stream));
+      CU(c, cudaMemsetAsync(c->ll_vhat, 0, sizeof(unsigned long long) * 2 * (size_t)dp, c->stream));
+      c->ll_tag = 0;
+    }
+    pa.tag_base = c->ll_tag;
     pa.v_tap = c->tap_u ? c->v_tap : nullptr;
     pa.alpc = kind; pa.tau1 = p[0]; pa.tau2 = p[1]; pa.alpha = p[2]; pa.inv4L = p[3];
     pa.y = c->yv; pa.z = c->zv; pa.ysum = c->ysum; pa.xt = c->xt; pa.vhat = c->vhat;
-    CU(c, cudaMemsetAsync(c->flags, 0, (512 * 16 + 1) * sizeof(unsigned long long), c->stream));
+    CU(c, cudaMemsetAsync(pa.abort_flag, 0, sizeof(unsigned long long), c->stream));
     cudaError_t e;
     { ProfScope ps_(c, LPC_KERNEL_INNER_LOOP); e = launch_persist(pa, kind == 0 ? c->persistSmem : c->apersistSmem, c->stream); }
     if (e == cudaSuccess) {
       done = count;
       c->persist_launches += 1;
+      c->ll_tag += (uint32_t)count;
     } else {
       cudaGetLastError();  // clear the refusal and use the per-step path
       if (kind == 0) c->persist_ok = false; else c->apersist_ok = false;
@@ -509,15 +525,22 @@ int lpc_init(lpc_ctx** out, const float* X, const float* y, int64_t n, int32_t d
   if (model && rc == LPC_OK) {
     const size_t dd = (size_t)d;
     A(dalloc(c, &c->x, dd)); A(dalloc(c, &c->xt, dd)); A(dalloc(c, &c->mu, dd)); A(dalloc(c, &c->margins, (size_t)n));
-    A(dalloc(c, &c->yv, dd)); A(dalloc(c, &c->zv, dd)); A(dalloc(c, &c->ysum, dd)); A(dalloc(c, &c->vhat, 2 * dd));  // two halves: the persistent loop alternates between them
+    A(dalloc(c, &c->yv, dd)); A(dalloc(c, &c->zv, dd)); A(dalloc(c, &c->ysum, dd)); A(dalloc(c, &c->vhat, dd));
     A(dalloc(c, &c->v_tap, dd));
-    A(dalloc(c, &c->delta, 2 * (size_t)N));  // two halves: the persistent loop alternates between them
+    A(dalloc(c, &c->delta, (size_t)N));
     A(dalloc(c, &c->clipped, (size_t)N));
     A(dalloc(c, &c->clipped_part, (size_t)N * inner_clipped_stride()));
     A(dalloc(c, &c->flags, 512 * 16 + 1));
+    {
+      int dp = 32;
+      while (dp < d) dp <<= 1;
+      c->ll_wpg = (b <= 4) ? 1 : (b <= 8) ? 2 : (b <= 16) ? 4 : 8;
+      A(dalloc(c, &c->ll, 2 * (size_t)N * (size_t)(dp / 8) * c->ll_wpg));
+      A(dalloc(c, &c->ll_vhat, 2 * (size_t)dp));
+    }
     A(dalloc(c, &c->idx_tap, (size_t)(N + 1) * B)); A(dalloc(c, &c->coef_tap, (size_t)(N + 1) * B));
     if (rc == LPC_OK) rc = make_plan(c, c->inner_seg, d, b, nullptr, 1);
-    if (rc == LPC_OK) A(dalloc(c, &c->codes, 2 * (size_t)N * (size_t)c->inner_seg.stride_words));
+    if (rc == LPC_OK) A(dalloc(c, &c->codes, (size_t)N * (size_t)c->inner_seg.stride_words));
     c->dpad = snapshot_dpad(d);
     snapshot_plan(d, c->max_smem, &c->snapR, &c->snapStages, &c->snapSmem);
     c->snapGrid = c->sm_count;
@@ -538,7 +561,7 @@ int lpc_destroy(lpc_ctx* c) {
   for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
   void* ptrs[] = {c->x, c->xt, c->mu, c->margins, c->yv, c->zv, c->ysum, c->vhat, c->v_tap, c->u_tap, c->codes,
                   c->delta, c->clipped_part, c->clipped, c->idx_tap, c->coef_tap, c->k_dev, c->dev_status, c->f_dev,
-                  c->partial_mu, c->partial_f, c->flags, c->q_pmax, c->q_ps1, c->q_ps2, c->q_scales, c->q_clip};
+                  c->partial_mu, c->partial_f, c->flags, c->ll, c->ll_vhat, c->q_pmax, c->q_ps1, c->q_ps2, c->q_scales, c->q_clip};
   for (void* p : ptrs)
     if (p) cudaFree(p);
   free_plan(c->inner_seg);

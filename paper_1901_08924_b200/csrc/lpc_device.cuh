@@ -220,6 +220,41 @@ __device__ __forceinline__ float index_as_float(uint32_t code, int b) {
   return __fsub_rn(biased, 8388608.f + (float)(1 << (b - 1)));
 }
 
+// The signed codebook indices of the 8 codes of one coordinate group (8 * BITS payload bits in `lo`), as exact
+// floats, for the fixed widths.  The codes are moved into the mantissa of 2^23 by byte permutes (one integer
+// instruction per code after a few shared masks), then one exact subtraction removes 2^23 and the offset.
+template <int BITS>
+__device__ __forceinline__ void decode8(uint64_t lo, float* k) {
+  static_assert(BITS == 1 || BITS == 2 || BITS == 4 || BITS == 8, "fixed widths only");
+  constexpr uint32_t MAGIC = 0x4B000000u;  // 2^23
+  if constexpr (BITS == 1) {
+#pragma unroll
+    for (int e = 0; e < 8; ++e) k[e] = ((uint32_t)lo >> e) & 1u ? 1.0f : -1.0f;
+  } else {
+    constexpr float C = 8388608.f + (float)(1 << (BITS - 1));
+    if constexpr (BITS == 8) {
+      const uint32_t w0 = (uint32_t)lo, w1 = (uint32_t)(lo >> 32);
+#pragma unroll
+      for (int e = 0; e < 8; ++e)
+        k[e] = __fsub_rn(__uint_as_float(__byte_perm(e < 4 ? w0 : w1, MAGIC, 0x7440u + (e & 3))), C);
+    } else if constexpr (BITS == 4) {
+      const uint32_t w = (uint32_t)lo;
+      const uint32_t ev = w & 0x0F0F0F0Fu, od = (w >> 4) & 0x0F0F0F0Fu;
+#pragma unroll
+      for (int e = 0; e < 8; ++e)
+        k[e] = __fsub_rn(__uint_as_float(__byte_perm((e & 1) ? od : ev, MAGIC, 0x7440u + (e >> 1))), C);
+    } else {  // 2 bits: code e sits in byte e/4 of (w >> 2 (e%4)) & 0x0303
+      const uint32_t w = (uint32_t)lo;
+      uint32_t x[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) x[j] = (w >> (2 * j)) & 0x0303u;
+#pragma unroll
+      for (int e = 0; e < 8; ++e)
+        k[e] = __fsub_rn(__uint_as_float(__byte_perm(x[e & 3], MAGIC, 0x7440u + (e >> 2))), C);
+    }
+  }
+}
+
 __device__ __forceinline__ float soft_threshold(float w, float kappa) {
   const float a = fmaxf(__fsub_rn(fabsf(w), kappa), 0.f);
   return copysignf(a, w);

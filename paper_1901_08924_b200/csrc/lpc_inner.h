@@ -42,13 +42,20 @@ struct PersistArgs {
   int count;
   float eta;
   float lambda_l1;
-  unsigned long long* pub;   // 2 x 256 publication words (step count | delta << 32), 128 bytes apart, zero at launch
+  // Exchange buffers of tagged 64-bit words (payload | tag << 32), two step-parity halves each; a word is valid
+  // for step t of this launch when its tag equals tag_base + t + 1.  Tags only grow from launch to launch, so
+  // stale words never match and the buffers need no clearing between launches.
+  unsigned long long* pub;   // scale delta: 2 x 256 words, 128 bytes apart, word (worker * CS + rank)
+  unsigned long long* ll;    // codes: 2 x N x (CS*SL/8) groups x wpg words
+  unsigned long long* ll_vhat;  // Algorithm 2's second estimator: 2 x CS*SL words
+  uint32_t tag_base;
+  int wpg;                   // words per group of 8 coordinates: 1 (b <= 4), 2 (b <= 8), 4 (b <= 16), 8 (b = 32)
   unsigned int* abort_flag;  // zero at launch; set when a bounded wait ran out
   float* x_out;              // iterate after `count` steps (may alias in.x)
   float* v_tap;              // nullable: v of the last step
   int nbuf;                  // shared-memory row buffers: 2 (prefetch a step ahead) or 1
   // Algorithm 2 (alpc = 1): in.x is not read; y, z, ysum are read at entry and written at exit, xt is the
-  // snapshot, vhat has two halves of d floats (step parity), x_out receives the last coupled point
+  // snapshot, vhat (d floats) receives the last step's second estimator, x_out the last coupled point
   int alpc;
   float tau1, tau2, alpha, inv4L;
   float* y;

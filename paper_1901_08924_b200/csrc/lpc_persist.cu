@@ -4,20 +4,26 @@
 // "all workers' codes of step t -> x_{t+1} -> margins -> u -> scale -> codes of step t+1" is strictly
 // serial.  Launching kernels per step pays a launch + drain for every link of that chain.  Here the
 // grid stays resident for `count` steps (one cluster per worker, one CTA per SM, launched
-// cooperatively so that co-residency is guaranteed) and the only grid-wide dependency per step is a
-// wait on publication words:
+// cooperatively so that co-residency is guaranteed) and the only grid-wide dependency per step is the
+// arrival of the other workers' messages:
 //   - every CTA keeps its slice of x and of mu in REGISTERS across steps;
 //   - the rows of step t+1 do not depend on step t (sampling is counter-based), so they are sampled
 //     and fetched by bulk copies (TMA) into the other half of a double buffer while step t computes;
 //     labels and cached snapshot margins of those rows travel in registers of the thread that owns the
 //     minibatch slot;
-//   - when a CTA has stored the codes of its slice it publishes (step, delta) in one 64-bit release
-//     store to a word with a cache line of its own; at the top of the next step thread i of every CTA
-//     waits for the word of worker i's CTA of the same rank (acquire), then the CTA decodes all workers'
-//     codes for ITS slice with L1-bypassing loads, averages, adds mu and applies the proximal step in
-//     registers.  Codes and publication words are double-buffered by step parity, because a fast CTA may
-//     store step t+1 while a slow one still decodes step t.
-// Every wait is bounded; when one runs out the CTA records a timeout in the status word, raises a global
+//   - the codes travel between CTAs as self-validating 64-bit words: 32 bits of payload (the codes of 8
+//     coordinates, or part of them) and a 32-bit tag that names the step (unique across launches).  Aligned
+//     64-bit stores are single-copy atomic, so a reader that sees the tag it expects also sees the payload:
+//     no fence, no flag and no block barrier sit between "codes stored" and "codes read".  The scale delta of
+//     a worker travels the same way (delta | tag), one word per CTA, and so does the full-precision second
+//     estimator of Algorithm 2 (value | tag per coordinate).  At the top of a step every thread loads, for
+//     ITS 8 coordinates, the words of all workers (all loads in flight together), repeats until every tag
+//     matches, then averages, adds mu and applies the proximal step in registers.  The exchange buffers are
+//     double-buffered by step parity, because a fast CTA may store step t+1 while a slow one still reads
+//     step t (it cannot get further ahead: storing step t+2 needs every reader's step t+1).
+//   - only the last step also writes the packed codes, delta and the second estimator in their documented
+//     layouts, for the caller.
+// Every wait is bounded; when one runs out the thread records a timeout in the status word, raises a global
 // abort flag that makes every other wait return at once, and the loop finishes without hanging (all CTAs
 // still execute the same cluster barriers).
 //
@@ -55,19 +61,21 @@ struct PSmem {
   float ws1[PMAXP * 8], ws2[PMAXP * 8];
   uint32_t wmax[8];
   uint32_t wclip[8];
-  float sdelta[PMAXFLAGS];
   Scale scale;
   __align__(16) uint8_t stage[PT * 16];
 };
 
-__device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p) {
+// Tagged 64-bit words (payload | tag << 32): relaxed, device scope, one indivisible access each.
+__device__ __forceinline__ unsigned long long ld_word(const unsigned long long* p) {
   unsigned long long v;
-  asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+  asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
   return v;
 }
-__device__ __forceinline__ void st_release_u64(unsigned long long* p, unsigned long long v) {
-  asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+__device__ __forceinline__ void st_word(unsigned long long* p, uint32_t payload, uint32_t tag) {
+  const unsigned long long v = (unsigned long long)payload | ((unsigned long long)tag << 32);
+  asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
+__device__ __forceinline__ uint32_t word_tag(unsigned long long w) { return (uint32_t)(w >> 32); }
 __device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int* p) {
   unsigned int v;
   asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
@@ -75,36 +83,6 @@ __device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int* p) {
 }
 __device__ __forceinline__ void st_release_u32(unsigned int* p, unsigned int v) {
   asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
-}
-
-// The 8*b bits of coordinate group g of a stream.  CG = true: from global memory around L1 (other SMs wrote
-// them during this launch); CG = false: from a copy staged in shared memory.
-template <int BITS, bool CG>
-__device__ __forceinline__ void load_chunk(const uint32_t* w, int64_t g, int b, int64_t limit_words, uint64_t& lo,
-                                           uint64_t& hi) {
-  hi = 0;
-  if (BITS == 8) {
-    const uint2* q = reinterpret_cast<const uint2*>(w + g * 2);
-    const uint2 t = CG ? __ldcg(q) : *q;
-    lo = (uint64_t)t.x | ((uint64_t)t.y << 32);
-  } else if (BITS == 4) {
-    lo = CG ? __ldcg(w + g) : w[g];
-  } else if (BITS == 2) {
-    const unsigned short* q = reinterpret_cast<const unsigned short*>(w) + g;
-    lo = CG ? __ldcg(q) : *q;
-  } else if (BITS == 1) {
-    const unsigned char* q = reinterpret_cast<const unsigned char*>(w) + g;
-    lo = CG ? __ldcg(q) : *q;
-  } else {
-    const unsigned char* bytes = reinterpret_cast<const unsigned char*>(w);
-    const int64_t b0 = g * b, limit = limit_words * 4;
-    lo = 0;
-    for (int i = 0; i < b; ++i) {
-      uint64_t v = 0;
-      if (b0 + i < limit) v = CG ? __ldcg(bytes + b0 + i) : bytes[b0 + i];
-      if (i < 8) lo |= v << (8 * i); else hi |= v << (8 * (i - 8));
-    }
-  }
 }
 
 __device__ __forceinline__ uint32_t extract_bits(uint64_t lo, uint64_t hi, int pos, int b) {
@@ -171,7 +149,6 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
   const float invB = __fdiv_rn(1.0f, (float)B);
   const float kappa = mul_rn(pa.eta, pa.lambda_l1);
   const uint32_t zero_code = (b == 1) ? 0u : (1u << (b - 1));
-  const int64_t codes_buf = (int64_t)N * a.stride_words;  // one parity half of the code buffer
 
   if (tid == 0) {
     mbar_init(&sm.bar[0], 1);
@@ -247,37 +224,19 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
     }
   };
 
-  // Waits until step target-1 has been published by the CTAs that wrote this slice's codes (those of the same
-  // rank in every worker's cluster), then applies that step's update to xr:
-  //   x <- prox_{eta h}(x - eta (mean_i delta_i k_i + mu)).
+  // Applies step target-1's update to this thread's coordinates:
+  //   x <- prox_{eta h}(x - eta (mean_i delta_i k_i + mu))      (Algorithm 2: the y and z updates).
+  // The words of all workers for the thread's 8 coordinates are loaded together (one L2 round trip) and
+  // re-loaded until every tag names step target-1; LLCH workers are handled per round.
+  constexpr int WMAX = (BITS == 0) ? 8 : (BITS == 8 ? 2 : 1);  // tagged words per group of 8 coordinates
+  constexpr int LLCH = (BITS == 0) ? 4 : 16;
+  const int wpg = (BITS == 0) ? pa.wpg : WMAX;
+  const size_t groups = (size_t)(CS * SL) >> 3;
   auto apply_update = [&](unsigned int target) {
     const int rpar = (pa.count - (int)target) & 1;  // parity half that holds step target-1
-    const unsigned long long* words = pa.pub + (size_t)rpar * PMAXFLAGS * PUB_STRIDE;
-    if (tid < N + (ALPC ? 1 : 0)) {  // thread i watches cluster i (in Algorithm 2 one more: the J cluster)
-      const unsigned long long* f = words + (size_t)(tid * CS + rank) * PUB_STRIDE;
-      unsigned long long w = 0;
-      uint64_t t0 = 0;
-      for (uint32_t it = 0;; ++it) {
-        w = ld_acquire_u64(f);
-        if ((unsigned int)w >= target) break;
-        if ((it & 63u) == 63u) {
-          if (ld_acquire_u32(pa.abort_flag) != 0u) break;
-          const uint64_t now = global_ns();
-          if (t0 == 0) t0 = now;
-          else if (now - t0 > 2000000000ull) {
-            atomicOr(a.dev_status, DEV_TIMEOUT);
-            st_release_u32(pa.abort_flag, 1u);
-            break;
-          }
-        }
-      }
-      sm.sdelta[tid] = __uint_as_float((unsigned int)(w >> 32));
-    }
-    const uint32_t* codes_in = a.codes + rpar * codes_buf;
-    __syncthreads();
-#ifdef LPC_TRACE
-    { const int t = (int)target; LPC_TRACE_MARK(3); }
-#endif
+    const uint32_t tag = pa.tag_base + target;
+    const unsigned long long* dwords = pa.pub + ((size_t)rpar * PMAXFLAGS + rank) * PUB_STRIDE;
+    const unsigned long long* ll_in = pa.ll + (size_t)rpar * N * groups * wpg;
 #pragma unroll
     for (int p = 0; p < NP; ++p) {
       const int off = p * PGROUP + tid * 8;
@@ -286,30 +245,84 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
       float acc[8];
 #pragma unroll
       for (int e = 0; e < 8; ++e) acc[e] = 0.f;
-      if (b == 32) {
-        for (int i = 0; i < N; ++i) {
-          const float di = sm.sdelta[i];
-          const uint32_t* wi = codes_in + (int64_t)i * a.stride_words;
+      unsigned long long vw[ALPC ? 8 : 1];
+#pragma unroll 1
+      for (int i0 = 0; i0 < N; i0 += LLCH) {
+        unsigned long long dw[LLCH], cw[LLCH][WMAX];
+        uint64_t t0 = 0;
+        for (uint32_t it = 0;; ++it) {
 #pragma unroll
-          for (int e = 0; e < 8; ++e) {
-            float val = 0.f;
-            if (c + e < d) val = __uint_as_float(__ldcg(wi + c + e));
-            acc[e] = add_rn(acc[e], mul_rn(di, val));
+          for (int j = 0; j < LLCH; ++j) {
+            const int i = min(i0 + j, N - 1);  // the tail repeats the last worker: harmless
+            dw[j] = ld_word(dwords + (size_t)i * CS * PUB_STRIDE);
+            const unsigned long long* q = ll_in + ((size_t)i * groups + (size_t)(c >> 3)) * wpg;
+#pragma unroll
+            for (int w = 0; w < WMAX; ++w) cw[j][w] = (w < wpg) ? ld_word(q + w) : ((unsigned long long)tag << 32);
+          }
+          if constexpr (ALPC) {
+            if (i0 == 0) {
+#pragma unroll
+              for (int e = 0; e < 8; ++e) vw[e] = ld_word(pa.ll_vhat + (size_t)rpar * groups * 8 + c + e);
+            }
+          }
+          bool ok = true;
+#pragma unroll
+          for (int j = 0; j < LLCH; ++j) {
+            ok = ok && word_tag(dw[j]) == tag;
+#pragma unroll
+            for (int w = 0; w < WMAX; ++w) ok = ok && word_tag(cw[j][w]) == tag;
+          }
+          if constexpr (ALPC) {
+            if (i0 == 0) {
+#pragma unroll
+              for (int e = 0; e < 8; ++e) ok = ok && word_tag(vw[e]) == tag;
+            }
+          }
+#ifdef LPC_TRACE
+          if (i0 == 0 && p == 0 && blockIdx.x == 0 && blockIdx.y == 0 && tid == 0 && target >= 8 && target < 72)
+            g_trace[(target - 8) * 16 + 15] = it + 1;
+#endif
+          if (ok) break;
+          if ((it & 63u) == 63u) {
+            if (ld_acquire_u32(pa.abort_flag) != 0u) break;
+            const uint64_t now = global_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > 2000000000ull) {
+              atomicOr(a.dev_status, DEV_TIMEOUT);
+              st_release_u32(pa.abort_flag, 1u);
+              break;
+            }
           }
         }
-      } else {
-        // all workers' loads are issued before the first is used: one L2 round trip instead of several
-#pragma unroll 16
-        for (int i = 0; i < N; ++i) {
-          const float di = sm.sdelta[i];
-          uint64_t lo, hi;
-          load_chunk<BITS, true>(codes_in + (int64_t)i * a.stride_words, c >> 3, b, a.pad_words, lo, hi);
+#ifdef LPC_TRACE
+        if (i0 == 0 && p == 0) { const int t = (int)target; LPC_TRACE_MARK(3); }
+#endif
+        {
 #pragma unroll
-          for (int e = 0; e < 8; ++e) {
-            uint32_t code;
-            if constexpr (BITS == 0) code = extract_bits(lo, hi, e * b, b);
-            else code = (uint32_t)(lo >> (e * BITS)) & ((1u << BITS) - 1u);
-            acc[e] = add_rn(acc[e], mul_rn(di, index_as_float(code, b)));
+          for (int j = 0; j < LLCH; ++j) {
+            if (i0 + j < N) {
+              const float di = __uint_as_float((uint32_t)dw[j]);
+              if (b == 32) {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                  const float val = (c + e < d && e < WMAX) ? __uint_as_float((uint32_t)cw[j][e < WMAX ? e : 0]) : 0.f;
+                  acc[e] = add_rn(acc[e], mul_rn(di, val));
+                }
+              } else {
+                uint64_t lo = (uint64_t)(uint32_t)cw[j][0], hi = 0;
+                if constexpr (WMAX >= 2) lo |= (uint64_t)(uint32_t)cw[j][1] << 32;
+                if constexpr (WMAX >= 4) hi = (uint64_t)(uint32_t)cw[j][2] | ((uint64_t)(uint32_t)cw[j][3] << 32);
+                float kf[8];
+                if constexpr (BITS == 0) {
+#pragma unroll
+                  for (int e = 0; e < 8; ++e) kf[e] = index_as_float(extract_bits(lo, hi, e * b, b), b);
+                } else {
+                  decode8<BITS ? BITS : 1>(lo, kf);
+                }
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[e] = add_rn(acc[e], mul_rn(di, kf[e]));
+              }
+            }
           }
         }
       }
@@ -318,7 +331,7 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
         if (c + e < d) {
           const float v = add_rn(mul_rn(acc[e], invN), mur[p][e]);
           if constexpr (ALPC) {  // steps 12-13 of Algorithm 2
-            const float vh = __ldcg(pa.vhat + rpar * d + c + e);
+            const float vh = __uint_as_float((uint32_t)vw[e]);
             yr[p][e] = soft_threshold(__fsub_rn(xr[p][e], mul_rn(pa.inv4L, v)), kappa_y);
             zr[p][e] = soft_threshold(__fsub_rn(zr[p][e], mul_rn(pa.alpha, vh)), kappa_z);
             sr[p][e] = add_rn(sr[p][e], yr[p][e]);
@@ -337,8 +350,10 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
     const uint32_t row_parity = (nbuf == 2) ? (uint32_t)((t >> 1) & 1) : (uint32_t)(t & 1);
     const uint64_t k = a.k_base + (uint64_t)t;
     const float* buf = rows + s * buf_floats;
-    const int wpar = (pa.count - 1 - t) & 1;  // the last step lands in parity half 0
-    uint32_t* out = a.codes + wpar * codes_buf + (int64_t)worker * a.stride_words;
+    const int wpar = (pa.count - 1 - t) & 1;  // parity half of the exchange buffers this step writes
+    const bool last = (t == pa.count - 1);    // the last step also leaves its messages in the documented layouts
+    const uint32_t tag = pa.tag_base + (uint32_t)(t + 1);
+    uint32_t* out = a.codes + (int64_t)worker * a.stride_words;
     LPC_TRACE_MARK(0);
     row_cur = row_next; y_cur = y_next; ms_cur = ms_next;
     if (nbuf == 2 && t + 1 < pa.count) prefetch(t + 1);
@@ -456,14 +471,20 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
 #pragma unroll
       for (int p = 0; p < NP; ++p) {
         const int off = p * PGROUP + tid * 8;
+        if (off < SL) {
+          unsigned long long* q = pa.ll_vhat + (size_t)wpar * groups * 8 + c0 + off;
 #pragma unroll
-        for (int e = 0; e < 8; ++e)
-          if (off + e < width) pa.vhat[wpar * d + c0 + off + e] = add_rn(u[p][e], mur[p][e]);
+          for (int e = 0; e < 8; ++e) {
+            const float vh = add_rn(u[p][e], mur[p][e]);
+            st_word(q + e, __float_as_uint(vh), tag);
+            if (last && off + e < width) pa.vhat[c0 + off + e] = vh;
+          }
+        }
       }
-      __syncthreads();  // the slice of v^ is stored and nobody reads the row buffer any more
-      if (nbuf == 1 && t + 1 < pa.count) prefetch(t + 1);
-      if (tid == 0)
-        st_release_u64(pa.pub + ((size_t)wpar * PMAXFLAGS + worker * CS + rank) * PUB_STRIDE, (unsigned long long)(unsigned int)(t + 1));
+      if (nbuf == 1) {
+        __syncthreads();  // nobody reads the row buffer any more
+        if (t + 1 < pa.count) prefetch(t + 1);
+      }
       continue;
     }
     // scale (Eq. 2)
@@ -513,8 +534,10 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
       float S1 = 0.f, S2 = 0.f;
       if (a.clip_mode == CLIP_STD) { S1 = tree_small(sm.s1part, CS); S2 = tree_small(sm.s2part, CS); }
       sm.scale = scale_out_of_line(m, S1, S2, d, b, a.clip_mode, a.clip_value);
+      // delta travels as a tagged word, one per CTA: the readers of rank r take every worker's rank-r word
+      st_word(pa.pub + ((size_t)wpar * PMAXFLAGS + worker * CS + rank) * PUB_STRIDE, __float_as_uint(sm.scale.delta), tag);
       if (rank == 0) {
-        a.delta[wpar * N + worker] = sm.scale.delta;
+        if (last) a.delta[worker] = sm.scale.delta;
         if (sm.scale.flags & 2u) atomicOr(a.dev_status, DEV_NONFINITE);
       }
     }
@@ -523,13 +546,15 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
     LPC_TRACE_MARK(12);
     const bool degenerate = (sc.flags & 1u) != 0;
 
-    // quantize (Section 2.2) and pack
+    // quantize (Section 2.2), pack, and send the codes of each group of 8 coordinates as tagged words
+    unsigned long long* ll_out = pa.ll + ((size_t)wpar * N + worker) * groups * wpg;
     uint32_t nclip = 0;
 #pragma unroll
     for (int p = 0; p < NP; ++p) {
       const int off = p * PGROUP + tid * 8;
       const int c = c0 + off;
       const bool mine = off < SL;
+      unsigned long long* q = ll_out + (size_t)(c >> 3) * wpg;
       if (b == 32) {
         if (mine) {
 #pragma unroll
@@ -539,7 +564,9 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
               if (v > sc.T) { v = sc.T; ++nclip; }
               if (v < -sc.T) { v = -sc.T; ++nclip; }
             }
-            if (c + e < a.pad_words) out[c + e] = (c + e < d) ? __float_as_uint(v) : 0u;
+            const uint32_t bits = (c + e < d) ? __float_as_uint(v) : 0u;
+            st_word(q + e, bits, tag);
+            if (last && c + e < a.pad_words) out[c + e] = bits;
           }
         }
         continue;
@@ -565,6 +592,16 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
           }
         }
       }
+      if (mine) {
+        st_word(q, (uint32_t)lo, tag);
+        if (WMAX >= 2 && wpg >= 2) st_word(q + 1, (uint32_t)(lo >> 32), tag);
+        if (WMAX >= 4 && wpg >= 4) {
+          st_word(q + 2, (uint32_t)hi, tag);
+          st_word(q + 3, (uint32_t)(hi >> 32), tag);
+        }
+      }
+      if (!last) continue;
+      // the caller's copy of the last messages: the packed little-endian bit stream
       if (BITS == 8) {
         const int64_t w = (int64_t)(c >> 3) * 2;
         if (mine && w < a.pad_words) *reinterpret_cast<uint2*>(out + w) = make_uint2((uint32_t)lo, (uint32_t)(lo >> 32));
@@ -595,17 +632,16 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
           if (w0 + w < a.pad_words) out[w0 + w] = st[w];
       }
     }
-    nclip = __reduce_add_sync(0xFFFFFFFFu, nclip);
-    if (lane == 0) sm.wclip[warp] = nclip;
-    __syncthreads();  // every thread of this CTA has stored its codes
     LPC_TRACE_MARK(13);
-    if (tid == 0) {
-      uint32_t tc = 0;
-      for (int w = 0; w < 8; ++w) tc += sm.wclip[w];
-      a.clipped_part[worker * PMAXCS + rank] = tc;
-      // publish step t: (step count, delta) in one word; the release store orders every code stored above
-      st_release_u64(pa.pub + ((size_t)wpar * PMAXFLAGS + worker * CS + rank) * PUB_STRIDE,
-                     (unsigned long long)(unsigned int)(t + 1) | ((unsigned long long)__float_as_uint(sc.delta) << 32));
+    if (last) {  // clipped-coordinate count of the last step, for the caller
+      nclip = __reduce_add_sync(0xFFFFFFFFu, nclip);
+      if (lane == 0) sm.wclip[warp] = nclip;
+      __syncthreads();
+      if (tid == 0) {
+        uint32_t tc = 0;
+        for (int w = 0; w < 8; ++w) tc += sm.wclip[w];
+        a.clipped_part[worker * PMAXCS + rank] = tc;
+      }
     }
     LPC_TRACE_MARK(14);
   }
