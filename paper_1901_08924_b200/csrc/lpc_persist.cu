@@ -55,9 +55,10 @@ struct PSmem {
   uint64_t bar[2];
   float coef[PMAXB];
   float wpart[PMAXB * PMAXP * 8];
-  float mpart[PMAXB * PMAXCS];
-  float s1part[PMAXCS], s2part[PMAXCS];
-  uint32_t maxpart[PMAXCS];
+  // cluster exchange slots, written by the peers through distributed shared memory as tagged words, two
+  // step-parity halves: margin partial sums (slot b * PMAXCS + rank) and statistics (max, S1, S2 per rank)
+  unsigned long long mx[2][PMAXB * PMAXCS];
+  unsigned long long sx[2][3 * PMAXCS];
   float ws1[PMAXP * 8], ws2[PMAXP * 8];
   uint32_t wmax[8];
   uint32_t wclip[8];
@@ -76,6 +77,19 @@ __device__ __forceinline__ void st_word(unsigned long long* p, uint32_t payload,
   asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
 __device__ __forceinline__ uint32_t word_tag(unsigned long long w) { return (uint32_t)(w >> 32); }
+// The same kind of word in shared memory: stored into CTA `cta` of the cluster at the address that `slot` has in
+// this CTA, read back from this CTA's own shared memory.
+__device__ __forceinline__ void st_cluster_word(const unsigned long long* slot, uint32_t cta, uint32_t payload, uint32_t tag) {
+  const unsigned long long v = (unsigned long long)payload | ((unsigned long long)tag << 32);
+  uint32_t remote;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(slot)), "r"(cta));
+  asm volatile("st.relaxed.cluster.shared::cluster.u64 [%0], %1;" ::"r"(remote), "l"(v) : "memory");
+}
+__device__ __forceinline__ unsigned long long ld_shared_word(const unsigned long long* slot) {
+  unsigned long long v;
+  asm volatile("ld.relaxed.cluster.shared::cta.u64 %0, [%1];" : "=l"(v) : "r"(smem_u32(slot)) : "memory");
+  return v;
+}
 __device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int* p) {
   unsigned int v;
   asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
@@ -155,6 +169,9 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
     mbar_init(&sm.bar[1], 1);
     mbar_fence_init();
   }
+  // no exchange slot may look valid before a peer has written it: tags start at 1
+  for (int i = tid; i < 2 * PMAXB * PMAXCS; i += PT) (&sm.mx[0][0])[i] = 0ull;
+  for (int i = tid; i < 2 * 3 * PMAXCS; i += PT) (&sm.sx[0][0])[i] = 0ull;
   asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   __syncthreads();
 
@@ -224,6 +241,22 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
     }
   };
 
+  // Every spin in this kernel ends: after about two seconds without progress the thread records a timeout and
+  // raises the abort flag, which ends all other spins at their next look at it.
+  auto wait_expired = [&](uint32_t it, uint64_t& t0) -> bool {
+    if ((it & 63u) != 63u) return false;
+    if (ld_acquire_u32(pa.abort_flag) != 0u) return true;
+    const uint64_t now = global_ns();
+    if (t0 == 0) {
+      t0 = now;
+      return false;
+    }
+    if (now - t0 <= 2000000000ull) return false;
+    atomicOr(a.dev_status, DEV_TIMEOUT);
+    st_release_u32(pa.abort_flag, 1u);
+    return true;
+  };
+
   // Applies step target-1's update to this thread's coordinates:
   //   x <- prox_{eta h}(x - eta (mean_i delta_i k_i + mu))      (Algorithm 2: the y and z updates).
   // The words of all workers for the thread's 8 coordinates are loaded together (one L2 round trip) and
@@ -282,17 +315,7 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
           if (i0 == 0 && p == 0 && blockIdx.x == 0 && blockIdx.y == 0 && tid == 0 && target >= 8 && target < 72)
             g_trace[(target - 8) * 16 + 15] = it + 1;
 #endif
-          if (ok) break;
-          if ((it & 63u) == 63u) {
-            if (ld_acquire_u32(pa.abort_flag) != 0u) break;
-            const uint64_t now = global_ns();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > 2000000000ull) {
-              atomicOr(a.dev_status, DEV_TIMEOUT);
-              st_release_u32(pa.abort_flag, 1u);
-              break;
-            }
-          }
+          if (ok || wait_expired(it, t0)) break;
         }
 #ifdef LPC_TRACE
         if (i0 == 0 && p == 0) { const int t = (int)target; LPC_TRACE_MARK(3); }
@@ -410,15 +433,32 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
     }
     __syncthreads();
     LPC_TRACE_MARK(6);
+    // Cluster exchange of the margin partial sums: every CTA stores its partial sum of row b into slot (b, rank)
+    // of every CTA of the cluster, tagged with the step; the owner of row b waits until its slots carry the tag.
+    const int xpar = t & 1;
     if (tid < B) {
       float part = tree8(&sm.wpart[tid * NP * 8]);
       if (NP == 2) part = add_rn(part, tree8(&sm.wpart[(tid * NP + 1) * 8]));
-      for (int q = 0; q < CS; ++q) cluster.map_shared_rank(sm.mpart, q)[tid * PMAXCS + rank] = part;
-    }
-    cluster.sync();
-    LPC_TRACE_MARK(7);
-    if (tid < B) {
-      const float m = tree_small(&sm.mpart[tid * PMAXCS], CS);
+      float m = part;
+      if (CS > 1) {
+        for (int q = 0; q < CS; ++q) st_cluster_word(&sm.mx[xpar][tid * PMAXCS + rank], (uint32_t)q, __float_as_uint(part), tag);
+        unsigned long long w[PMAXCS];
+        uint64_t t0 = 0;
+        for (uint32_t it = 0;; ++it) {
+          bool ok = true;
+#pragma unroll
+          for (int q = 0; q < PMAXCS; ++q) {
+            w[q] = (q < CS) ? ld_shared_word(&sm.mx[xpar][tid * PMAXCS + q]) : ((unsigned long long)tag << 32);
+            ok = ok && word_tag(w[q]) == tag;
+          }
+          if (ok || wait_expired(it, t0)) break;
+        }
+        float mp[PMAXCS];
+#pragma unroll
+        for (int q = 0; q < PMAXCS; ++q) mp[q] = __uint_as_float((uint32_t)w[q]);
+        m = tree_small(mp, CS);
+      }
+      LPC_TRACE_MARK(7);
       const float c = coef_out_of_line(a.loss, m, ms_cur, y_cur);
       sm.coef[tid] = c;
       if (rank == 0 && t == pa.count - 1) {
@@ -520,19 +560,38 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
         s2 = tree8(sm.ws2);
         if (NP == 2) { s1 = add_rn(s1, tree8(sm.ws1 + 8)); s2 = add_rn(s2, tree8(sm.ws2 + 8)); }
       }
-      for (int q = 0; q < CS; ++q) {
-        cluster.map_shared_rank(sm.maxpart, q)[rank] = m;
-        cluster.map_shared_rank(sm.s1part, q)[rank] = s1;
-        cluster.map_shared_rank(sm.s2part, q)[rank] = s2;
+      LPC_TRACE_MARK(11);
+      float S1 = s1, S2 = s2;
+      if (CS > 1) {  // the same exchange for the statistics: (max |u|, S1, S2) of every rank
+        for (int q = 0; q < CS; ++q) {
+          st_cluster_word(&sm.sx[xpar][0 * PMAXCS + rank], (uint32_t)q, m, tag);
+          st_cluster_word(&sm.sx[xpar][1 * PMAXCS + rank], (uint32_t)q, __float_as_uint(s1), tag);
+          st_cluster_word(&sm.sx[xpar][2 * PMAXCS + rank], (uint32_t)q, __float_as_uint(s2), tag);
+        }
+        unsigned long long w[3][PMAXCS];
+        uint64_t t0 = 0;
+        for (uint32_t it = 0;; ++it) {
+          bool ok = true;
+#pragma unroll
+          for (int j = 0; j < 3; ++j) {
+#pragma unroll
+            for (int q = 0; q < PMAXCS; ++q) {
+              w[j][q] = (q < CS) ? ld_shared_word(&sm.sx[xpar][j * PMAXCS + q]) : ((unsigned long long)tag << 32);
+              ok = ok && word_tag(w[j][q]) == tag;
+            }
+          }
+          if (ok || wait_expired(it, t0)) break;
+        }
+        float p1[PMAXCS], p2[PMAXCS];
+        m = 0;
+#pragma unroll
+        for (int q = 0; q < PMAXCS; ++q) {
+          m = max(m, (uint32_t)w[0][q]);
+          p1[q] = __uint_as_float((uint32_t)w[1][q]);
+          p2[q] = __uint_as_float((uint32_t)w[2][q]);
+        }
+        if (a.clip_mode == CLIP_STD) { S1 = tree_small(p1, CS); S2 = tree_small(p2, CS); }
       }
-    }
-    cluster.sync();
-    LPC_TRACE_MARK(11);
-    if (tid == 0) {
-      uint32_t m = 0;
-      for (int q = 0; q < CS; ++q) m = max(m, sm.maxpart[q]);
-      float S1 = 0.f, S2 = 0.f;
-      if (a.clip_mode == CLIP_STD) { S1 = tree_small(sm.s1part, CS); S2 = tree_small(sm.s2part, CS); }
       sm.scale = scale_out_of_line(m, S1, S2, d, b, a.clip_mode, a.clip_value);
       // delta travels as a tagged word, one per CTA: the readers of rank r take every worker's rank-r word
       st_word(pa.pub + ((size_t)wpar * PMAXFLAGS + worker * CS + rank) * PUB_STRIDE, __float_as_uint(sm.scale.delta), tag);
