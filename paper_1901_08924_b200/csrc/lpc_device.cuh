@@ -145,8 +145,17 @@ __device__ __forceinline__ Scale make_scale(uint32_t max_bits, float S1, float S
   if (clip_mode == CLIP_LAMBDA) {
     T = mul_rn(clip_value, M);
   } else if (clip_mode == CLIP_STD) {
-    const double mean = __ddiv_rn((double)S1, (double)len);
-    double var = __dsub_rn(__ddiv_rn((double)S2, (double)len), __dmul_rn(mean, mean));
+    double mean, ex2;
+    if (len > 0 && (len & (len - 1)) == 0) {
+      // a power-of-two length: multiplying by 2^-log2(len) is the same exact operation as the division
+      const double inv = __longlong_as_double((long long)(1023 - (63 - __clzll(len))) << 52);
+      mean = __dmul_rn((double)S1, inv);
+      ex2 = __dmul_rn((double)S2, inv);
+    } else {
+      mean = __ddiv_rn((double)S1, (double)len);
+      ex2 = __ddiv_rn((double)S2, (double)len);
+    }
+    double var = __dsub_rn(ex2, __dmul_rn(mean, mean));
     if (var < 0.0) var = 0.0;
     double t = __dmul_rn((double)clip_value, __dsqrt_rn(var));
     if (t > (double)M) t = (double)M;
