@@ -256,6 +256,7 @@ def run_ours(args):
         ctx.close()
         torch.cuda.empty_cache()
         out["alpc"] = alpc_bench(dev)
+        out["fused_large_batch"] = fused_large_batch_bench(dev, peak)
     elif rank == 0:
         out["e2e"] = None
     ctx.close()
@@ -343,6 +344,35 @@ def quantize_aggregate_bench(dev, peak, log2_len=26, dnn=True):
         "combined_gbs": round((bq + ba) / (tq + ta) * 1e-6, 1)}
     q.close()
     return res
+
+
+def fused_large_batch_bench(dev, peak, n=65536, steps=30):
+    """The fused worker kernel (sampling, SVRG difference, scale, quantize, pack) where it is bandwidth-bound: the ALPC
+    workload's shape (d = 8,192, N = 32, logistic) with the minibatch raised to B = 256 rows per worker, so that one
+    step gathers N*B*d*4 = 268 MB of rows.  Times come from the library's per-kernel event profile."""
+    import torch
+    from paper_1901_08924_b200 import lpc, synth
+    d, N, B = 8192, 32, 256
+    X, y, _ = synth.linear_problem(n, d, loss="logistic", sparsity=0.02, noise=0.1, seed=1, col_scale_range=(0.1, 10.0),
+                                   device=dev)
+    out = {"workload": "fused_step_logistic_%dx8192_N32_B256" % n, "row_bytes_per_step": N * B * d * 4}
+    for b in (2, 8):
+        ctx = lpc.Context(X, y, lpc.LOGISTIC, 1e-5, N, B, b, lpc.CLIP_STD, 2.0, 0)
+        ctx.snapshot_full_grad()
+        ctx.inner_steps(1e-3, 0, 5)
+        ctx.set_option(lpc.OPT_PROFILE, 1)
+        ctx.inner_steps(1e-3, 5, steps)
+        ctx.sync_status()
+        prof = ctx.get_profile()
+        tw = prof["worker"][0] / prof["worker"][1]
+        ta = prof["aggregate"][0] / prof["aggregate"][1]
+        bw = N * B * d * 4 + N * B * 8 + N * (d * b // 8 + 4)
+        out["b%d" % b] = {"worker_us": round(tw * 1e3, 2), "worker_gbs": round(bw / tw * 1e-6, 1),
+                          "worker_frac": round(bw / tw * 1e-6 / peak, 4), "aggregate_us": round(ta * 1e3, 2),
+                          "ring_stages": ctx.query(lpc.INFO_STEP_RING_STAGES),
+                          "cluster_size": ctx.query(lpc.INFO_STEP_CLUSTER_SIZE)}
+        ctx.close()
+    return out
 
 
 def alpc_bench(dev):
@@ -479,8 +509,15 @@ def main():
     ap.add_argument("--per-step-kernels", action="store_true",
                     help="run the inner loop as per-step kernels (graph replay) instead of the one-launch loop; "
                          "for profiler captures, which cannot replay the cooperative launch")
+    ap.add_argument("--fused-large-batch-only", type=int, default=0, metavar="ROWS",
+                    help="run only the large-minibatch leg of the fused worker kernel on a ROWS x 8192 matrix "
+                         "(a small case for profiler captures)")
     args = ap.parse_args()
-    if args.quantize_aggregate_only:
+    if args.fused_large_batch_only:
+        import torch
+        peak, _ = read_peak()
+        print(json.dumps(fused_large_batch_bench(torch.device("cuda", 0), peak, n=args.fused_large_batch_only, steps=4)))
+    elif args.quantize_aggregate_only:
         import torch
         peak, _ = read_peak()
         print(json.dumps(quantize_aggregate_bench(torch.device("cuda", 0), peak, args.quantize_aggregate_only, dnn=False)))

@@ -103,7 +103,9 @@ typedef struct lpc_ctx lpc_ctx;
  *   y        n labels / targets
  *   n        rows; must be a multiple of N.  Worker i owns rows [i*n/N, (i+1)*n/N).
  *   d        features, multiple of 4, at most 16384
- *   N        simulated workers, 1..1024;  B minibatch size per worker, 1..64
+ *   N        simulated workers, 1..1024;  B minibatch size per worker, 1..1024 (up to 64 rows per worker stay
+ *            resident on chip and the one-launch loops are available; larger minibatches stream through
+ *            the per-step kernel)
  *   b        bits per coordinate: 1..16 or 32 (32 = full precision, the codes are the floats)
  *   seed     key of every random stream (minibatches, shared batch J, stochastic rounding)
  *   stream   cudaStream_t (NULL = default stream)
@@ -218,6 +220,7 @@ int lpc_objective(lpc_ctx* ctx, const float* x, double* P_out);
 #define LPC_INFO_ALPC_LOOP_CLUSTER_SIZE 5  /* as LOOP_CLUSTER_SIZE, for the one-launch loop of Algorithm 2 */
 #define LPC_INFO_LOOP_ROW_BUFFERS 6        /* sampled-row buffers per CTA of the one-launch loop (1 or 2; 0: not available) */
 #define LPC_INFO_ALPC_LOOP_ROW_BUFFERS 7   /* the same for the loop of Algorithm 2 */
+#define LPC_INFO_STEP_RING_STAGES 8        /* per-step kernel: 0 = minibatch rows resident on chip, else ring stages they stream through */
 int lpc_query(const lpc_ctx* ctx, int what, int64_t* out);
 
 /* Per-kernel device time measured with CUDA events on the context's stream while LPC_OPT_PROFILE is

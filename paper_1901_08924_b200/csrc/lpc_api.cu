@@ -79,6 +79,7 @@ struct lpc_ctx {
   bool inner_ok = false;
   int CS = 1, SL = 0;
   size_t innerSmem = 0;
+  int innerStages = 0;  // 0: minibatch rows resident in shared memory; > 0: streamed through that many stages
   SegPlan inner_seg;  // one segment of length d for the aggregator
   // persistent inner loop
   bool persist_ok = false, apersist_ok = false;  // Algorithm 1 loop / Algorithm 2 loop
@@ -294,7 +295,7 @@ InnerArgs inner_args(lpc_ctx* c, uint64_t k_base, const uint64_t* k_dev, int has
   a.codes = c->codes; a.stride_words = c->inner_seg.stride_words; a.pad_words = c->inner_seg.stride_words;
   a.delta = c->delta; a.clipped_part = c->clipped_part;
   a.idx_tap = c->idx_tap; a.coef_tap = c->coef_tap; a.u_tap = c->tap_u ? c->u_tap : nullptr;
-  a.dev_status = c->dev_status; a.CS = c->CS; a.SL = c->SL;
+  a.dev_status = c->dev_status; a.CS = c->CS; a.SL = c->SL; a.stream_stages = c->innerStages;
   return a;
 }
 
@@ -311,8 +312,9 @@ AggArgs agg_args(lpc_ctx* c, const SegPlan& p, const uint32_t* codes, const floa
 int replan_inner(lpc_ctx* c) {
   size_t smem = 0;
   int cs = 1, sl = 0;
-  c->inner_ok = inner_plan(c->d, c->B, c->want_cs, c->max_smem, &cs, &sl, &smem);
-  if (c->inner_ok) { c->CS = cs; c->SL = sl; c->innerSmem = smem; }
+  int stages = 0;
+  c->inner_ok = inner_plan(c->d, c->B, c->want_cs, c->max_smem, &cs, &sl, &smem, &stages);
+  if (c->inner_ok) { c->CS = cs; c->SL = sl; c->innerSmem = smem; c->innerStages = stages; }
   int nbuf = 2;
   c->persist_ok = persist_plan(c->d, c->N, c->B, c->b, 0, c->want_cs, c->max_smem, &cs, &sl, &smem, &nbuf);
   if (c->persist_ok) { c->pCS = cs; c->pSL = sl; c->persistSmem = smem; c->pNbuf = nbuf; }
@@ -723,6 +725,7 @@ int lpc_query(const lpc_ctx* c, int what, int64_t* out) {
     case LPC_INFO_ALPC_LOOP_CLUSTER_SIZE: *out = c->apersist_ok ? c->aCS : 0; return LPC_OK;
     case LPC_INFO_LOOP_ROW_BUFFERS: *out = c->persist_ok ? c->pNbuf : 0; return LPC_OK;
     case LPC_INFO_ALPC_LOOP_ROW_BUFFERS: *out = c->apersist_ok ? c->aNbuf : 0; return LPC_OK;
+    case LPC_INFO_STEP_RING_STAGES: *out = c->inner_ok ? c->innerStages : 0; return LPC_OK;
     case LPC_INFO_LOOP_LAUNCHES: *out = c->persist_launches; return LPC_OK;
     case LPC_INFO_SNAPSHOT_ROWS_PER_TILE: *out = c->snapR; return LPC_OK;
     case LPC_INFO_SNAPSHOT_STAGES: *out = c->snapStages; return LPC_OK;

@@ -13,6 +13,14 @@
 // way, and after a second cluster barrier every CTA derives the same scale and quantizes its slice.
 // In ALPC-SVRG one more cluster handles the shared batch J and stores v^ = u_J + mu in full
 // precision.  No load with cluster multicast is used; each CTA fetches its own slice.
+//
+// Large minibatches (STREAM = true: more rows than shared memory holds, up to 1024 per worker) stream the
+// rows instead, in batch order, through a ring of small stages filled by bulk copies, with no block barrier
+// in the loop.  Half of the warps take the margin partial sums (one warp per row of a group, over the whole
+// slice, reduced by shuffles alone) and send them to the cluster as tagged words through distributed shared
+// memory; the other half own the coordinates of u, wait for the partial sums of all CTAs, form the
+// coefficients and add the rows -- still in shared memory -- into u, then hand the stage back to be
+// refilled.  Each row is read from HBM once and the kernel runs at the rate of the bulk copies.
 #include <cooperative_groups.h>
 
 #include "lpc_device.cuh"
@@ -28,6 +36,11 @@ constexpr int IGROUP = IT * 8;    // coordinates per pass
 constexpr int MAXP = 4;           // passes per CTA: SL <= 8192
 constexpr int MAXB = 64;          // minibatch rows
 constexpr int MAXCS = 8;
+// streaming path
+constexpr int SG = 4;             // rows per ring stage
+constexpr int SSLOTS = 16;        // exchange slots (a peer's margins run at most 2 * SMAXR - 2 groups ahead of this CTA's u)
+constexpr int SMAXR = 8;          // ring stages at most
+constexpr int SMAXB = 1024;       // rows per worker at most
 
 struct Smem {
   uint64_t bar;
@@ -45,18 +58,50 @@ struct Smem {
   Scale scale;
   int load_ok;
   __align__(16) uint8_t stage[IT * 16];
+  // streaming path: one mbarrier per ring stage; tagged partial sums of the groups in flight (written by peers)
+  uint64_t sbar[SMAXR];           // stage filled (bulk-copy bytes)
+  uint64_t ebar[SMAXR];           // stage consumed (one arrival per warp that adds rows into u)
+  unsigned long long sx[SSLOTS][SG * MAXCS];
 };
 
-template <int BITS>  // 1, 2, 4, 8: fixed-width packing; 0: b from the arguments (1..16 or 32)
+// Tagged 64-bit words (payload | tag << 32) stored into the shared memory of CTA `cta` of the cluster at the
+// address `slot` has in this CTA; a reader that sees the tag it expects also sees the payload.
+__device__ __forceinline__ void st_cluster_word(const unsigned long long* slot, uint32_t cta, uint32_t payload, uint32_t tag) {
+  const unsigned long long v = (unsigned long long)payload | ((unsigned long long)tag << 32);
+  uint32_t remote;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(slot)), "r"(cta));
+  asm volatile("st.relaxed.cluster.shared::cluster.u64 [%0], %1;" ::"r"(remote), "l"(v) : "memory");
+}
+__device__ __forceinline__ unsigned long long ld_shared_word(const unsigned long long* slot) {
+  unsigned long long v;
+  asm volatile("ld.relaxed.cluster.shared::cta.u64 %0, [%1];" : "=l"(v) : "r"(smem_u32(slot)) : "memory");
+  return v;
+}
+
+// BITS: 1, 2, 4, 8 fixed-width packing; 0: b from the arguments (1..16 or 32).
+// STREAM: rows pass through a ring of stages (large minibatches; one pass, SL <= IGROUP) instead of all being resident.
+template <int BITS, bool STREAM>
 __global__ void __launch_bounds__(IT) inner_kernel(InnerArgs a) {
   cg::cluster_group cluster = cg::this_cluster();
   extern __shared__ __align__(16) unsigned char smem_raw[];
   Smem& sm = *reinterpret_cast<Smem*>(smem_raw);
-  float* rows = reinterpret_cast<float*>(smem_raw + ((sizeof(Smem) + 15) & ~(size_t)15));  // B x SL
+  unsigned char* dyn = smem_raw + ((sizeof(Smem) + 15) & ~(size_t)15);
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int rank = (int)cluster.block_rank();
   const int CS = a.CS, SL = a.SL, B = a.B, d = a.d;
+  // sampled rows, their labels and cached snapshot margins; the row data (resident: B x SL; streaming: the ring)
+  int64_t* s_idx = sm.idx;
+  float* s_yv = sm.yv;
+  float* s_ms = sm.msnap;
+  float* rows = reinterpret_cast<float*>(dyn);
+  if constexpr (STREAM) {
+    const int Bp = (B + 3) & ~3;
+    s_idx = reinterpret_cast<int64_t*>(dyn);
+    s_yv = reinterpret_cast<float*>(s_idx + Bp);
+    s_ms = s_yv + Bp;
+    rows = s_ms + Bp;
+  }
   const int worker = blockIdx.y;
   const bool is_J = (worker == a.N);
   const uint64_t k = a.k_base + (a.k_dev ? *a.k_dev : 0ull);
@@ -66,30 +111,39 @@ __global__ void __launch_bounds__(IT) inner_kernel(InnerArgs a) {
   const int width = max(0, min(SL, d - c0));        // coordinates of the slice that exist
 
   // ---- sampling (Algorithm 1 step 6): slot a uses word 0 of block a of the batch stream -----------------
-  if (tid < B) {
+  for (int slot = tid; slot < B; slot += IT) {
     int64_t lo, span;
     uint32_t tag, wk;
     if (is_J) { lo = 0; span = a.n; tag = TAG_BATCH_J; wk = 0; }
     else if (a.sample_global) { lo = 0; span = a.n; tag = TAG_BATCH; wk = (uint32_t)worker; }
     else { span = a.n / a.N; lo = (int64_t)worker * span; tag = TAG_BATCH; wk = (uint32_t)worker; }
-    const U4 r = stream_block(a.seed, tag, wk, k, (uint32_t)tid);
+    const U4 r = stream_block(a.seed, tag, wk, k, (uint32_t)slot);
     const int64_t row = lo + (int64_t)(((uint64_t)r.x * (uint64_t)span) >> 32);
-    sm.idx[tid] = row;
-    sm.yv[tid] = a.y[row];
-    sm.msnap[tid] = a.margins[row];
+    s_idx[slot] = row;
+    s_yv[slot] = a.y[row];
+    s_ms[slot] = a.margins[row];
   }
   if (tid == 0) {
     mbar_init(&sm.bar, 1);
+    if constexpr (STREAM) {
+      for (int r = 0; r < SMAXR; ++r) {
+        mbar_init(&sm.sbar[r], 1);
+        mbar_init(&sm.ebar[r], IT / 32 - SG);
+      }
+    }
     mbar_fence_init();
+  }
+  if constexpr (STREAM) {  // no exchange slot may look valid before a peer has written it: tags start at 1
+    for (int i = tid; i < SSLOTS * SG * MAXCS; i += IT) (&sm.sx[0][0])[i] = 0ull;
   }
   // Every CTA of the cluster announces that it is running; peers wait for this before their first
   // store into this CTA's shared memory.
   asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   __syncthreads();
-  if (tid == 0 && width > 0) {
+  if (!STREAM && tid == 0 && width > 0) {
     const uint32_t bytes = (uint32_t)width * 4u;
     mbar_expect_tx(&sm.bar, bytes * (uint32_t)B);
-    for (int r = 0; r < B; ++r) bulk_load(rows + (size_t)r * SL, a.X + sm.idx[r] * (int64_t)d + c0, bytes, &sm.bar);
+    for (int r = 0; r < B; ++r) bulk_load(rows + (size_t)r * SL, a.X + s_idx[r] * (int64_t)d + c0, bytes, &sm.bar);
   }
 
   // ---- this thread's coordinates and the iterate at them ---------------------------------------------------
@@ -110,7 +164,7 @@ __global__ void __launch_bounds__(IT) inner_kernel(InnerArgs a) {
   }
 
   bool ok = true;
-  if (width > 0) ok = mbar_wait(&sm.bar, 0);
+  if (!STREAM && width > 0) ok = mbar_wait(&sm.bar, 0);
   if (!ok) {
     atomicOr(a.dev_status, DEV_TIMEOUT);
     ok = mbar_wait(&sm.bar, 0);  // one more bounded chance for the copies in flight before going on
@@ -130,6 +184,169 @@ __global__ void __launch_bounds__(IT) inner_kernel(InnerArgs a) {
     }
   };
 
+  const float invB = __fdiv_rn(1.0f, (float)B);
+  float u[MAXP][8];
+  if constexpr (STREAM) {
+    // ---- streaming: groups of SG rows in batch order through a ring of R stages, no block barrier inside.
+    // Warps 0..SG-1 take the margin partial sums (warp w: row w of every group, over the whole slice) and send
+    // them to the cluster; warps SG..7 own the coordinates of u: per group they collect the partial sums of all
+    // CTAs, form the coefficients and add the rows, then hand the stage back to be refilled. ----------------------
+#pragma unroll
+    for (int p = 0; p < MAXP; ++p) {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) u[p][e] = 0.f;
+    }
+    const int R = a.stream_stages;
+    const int ngroups = (B + SG - 1) / SG;
+    const uint32_t row_bytes = (uint32_t)width * 4u;
+    auto issue = [&](int g) {  // one thread: the rows of group g into stage g % R
+      const int s = g % R;
+      const int cnt = min(SG, B - g * SG);
+      mbar_expect_tx(&sm.sbar[s], row_bytes * (uint32_t)cnt);
+      for (int j = 0; j < cnt; ++j)
+        bulk_load(rows + ((size_t)s * SG + j) * SL, a.X + s_idx[g * SG + j] * (int64_t)d + c0, row_bytes, &sm.sbar[s]);
+    };
+    if (tid == 0 && width > 0) {
+      for (int g = 0; g < min(R, ngroups); ++g) issue(g);
+    }
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");  // all peers have started
+    bool gave_up = false;  // after one wait ran out this thread waits no more (the status word says so)
+    auto wait_stage = [&](int g) {
+      if (width > 0 && !gave_up && !mbar_wait(&sm.sbar[g % R], (uint32_t)((g / R) & 1))) {
+        atomicOr(a.dev_status, DEV_TIMEOUT);
+        gave_up = true;
+      }
+    };
+    constexpr int CH = IGROUP / 8 / 32;  // 8-coordinate chunks per lane when one warp covers a slice: 8
+    constexpr int AT = IT - SG * 32;     // threads that own the coordinates of u
+    constexpr int UC = IGROUP / 8 / AT;  // chunks per such thread: 2
+    float ua[UC][8];
+#pragma unroll
+    for (int q = 0; q < UC; ++q)
+#pragma unroll
+      for (int e = 0; e < 8; ++e) ua[q][e] = 0.f;
+    if (warp < SG) {
+      // -- margins: lane l holds x for chunks l, l+32, ..., the leaves of the tree in coordinate order are
+      // (chunk, element); per chunk tree8, then the tree over the 32 lanes for every chunk row, then over the rows
+      float xs[CH][8];
+#pragma unroll
+      for (int q = 0; q < CH; ++q) {
+        const int off = (q * 32 + lane) * 8;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) xs[q][e] = (off + e < width) ? a.x[c0 + off + e] : 0.f;
+      }
+#pragma unroll 1
+      for (int g = 0; g < ngroups; ++g) {
+        const int cnt = min(SG, B - g * SG);
+        wait_stage(g);
+        if (warp < cnt) {
+          float sv[CH];
+#pragma unroll
+          for (int q = 0; q < CH; ++q) {
+            float v[8], pr[8];
+            row8((g % R) * SG + warp, (q * 32 + lane) * 8, v);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) pr[e] = mul_rn(v[e], xs[q][e]);
+            sv[q] = tree8(pr);
+          }
+          WarpHalving<CH, 0>::run(sv, lane);  // lane holds the 32-lane tree sum of chunk row halving_index<3>(lane)
+          float part = sv[0];
+          part = add_rn(part, __shfl_xor_sync(0xFFFFFFFFu, part, 4));  // rows 2k, 2k+1
+          part = add_rn(part, __shfl_xor_sync(0xFFFFFFFFu, part, 2));
+          part = add_rn(part, __shfl_xor_sync(0xFFFFFFFFu, part, 1));
+          if (lane < CS)
+            st_cluster_word(&sm.sx[g % SSLOTS][warp * MAXCS + rank], (uint32_t)lane, __float_as_uint(part), (uint32_t)(g + 1));
+        }
+      }
+    } else {
+      // -- u: thread t of these warps owns chunks t and t + 128 of the slice
+      const int t = tid - SG * 32;
+#pragma unroll 1
+      for (int g = 0; g < ngroups; ++g) {
+        const int cnt = min(SG, B - g * SG);
+        const int s = g % R;
+        float c_mine = 0.f;
+        if (lane < cnt) {  // lane j: the coefficient of row j of the group (every warp forms all of them)
+          float mp[MAXCS];
+          uint64_t t0 = 0;
+          for (uint32_t it = 0;; ++it) {
+            bool all = true;
+#pragma unroll
+            for (int q = 0; q < MAXCS; ++q) {
+              mp[q] = 0.f;
+              if (q < CS) {
+                const unsigned long long w = ld_shared_word(&sm.sx[g % SSLOTS][lane * MAXCS + q]);
+                all = all && (uint32_t)(w >> 32) == (uint32_t)(g + 1);
+                mp[q] = __uint_as_float((uint32_t)w);
+              }
+            }
+            if (all || gave_up) break;
+            if ((it & 63u) == 63u) {
+              const uint64_t now = global_ns();
+              if (t0 == 0) t0 = now;
+              else if (now - t0 > 2000000000ull) {
+                atomicOr(a.dev_status, DEV_TIMEOUT);
+                gave_up = true;
+              }
+            }
+          }
+          const int slot = g * SG + lane;
+          const float m = (CS == 1) ? mp[0] : (CS == 2) ? add_rn(mp[0], mp[1]) : (CS == 4) ? tree4(mp[0], mp[1], mp[2], mp[3]) : tree8(mp);
+          c_mine = __fsub_rn(loss_deriv(a.loss, m, s_yv[slot]), loss_deriv(a.loss, s_ms[slot], s_yv[slot]));
+          if (rank == 0 && warp == SG) {
+            if (a.idx_tap) a.idx_tap[(int64_t)worker * B + slot] = s_idx[slot];
+            if (a.coef_tap) a.coef_tap[(int64_t)worker * B + slot] = c_mine;
+          }
+        }
+        __syncwarp();
+        wait_stage(g);
+#pragma unroll
+        for (int j = 0; j < SG; ++j) {
+          const float c = __shfl_sync(0xFFFFFFFFu, c_mine, j);
+          if (j < cnt) {
+#pragma unroll
+            for (int q = 0; q < UC; ++q) {
+              float v[8];
+              row8(s * SG + j, (q * AT + t) * 8, v);
+#pragma unroll
+              for (int e = 0; e < 8; ++e) ua[q][e] = add_rn(ua[q][e], mul_rn(c, v[e]));
+            }
+          }
+        }
+        // hand the stage back: when all warps of this side are done with it, one thread refills it
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.ebar[s]);
+        if (t == 0 && g + R < ngroups) {
+          if (!gave_up && !mbar_wait(&sm.ebar[s], (uint32_t)((g / R) & 1))) {
+            atomicOr(a.dev_status, DEV_TIMEOUT);
+            gave_up = true;
+          }
+          if (width > 0) issue(g + R);
+        }
+      }
+    }
+    __syncthreads();  // both sides are done with the ring: it now carries u to the usual owner of each coordinate
+    if (warp >= SG) {
+      const int t = tid - SG * 32;
+#pragma unroll
+      for (int q = 0; q < UC; ++q) {
+        if ((q * AT + t) * 8 < SL) {  // the ring holds at least one slice
+          float* dst = rows + (q * AT + t) * 8;
+          *reinterpret_cast<float4*>(dst) = make_float4(ua[q][0], ua[q][1], ua[q][2], ua[q][3]);
+          *reinterpret_cast<float4*>(dst + 4) = make_float4(ua[q][4], ua[q][5], ua[q][6], ua[q][7]);
+        }
+      }
+    }
+    __syncthreads();
+    if (tid * 8 < SL) {
+      const float4 v0 = *reinterpret_cast<const float4*>(rows + tid * 8);
+      const float4 v1 = *reinterpret_cast<const float4*>(rows + tid * 8 + 4);
+      u[0][0] = v0.x; u[0][1] = v0.y; u[0][2] = v0.z; u[0][3] = v0.w;
+      u[0][4] = v1.x; u[0][5] = v1.y; u[0][6] = v1.z; u[0][7] = v1.w;
+    }
+#pragma unroll
+    for (int e = 0; e < 8; ++e) u[0][e] = mul_rn(u[0][e], invB);
+  } else {
   // ---- margins <X_a, x>: balanced tree over the column index ---------------------------------------------------
   for (int r = 0; r < B; ++r) {
 #pragma unroll
@@ -165,20 +382,18 @@ __global__ void __launch_bounds__(IT) inner_kernel(InnerArgs a) {
   cluster.sync();
   if (tid < B) {
     const float m = smem_tree_sum(&sm.mpart[tid * MAXCS], CS);
-    const float g_cur = loss_deriv(a.loss, m, sm.yv[tid]);
-    const float g_snap = loss_deriv(a.loss, sm.msnap[tid], sm.yv[tid]);
+    const float g_cur = loss_deriv(a.loss, m, s_yv[tid]);
+    const float g_snap = loss_deriv(a.loss, s_ms[tid], s_yv[tid]);
     const float c = __fsub_rn(g_cur, g_snap);
     sm.coef[tid] = c;
     if (rank == 0) {
-      if (a.idx_tap) a.idx_tap[(int64_t)worker * B + tid] = sm.idx[tid];
+      if (a.idx_tap) a.idx_tap[(int64_t)worker * B + tid] = s_idx[tid];
       if (a.coef_tap) a.coef_tap[(int64_t)worker * B + tid] = c;
     }
   }
   __syncthreads();
 
   // ---- u = (1/B) sum_a c_a X_a, summed in batch order (Algorithm 1 step 6) ------------------------------------
-  const float invB = __fdiv_rn(1.0f, (float)B);
-  float u[MAXP][8];
 #pragma unroll
   for (int p = 0; p < MAXP; ++p) {
 #pragma unroll
@@ -194,6 +409,8 @@ __global__ void __launch_bounds__(IT) inner_kernel(InnerArgs a) {
 #pragma unroll
       for (int e = 0; e < 8; ++e) u[p][e] = mul_rn(u[p][e], invB);
     }
+  }
+
   }
 
   if (is_J) {  // double sampling: v^ = u_J + mu in full precision, nothing quantized
@@ -360,9 +577,9 @@ __global__ void __launch_bounds__(IT) inner_kernel(InnerArgs a) {
   }
 }
 
-template <int BITS>
+template <int BITS, bool STREAM>
 cudaError_t launch_t(const InnerArgs& a, size_t smem, cudaStream_t st) {
-  cudaError_t e = cudaFuncSetAttribute(inner_kernel<BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t e = cudaFuncSetAttribute(inner_kernel<BITS, STREAM>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)a.CS, (unsigned)(a.N + (a.has_J ? 1 : 0)), 1);
@@ -376,7 +593,7 @@ cudaError_t launch_t(const InnerArgs& a, size_t smem, cudaStream_t st) {
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, inner_kernel<BITS>, a);
+  return cudaLaunchKernelEx(&cfg, inner_kernel<BITS, STREAM>, a);
 }
 
 __global__ void clipped_sum_kernel(const uint32_t* __restrict__ part, int N, uint32_t* __restrict__ out) {
@@ -407,38 +624,62 @@ __global__ void mean_y_kernel(float* __restrict__ ysum, float inv_m, int d, floa
 
 }  // namespace
 
-int inner_max_b() { return MAXB; }
+int inner_max_b() { return SMAXB; }
 int inner_clipped_stride() { return MAXCS; }
 
-// Picks the cluster size and slice width.  Returns false when d is too large for the fused kernel.
-bool inner_plan(int d, int B, int want_cs, int max_smem, int* CS_out, int* SL_out, size_t* smem_out) {
+// Picks the cluster size and slice width, and whether the rows stay resident in shared memory (stages = 0) or
+// stream through a ring of `stages` stages of SG rows.  Returns false when d is too large for the fused kernel.
+bool inner_plan(int d, int B, int want_cs, int max_smem, int* CS_out, int* SL_out, size_t* smem_out, int* stages_out) {
   int P = 1;
   while (P < d) P <<= 1;
   if (P < 32) P = 32;
+  const size_t fixed = (sizeof(Smem) + 15) & ~(size_t)15;
+  if (B <= MAXB) {
+    for (int cs = 1; cs <= MAXCS; cs <<= 1) {
+      if (want_cs > 0 && cs != want_cs) continue;
+      const int SL = P / cs;
+      if (SL < 32) break;
+      if (SL > IGROUP * MAXP) continue;
+      const size_t smem = fixed + (size_t)B * SL * 4;
+      if (smem > (size_t)max_smem) continue;
+      // automatic choice: the first (smallest) cluster whose slice is covered in one pass
+      if (want_cs > 0 || SL <= IGROUP || cs == MAXCS) {
+        *CS_out = cs; *SL_out = SL; *smem_out = smem; *stages_out = 0;
+        return true;
+      }
+    }
+  }
+  if (B > SMAXB) return false;
+  // streaming: one pass per CTA (SL <= IGROUP), as many ring stages as shared memory holds
+  const size_t meta = (size_t)((B + 3) & ~3) * 16;
   for (int cs = 1; cs <= MAXCS; cs <<= 1) {
     if (want_cs > 0 && cs != want_cs) continue;
     const int SL = P / cs;
     if (SL < 32) break;
-    if (SL > IGROUP * MAXP) continue;
-    const size_t smem = ((sizeof(Smem) + 15) & ~(size_t)15) + (size_t)B * SL * 4;
-    if (smem > (size_t)max_smem) continue;
-    // automatic choice: the first (smallest) cluster whose slice is covered in one pass
-    if (want_cs > 0 || SL <= IGROUP || cs == MAXCS) {
-      *CS_out = cs; *SL_out = SL; *smem_out = smem;
-      return true;
-    }
+    if (SL > IGROUP) continue;
+    const size_t stage = (size_t)SG * SL * 4;
+    if (fixed + meta + 3 * stage > (size_t)max_smem) continue;
+    int R = (int)(((size_t)max_smem - fixed - meta) / stage);
+    if (R > SMAXR) R = SMAXR;
+    *CS_out = cs; *SL_out = SL; *smem_out = fixed + meta + (size_t)R * stage; *stages_out = R;
+    return true;
   }
   return false;
 }
 
-cudaError_t launch_inner(const InnerArgs& a, size_t smem, cudaStream_t st) {
+template <bool STREAM>
+cudaError_t launch_s(const InnerArgs& a, size_t smem, cudaStream_t st) {
   switch (a.b) {
-    case 1: return launch_t<1>(a, smem, st);
-    case 2: return launch_t<2>(a, smem, st);
-    case 4: return launch_t<4>(a, smem, st);
-    case 8: return launch_t<8>(a, smem, st);
-    default: return launch_t<0>(a, smem, st);
+    case 1: return launch_t<1, STREAM>(a, smem, st);
+    case 2: return launch_t<2, STREAM>(a, smem, st);
+    case 4: return launch_t<4, STREAM>(a, smem, st);
+    case 8: return launch_t<8, STREAM>(a, smem, st);
+    default: return launch_t<0, STREAM>(a, smem, st);
   }
+}
+
+cudaError_t launch_inner(const InnerArgs& a, size_t smem, cudaStream_t st) {
+  return a.stream_stages > 0 ? launch_s<true>(a, smem, st) : launch_s<false>(a, smem, st);
 }
 
 cudaError_t launch_clipped_sum(const uint32_t* part, int N, uint32_t* out, cudaStream_t st) {

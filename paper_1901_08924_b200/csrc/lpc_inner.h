@@ -34,6 +34,7 @@ struct InnerArgs {
   unsigned int* dev_status;
   int CS;                  // CTAs per cluster
   int SL;                  // coordinates per CTA slice
+  int stream_stages;       // 0: the B rows are resident in shared memory; > 0: they stream through that many ring stages
 };
 
 // Arguments of the persistent inner loop (lpc_persist.cu): `count` steps k_base, k_base+1, ... in one launch.
@@ -70,7 +71,7 @@ cudaError_t launch_persist(const PersistArgs& pa, size_t smem, cudaStream_t st);
 
 int inner_max_b();
 int inner_clipped_stride();
-bool inner_plan(int d, int B, int want_cs, int max_smem, int* CS_out, int* SL_out, size_t* smem_out);
+bool inner_plan(int d, int B, int want_cs, int max_smem, int* CS_out, int* SL_out, size_t* smem_out, int* stages_out);
 cudaError_t launch_inner(const InnerArgs& a, size_t smem, cudaStream_t st);
 cudaError_t launch_clipped_sum(const uint32_t* part, int N, uint32_t* out, cudaStream_t st);
 cudaError_t launch_coupling(const float* z, const float* xt, const float* y, float tau1, float tau2, int d, float* x,

@@ -19,7 +19,7 @@ CLIP_NONE, CLIP_LAMBDA, CLIP_STD = 0, 1, 2
  BUF_COEF, BUF_U, BUF_V, BUF_VHAT) = range(15)
 OPT_SAMPLE_GLOBAL, OPT_TAP_U, OPT_CLUSTER_SIZE, OPT_USE_GRAPH, OPT_PROFILE, OPT_PERSISTENT = 0, 1, 2, 3, 4, 5
 (INFO_STEP_CLUSTER_SIZE, INFO_LOOP_CLUSTER_SIZE, INFO_LOOP_LAUNCHES, INFO_SNAPSHOT_ROWS_PER_TILE, INFO_SNAPSHOT_STAGES,
- INFO_ALPC_LOOP_CLUSTER_SIZE, INFO_LOOP_ROW_BUFFERS, INFO_ALPC_LOOP_ROW_BUFFERS) = range(8)
+ INFO_ALPC_LOOP_CLUSTER_SIZE, INFO_LOOP_ROW_BUFFERS, INFO_ALPC_LOOP_ROW_BUFFERS, INFO_STEP_RING_STAGES) = range(9)
 KERNEL_NAMES = ["snapshot", "worker", "aggregate", "quant_stats", "quant_pack", "other", "inner_loop"]
 
 # every symbol that include/lpc.h declares: (name, restype, argtypes)

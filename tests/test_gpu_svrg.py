@@ -105,6 +105,9 @@ def _check_step(P, ctx, k, eta, x, xs, mu):
     dict(n=256, d=1000, N=4, B=3, b=3), dict(n=128, d=2048, N=2, B=8, b=8), dict(n=128, d=4096, N=16, B=8, b=4),
     dict(n=64, d=8192, N=4, B=16, b=2), dict(n=64, d=5000, N=2, B=4, b=1), dict(n=64, d=3000, N=2, B=4, b=32),
     dict(n=64, d=12288, N=2, B=2, b=5), dict(n=32, d=16384, N=2, B=2, b=4),
+    # minibatches larger than shared memory holds: the rows stream through the ring in batch order
+    dict(n=2048, d=1000, N=2, B=101, b=4), dict(n=1024, d=4096, N=4, B=256, b=4), dict(n=512, d=8192, N=2, B=65, b=2),
+    dict(n=4096, d=256, N=2, B=1024, b=8), dict(n=256, d=16384, N=2, B=70, b=3),
 ])
 def test_inner_step_chain_of_custody(loss, cfg):
     c = dict(cfg)
@@ -288,7 +291,7 @@ def test_multi_step_paths_equal_single_launches(cfg, mode):
 
 @pytest.mark.parametrize("loss", ["least_squares", "logistic"])
 @pytest.mark.parametrize("cfg", [dict(n=128, d=1000, N=4, B=2, b=2), dict(n=128, d=8192, N=4, B=16, b=8),
-                                 dict(n=64, d=4096, N=2, B=4, b=4)])
+                                 dict(n=64, d=4096, N=2, B=4, b=4), dict(n=1024, d=2048, N=2, B=130, b=4)])
 def test_alpc_step_chain_of_custody(loss, cfg):
     c = dict(cfg)
     P, ctx = _setup(c.pop("n"), c.pop("d"), loss, lam=1e-3, **c)
