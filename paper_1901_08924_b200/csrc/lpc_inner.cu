@@ -41,6 +41,10 @@ constexpr int SG = 4;             // rows per ring stage
 constexpr int SSLOTS = 16;        // exchange slots (a peer's margins run at most 2 * SMAXR - 2 groups ahead of this CTA's u)
 constexpr int SMAXR = 8;          // ring stages at most
 constexpr int SMAXB = 1024;       // rows per worker at most
+constexpr int SDW = 8;            // warps that take margin partial sums: SDW / SG groups in flight on that side
+constexpr int SUW = 8;            // warps that own the coordinates of u
+constexpr int SCW = 2;            // warps that form coefficients and refill stages (they alternate groups)
+constexpr int SNT = (SDW + SUW + SCW) * 32;  // threads of the streaming kernel
 
 struct Smem {
   uint64_t bar;
@@ -62,6 +66,7 @@ struct Smem {
   uint64_t sbar[SMAXR];           // stage filled (bulk-copy bytes)
   uint64_t ebar[SMAXR];           // stage consumed (one arrival per warp that adds rows into u)
   unsigned long long sx[SSLOTS][SG * MAXCS];
+  unsigned long long cw[SSLOTS][SG];  // coefficients of the groups in flight, tagged, written by this CTA's own warp
 };
 
 // Tagged 64-bit words (payload | tag << 32) stored into the shared memory of CTA `cta` of the cluster at the
@@ -74,20 +79,21 @@ __device__ __forceinline__ void st_cluster_word(const unsigned long long* slot, 
 }
 __device__ __forceinline__ unsigned long long ld_shared_word(const unsigned long long* slot) {
   unsigned long long v;
-  asm volatile("ld.relaxed.cluster.shared::cta.u64 %0, [%1];" : "=l"(v) : "r"(smem_u32(slot)) : "memory");
+  asm volatile("ld.volatile.shared::cta.u64 %0, [%1];" : "=l"(v) : "r"(smem_u32(slot)) : "memory");
   return v;
 }
 
 // BITS: 1, 2, 4, 8 fixed-width packing; 0: b from the arguments (1..16 or 32).
 // STREAM: rows pass through a ring of stages (large minibatches; one pass, SL <= IGROUP) instead of all being resident.
 template <int BITS, bool STREAM>
-__global__ void __launch_bounds__(IT) inner_kernel(InnerArgs a) {
+__global__ void __launch_bounds__(STREAM ? SNT : IT) inner_kernel(InnerArgs a) {
   cg::cluster_group cluster = cg::this_cluster();
   extern __shared__ __align__(16) unsigned char smem_raw[];
   Smem& sm = *reinterpret_cast<Smem*>(smem_raw);
   unsigned char* dyn = smem_raw + ((sizeof(Smem) + 15) & ~(size_t)15);
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  constexpr int NT = STREAM ? SNT : IT;  // the streaming path runs more warps, specialised by role
   const int rank = (int)cluster.block_rank();
   const int CS = a.CS, SL = a.SL, B = a.B, d = a.d;
   // sampled rows, their labels and cached snapshot margins; the row data (resident: B x SL; streaming: the ring)
@@ -111,7 +117,7 @@ __global__ void __launch_bounds__(IT) inner_kernel(InnerArgs a) {
   const int width = max(0, min(SL, d - c0));        // coordinates of the slice that exist
 
   // ---- sampling (Algorithm 1 step 6): slot a uses word 0 of block a of the batch stream -----------------
-  for (int slot = tid; slot < B; slot += IT) {
+  for (int slot = tid; slot < B; slot += NT) {
     int64_t lo, span;
     uint32_t tag, wk;
     if (is_J) { lo = 0; span = a.n; tag = TAG_BATCH_J; wk = 0; }
@@ -122,19 +128,21 @@ __global__ void __launch_bounds__(IT) inner_kernel(InnerArgs a) {
     s_idx[slot] = row;
     s_yv[slot] = a.y[row];
     s_ms[slot] = a.margins[row];
+    if constexpr (STREAM) s_ms[slot] = loss_deriv(a.loss, a.margins[row], s_yv[slot]);  // the snapshot side of the coefficient
   }
   if (tid == 0) {
     mbar_init(&sm.bar, 1);
     if constexpr (STREAM) {
       for (int r = 0; r < SMAXR; ++r) {
         mbar_init(&sm.sbar[r], 1);
-        mbar_init(&sm.ebar[r], IT / 32 - SG);
+        mbar_init(&sm.ebar[r], SUW);
       }
     }
     mbar_fence_init();
   }
   if constexpr (STREAM) {  // no exchange slot may look valid before a peer has written it: tags start at 1
-    for (int i = tid; i < SSLOTS * SG * MAXCS; i += IT) (&sm.sx[0][0])[i] = 0ull;
+    for (int i = tid; i < SSLOTS * SG * MAXCS; i += NT) (&sm.sx[0][0])[i] = 0ull;
+    for (int i = tid; i < SSLOTS * SG; i += NT) (&sm.cw[0][0])[i] = 0ull;
   }
   // Every CTA of the cluster announces that it is running; peers wait for this before their first
   // store into this CTA's shared memory.
@@ -188,9 +196,9 @@ __global__ void __launch_bounds__(IT) inner_kernel(InnerArgs a) {
   float u[MAXP][8];
   if constexpr (STREAM) {
     // ---- streaming: groups of SG rows in batch order through a ring of R stages, no block barrier inside.
-    // Warps 0..SG-1 take the margin partial sums (warp w: row w of every group, over the whole slice) and send
-    // them to the cluster; warps SG..7 own the coordinates of u: per group they collect the partial sums of all
-    // CTAs, form the coefficients and add the rows, then hand the stage back to be refilled. ----------------------
+    // The first SDW warps take the margin partial sums (one warp per row, over the whole slice) and send them to
+    // the cluster; the last SCW warps turn the partial sums of all CTAs into coefficients and refill the stages;
+    // the SUW warps in between own the coordinates of u and add the rows, then hand the stage back. ----------------------
 #pragma unroll
     for (int p = 0; p < MAXP; ++p) {
 #pragma unroll
@@ -212,21 +220,22 @@ __global__ void __launch_bounds__(IT) inner_kernel(InnerArgs a) {
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");  // all peers have started
     bool gave_up = false;  // after one wait ran out this thread waits no more (the status word says so)
     auto wait_stage = [&](int g) {
-      if (width > 0 && !gave_up && !mbar_wait(&sm.sbar[g % R], (uint32_t)((g / R) & 1))) {
+      if (width > 0 && !gave_up && !mbar_test(&sm.sbar[g % R], (uint32_t)((g / R) & 1)) &&
+          !mbar_wait(&sm.sbar[g % R], (uint32_t)((g / R) & 1))) {
         atomicOr(a.dev_status, DEV_TIMEOUT);
         gave_up = true;
       }
     };
     constexpr int CH = IGROUP / 8 / 32;  // 8-coordinate chunks per lane when one warp covers a slice: 8
-    constexpr int AT = IT - SG * 32;     // threads that own the coordinates of u
-    constexpr int UC = IGROUP / 8 / AT;  // chunks per such thread: 2
+    constexpr int AT = SUW * 32;         // threads that own the coordinates of u
+    constexpr int UC = IGROUP / 8 / AT;  // chunks per such thread
     float ua[UC][8];
 #pragma unroll
     for (int q = 0; q < UC; ++q)
 #pragma unroll
       for (int e = 0; e < 8; ++e) ua[q][e] = 0.f;
-    if (warp < SG) {
-      // -- margins: lane l holds x for chunks l, l+32, ..., the leaves of the tree in coordinate order are
+    if (warp < SDW) {
+      // -- margins (warp w: row w % SG of the groups g = w / SG, w / SG + SDW / SG, ...): lane l holds x for chunks l, l+32, ..., the leaves of the tree in coordinate order are
       // (chunk, element); per chunk tree8, then the tree over the 32 lanes for every chunk row, then over the rows
       float xs[CH][8];
 #pragma unroll
@@ -235,16 +244,17 @@ __global__ void __launch_bounds__(IT) inner_kernel(InnerArgs a) {
 #pragma unroll
         for (int e = 0; e < 8; ++e) xs[q][e] = (off + e < width) ? a.x[c0 + off + e] : 0.f;
       }
+      const int myrow = warp % SG;
 #pragma unroll 1
-      for (int g = 0; g < ngroups; ++g) {
+      for (int g = warp / SG; g < ngroups; g += SDW / SG) {
         const int cnt = min(SG, B - g * SG);
         wait_stage(g);
-        if (warp < cnt) {
+        if (myrow < cnt) {
           float sv[CH];
 #pragma unroll
           for (int q = 0; q < CH; ++q) {
             float v[8], pr[8];
-            row8((g % R) * SG + warp, (q * 32 + lane) * 8, v);
+            row8((g % R) * SG + myrow, (q * 32 + lane) * 8, v);
 #pragma unroll
             for (int e = 0; e < 8; ++e) pr[e] = mul_rn(v[e], xs[q][e]);
             sv[q] = tree8(pr);
@@ -255,18 +265,18 @@ __global__ void __launch_bounds__(IT) inner_kernel(InnerArgs a) {
           part = add_rn(part, __shfl_xor_sync(0xFFFFFFFFu, part, 2));
           part = add_rn(part, __shfl_xor_sync(0xFFFFFFFFu, part, 1));
           if (lane < CS)
-            st_cluster_word(&sm.sx[g % SSLOTS][warp * MAXCS + rank], (uint32_t)lane, __float_as_uint(part), (uint32_t)(g + 1));
+            st_cluster_word(&sm.sx[g % SSLOTS][myrow * MAXCS + rank], (uint32_t)lane, __float_as_uint(part), (uint32_t)(g + 1));
         }
       }
-    } else {
-      // -- u: thread t of these warps owns chunks t and t + 128 of the slice
-      const int t = tid - SG * 32;
+    } else if (warp >= SDW + SUW) {
+      // -- coefficients and refills (warp c of this side takes the groups c, c + SCW, ...): lane j collects the partial sums of row j of a group from all CTAs
+      // of the cluster and publishes the coefficient l'(m) - l'(m~) to the update side; lane 0 refills a stage as
+      // soon as the update side has handed it back.  Running in a warp of its own, the fp64 loss derivative and
+      // the barrier waits delay neither the margins nor the updates.
 #pragma unroll 1
-      for (int g = 0; g < ngroups; ++g) {
+      for (int g = warp - (SDW + SUW); g < ngroups; g += SCW) {
         const int cnt = min(SG, B - g * SG);
-        const int s = g % R;
-        float c_mine = 0.f;
-        if (lane < cnt) {  // lane j: the coefficient of row j of the group (every warp forms all of them)
+        if (lane < cnt) {
           float mp[MAXCS];
           uint64_t t0 = 0;
           for (uint32_t it = 0;; ++it) {
@@ -292,10 +302,45 @@ __global__ void __launch_bounds__(IT) inner_kernel(InnerArgs a) {
           }
           const int slot = g * SG + lane;
           const float m = (CS == 1) ? mp[0] : (CS == 2) ? add_rn(mp[0], mp[1]) : (CS == 4) ? tree4(mp[0], mp[1], mp[2], mp[3]) : tree8(mp);
-          c_mine = __fsub_rn(loss_deriv(a.loss, m, s_yv[slot]), loss_deriv(a.loss, s_ms[slot], s_yv[slot]));
-          if (rank == 0 && warp == SG) {
+          const float c = __fsub_rn(loss_deriv(a.loss, m, s_yv[slot]), s_ms[slot]);
+          st_cluster_word(&sm.cw[g % SSLOTS][lane], (uint32_t)rank, __float_as_uint(c), (uint32_t)(g + 1));
+          if (rank == 0) {
             if (a.idx_tap) a.idx_tap[(int64_t)worker * B + slot] = s_idx[slot];
-            if (a.coef_tap) a.coef_tap[(int64_t)worker * B + slot] = c_mine;
+            if (a.coef_tap) a.coef_tap[(int64_t)worker * B + slot] = c;
+          }
+        }
+        if (lane == 0 && g >= SCW && g - SCW + R < ngroups) {  // an earlier group of this warp, added into u by now
+          const int h = g - SCW;
+          if (!gave_up && !mbar_wait(&sm.ebar[h % R], (uint32_t)((h / R) & 1))) {
+            atomicOr(a.dev_status, DEV_TIMEOUT);
+            gave_up = true;
+          }
+          if (width > 0) issue(h + R);
+        }
+        __syncwarp();
+      }
+    } else {
+      // -- u: thread t of these warps owns chunk t (+ AT, ...) of the slice
+      const int t = tid - SDW * 32;
+#pragma unroll 1
+      for (int g = 0; g < ngroups; ++g) {
+        const int cnt = min(SG, B - g * SG);
+        const int s = g % R;
+        float c_mine = 0.f;
+        if (lane < cnt) {  // lane j fetches the coefficient of row j
+          uint64_t t0 = 0;
+          for (uint32_t it = 0;; ++it) {
+            const unsigned long long w = ld_shared_word(&sm.cw[g % SSLOTS][lane]);
+            c_mine = __uint_as_float((uint32_t)w);
+            if ((uint32_t)(w >> 32) == (uint32_t)(g + 1) || gave_up) break;
+            if ((it & 63u) == 63u) {
+              const uint64_t now = global_ns();
+              if (t0 == 0) t0 = now;
+              else if (now - t0 > 2000000000ull) {
+                atomicOr(a.dev_status, DEV_TIMEOUT);
+                gave_up = true;
+              }
+            }
           }
         }
         __syncwarp();
@@ -313,21 +358,13 @@ __global__ void __launch_bounds__(IT) inner_kernel(InnerArgs a) {
             }
           }
         }
-        // hand the stage back: when all warps of this side are done with it, one thread refills it
         __syncwarp();
-        if (lane == 0) mbar_arrive(&sm.ebar[s]);
-        if (t == 0 && g + R < ngroups) {
-          if (!gave_up && !mbar_wait(&sm.ebar[s], (uint32_t)((g / R) & 1))) {
-            atomicOr(a.dev_status, DEV_TIMEOUT);
-            gave_up = true;
-          }
-          if (width > 0) issue(g + R);
-        }
+        if (lane == 0) mbar_arrive(&sm.ebar[s]);  // this warp is done with the stage
       }
     }
     __syncthreads();  // both sides are done with the ring: it now carries u to the usual owner of each coordinate
-    if (warp >= SG) {
-      const int t = tid - SG * 32;
+    if (warp >= SDW && warp < SDW + SUW) {
+      const int t = tid - SDW * 32;
 #pragma unroll
       for (int q = 0; q < UC; ++q) {
         if ((q * AT + t) * 8 < SL) {  // the ring holds at least one slice
@@ -338,7 +375,7 @@ __global__ void __launch_bounds__(IT) inner_kernel(InnerArgs a) {
       }
     }
     __syncthreads();
-    if (tid * 8 < SL) {
+    if (tid < IT && tid * 8 < SL) {
       const float4 v0 = *reinterpret_cast<const float4*>(rows + tid * 8);
       const float4 v1 = *reinterpret_cast<const float4*>(rows + tid * 8 + 4);
       u[0][0] = v0.x; u[0][1] = v0.y; u[0][2] = v0.z; u[0][3] = v0.w;
@@ -450,12 +487,12 @@ __global__ void __launch_bounds__(IT) inner_kernel(InnerArgs a) {
         for (int e = 0; e < 8; ++e) sq[e] = mul_rn(u[p][e], u[p][e]);
         const float s1 = warp_tree_sum(tree8(u[p]));
         const float s2 = warp_tree_sum(tree8(sq));
-        if (lane == 0) { sm.ws1[p * 8 + warp] = s1; sm.ws2[p * 8 + warp] = s2; }
+        if (lane == 0 && warp < IT / 32) { sm.ws1[p * 8 + warp] = s1; sm.ws2[p * 8 + warp] = s2; }
       }
     }
   }
   mx = warp_max_u32(mx);
-  if (lane == 0) sm.wmax[warp] = mx;
+  if (lane == 0 && warp < IT / 32) sm.wmax[warp] = mx;
   __syncthreads();
   if (tid == 0) {
     uint32_t m = 0;
@@ -558,17 +595,17 @@ __global__ void __launch_bounds__(IT) inner_kernel(InnerArgs a) {
     } else {
       if (p > 0) __syncthreads();
       for (int i = 0; i < b; ++i)
-        sm.stage[tid * b + i] = (uint8_t)((i < 8) ? (lo >> (8 * i)) : (hi >> (8 * (i - 8))));
+        if (tid < IT) sm.stage[tid * b + i] = (uint8_t)((i < 8) ? (lo >> (8 * i)) : (hi >> (8 * (i - 8))));
       __syncthreads();
       const int span = min(IGROUP, SL - p * IGROUP);           // coordinates of this pass (multiple of 32)
       const int64_t w0 = (int64_t)((c0 + p * IGROUP) >> 5) * b;  // exact: the pass starts on a multiple of 32
       const uint32_t* st = reinterpret_cast<const uint32_t*>(sm.stage);
-      for (int w = tid; w < (span / 32) * b; w += IT)
+      for (int w = tid; w < (span / 32) * b && tid < IT; w += IT)
         if (w0 + w < a.pad_words) out[w0 + w] = st[w];
     }
   }
   nclip = __reduce_add_sync(0xFFFFFFFFu, nclip);
-  if (lane == 0) sm.wclip[warp] = nclip;
+  if (lane == 0 && warp < IT / 32) sm.wclip[warp] = nclip;
   __syncthreads();
   if (tid == 0) {
     uint32_t t = 0;
@@ -583,7 +620,7 @@ cudaError_t launch_t(const InnerArgs& a, size_t smem, cudaStream_t st) {
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)a.CS, (unsigned)(a.N + (a.has_J ? 1 : 0)), 1);
-  cfg.blockDim = dim3(IT, 1, 1);
+  cfg.blockDim = dim3(STREAM ? SNT : IT, 1, 1);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
