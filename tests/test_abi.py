@@ -57,7 +57,7 @@ def test_init_rejects_bad_arguments_before_touching_the_device(lpc):
         dict(N=0), dict(N=2000), dict(b=0), dict(b=17), dict(b=31), dict(clip_mode=5),
         dict(clip_mode=lpc.CLIP_LAMBDA, clip_value=1.5), dict(clip_mode=lpc.CLIP_LAMBDA, clip_value=0.0),
         dict(clip_mode=lpc.CLIP_STD, clip_value=-1.0), dict(lam=-1.0), dict(d=1002), dict(d=2), dict(d=32768),
-        dict(n=4001), dict(B=0), dict(B=100), dict(loss=7), dict(X=C.c_void_p((1 << 20) + 4)),
+        dict(n=4001), dict(B=0), dict(B=1025), dict(loss=7), dict(X=C.c_void_p((1 << 20) + 4)),
     ]
     for kw in bad:
         a = dict(X=fake, y=fake, n=4000, d=1000, loss=0, lam=1e-4, N=4, B=1, b=2, clip_mode=2, clip_value=2.5)
