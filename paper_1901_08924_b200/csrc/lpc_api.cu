@@ -840,3 +840,10 @@ int lpc_svrg_run_host(const float* X_host, const float* y_host, int64_t n, int32
 }
 
 }  // extern "C"
+
+#ifdef LPC_TRACE
+namespace lpc { cudaError_t read_stream_trace(unsigned long long* host_out); }
+extern "C" int lpc_debug_stream_trace(unsigned long long* host_out) {
+  return lpc::read_stream_trace(host_out) == cudaSuccess ? LPC_OK : LPC_ERR_CUDA;
+}
+#endif

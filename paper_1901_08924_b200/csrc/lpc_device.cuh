@@ -27,10 +27,9 @@ __device__ __forceinline__ U4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c
                                             uint32_t k0, uint32_t k1) {
 #pragma unroll
   for (int r = 0; r < 10; ++r) {
-    const uint64_t p0 = (uint64_t)0xD2511F53u * (uint64_t)c0;  // one wide multiply gives both halves
-    const uint64_t p1 = (uint64_t)0xCD9E8D57u * (uint64_t)c2;
-    const uint32_t hi0 = (uint32_t)(p0 >> 32), lo0 = (uint32_t)p0;
-    const uint32_t hi1 = (uint32_t)(p1 >> 32), lo1 = (uint32_t)p1;
+    // the two halves of each 32x32 product as separate multiplies: fewer instructions here than the 64-bit form
+    const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
     c0 = hi1 ^ c1 ^ k0;
     c1 = lo1;
     c2 = hi0 ^ c3 ^ k1;
@@ -186,27 +185,54 @@ __device__ __forceinline__ Scale make_scale(uint32_t max_bits, float S1, float S
 // frac(s) = s - floor(s), taken exactly (rule 1):   up  <=>  r16 + 0.5 < frac(s) * 65536.
 //
 // The decision is evaluated in fixed point, exactly and with few instructions (the quantize pass is bound
-// by instruction issue).  Z = ceil(s * 2^17) is exact (a power-of-two scaling and one conversion).  Then
+// by instruction issue, and there by the integer/logic pipe).  With Z = ceil(s * 2^17), which is exact
+// (a power-of-two scaling and one directed rounding),
 //   A := ceil(s * 65536 - 1/2) = floor(Z / 2),
 //   r16 + 1/2 < frac(s) * 65536   <=>   r16 < A - 65536 * floor(s)          (r16 is an integer),
-//   floor(s) + [r16 < A - 65536 floor(s)] = floor((A + 65535 - r16) / 65536)  (0 <= r16 <= 65535),
-// and both floors are arithmetic right shifts.
+//   floor(s) + [r16 < A - 65536 floor(s)] = floor((A + 65535 - r16) / 65536)  (0 <= r16 <= 65535)
+//                                         = floor((Z + 131070 - 2 r16) / 2^17),
+// and the floor is a right shift.
+//
+// b <= 4: Z is formed in the mantissa of a float instead of by a conversion.  One fused multiply-add with
+// round-up, t = RU(s * 2^17 + K), has an exact product and a single directed rounding; K is an integer
+// that keeps t inside the binade [2^23, 2^24) where floats are the integers, so t = K + Z and the bit
+// pattern of t is bits(K) + Z.  K also carries the constants 131070 and 2^17 * 2^(b-1), and bits(1.5 * 2^23)
+// = 0x4B400000 = 0x25A0 * 2^17, hence
+//   (bits(t) - 2 r16) >> 17  =  0x25A0 + code,        code = floor(s) + up + 2^(b-1).
+// quantize_raw returns that biased value; QRAW_BIAS is removed once per packed word.
+constexpr uint32_t QRAW_BIAS = 0x25A0u;
+
+template <int B_>
+__device__ __forceinline__ uint32_t quantize_raw(float u, float rdelta, uint32_t r16) {
+  static_assert(B_ >= 1 && B_ <= 4, "the mantissa form covers b <= 4");
+  float s = mul_rn(u, rdelta);
+  if constexpr (B_ == 1) {
+    // two code points: position between them ((s + 1) / 2) * 65536 = (s + 1) * 32768, s + 1 rounded to fp32
+    s = add_rn(fminf(fmaxf(s, -1.f), 1.f), 1.f);
+    const float t = __fmaf_ru(s, 65536.f, 12582912.f + 131070.f);
+    return (__float_as_uint(t) - 2u * r16) >> 17;
+  } else {
+    constexpr float lo = -(float)(1 << (B_ - 1));
+    constexpr float hi = (float)((1 << (B_ - 1)) - 1);
+    constexpr float K = 12582912.f + 131070.f + (float)(131072 << (B_ - 1));
+    s = fminf(fmaxf(s, lo), hi);  // projection onto the hull (rule 2)
+    const float t = __fmaf_ru(s, 131072.f, K);
+    return (__float_as_uint(t) - 2u * r16) >> 17;
+  }
+}
+
 template <int B_>
 __device__ __forceinline__ uint32_t quantize_code(float u, float rdelta, uint32_t r16) {
   static_assert(B_ >= 1 && B_ <= 8, "32-bit fixed point covers b <= 8");
-  if constexpr (B_ == 1) {
-    float s = mul_rn(u, rdelta);
-    s = fminf(fmaxf(s, -1.f), 1.f);
-    // position between the two code points, ((s + 1) / 2) * 65536 = (s + 1) * 32768 with s + 1 rounded to fp32
-    const int A = __float2int_ru(mul_rn(add_rn(s, 1.f), 65536.f)) >> 1;  // ceil(t - 1/2), in [0, 65536]
-    return ((int)r16 < A) ? 1u : 0u;
+  if constexpr (B_ <= 4) {
+    return quantize_raw<B_>(u, rdelta, r16) - QRAW_BIAS;
   } else {
     constexpr float lo = -(float)(1 << (B_ - 1));
     constexpr float hi = (float)((1 << (B_ - 1)) - 1);
     float s = mul_rn(u, rdelta);
-    s = fminf(fmaxf(s, lo), hi);  // projection onto the hull (rule 2)
-    const int A = __float2int_ru(mul_rn(s, 131072.f)) >> 1;
-    return (uint32_t)((A + (65535 + (65536 << (B_ - 1))) - (int)r16) >> 16);  // floor(s) + up + 2^(b-1)
+    s = fminf(fmaxf(s, lo), hi);
+    const int Z = __float2int_ru(mul_rn(s, 131072.f));
+    return (uint32_t)((Z + (131070 + (131072 << (B_ - 1))) - 2 * (int)r16) >> 17);
   }
 }
 
@@ -273,6 +299,43 @@ __device__ __forceinline__ float soft_threshold(float w, float kappa) {
 __device__ __forceinline__ uint32_t lane16(const U4& r, int e) {
   const uint32_t w = (e < 2) ? r.x : (e < 4) ? r.y : (e < 6) ? r.z : r.w;
   return (e & 1) ? (w >> 16) : (w & 0xFFFFu);
+}
+
+// One more coordinate outside the hull [lower, T]: two compares and a predicated float add, which keeps the
+// count off the integer pipe (exact: a thread counts far fewer than 2^24 coordinates).
+__device__ __forceinline__ void count_outside(float& cnt, float u, float T, float lower) {
+  asm("{\n\t.reg .pred p;\n\t"
+      "setp.gt.f32 p, %1, %2;\n\t"
+      "setp.lt.or.f32 p, %1, %3, p;\n\t"
+      "@p add.rn.f32 %0, %0, 0f3F800000;\n\t}"
+      : "+f"(cnt)
+      : "f"(u), "f"(T), "f"(lower));
+}
+
+// The 8 * BITS packed bits of one coordinate group (code e in bits [e BITS, (e+1) BITS)) from its eight values
+// and its Philox block; `cnt` grows by the number of values outside the hull when COUNT is set.
+template <int BITS, bool COUNT>
+__device__ __forceinline__ uint64_t quantize_group8(const float* v, float rdelta, const U4& r, float T, float lower,
+                                                    float& cnt) {
+  static_assert(BITS == 1 || BITS == 2 || BITS == 4 || BITS == 8, "fixed widths only");
+  uint32_t w0 = 0, w1 = 0;
+#pragma unroll
+  for (int e = 0; e < 8; ++e) {
+    if (COUNT) count_outside(cnt, v[e], T, lower);
+    uint32_t c;
+    if constexpr (BITS <= 4) c = quantize_raw<BITS>(v[e], rdelta, lane16(r, e));  // biased by QRAW_BIAS
+    else c = quantize_code<BITS>(v[e], rdelta, lane16(r, e));
+    // multiply-add form: the shift rides on the multiplier pipe, and biased values may carry into higher fields
+    if (e * BITS < 32) w0 += c * (1u << ((e * BITS) & 31));
+    else w1 += c * (1u << ((e * BITS) & 31));
+  }
+  if constexpr (BITS <= 4) {
+    uint32_t bias = 0;  // sum of the biases at the eight field positions, modulo 2^32
+#pragma unroll
+    for (int e = 0; e < 8; ++e) bias += QRAW_BIAS << (e * BITS);
+    w0 -= bias;
+  }
+  return (uint64_t)w0 | ((uint64_t)w1 << 32);
 }
 
 // ---- mbarrier / bulk-copy (TMA) wrappers ---------------------------------------------------------------

@@ -83,6 +83,17 @@ __device__ __forceinline__ unsigned long long ld_shared_word(const unsigned long
   return v;
 }
 
+// Phase timestamps of the streaming path of one CTA, for latency studies; compiled in only with -DLPC_TRACE.
+#ifdef LPC_TRACE
+__device__ unsigned long long g_stream_trace[64 * 8];
+#define LPC_STREAM_MARK(g, i)                                                                       \
+  do {                                                                                              \
+    if (blockIdx.x == 0 && blockIdx.y == 0 && (g) < 64) g_stream_trace[(g) * 8 + (i)] = global_ns(); \
+  } while (0)
+#else
+#define LPC_STREAM_MARK(g, i) do { } while (0)
+#endif
+
 // BITS: 1, 2, 4, 8 fixed-width packing; 0: b from the arguments (1..16 or 32).
 // STREAM: rows pass through a ring of stages (large minibatches; one pass, SL <= IGROUP) instead of all being resident.
 template <int BITS, bool STREAM>
@@ -213,6 +224,7 @@ __global__ void __launch_bounds__(STREAM ? SNT : IT) inner_kernel(InnerArgs a) {
       mbar_expect_tx(&sm.sbar[s], row_bytes * (uint32_t)cnt);
       for (int j = 0; j < cnt; ++j)
         bulk_load(rows + ((size_t)s * SG + j) * SL, a.X + s_idx[g * SG + j] * (int64_t)d + c0, row_bytes, &sm.sbar[s]);
+      LPC_STREAM_MARK(g, 6);
     };
     if (tid == 0 && width > 0) {
       for (int g = 0; g < min(R, ngroups); ++g) issue(g);
@@ -249,6 +261,7 @@ __global__ void __launch_bounds__(STREAM ? SNT : IT) inner_kernel(InnerArgs a) {
       for (int g = warp / SG; g < ngroups; g += SDW / SG) {
         const int cnt = min(SG, B - g * SG);
         wait_stage(g);
+        if (myrow == 0 && lane == 0) LPC_STREAM_MARK(g, 0);
         if (myrow < cnt) {
           float sv[CH];
 #pragma unroll
@@ -266,6 +279,7 @@ __global__ void __launch_bounds__(STREAM ? SNT : IT) inner_kernel(InnerArgs a) {
           part = add_rn(part, __shfl_xor_sync(0xFFFFFFFFu, part, 1));
           if (lane < CS)
             st_cluster_word(&sm.sx[g % SSLOTS][myrow * MAXCS + rank], (uint32_t)lane, __float_as_uint(part), (uint32_t)(g + 1));
+          if (myrow == 0 && lane == 0) LPC_STREAM_MARK(g, 1);
         }
       }
     } else if (warp >= SDW + SUW) {
@@ -300,10 +314,12 @@ __global__ void __launch_bounds__(STREAM ? SNT : IT) inner_kernel(InnerArgs a) {
               }
             }
           }
+          if (lane == 0) LPC_STREAM_MARK(g, 2);
           const int slot = g * SG + lane;
           const float m = (CS == 1) ? mp[0] : (CS == 2) ? add_rn(mp[0], mp[1]) : (CS == 4) ? tree4(mp[0], mp[1], mp[2], mp[3]) : tree8(mp);
           const float c = __fsub_rn(loss_deriv(a.loss, m, s_yv[slot]), s_ms[slot]);
           st_cluster_word(&sm.cw[g % SSLOTS][lane], (uint32_t)rank, __float_as_uint(c), (uint32_t)(g + 1));
+          if (lane == 0) LPC_STREAM_MARK(g, 3);
           if (rank == 0) {
             if (a.idx_tap) a.idx_tap[(int64_t)worker * B + slot] = s_idx[slot];
             if (a.coef_tap) a.coef_tap[(int64_t)worker * B + slot] = c;
@@ -345,6 +361,7 @@ __global__ void __launch_bounds__(STREAM ? SNT : IT) inner_kernel(InnerArgs a) {
         }
         __syncwarp();
         wait_stage(g);
+        if (t == 0) LPC_STREAM_MARK(g, 4);
 #pragma unroll
         for (int j = 0; j < SG; ++j) {
           const float c = __shfl_sync(0xFFFFFFFFu, c_mine, j);
@@ -360,6 +377,7 @@ __global__ void __launch_bounds__(STREAM ? SNT : IT) inner_kernel(InnerArgs a) {
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(&sm.ebar[s]);  // this warp is done with the stage
+        if (t == 0) LPC_STREAM_MARK(g, 5);
       }
     }
     __syncthreads();  // both sides are done with the ring: it now carries u to the usual owner of each coordinate
@@ -718,6 +736,12 @@ cudaError_t launch_s(const InnerArgs& a, size_t smem, cudaStream_t st) {
 cudaError_t launch_inner(const InnerArgs& a, size_t smem, cudaStream_t st) {
   return a.stream_stages > 0 ? launch_s<true>(a, smem, st) : launch_s<false>(a, smem, st);
 }
+
+#ifdef LPC_TRACE
+cudaError_t read_stream_trace(unsigned long long* host_out) {
+  return cudaMemcpyFromSymbol(host_out, g_stream_trace, sizeof(unsigned long long) * 64 * 8);
+}
+#endif
 
 cudaError_t launch_clipped_sum(const uint32_t* part, int N, uint32_t* out, cudaStream_t st) {
   clipped_sum_kernel<<<(N + 127) / 128, 128, 0, st>>>(part, N, out);

@@ -152,9 +152,80 @@ __global__ void __launch_bounds__(QT) finish_kernel(QuantArgs a) {
 // BITS = 1, 2, 4, 8: register/shuffle packing with direct coalesced stores.
 // BITS = 0: any b in 1..16 read from the arguments; each thread's 8*b bits are b whole bytes, staged
 //           through shared memory and written out as words.
+// A CTA takes a run of QRUN consecutive tiles of one worker.  Runs that consist of whole tiles of one segment of
+// 16-byte aligned vectors (all but a segment's last tiles) go through a software-pipelined loop: the loads of the
+// next sweeps are in flight while the current ones are quantized, nothing is tested per group and every index is a
+// small offset from the run's base.  Everything else goes tile by tile through the general code.
+constexpr int QRUN = 8;
+
+template <int BITS>
+__device__ __forceinline__ void store_group(uint32_t* __restrict__ ot, int g, int lane, uint64_t lo) {
+  if (BITS == 8) {
+    *reinterpret_cast<uint2*>(ot + 2 * g) = make_uint2((uint32_t)lo, (uint32_t)(lo >> 32));
+  } else if (BITS == 4) {
+    ot[g] = (uint32_t)lo;
+  } else if (BITS == 2) {
+    const uint32_t next = __shfl_down_sync(0xFFFFFFFFu, (uint32_t)lo, 1);
+    if ((lane & 1) == 0) ot[g >> 1] = (uint32_t)lo | (next << 16);
+  } else {
+    const uint32_t mine = (uint32_t)lo;
+    const uint32_t n1 = __shfl_down_sync(0xFFFFFFFFu, mine, 1);
+    const uint32_t n2 = __shfl_down_sync(0xFFFFFFFFu, mine, 2);
+    const uint32_t n3 = __shfl_down_sync(0xFFFFFFFFu, mine, 3);
+    if ((lane & 3) == 0) ot[g >> 2] = mine | (n1 << 8) | (n2 << 16) | (n3 << 24);
+  }
+}
+
+// `nsweeps` sweeps of QGROUP coordinates from pt/qt (this thread's first group); HAS_Q: u = p - q.
+// A step covers SW sweeps (2 without a subtrahend, 1 with), i.e. four 16-byte loads per thread; the loads of step
+// i + 1 are issued before step i is quantized.
+template <int BITS, bool COUNT, bool HAS_Q>
+__device__ __forceinline__ void quantize_run(const QuantArgs& a, const ScaleRec& sc, const float* __restrict__ pt,
+                                             const float* __restrict__ qt, uint32_t block0, uint32_t* __restrict__ ot,
+                                             int nsweeps, int worker, int tid, int lane, float& fclip) {
+  constexpr int SW = HAS_Q ? 1 : 2;
+  const int nsteps = nsweeps / SW;  // a tile has QITER = 4 sweeps, so this is exact
+  float4 cur[4], nxt[4];
+  auto load = [&](float4* dst, int step) {
+#pragma unroll
+    for (int w = 0; w < SW; ++w) {
+      const int off = (step * SW + w) * QGROUP;
+      dst[2 * w] = __ldcs(reinterpret_cast<const float4*>(pt + off));
+      dst[2 * w + 1] = __ldcs(reinterpret_cast<const float4*>(pt + off + 4));
+      if (HAS_Q) {
+        dst[2] = __ldcs(reinterpret_cast<const float4*>(qt + off));
+        dst[3] = __ldcs(reinterpret_cast<const float4*>(qt + off + 4));
+      }
+    }
+  };
+  auto work = [&](const float4* src, int step) {
+#pragma unroll
+    for (int w = 0; w < SW; ++w) {
+      float v[8] = {src[2 * w].x, src[2 * w].y, src[2 * w].z, src[2 * w].w,
+                    src[2 * w + 1].x, src[2 * w + 1].y, src[2 * w + 1].z, src[2 * w + 1].w};
+      if (HAS_Q) {
+        v[0] = __fsub_rn(v[0], src[2].x); v[1] = __fsub_rn(v[1], src[2].y); v[2] = __fsub_rn(v[2], src[2].z);
+        v[3] = __fsub_rn(v[3], src[2].w); v[4] = __fsub_rn(v[4], src[3].x); v[5] = __fsub_rn(v[5], src[3].y);
+        v[6] = __fsub_rn(v[6], src[3].z); v[7] = __fsub_rn(v[7], src[3].w);
+      }
+      const int g = (step * SW + w) * (QGROUP / 8) + tid;  // coordinate group inside the run
+      const U4 r = stream_block(a.seed, TAG_ROUND, (uint32_t)worker, a.k, block0 + (uint32_t)g);
+      const uint64_t lo = quantize_group8<BITS, COUNT>(v, sc.rdelta, r, sc.T, sc.lower, fclip);
+      store_group<BITS>(ot, g, lane, lo);
+    }
+  };
+  load(cur, 0);
+#pragma unroll 1
+  for (int step = 0; step < nsteps; step += 2) {  // nsteps is even: a tile is 2 or 4 steps
+    load(nxt, step + 1);
+    work(cur, step);
+    if (step + 2 < nsteps) load(cur, step + 2);
+    work(nxt, step + 1);
+  }
+}
+
 template <int BITS, bool COUNT>
-__global__ void __launch_bounds__(QT) quantize_kernel(QuantArgs a) {
-  const int tile = blockIdx.x, worker = blockIdx.y;
+__device__ __forceinline__ void quantize_tile(const QuantArgs& a, int tile, int worker, uint8_t* stage) {
   const int seg = a.tile_seg ? a.tile_seg[tile] : 0;
   const SegInfo s = a.segs[seg];
   const int64_t tstart = (int64_t)(tile - s.tile_first) * TILE;
@@ -168,9 +239,8 @@ __global__ void __launch_bounds__(QT) quantize_kernel(QuantArgs a) {
   const uint32_t zero_code = (b == 1) ? 0u : (1u << (b - 1));
   uint32_t* out = a.codes + (int64_t)worker * a.stride_words + s.word_off;
 
-  __shared__ __align__(16) uint8_t stage[BITS == 0 ? QT * 16 : 16];
-
   uint32_t nclip = 0;
+  float fclip = 0.f;
 #pragma unroll
   for (int it = 0; it < QITER; ++it) {
     const int64_t sweep0 = tstart + (int64_t)it * QGROUP;  // first coordinate of this sweep (segment-local)
@@ -183,16 +253,9 @@ __global__ void __launch_bounds__(QT) quantize_kernel(QuantArgs a) {
       if (!degenerate) {
         const U4 r = stream_block(a.seed, TAG_ROUND, (uint32_t)worker, a.k, s.block_base + (uint32_t)(j >> 3));
         if constexpr (BITS != 0) {
-          // all eight coordinates are computed without bounds tests; codes past the end are masked off below
-          uint32_t w0 = 0, w1 = 0;
-#pragma unroll
-          for (int e = 0; e < 8; ++e) {
-            const uint32_t code = quantize_code<BITS ? BITS : 1>(v[e], sc.rdelta, lane16(r, e));
-            if (COUNT) nclip += (v[e] > sc.T || v[e] < sc.lower) ? 1u : 0u;  // zero padding is never counted
-            if (e * BITS < 32) w0 += code << ((e * BITS) & 31);
-            else w1 += code << ((e * BITS) & 31);
-          }
-          lo = (uint64_t)w0 | ((uint64_t)w1 << 32);
+          // all eight coordinates are computed without bounds tests (zero padding is inside the hull and is
+          // never counted); codes past the end are masked off below
+          lo = quantize_group8<BITS ? BITS : 1, COUNT>(v, sc.rdelta, r, sc.T, sc.lower, fclip);
           if (nvalid < 8) lo &= (1ull << (nvalid * BITS)) - 1ull;
         } else {
 #pragma unroll
@@ -253,9 +316,48 @@ __global__ void __launch_bounds__(QT) quantize_kernel(QuantArgs a) {
         if (w0 + w < s.pad_words) out[w0 + w] = st[w];
     }
   }
-  nclip = __reduce_add_sync(0xFFFFFFFFu, nclip);
+  nclip = __reduce_add_sync(0xFFFFFFFFu, nclip + (uint32_t)fclip);
   if (COUNT && lane == 0 && nclip) atomicAdd(&a.clipped_out[(int64_t)worker * a.nseg + seg], nclip);
 }
+
+template <int BITS, bool COUNT>
+__global__ void __launch_bounds__(QT, 4) quantize_kernel(QuantArgs a) {
+  const int worker = blockIdx.y;
+  const int tile0 = blockIdx.x * QRUN;
+  const int ntl = min(QRUN, a.ntiles - tile0);
+  __shared__ __align__(16) uint8_t stage[BITS == 0 ? QT * 16 : 16];
+  if constexpr (BITS != 0) {
+    const int seg = a.tile_seg ? a.tile_seg[tile0] : 0;
+    const int seg_last = a.tile_seg ? a.tile_seg[tile0 + ntl - 1] : 0;  // tiles are numbered segment by segment
+    if (seg == seg_last) {
+      const SegInfo s = a.segs[seg];
+      const int64_t tstart = (int64_t)(tile0 - s.tile_first) * TILE;
+      const float* p = a.U + (int64_t)worker * a.ld + s.off;
+      const float* q = a.U_sub ? a.U_sub + (int64_t)worker * a.ld + s.off : nullptr;
+      const ScaleRec sc = a.scales[(int64_t)worker * a.nseg + seg];
+      if (aligned16(p) && (!q || aligned16(q)) && !(sc.flags & 1u) && tstart + (int64_t)ntl * TILE <= s.len) {
+        const int tid = threadIdx.x, lane = tid & 31;
+        const uint32_t block0 = s.block_base + (uint32_t)(tstart >> 3);
+        uint32_t* ot = a.codes + (int64_t)worker * a.stride_words + s.word_off + (tstart >> 5) * BITS;
+        float fclip = 0.f;
+        if (q)
+          quantize_run<BITS ? BITS : 1, COUNT, true>(a, sc, p + tstart + tid * 8, q + tstart + tid * 8, block0, ot,
+                                                     ntl * QITER, worker, tid, lane, fclip);
+        else
+          quantize_run<BITS ? BITS : 1, COUNT, false>(a, sc, p + tstart + tid * 8, nullptr, block0, ot, ntl * QITER,
+                                                      worker, tid, lane, fclip);
+        const uint32_t nclip = __reduce_add_sync(0xFFFFFFFFu, (uint32_t)fclip);
+        if (COUNT && lane == 0 && nclip) atomicAdd(&a.clipped_out[(int64_t)worker * a.nseg + seg], nclip);
+        return;
+      }
+    }
+  }
+  for (int t = 0; t < ntl; ++t) {
+    if (BITS == 0 && t > 0) __syncthreads();  // the staging buffer is reused from tile to tile
+    quantize_tile<BITS, COUNT>(a, tile0 + t, worker, stage);
+  }
+}
+
 
 // b = 32: the message is the vector itself (clamped to [-T, T] when a clip rule is set).
 __global__ void __launch_bounds__(QT) bypass_kernel(QuantArgs a) {
@@ -320,23 +422,25 @@ cudaError_t launch_quantize_pack(const QuantArgs& a, cudaStream_t st, LaunchHook
     ~Close() { if (h) h(u, 4, 0); }
   } close_{hook, user};
   if (hook) hook(user, 4 /* LPC_KERNEL_QUANT_PACK */, 1);
+  const dim3 grid_tiles = grid;  // one tile per CTA: the statistics pass and the full-precision bypass
+  const dim3 grid_runs((unsigned)((a.ntiles + QRUN - 1) / QRUN), (unsigned)a.N);  // QRUN tiles per CTA
   if (a.count_clipped) {
     switch (a.b) {
-      case 1: quantize_kernel<1, true><<<grid, block, 0, st>>>(a); break;
-      case 2: quantize_kernel<2, true><<<grid, block, 0, st>>>(a); break;
-      case 4: quantize_kernel<4, true><<<grid, block, 0, st>>>(a); break;
-      case 8: quantize_kernel<8, true><<<grid, block, 0, st>>>(a); break;
-      case 32: bypass_kernel<<<grid, block, 0, st>>>(a); break;
-      default: quantize_kernel<0, true><<<grid, block, 0, st>>>(a); break;
+      case 1: quantize_kernel<1, true><<<grid_runs, block, 0, st>>>(a); break;
+      case 2: quantize_kernel<2, true><<<grid_runs, block, 0, st>>>(a); break;
+      case 4: quantize_kernel<4, true><<<grid_runs, block, 0, st>>>(a); break;
+      case 8: quantize_kernel<8, true><<<grid_runs, block, 0, st>>>(a); break;
+      case 32: bypass_kernel<<<grid_tiles, block, 0, st>>>(a); break;
+      default: quantize_kernel<0, true><<<grid_runs, block, 0, st>>>(a); break;
     }
   } else {
     switch (a.b) {
-      case 1: quantize_kernel<1, false><<<grid, block, 0, st>>>(a); break;
-      case 2: quantize_kernel<2, false><<<grid, block, 0, st>>>(a); break;
-      case 4: quantize_kernel<4, false><<<grid, block, 0, st>>>(a); break;
-      case 8: quantize_kernel<8, false><<<grid, block, 0, st>>>(a); break;
-      case 32: bypass_kernel<<<grid, block, 0, st>>>(a); break;
-      default: quantize_kernel<0, false><<<grid, block, 0, st>>>(a); break;
+      case 1: quantize_kernel<1, false><<<grid_runs, block, 0, st>>>(a); break;
+      case 2: quantize_kernel<2, false><<<grid_runs, block, 0, st>>>(a); break;
+      case 4: quantize_kernel<4, false><<<grid_runs, block, 0, st>>>(a); break;
+      case 8: quantize_kernel<8, false><<<grid_runs, block, 0, st>>>(a); break;
+      case 32: bypass_kernel<<<grid_tiles, block, 0, st>>>(a); break;
+      default: quantize_kernel<0, false><<<grid_runs, block, 0, st>>>(a); break;
     }
   }
   return cudaGetLastError();
