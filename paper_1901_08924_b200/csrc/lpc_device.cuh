@@ -364,7 +364,12 @@ __device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait: returns false when the phase did not complete within about two seconds.
+// Bounded wait: returns false when the phase did not complete within about two seconds.  One try suspends the
+// thread for at most LPC_WAIT_HINT_NS nanoseconds before it looks again: with the system's default limit a waiter
+// noticed a completed phase more than a microsecond late.
+#ifndef LPC_WAIT_HINT_NS
+#define LPC_WAIT_HINT_NS 100u
+#endif
 __device__ __forceinline__ uint64_t global_ns() {
   uint64_t t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
@@ -377,10 +382,10 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint64
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
-        : "r"(addr), "r"(parity)
+        : "r"(addr), "r"(parity), "r"(LPC_WAIT_HINT_NS)
         : "memory");
     if (ok) return true;
     if ((it & 255u) == 255u) {
@@ -389,6 +394,38 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint64
       else if (now - t0 > limit_ns) return false;
     }
   }
+}
+// Same bounded wait with acquire semantics at cluster scope: for phases completed by stores of other CTAs of the
+// cluster (st_async_cluster below).
+__device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity, uint64_t limit_ns = 2000000000ull) {
+  const uint32_t addr = smem_u32(bar);
+  uint64_t t0 = 0;
+  for (uint32_t it = 0;; ++it) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(addr), "r"(parity), "r"(LPC_WAIT_HINT_NS)
+        : "memory");
+    if (ok) return true;
+    if ((it & 255u) == 255u) {
+      const uint64_t now = global_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > limit_ns) return false;
+    }
+  }
+}
+// A 32-bit store into the shared memory of CTA `cta` of the cluster, at the address `slot` has in this CTA, that
+// counts 4 bytes on that CTA's mbarrier `bar` (same offset there) when it lands: data and signal in one message.
+__device__ __forceinline__ void st_async_cluster(const void* slot, const uint64_t* bar, uint32_t cta, uint32_t value) {
+  uint32_t rslot, rbar;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(rslot) : "r"(smem_u32(slot)), "r"(cta));
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(rbar) : "r"(smem_u32(bar)), "r"(cta));
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];" ::"r"(rslot), "r"(value),
+               "r"(rbar)
+               : "memory");
 }
 // One-dimensional bulk copy global -> this CTA's shared memory, completion counted on `bar`.
 // dst, src 16-byte aligned, bytes a multiple of 16.

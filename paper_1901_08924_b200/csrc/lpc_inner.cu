@@ -16,11 +16,12 @@
 //
 // Large minibatches (STREAM = true: more rows than shared memory holds, up to 1024 per worker) stream the
 // rows instead, in batch order, through a ring of small stages filled by bulk copies, with no block barrier
-// in the loop.  Half of the warps take the margin partial sums (one warp per row of a group, over the whole
-// slice, reduced by shuffles alone) and send them to the cluster as tagged words through distributed shared
-// memory; the other half own the coordinates of u, wait for the partial sums of all CTAs, form the
-// coefficients and add the rows -- still in shared memory -- into u, then hand the stage back to be
-// refilled.  Each row is read from HBM once and the kernel runs at the rate of the bulk copies.
+// in the loop.  The warps are specialised: eight take the margin partial sums (one warp per row of a group, over
+// the whole slice, reduced by shuffles alone) and send them to every CTA of the cluster as asynchronous stores that
+// count on the receiver's mbarrier of that group; two turn the complete margins into coefficients; eight own the
+// coordinates of u and add the rows -- still in shared memory -- into u, then hand the stage back; one refills
+// the stages.  Every hand-over is an mbarrier phase, so waiting warps sleep in hardware and take no issue slots or
+// shared-memory bandwidth from the working ones.  Each row is read from HBM once.
 #include <cooperative_groups.h>
 
 #include "lpc_device.cuh"
@@ -43,8 +44,9 @@ constexpr int SMAXR = 8;          // ring stages at most
 constexpr int SMAXB = 1024;       // rows per worker at most
 constexpr int SDW = 8;            // warps that take margin partial sums: SDW / SG groups in flight on that side
 constexpr int SUW = 8;            // warps that own the coordinates of u
-constexpr int SCW = 2;            // warps that form coefficients and refill stages (they alternate groups)
-constexpr int SNT = (SDW + SUW + SCW) * 32;  // threads of the streaming kernel
+constexpr int SCW = 2;            // warps that form coefficients (they alternate groups)
+constexpr int SPW = 1;            // warp that refills the ring
+constexpr int SNT = (SDW + SUW + SCW + SPW) * 32;  // threads of the streaming kernel
 
 struct Smem {
   uint64_t bar;
@@ -62,26 +64,16 @@ struct Smem {
   Scale scale;
   int load_ok;
   __align__(16) uint8_t stage[IT * 16];
-  // streaming path: one mbarrier per ring stage; tagged partial sums of the groups in flight (written by peers)
+  // streaming path: every hand-over is an mbarrier phase, so a waiting warp sleeps in hardware instead of polling
   uint64_t sbar[SMAXR];           // stage filled (bulk-copy bytes)
   uint64_t ebar[SMAXR];           // stage consumed (one arrival per warp that adds rows into u)
-  unsigned long long sx[SSLOTS][SG * MAXCS];
-  unsigned long long cw[SSLOTS][SG];  // coefficients of the groups in flight, tagged, written by this CTA's own warp
+  uint64_t pbar[SSLOTS];          // margin partial sums of a group have arrived from every CTA (bytes of their stores)
+  uint64_t cbar[SSLOTS];          // coefficients of a group are in `coefs`
+  __align__(16) float parts[SSLOTS][SG * MAXCS * 4];  // quarter-slice partial sums of the groups in flight (written by all CTAs of the cluster)
+  __align__(16) float coefs[SSLOTS][SG];
+  int stream_fail;                // a bounded wait ran out somewhere in this CTA
+  int issued;                     // groups whose bulk copies have been issued
 };
-
-// Tagged 64-bit words (payload | tag << 32) stored into the shared memory of CTA `cta` of the cluster at the
-// address `slot` has in this CTA; a reader that sees the tag it expects also sees the payload.
-__device__ __forceinline__ void st_cluster_word(const unsigned long long* slot, uint32_t cta, uint32_t payload, uint32_t tag) {
-  const unsigned long long v = (unsigned long long)payload | ((unsigned long long)tag << 32);
-  uint32_t remote;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(slot)), "r"(cta));
-  asm volatile("st.relaxed.cluster.shared::cluster.u64 [%0], %1;" ::"r"(remote), "l"(v) : "memory");
-}
-__device__ __forceinline__ unsigned long long ld_shared_word(const unsigned long long* slot) {
-  unsigned long long v;
-  asm volatile("ld.volatile.shared::cta.u64 %0, [%1];" : "=l"(v) : "r"(smem_u32(slot)) : "memory");
-  return v;
-}
 
 // Phase timestamps of the streaming path of one CTA, for latency studies; compiled in only with -DLPC_TRACE.
 #ifdef LPC_TRACE
@@ -137,9 +129,10 @@ __global__ void __launch_bounds__(STREAM ? SNT : IT) inner_kernel(InnerArgs a) {
     const U4 r = stream_block(a.seed, tag, wk, k, (uint32_t)slot);
     const int64_t row = lo + (int64_t)(((uint64_t)r.x * (uint64_t)span) >> 32);
     s_idx[slot] = row;
-    s_yv[slot] = a.y[row];
-    s_ms[slot] = a.margins[row];
-    if constexpr (STREAM) s_ms[slot] = loss_deriv(a.loss, a.margins[row], s_yv[slot]);  // the snapshot side of the coefficient
+    if constexpr (!STREAM) {
+      s_yv[slot] = a.y[row];
+      s_ms[slot] = a.margins[row];
+    }
   }
   if (tid == 0) {
     mbar_init(&sm.bar, 1);
@@ -148,15 +141,17 @@ __global__ void __launch_bounds__(STREAM ? SNT : IT) inner_kernel(InnerArgs a) {
         mbar_init(&sm.sbar[r], 1);
         mbar_init(&sm.ebar[r], SUW);
       }
+      for (int r = 0; r < SSLOTS; ++r) {
+        mbar_init(&sm.pbar[r], 1);
+        mbar_init(&sm.cbar[r], 1);
+      }
+      sm.stream_fail = 0;
+      sm.issued = 0;
     }
     mbar_fence_init();
   }
-  if constexpr (STREAM) {  // no exchange slot may look valid before a peer has written it: tags start at 1
-    for (int i = tid; i < SSLOTS * SG * MAXCS; i += NT) (&sm.sx[0][0])[i] = 0ull;
-    for (int i = tid; i < SSLOTS * SG; i += NT) (&sm.cw[0][0])[i] = 0ull;
-  }
-  // Every CTA of the cluster announces that it is running; peers wait for this before their first
-  // store into this CTA's shared memory.
+  // Every CTA of the cluster announces that it is running (its barriers exist); peers wait for this before their
+  // first store into this CTA's shared memory.
   asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   __syncthreads();
   if (!STREAM && tid == 0 && width > 0) {
@@ -218,178 +213,218 @@ __global__ void __launch_bounds__(STREAM ? SNT : IT) inner_kernel(InnerArgs a) {
     const int R = a.stream_stages;
     const int ngroups = (B + SG - 1) / SG;
     const uint32_t row_bytes = (uint32_t)width * 4u;
-    auto issue = [&](int g) {  // one thread: the rows of group g into stage g % R
+    // One warp: the rows of group g into stage g % R.  Lane 0 arms the stage's barrier with the byte count, lane j
+    // issues the copy of row j: a bulk copy occupies its issuing thread for a noticeable time, so the rows of a
+    // group are issued side by side.
+    auto issue = [&](int g, int lane_in_group) {
       const int s = g % R;
       const int cnt = min(SG, B - g * SG);
-      mbar_expect_tx(&sm.sbar[s], row_bytes * (uint32_t)cnt);
-      for (int j = 0; j < cnt; ++j)
-        bulk_load(rows + ((size_t)s * SG + j) * SL, a.X + s_idx[g * SG + j] * (int64_t)d + c0, row_bytes, &sm.sbar[s]);
-      LPC_STREAM_MARK(g, 6);
+      if (lane_in_group == 0) {
+        mbar_expect_tx(&sm.sbar[s], row_bytes * (uint32_t)cnt);
+        sm.issued = g + 1;
+      }
+      if (lane_in_group < cnt)
+        bulk_load(rows + ((size_t)s * SG + lane_in_group) * SL, a.X + s_idx[g * SG + lane_in_group] * (int64_t)d + c0,
+                  row_bytes, &sm.sbar[s]);
+      if (lane_in_group == 0) LPC_STREAM_MARK(g, 6);
     };
-    if (tid == 0 && width > 0) {
-      for (int g = 0; g < min(R, ngroups); ++g) issue(g);
+    static_assert(SMAXR * SG <= 32, "the first fills are issued by one warp, one row per lane");
+    if (warp == 0 && width > 0) {  // the first fills start before anything else of the step
+      const int g = lane / SG;
+      if (g < min(R, ngroups)) issue(g, lane % SG);
+    }
+    // labels and the snapshot side of the coefficients, l'(m~_a): needed only once the first margins are complete
+    for (int slot = tid; slot < B; slot += NT) {
+      const int64_t row = s_idx[slot];
+      const float yv = a.y[row];
+      s_yv[slot] = yv;
+      s_ms[slot] = loss_deriv(a.loss, a.margins[row], yv);
     }
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");  // all peers have started
+    __syncthreads();
     bool gave_up = false;  // after one wait ran out this thread waits no more (the status word says so)
-    auto wait_stage = [&](int g) {
-      if (width > 0 && !gave_up && !mbar_test(&sm.sbar[g % R], (uint32_t)((g / R) & 1)) &&
-          !mbar_wait(&sm.sbar[g % R], (uint32_t)((g / R) & 1))) {
+    auto wait_on = [&](uint64_t* bar, uint32_t parity, bool from_cluster) {
+      if (gave_up) return;
+      if (!from_cluster && mbar_test(bar, parity)) return;
+      const bool ok = from_cluster ? mbar_wait_cluster(bar, parity) : mbar_wait(bar, parity);
+      if (!ok) {
         atomicOr(a.dev_status, DEV_TIMEOUT);
+        sm.stream_fail = 1;
         gave_up = true;
       }
     };
-    constexpr int CH = IGROUP / 8 / 32;  // 8-coordinate chunks per lane when one warp covers a slice: 8
+    auto wait_stage = [&](int g) {
+      if (width > 0) wait_on(&sm.sbar[g % R], (uint32_t)((g / R) & 1), false);
+    };
+    // Shared-memory reads are laid out so that a warp's 16-byte loads touch consecutive addresses (no bank
+    // conflicts): the ring is read twice per row and written once, and that traffic is what bounds a group.
+    constexpr int NBK = IGROUP / 128;    // blocks of 128 coordinates per slice: 16; a lane takes 4 coordinates of each
     constexpr int AT = SUW * 32;         // threads that own the coordinates of u
-    constexpr int UC = IGROUP / 8 / AT;  // chunks per such thread
-    float ua[UC][8];
+    constexpr int UC = IGROUP / 4 / AT;  // 4-coordinate pieces per such thread: 2, IGROUP / UC apart
+    float ua[UC][4];
 #pragma unroll
     for (int q = 0; q < UC; ++q)
 #pragma unroll
-      for (int e = 0; e < 8; ++e) ua[q][e] = 0.f;
+      for (int e = 0; e < 4; ++e) ua[q][e] = 0.f;
+    const bool full = (width == IGROUP);  // the usual case: every column of the slice exists, nothing to test per load
+    auto row4 = [&](int r, int off) {  // four row values of the slice (zero outside the existing columns)
+      return (off < width) ? *reinterpret_cast<const float4*>(rows + (size_t)r * SL + off) : make_float4(0.f, 0.f, 0.f, 0.f);
+    };
     if (warp < SDW) {
-      // -- margins (warp w: row w % SG of the groups g = w / SG, w / SG + SDW / SG, ...): lane l holds x for chunks l, l+32, ..., the leaves of the tree in coordinate order are
-      // (chunk, element); per chunk tree8, then the tree over the 32 lanes for every chunk row, then over the rows
-      float xs[CH][8];
+      // -- margins: the SMW = 4 warps of a side share a group, warp w of them taking the blocks 4 w .. 4 w + 3 (a quarter
+      // of the slice) of all rows of the group; the two sides alternate groups.  Lane l holds x for the coordinates
+      // 128 q + 4 l .. + 3 of its blocks q.  The leaves of the tree in coordinate order: four products per lane
+      // (tree4), then the tree over the 32 lanes of a block, then the tree over the four blocks; the quarter sums go to
+      // every CTA of the cluster as stores that count on that CTA's barrier of the group, and are combined there.
+      // Sixteen independent 16-byte loads and one reduction per group keep a warp's dependent chains short.
+      constexpr int SMW = 4, QB = NBK / SMW;  // warps per side; blocks per warp
+      static_assert(SDW == 2 * SMW && QB * SG == 16, "one 16-value recursive-halving reduction per group");
+      const int wq = warp % SMW;
+      float4 xs[QB];
 #pragma unroll
-      for (int q = 0; q < CH; ++q) {
-        const int off = (q * 32 + lane) * 8;
-#pragma unroll
-        for (int e = 0; e < 8; ++e) xs[q][e] = (off + e < width) ? a.x[c0 + off + e] : 0.f;
+      for (int q = 0; q < QB; ++q) {
+        const int off = (wq * QB + q) * 128 + lane * 4;  // width is a multiple of 4
+        xs[q] = (off < width) ? *reinterpret_cast<const float4*>(a.x + c0 + off) : make_float4(0.f, 0.f, 0.f, 0.f);
       }
-      const int myrow = warp % SG;
+      // after the reduction lane l holds the sum of row halving_index<2>(l & 3); lane l sends it to CTA l >> 2
+      const int myrow = ((lane & 1) << 1) | ((lane >> 1) & 1);
 #pragma unroll 1
-      for (int g = warp / SG; g < ngroups; g += SDW / SG) {
+      for (int g = warp / SMW; g < ngroups; g += SDW / SMW) {
         const int cnt = min(SG, B - g * SG);
         wait_stage(g);
-        if (myrow == 0 && lane == 0) LPC_STREAM_MARK(g, 0);
-        if (myrow < cnt) {
-          float sv[CH];
+        if (warp < 2 * SMW && wq == 0 && lane == 0) LPC_STREAM_MARK(g, 0);
+        float4 v[SG][QB];  // all sixteen loads first
+        if (full) {
+          const float* src = rows + (size_t)((g % R) * SG) * SL + wq * QB * 128 + lane * 4;
 #pragma unroll
-          for (int q = 0; q < CH; ++q) {
-            float v[8], pr[8];
-            row8((g % R) * SG + myrow, (q * 32 + lane) * 8, v);
+          for (int j = 0; j < SG; ++j)
 #pragma unroll
-            for (int e = 0; e < 8; ++e) pr[e] = mul_rn(v[e], xs[q][e]);
-            sv[q] = tree8(pr);
-          }
-          WarpHalving<CH, 0>::run(sv, lane);  // lane holds the 32-lane tree sum of chunk row halving_index<3>(lane)
-          float part = sv[0];
-          part = add_rn(part, __shfl_xor_sync(0xFFFFFFFFu, part, 4));  // rows 2k, 2k+1
-          part = add_rn(part, __shfl_xor_sync(0xFFFFFFFFu, part, 2));
-          part = add_rn(part, __shfl_xor_sync(0xFFFFFFFFu, part, 1));
-          if (lane < CS)
-            st_cluster_word(&sm.sx[g % SSLOTS][myrow * MAXCS + rank], (uint32_t)lane, __float_as_uint(part), (uint32_t)(g + 1));
-          if (myrow == 0 && lane == 0) LPC_STREAM_MARK(g, 1);
+            for (int q = 0; q < QB; ++q) v[j][q] = *reinterpret_cast<const float4*>(src + j * SL + q * 128);
+        } else {
+#pragma unroll
+          for (int j = 0; j < SG; ++j)
+#pragma unroll
+            for (int q = 0; q < QB; ++q) v[j][q] = row4((g % R) * SG + j, (wq * QB + q) * 128 + lane * 4);
         }
+        float sv[SG * QB];
+#pragma unroll
+        for (int j = 0; j < SG; ++j)
+#pragma unroll
+          for (int q = 0; q < QB; ++q)
+            sv[j * QB + q] = tree4(mul_rn(v[j][q].x, xs[q].x), mul_rn(v[j][q].y, xs[q].y), mul_rn(v[j][q].z, xs[q].z),
+                                   mul_rn(v[j][q].w, xs[q].w));
+        WarpHalving<SG * QB, 0>::run(sv, lane);  // lane holds the 32-lane tree sum of (row, block) halving_index<4>(lane)
+        float part = sv[0];
+        part = add_rn(part, __shfl_xor_sync(0xFFFFFFFFu, part, 8));  // blocks 2k, 2k+1 of the row
+        part = add_rn(part, __shfl_xor_sync(0xFFFFFFFFu, part, 4));
+        if ((lane >> 2) < CS && myrow < cnt)
+          st_async_cluster(&sm.parts[g % SSLOTS][(myrow * MAXCS + rank) * SMW + wq], &sm.pbar[g % SSLOTS],
+                           (uint32_t)(lane >> 2), __float_as_uint(part));
+        if (wq == 0 && lane == 0) LPC_STREAM_MARK(g, 1);
       }
-    } else if (warp >= SDW + SUW) {
-      // -- coefficients and refills (warp c of this side takes the groups c, c + SCW, ...): lane j collects the partial sums of row j of a group from all CTAs
-      // of the cluster and publishes the coefficient l'(m) - l'(m~) to the update side; lane 0 refills a stage as
-      // soon as the update side has handed it back.  Running in a warp of its own, the fp64 loss derivative and
-      // the barrier waits delay neither the margins nor the updates.
-#pragma unroll 1
-      for (int g = warp - (SDW + SUW); g < ngroups; g += SCW) {
-        const int cnt = min(SG, B - g * SG);
-        if (lane < cnt) {
-          float mp[MAXCS];
-          uint64_t t0 = 0;
-          for (uint32_t it = 0;; ++it) {
-            bool all = true;
-#pragma unroll
-            for (int q = 0; q < MAXCS; ++q) {
-              mp[q] = 0.f;
-              if (q < CS) {
-                const unsigned long long w = ld_shared_word(&sm.sx[g % SSLOTS][lane * MAXCS + q]);
-                all = all && (uint32_t)(w >> 32) == (uint32_t)(g + 1);
-                mp[q] = __uint_as_float((uint32_t)w);
-              }
-            }
-            if (all || gave_up) break;
-            if ((it & 63u) == 63u) {
-              const uint64_t now = global_ns();
-              if (t0 == 0) t0 = now;
-              else if (now - t0 > 2000000000ull) {
-                atomicOr(a.dev_status, DEV_TIMEOUT);
-                gave_up = true;
-              }
-            }
-          }
-          if (lane == 0) LPC_STREAM_MARK(g, 2);
-          const int slot = g * SG + lane;
-          const float m = (CS == 1) ? mp[0] : (CS == 2) ? add_rn(mp[0], mp[1]) : (CS == 4) ? tree4(mp[0], mp[1], mp[2], mp[3]) : tree8(mp);
-          const float c = __fsub_rn(loss_deriv(a.loss, m, s_yv[slot]), s_ms[slot]);
-          st_cluster_word(&sm.cw[g % SSLOTS][lane], (uint32_t)rank, __float_as_uint(c), (uint32_t)(g + 1));
-          if (lane == 0) LPC_STREAM_MARK(g, 3);
-          if (rank == 0) {
-            if (a.idx_tap) a.idx_tap[(int64_t)worker * B + slot] = s_idx[slot];
-            if (a.coef_tap) a.coef_tap[(int64_t)worker * B + slot] = c;
-          }
-        }
-        if (lane == 0 && g >= SCW && g - SCW + R < ngroups) {  // an earlier group of this warp, added into u by now
-          const int h = g - SCW;
-          if (!gave_up && !mbar_wait(&sm.ebar[h % R], (uint32_t)((h / R) & 1))) {
-            atomicOr(a.dev_status, DEV_TIMEOUT);
-            gave_up = true;
-          }
-          if (width > 0) issue(h + R);
-        }
-        __syncwarp();
-      }
-    } else {
-      // -- u: thread t of these warps owns chunk t (+ AT, ...) of the slice
+    } else if (warp < SDW + SUW) {
+      // -- u: thread t of these warps owns the coordinates 4 t .. 4 t + 3 of each half of the slice
       const int t = tid - SDW * 32;
 #pragma unroll 1
       for (int g = 0; g < ngroups; ++g) {
         const int cnt = min(SG, B - g * SG);
         const int s = g % R;
-        float c_mine = 0.f;
-        if (lane < cnt) {  // lane j fetches the coefficient of row j
-          uint64_t t0 = 0;
-          for (uint32_t it = 0;; ++it) {
-            const unsigned long long w = ld_shared_word(&sm.cw[g % SSLOTS][lane]);
-            c_mine = __uint_as_float((uint32_t)w);
-            if ((uint32_t)(w >> 32) == (uint32_t)(g + 1) || gave_up) break;
-            if ((it & 63u) == 63u) {
-              const uint64_t now = global_ns();
-              if (t0 == 0) t0 = now;
-              else if (now - t0 > 2000000000ull) {
-                atomicOr(a.dev_status, DEV_TIMEOUT);
-                gave_up = true;
-              }
-            }
-          }
-        }
-        __syncwarp();
+        wait_on(&sm.cbar[g % SSLOTS], (uint32_t)((g / SSLOTS) & 1), false);
         wait_stage(g);
         if (t == 0) LPC_STREAM_MARK(g, 4);
+        const float4 c4 = *reinterpret_cast<const float4*>(sm.coefs[g % SSLOTS]);
+        const float cj[SG] = {c4.x, c4.y, c4.z, c4.w};
+        float4 v[SG][UC];  // all loads of the group first (rows past a ragged end are read and not used)
+        if (full) {
+          const float* src = rows + (size_t)(s * SG) * SL + t * 4;
+#pragma unroll
+          for (int j = 0; j < SG; ++j)
+#pragma unroll
+            for (int q = 0; q < UC; ++q) v[j][q] = *reinterpret_cast<const float4*>(src + j * SL + q * (IGROUP / UC));
+        } else {
+#pragma unroll
+          for (int j = 0; j < SG; ++j)
+#pragma unroll
+            for (int q = 0; q < UC; ++q) v[j][q] = row4(s * SG + j, q * (IGROUP / UC) + t * 4);
+        }
 #pragma unroll
         for (int j = 0; j < SG; ++j) {
-          const float c = __shfl_sync(0xFFFFFFFFu, c_mine, j);
           if (j < cnt) {
 #pragma unroll
             for (int q = 0; q < UC; ++q) {
-              float v[8];
-              row8(s * SG + j, (q * AT + t) * 8, v);
-#pragma unroll
-              for (int e = 0; e < 8; ++e) ua[q][e] = add_rn(ua[q][e], mul_rn(c, v[e]));
+              ua[q][0] = add_rn(ua[q][0], mul_rn(cj[j], v[j][q].x));
+              ua[q][1] = add_rn(ua[q][1], mul_rn(cj[j], v[j][q].y));
+              ua[q][2] = add_rn(ua[q][2], mul_rn(cj[j], v[j][q].z));
+              ua[q][3] = add_rn(ua[q][3], mul_rn(cj[j], v[j][q].w));
             }
           }
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(&sm.ebar[s]);  // this warp is done with the stage
-        if (t == 0) LPC_STREAM_MARK(g, 5);
+#ifdef LPC_TRACE
+        if (lane == 0 && blockIdx.x == 0 && blockIdx.y == 0 && g < 64) atomicMax(&g_stream_trace[g * 8 + 5], global_ns());
+#endif
+      }
+    } else if (warp < SDW + SUW + SCW) {
+      // -- coefficients (warp c of this side takes the groups c, c + SCW, ...): lane j collects the partial sums of
+      // row j of a group from all CTAs of the cluster and leaves the coefficient l'(m) - l'(m~) for the update side.
+      // Running in warps of their own, the fp64 loss derivative delays neither the margins nor the updates.
+#pragma unroll 1
+      for (int g = warp - (SDW + SUW); g < ngroups; g += SCW) {
+        const int cnt = min(SG, B - g * SG);
+        const int sl = g % SSLOTS;
+        if (lane == 0) mbar_expect_tx(&sm.pbar[sl], (uint32_t)(CS * cnt * 16));  // this phase: one arrival and the bytes of 4 quarter sums per row and CTA
+        __syncwarp();
+        wait_on(&sm.pbar[sl], (uint32_t)((g / SSLOTS) & 1), true);
+        if (lane == 0) LPC_STREAM_MARK(g, 2);
+        if (lane < SG) {
+          float c = 0.f;
+          if (lane < cnt) {
+            float mp[MAXCS];
+#pragma unroll
+            for (int q = 0; q < MAXCS; ++q) {
+              const float4 pq = *reinterpret_cast<const float4*>(&sm.parts[sl][(lane * MAXCS + q) * 4]);
+              mp[q] = (q < CS) ? tree4(pq.x, pq.y, pq.z, pq.w) : 0.f;
+            }
+            const int slot = g * SG + lane;
+            const float m = (CS == 1) ? mp[0] : (CS == 2) ? add_rn(mp[0], mp[1]) : (CS == 4) ? tree4(mp[0], mp[1], mp[2], mp[3]) : tree8(mp);
+            c = __fsub_rn(loss_deriv(a.loss, m, s_yv[slot]), s_ms[slot]);
+            if (rank == 0) {
+              if (a.idx_tap) a.idx_tap[(int64_t)worker * B + slot] = s_idx[slot];
+              if (a.coef_tap) a.coef_tap[(int64_t)worker * B + slot] = c;
+            }
+          }
+          sm.coefs[sl][lane] = c;
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.cbar[sl]);
+        if (lane == 0) LPC_STREAM_MARK(g, 3);
+      }
+    } else {
+      // -- refills: a stage goes back to the bulk copies the moment the update side has handed it over
+#pragma unroll 1
+      for (int g = R; g < ngroups; ++g) {
+        const int h = g - R;
+        wait_on(&sm.ebar[h % R], (uint32_t)((h / R) & 1), false);
+        if (lane == 0) LPC_STREAM_MARK(g, 7);
+        if (gave_up) break;
+        if (width > 0 && lane < SG) issue(g, lane);
+        __syncwarp();
       }
     }
     __syncthreads();  // both sides are done with the ring: it now carries u to the usual owner of each coordinate
+    if (sm.stream_fail) {  // a wait ran out: give the copies still in flight a bounded chance to land before the ring is reused
+      if (tid == 0 && width > 0)
+        for (int g = max(0, sm.issued - R); g < sm.issued; ++g) mbar_wait(&sm.sbar[g % R], (uint32_t)((g / R) & 1), 100000000ull);
+      __syncthreads();
+    }
     if (warp >= SDW && warp < SDW + SUW) {
       const int t = tid - SDW * 32;
 #pragma unroll
       for (int q = 0; q < UC; ++q) {
-        if ((q * AT + t) * 8 < SL) {  // the ring holds at least one slice
-          float* dst = rows + (q * AT + t) * 8;
-          *reinterpret_cast<float4*>(dst) = make_float4(ua[q][0], ua[q][1], ua[q][2], ua[q][3]);
-          *reinterpret_cast<float4*>(dst + 4) = make_float4(ua[q][4], ua[q][5], ua[q][6], ua[q][7]);
-        }
+        const int off = q * (IGROUP / UC) + t * 4;
+        if (off < SL)  // the ring holds at least one slice
+          *reinterpret_cast<float4*>(rows + off) = make_float4(ua[q][0], ua[q][1], ua[q][2], ua[q][3]);
       }
     }
     __syncthreads();
