@@ -46,7 +46,8 @@ constexpr int SDW = 8;            // warps that take margin partial sums: SDW / 
 constexpr int SUW = 8;            // warps that own the coordinates of u
 constexpr int SCW = 2;            // warps that form coefficients (they alternate groups)
 constexpr int SPW = 1;            // warp that refills the ring
-constexpr int SNT = (SDW + SUW + SCW + SPW) * 32;  // threads of the streaming kernel
+constexpr int SMETAW = 1;         // warp that gathers labels and snapshot margins of the sampled rows, 32 rows per pass
+constexpr int SNT = (SDW + SUW + SCW + SPW + SMETAW) * 32;  // threads of the streaming kernel
 
 struct Smem {
   uint64_t bar;
@@ -69,6 +70,7 @@ struct Smem {
   uint64_t ebar[SMAXR];           // stage consumed (one arrival per warp that adds rows into u)
   uint64_t pbar[SSLOTS];          // margin partial sums of a group have arrived from every CTA (bytes of their stores)
   uint64_t cbar[SSLOTS];          // coefficients of a group are in `coefs`
+  uint64_t mbar_meta[SMAXB / 32]; // labels and snapshot-side derivatives of 32 sampled rows are in place (used once each)
   __align__(16) float parts[SSLOTS][SG * MAXCS * 4];  // quarter-slice partial sums of the groups in flight (written by all CTAs of the cluster)
   __align__(16) float coefs[SSLOTS][SG];
   int stream_fail;                // a bounded wait ran out somewhere in this CTA
@@ -77,13 +79,18 @@ struct Smem {
 
 // Phase timestamps of the streaming path of one CTA, for latency studies; compiled in only with -DLPC_TRACE.
 #ifdef LPC_TRACE
-__device__ unsigned long long g_stream_trace[64 * 8];
+__device__ unsigned long long g_stream_trace[64 * 8 + 16];  // per group: 8 marks; then 16 phase marks of the kernel
 #define LPC_STREAM_MARK(g, i)                                                                       \
   do {                                                                                              \
     if (blockIdx.x == 0 && blockIdx.y == 0 && (g) < 64) g_stream_trace[(g) * 8 + (i)] = global_ns(); \
   } while (0)
+#define LPC_PHASE_MARK(i)                                                                            \
+  do {                                                                                               \
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) g_stream_trace[64 * 8 + (i)] = global_ns(); \
+  } while (0)
 #else
 #define LPC_STREAM_MARK(g, i) do { } while (0)
+#define LPC_PHASE_MARK(i) do { } while (0)
 #endif
 
 // BITS: 1, 2, 4, 8 fixed-width packing; 0: b from the arguments (1..16 or 32).
@@ -96,6 +103,7 @@ __global__ void __launch_bounds__(STREAM ? SNT : IT) inner_kernel(InnerArgs a) {
   unsigned char* dyn = smem_raw + ((sizeof(Smem) + 15) & ~(size_t)15);
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  LPC_PHASE_MARK(0);
   constexpr int NT = STREAM ? SNT : IT;  // the streaming path runs more warps, specialised by role
   const int rank = (int)cluster.block_rank();
   const int CS = a.CS, SL = a.SL, B = a.B, d = a.d;
@@ -145,6 +153,7 @@ __global__ void __launch_bounds__(STREAM ? SNT : IT) inner_kernel(InnerArgs a) {
         mbar_init(&sm.pbar[r], 1);
         mbar_init(&sm.cbar[r], 1);
       }
+      for (int r = 0; r < (B + 31) / 32; ++r) mbar_init(&sm.mbar_meta[r], 1);
       sm.stream_fail = 0;
       sm.issued = 0;
     }
@@ -229,19 +238,14 @@ __global__ void __launch_bounds__(STREAM ? SNT : IT) inner_kernel(InnerArgs a) {
       if (lane_in_group == 0) LPC_STREAM_MARK(g, 6);
     };
     static_assert(SMAXR * SG <= 32, "the first fills are issued by one warp, one row per lane");
-    if (warp == 0 && width > 0) {  // the first fills start before anything else of the step
+    static_assert(SG * MAXCS == 32, "one lane per (row, CTA) pair when the coefficients are formed");
+    LPC_PHASE_MARK(1);
+    if (warp == SDW + SUW + SCW && width > 0) {  // the first fills start before anything else of the step
       const int g = lane / SG;
       if (g < min(R, ngroups)) issue(g, lane % SG);
     }
-    // labels and the snapshot side of the coefficients, l'(m~_a): needed only once the first margins are complete
-    for (int slot = tid; slot < B; slot += NT) {
-      const int64_t row = s_idx[slot];
-      const float yv = a.y[row];
-      s_yv[slot] = yv;
-      s_ms[slot] = loss_deriv(a.loss, a.margins[row], yv);
-    }
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");  // all peers have started
-    __syncthreads();
+    LPC_PHASE_MARK(3);
     bool gave_up = false;  // after one wait ran out this thread waits no more (the status word says so)
     auto wait_on = [&](uint64_t* bar, uint32_t parity, bool from_cluster) {
       if (gave_up) return;
@@ -375,32 +379,40 @@ __global__ void __launch_bounds__(STREAM ? SNT : IT) inner_kernel(InnerArgs a) {
         const int sl = g % SSLOTS;
         if (lane == 0) mbar_expect_tx(&sm.pbar[sl], (uint32_t)(CS * cnt * 16));  // this phase: one arrival and the bytes of 4 quarter sums per row and CTA
         __syncwarp();
+        wait_on(&sm.mbar_meta[(g * SG) / 32], 0u, false);
         wait_on(&sm.pbar[sl], (uint32_t)((g / SSLOTS) & 1), true);
         if (lane == 0) LPC_STREAM_MARK(g, 2);
-        if (lane < SG) {
-          float c = 0.f;
-          if (lane < cnt) {
-            float mp[MAXCS];
-#pragma unroll
-            for (int q = 0; q < MAXCS; ++q) {
-              const float4 pq = *reinterpret_cast<const float4*>(&sm.parts[sl][(lane * MAXCS + q) * 4]);
-              mp[q] = (q < CS) ? tree4(pq.x, pq.y, pq.z, pq.w) : 0.f;
-            }
-            const int slot = g * SG + lane;
-            const float m = (CS == 1) ? mp[0] : (CS == 2) ? add_rn(mp[0], mp[1]) : (CS == 4) ? tree4(mp[0], mp[1], mp[2], mp[3]) : tree8(mp);
-            c = __fsub_rn(loss_deriv(a.loss, m, s_yv[slot]), s_ms[slot]);
-            if (rank == 0) {
-              if (a.idx_tap) a.idx_tap[(int64_t)worker * B + slot] = s_idx[slot];
-              if (a.coef_tap) a.coef_tap[(int64_t)worker * B + slot] = c;
-            }
+        // lane (j, q) = (lane / MAXCS, lane % MAXCS): the tree over the four quarter sums of CTA q's slice for row j, then
+        // the tree over the CTAs by shuffles; lane (j, 0) ends with the margin of row j
+        {
+          const int j = lane / MAXCS, q = lane % MAXCS;
+          float mq = 0.f;
+          if (q < CS) {
+            const float4 pq = *reinterpret_cast<const float4*>(&sm.parts[sl][(j * MAXCS + q) * 4]);
+            mq = tree4(pq.x, pq.y, pq.z, pq.w);
           }
-          sm.coefs[sl][lane] = c;
+          // CS is a power of two: the tree over q = 0 .. CS-1
+          if (CS > 1) mq = add_rn(mq, __shfl_xor_sync(0xFFFFFFFFu, mq, 1));
+          if (CS > 2) mq = add_rn(mq, __shfl_xor_sync(0xFFFFFFFFu, mq, 2));
+          if (CS > 4) mq = add_rn(mq, __shfl_xor_sync(0xFFFFFFFFu, mq, 4));
+          if (q == 0) {
+            float c = 0.f;
+            if (j < cnt) {
+              const int slot = g * SG + j;
+              c = __fsub_rn(loss_deriv(a.loss, mq, s_yv[slot]), s_ms[slot]);
+              if (rank == 0) {
+                if (a.idx_tap) a.idx_tap[(int64_t)worker * B + slot] = s_idx[slot];
+                if (a.coef_tap) a.coef_tap[(int64_t)worker * B + slot] = c;
+              }
+            }
+            sm.coefs[sl][j] = c;
+          }
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(&sm.cbar[sl]);
         if (lane == 0) LPC_STREAM_MARK(g, 3);
       }
-    } else {
+    } else if (warp < SDW + SUW + SCW + SPW) {
       // -- refills: a stage goes back to the bulk copies the moment the update side has handed it over
 #pragma unroll 1
       for (int g = R; g < ngroups; ++g) {
@@ -410,6 +422,20 @@ __global__ void __launch_bounds__(STREAM ? SNT : IT) inner_kernel(InnerArgs a) {
         if (gave_up) break;
         if (width > 0 && lane < SG) issue(g, lane);
         __syncwarp();
+      }
+    } else {
+      // -- labels and the snapshot side of the coefficients, l'(m~_a), 32 sampled rows per pass, ahead of their use
+#pragma unroll 1
+      for (int base = 0; base < B; base += 32) {
+        const int slot = base + lane;
+        if (slot < B) {
+          const int64_t row = s_idx[slot];
+          const float yv = a.y[row];
+          s_yv[slot] = yv;
+          s_ms[slot] = loss_deriv(a.loss, a.margins[row], yv);
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.mbar_meta[base / 32]);
       }
     }
     __syncthreads();  // both sides are done with the ring: it now carries u to the usual owner of each coordinate
@@ -528,6 +554,7 @@ __global__ void __launch_bounds__(STREAM ? SNT : IT) inner_kernel(InnerArgs a) {
   }
 
   // ---- scale (Eq. 2): max |u| and, for the c*std rule, tree sums of u and u^2 ----------------------------------
+  LPC_PHASE_MARK(5);
   uint32_t mx = 0;
 #pragma unroll
   for (int p = 0; p < MAXP; ++p) {
@@ -577,6 +604,7 @@ __global__ void __launch_bounds__(STREAM ? SNT : IT) inner_kernel(InnerArgs a) {
     }
   }
   __syncthreads();
+  LPC_PHASE_MARK(6);
   const Scale sc = sm.scale;
   const bool degenerate = (sc.flags & 1u) != 0;
   const uint32_t zero_code = (b == 1) ? 0u : (1u << (b - 1));
@@ -665,6 +693,7 @@ __global__ void __launch_bounds__(STREAM ? SNT : IT) inner_kernel(InnerArgs a) {
     for (int w = 0; w < 8; ++w) t += sm.wclip[w];
     a.clipped_part[worker * MAXCS + rank] = t;
   }
+  LPC_PHASE_MARK(7);
 }
 
 template <int BITS, bool STREAM>
@@ -774,7 +803,7 @@ cudaError_t launch_inner(const InnerArgs& a, size_t smem, cudaStream_t st) {
 
 #ifdef LPC_TRACE
 cudaError_t read_stream_trace(unsigned long long* host_out) {
-  return cudaMemcpyFromSymbol(host_out, g_stream_trace, sizeof(unsigned long long) * 64 * 8);
+  return cudaMemcpyFromSymbol(host_out, g_stream_trace, sizeof(unsigned long long) * (64 * 8 + 16));
 }
 #endif
 
