@@ -349,29 +349,32 @@ def quantize_aggregate_bench(dev, peak, log2_len=26, dnn=True):
 def fused_large_batch_bench(dev, peak, n=65536, steps=30):
     """The fused worker kernel (sampling, SVRG difference, scale, quantize, pack) where it is bandwidth-bound: the ALPC
     workload's shape (d = 8,192, N = 32, logistic) with the minibatch raised to B = 256 rows per worker, so that one
-    step gathers N*B*d*4 = 268 MB of rows.  Times come from the library's per-kernel event profile."""
+    step gathers N*B*d*4 = 268 MB of rows, and to the kernel's limit of B = 1,024 (1.07 GB per step), where the
+    fixed cost of a launch (sampling, first fills, scale exchange, packing) weighs less.  Times come from the
+    library's per-kernel event profile."""
     import torch
     from paper_1901_08924_b200 import lpc, synth
-    d, N, B = 8192, 32, 256
+    d, N = 8192, 32
     X, y, _ = synth.linear_problem(n, d, loss="logistic", sparsity=0.02, noise=0.1, seed=1, col_scale_range=(0.1, 10.0),
                                    device=dev)
-    out = {"workload": "fused_step_logistic_%dx8192_N32_B256" % n, "row_bytes_per_step": N * B * d * 4}
-    for b in (2, 8):
-        ctx = lpc.Context(X, y, lpc.LOGISTIC, 1e-5, N, B, b, lpc.CLIP_STD, 2.0, 0)
-        ctx.snapshot_full_grad()
-        ctx.inner_steps(1e-3, 0, 5)
-        ctx.set_option(lpc.OPT_PROFILE, 1)
-        ctx.inner_steps(1e-3, 5, steps)
-        ctx.sync_status()
-        prof = ctx.get_profile()
-        tw = prof["worker"][0] / prof["worker"][1]
-        ta = prof["aggregate"][0] / prof["aggregate"][1]
-        bw = N * B * d * 4 + N * B * 8 + N * (d * b // 8 + 4)
-        out["b%d" % b] = {"worker_us": round(tw * 1e3, 2), "worker_gbs": round(bw / tw * 1e-6, 1),
-                          "worker_frac": round(bw / tw * 1e-6 / peak, 4), "aggregate_us": round(ta * 1e3, 2),
-                          "ring_stages": ctx.query(lpc.INFO_STEP_RING_STAGES),
-                          "cluster_size": ctx.query(lpc.INFO_STEP_CLUSTER_SIZE)}
-        ctx.close()
+    out = {"workload": "fused_step_logistic_%dx8192_N32" % n}
+    for B, bits in ((256, (2, 8)), (1024, (2,))):
+        for b in bits:
+            ctx = lpc.Context(X, y, lpc.LOGISTIC, 1e-5, N, B, b, lpc.CLIP_STD, 2.0, 0)
+            ctx.snapshot_full_grad()
+            ctx.inner_steps(1e-3, 0, 5)
+            ctx.set_option(lpc.OPT_PROFILE, 1)
+            ctx.inner_steps(1e-3, 5, steps)
+            ctx.sync_status()
+            prof = ctx.get_profile()
+            tw = prof["worker"][0] / prof["worker"][1]
+            ta = prof["aggregate"][0] / prof["aggregate"][1]
+            bw = N * B * d * 4 + N * B * 8 + N * (d * b // 8 + 4)
+            out["B%d_b%d" % (B, b)] = {"row_bytes_per_step": N * B * d * 4, "worker_us": round(tw * 1e3, 2),
+                                       "worker_gbs": round(bw / tw * 1e-6, 1), "worker_frac": round(bw / tw * 1e-6 / peak, 4),
+                                       "aggregate_us": round(ta * 1e3, 2), "ring_stages": ctx.query(lpc.INFO_STEP_RING_STAGES),
+                                       "cluster_size": ctx.query(lpc.INFO_STEP_CLUSTER_SIZE)}
+            ctx.close()
     return out
 
 

@@ -57,6 +57,18 @@ def _declare(L):
     L.orc_quantize_coord.argtypes = [C.c_float, C.c_float, C.c_int, C.c_uint32]
     L.orc_quantize_coord.restype = C.c_int
     L.orc_pack.argtypes = [_u32p, C.c_int64, C.c_int, _u32p]
+    L.orc_sum_bits_per_coordinate.argtypes = [C.c_int, C.c_int]
+    L.orc_sum_bits_per_coordinate.restype = C.c_int
+    L.orc_scheme_bits.argtypes = [C.c_int, C.c_int64, C.c_int, C.c_int]
+    L.orc_scheme_bits.restype = C.c_uint64
+    L.orc_quantize_pack_shared.argtypes = [_f32p, C.c_int, C.c_int64, C.c_int64, C.c_int, C.c_int, C.c_float, C.c_uint64,
+                                           C.c_uint64, _u32p, C.c_int64, _f32p, _u32p]
+    L.orc_quantize_pack_shared.restype = C.c_int
+    L.orc_server_reduce.argtypes = [_u32p, C.c_int64, C.c_int, C.c_int64, C.c_int, C.c_int, C.c_uint64, C.c_uint64, _u32p]
+    L.orc_server_reduce.restype = C.c_int
+    L.orc_unpack_scaled_prox.argtypes = [_u32p, C.c_float, C.c_int64, C.c_int, C.c_int, _f32p, _f32p, C.c_float, C.c_float,
+                                         _f32p, _f32p]
+    L.orc_unpack_scaled_prox.restype = None
     L.orc_pack.restype = None
     L.orc_unpack.argtypes = [_u32p, C.c_int64, C.c_int, _u32p]
     L.orc_unpack.restype = None
@@ -227,6 +239,62 @@ def unpack_average_prox(words, delta, length, b, mu, x, eta, lambda_l1, want_v=F
     ut = np.zeros(length, dtype=np.float32) if want_utilde else None
     lib().orc_unpack_average_prox(words.ctypes.data_as(_u32p), stride, pd, N, length, b, _ptr(mu_a, _f32p),
                                   xn.ctypes.data_as(_f32p), eta, lambda_l1, _ptr(v, _f32p), _ptr(ut, _f32p))
+    out = (xn,)
+    if want_v:
+        out += (v,)
+    if want_utilde:
+        out += (ut,)
+    return out if len(out) > 1 else xn
+
+
+SCHEME_A, SCHEME_B, SCHEME_C = 0, 1, 2
+
+
+def sum_bits_per_coordinate(b, N):
+    """Width of the server's sum stream under scheme (b): b + ceil(log2 N)."""
+    return int(lib().orc_sum_bits_per_coordinate(b, N))
+
+
+def scheme_bits(scheme, d, b, N):
+    """Bits of one communication step 2 under scheme (a), (b) or (c) (Table 1)."""
+    return int(lib().orc_scheme_bits(scheme, d, b, N))
+
+
+def quantize_pack_shared(U, b, clip_mode=CLIP_NONE, clip_value=1.0, seed=0, k=0):
+    """All N worker vectors (rows of U) with the unified scale of schemes (b)/(c).
+    Returns (words (N, W), delta, clipped (N,))."""
+    U = np.ascontiguousarray(U, dtype=np.float32)
+    N, length = U.shape
+    W = max(packed_words(length, b), 1)
+    words = np.zeros((N, W), dtype=np.uint32)
+    delta = np.zeros(1, dtype=np.float32)
+    clipped = np.zeros(N, dtype=np.uint32)
+    _check(lib().orc_quantize_pack_shared(U.ctypes.data_as(_f32p), N, length, length, b, clip_mode, clip_value, seed, k,
+                                          words.ctypes.data_as(_u32p), W, delta.ctypes.data_as(_f32p),
+                                          clipped.ctypes.data_as(_u32p)))
+    return words[:, : packed_words(length, b)], np.float32(delta[0]), clipped
+
+
+def server_reduce(words, length, b, requantize, seed=0, k=0):
+    """The server of scheme (b) (requantize False: index sums, b + ceil(log2 N) bits) or (c) (True: b bits)."""
+    words = np.ascontiguousarray(words, dtype=np.uint32)
+    N, stride = words.shape
+    bo = b if requantize else sum_bits_per_coordinate(b, N)
+    out = np.zeros(max(packed_words(length, bo), 1), dtype=np.uint32)
+    _check(lib().orc_server_reduce(words.ctypes.data_as(_u32p), stride, N, length, b, 1 if requantize else 0, seed, k,
+                                   out.ctypes.data_as(_u32p)))
+    return out[: packed_words(length, bo)]
+
+
+def unpack_scaled_prox(words, delta, length, bits, divisor, mu, x, eta, lambda_l1, want_v=False, want_utilde=False):
+    """A worker after the server's message: u~ = (delta * index) / divisor, then the proximal step."""
+    words = np.ascontiguousarray(words, dtype=np.uint32)
+    xn = np.array(x, dtype=np.float32, copy=True)
+    mu_a = None if mu is None else np.ascontiguousarray(mu, dtype=np.float32)
+    v = np.zeros(length, dtype=np.float32) if want_v else None
+    ut = np.zeros(length, dtype=np.float32) if want_utilde else None
+    lib().orc_unpack_scaled_prox(words.ctypes.data_as(_u32p), np.float32(delta), length, bits, divisor, _ptr(mu_a, _f32p),
+                                 xn.ctypes.data_as(_f32p), eta, lambda_l1, _ptr(v, _f32p), _ptr(ut, _f32p))
     out = (xn,)
     if want_v:
         out += (v,)

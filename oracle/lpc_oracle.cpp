@@ -42,6 +42,7 @@ constexpr int CLIP_STD = 2;     // T = min(c * std(u), ||u||_inf)  (the [-c sigm
 constexpr uint32_t TAG_ROUND = 0;    // stochastic-rounding stream
 constexpr uint32_t TAG_BATCH = 1;    // per-worker minibatch i_B
 constexpr uint32_t TAG_BATCH_J = 2;  // shared minibatch J of the double sampling
+constexpr uint32_t TAG_REQUANT = 4;   // the server's rounding variables under scheme (c)
 
 // ---------------------------------------------------------------------------------------
 // Philox4x32-10 (Salmon, Moraes, Dror, Shaw, "Parallel random numbers: as easy as 1, 2, 3",
@@ -392,6 +393,129 @@ void orc_unpack_average_prox(const uint32_t* words, int64_t stride_words, const 
 }
 
 float orc_soft_threshold(float w, float kappa) { return soft_threshold(w, kappa); }
+
+}  // extern "C"
+
+// ---------------------------------------------------------------------------------------
+// Parameter-server schemes (b) and (c) of Section 3.2.
+//
+// Both unify the scale first: delta_t = max_i delta_t^i, and every worker quantizes with delta_t
+// ("delta_t^i = delta_t for each i").  delta^i = T^i / levels is monotone in the threshold T^i, so the
+// shared scale is the scale of the worker with the largest threshold; a worker whose own vector is all
+// zero then simply sends zero codes on the shared grid.  If every worker is degenerate so is the result.
+//
+// (b) The server adds the signed grid indices, K_j = sum_i k_ij, which needs ceil(log2 N) more bits
+//     ("allows for an overflow of ceil(log N) bits"), and sends the sums back; a worker recovers
+//     u~_j = (delta_t * K_j) / N  (Eq. 3 with a common delta).  The sum is stored like any other code
+//     stream, in offset binary with b' = b + ceil(log2 N) bits: K_j + 2^(b'-1).
+// (c) The server averages and quantizes again with the same grid, u~ = Q_(delta_t,b)(avg) (Eq. 4):
+//     in grid units the average is s_j = K_j / N (one fp32 division), already inside the hull, and
+//     rule (1) of Section 2.2 rounds it with the server's own rounding stream; b bits go back.
+// The two-point extension b = 1 and the bypass b = 32 have no integer grid to add on: not offered.
+// ---------------------------------------------------------------------------------------
+int ceil_log2(int N) {
+  int r = 0;
+  while ((1 << r) < N) ++r;
+  return r;
+}
+
+extern "C" {
+
+int orc_sum_bits_per_coordinate(int b, int N) { return b + ceil_log2(N); }
+
+// Table 1: bits of one communication step 2.  scheme 0: (a) broadcast (32+bd)N(N-1);
+// 1: (b) N(64 + 2bd + d ceil(log N));  2: (c) N(64 + 2bd).
+uint64_t orc_scheme_bits(int scheme, int64_t d, int b, int N) {
+  const uint64_t bd = (uint64_t)b * (uint64_t)d;
+  if (scheme == 0) return (32u + bd) * (uint64_t)N * (uint64_t)(N - 1);
+  if (scheme == 1) return (uint64_t)N * (64u + 2u * bd + (uint64_t)d * (uint64_t)ceil_log2(N));
+  return (uint64_t)N * (64u + 2u * bd);
+}
+
+// Step 7 of Algorithm 1 for all N workers with the unified scale.  U: N vectors, vector i at U + i*ld.
+// words_out: N streams, stream i at words_out + i*stride_words.  delta_out: the one shared float.
+// clipped_out (nullable): N counts of coordinates outside the shared hull.
+int orc_quantize_pack_shared(const float* U, int N, int64_t len, int64_t ld, int b, int clip_mode,
+                             float clip_value, uint64_t seed, uint64_t k, uint32_t* words_out,
+                             int64_t stride_words, float* delta_out, uint32_t* clipped_out) {
+  if (len < 0 || N < 1 || b < 2 || b > 16) return ORC_ERR_INVALID;
+  Scale best;
+  bool have = false;
+  for (int i = 0; i < N; ++i) {
+    Scale sc;
+    const int rc = compute_scale(U + (int64_t)i * ld, len, b, clip_mode, clip_value, &sc);
+    if (rc != ORC_OK) return rc;
+    if (!sc.degenerate && (!have || sc.T > best.T)) { best = sc; have = true; }
+  }
+  *delta_out = have ? best.delta : 0.0f;
+  const int64_t W = packed_words(len, b);
+  for (int i = 0; i < N; ++i) {
+    const float* u = U + (int64_t)i * ld;
+    uint32_t* words = words_out + (int64_t)i * stride_words;
+    for (int64_t w = 0; w < W; ++w) words[w] = 0;
+    uint32_t clipped = 0;
+    for (int64_t j = 0; j < len; ++j) {
+      int kq = 0;
+      if (have) {
+        kq = quantize_coord(u[j], best.rdelta, b, rounding_bits(seed, (uint32_t)i, k, 0, j));
+        if (u[j] > best.T || u[j] < -(best.T + best.delta)) ++clipped;
+      }
+      put_code(words, j, b, code_of(kq, b));
+    }
+    if (clipped_out) clipped_out[i] = clipped;
+  }
+  return ORC_OK;
+}
+
+// The server of schemes (b) (requantize = 0) and (c) (requantize = 1).  out: one stream of
+// b + ceil(log2 N) bits per coordinate (b), or of b bits (c).
+int orc_server_reduce(const uint32_t* words, int64_t stride_words, int N, int64_t len, int b,
+                      int requantize, uint64_t seed, uint64_t k, uint32_t* out) {
+  if (len < 0 || N < 1 || b < 2 || b > 16) return ORC_ERR_INVALID;
+  const int bo = requantize ? b : b + ceil_log2(N);
+  if (bo > 16) return ORC_ERR_INVALID;
+  const int64_t W = packed_words(len, bo);
+  for (int64_t w = 0; w < W; ++w) out[w] = 0;
+  for (int64_t j = 0; j < len; ++j) {
+    int K = 0;
+    for (int i = 0; i < N; ++i) K += index_of(get_code(words + (int64_t)i * stride_words, j, b), b);
+    if (!requantize) {
+      put_code(out, j, bo, code_of(K, bo));
+    } else {
+      const float s = (float)K / (float)N;  // the average in grid units
+      uint32_t w4[4];
+      stream_block(seed, TAG_REQUANT, 0, k, (uint32_t)(j >> 3), w4);
+      const int lane = (int)(j & 7);
+      const uint32_t r16 = (w4[lane >> 1] >> (16 * (lane & 1))) & 0xFFFFu;
+      put_code(out, j, b, code_of(quantize_coord(s, 1.0f, b, r16), b));
+    }
+  }
+  return ORC_OK;
+}
+
+// A worker's side after the server's message: u~_j = (delta * index_j) / divisor, then Algorithm 1
+// steps 9-10 as in orc_unpack_average_prox.  Scheme (b): bits = b + ceil(log2 N), divisor = N;
+// scheme (c): bits = b, divisor = 1.
+void orc_unpack_scaled_prox(const uint32_t* words, float delta, int64_t len, int bits, int divisor,
+                            const float* mu, float* x_inout, float eta, float lambda_l1, float* v_out,
+                            float* utilde_out) {
+  const float inv = 1.0f / (float)divisor;
+  const float kappa = eta * lambda_l1;
+  for (int64_t j = 0; j < len; ++j) {
+    const float acc = 0.0f + decode_value(words, j, bits, delta);
+    const float ut = acc * inv;
+    const float v = ut + (mu ? mu[j] : 0.0f);
+    const float w = x_inout[j] - eta * v;
+    x_inout[j] = soft_threshold(w, kappa);
+    if (v_out) v_out[j] = v;
+    if (utilde_out) utilde_out[j] = ut;
+  }
+}
+
+}  // extern "C"
+
+extern "C" {
+
 
 // ---- linear model ---------------------------------------------------------------------
 

@@ -252,7 +252,7 @@ def test_pack_layout_and_round_trip(b):
 
 
 def test_bit_counts_match_table1():
-    rows = [l.split() for l in open(os.path.join(GOLDEN, "table1_bits.txt")) if l[0] != "#"]
+    rows = [l.split() for l in open(os.path.join(GOLDEN, "table1_bits.txt")) if l[0] != "#" and not l.startswith("ps")]
     for d, b, N, msg, bc in (map(int, r) for r in rows):
         assert orc.message_bits(d, b) == msg
         assert orc.broadcast_bits(d, b, N) == bc
