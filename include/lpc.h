@@ -82,6 +82,8 @@ typedef struct lpc_ctx lpc_ctx;
 #define LPC_OPT_USE_GRAPH 3     /* 1 (default): lpc_inner_steps replays a CUDA graph; 0: plain launches */
 #define LPC_OPT_PROFILE 4       /* 1: record CUDA events around every kernel launch (graph replay is off meanwhile) */
 
+#define LPC_OPT_SHARED_SCALE 6  /* 1: lpc_quantize_pack gives every worker the unified scale delta_t = max_i delta_t^i of the parameter-server schemes (b), (c) of Section 3.2; needs b in 2..16 */
+#define LPC_OPT_AVERAGE_DIVISOR 7 /* lpc_unpack_average_prox divides the decoded sum by this count instead of the context's N (0 = N): the worker count behind a server's sum stream */
 #define LPC_OPT_PERSISTENT 5    /* 1 (default): lpc_inner_steps runs the whole loop in one cooperative launch when it fits */
 
 /* kernel classes reported by lpc_get_profile */
@@ -190,6 +192,33 @@ int lpc_quantize_pack(lpc_ctx* ctx, const float* U, const float* U_sub, int64_t 
 int lpc_unpack_average_prox(lpc_ctx* ctx, const uint32_t* codes, const float* delta, int64_t len,
                             const int64_t* seg_offsets, int32_t nseg, const float* mu,
                             float* x_inout, float eta, float lambda_l1, float* v_out);
+
+/*
+ * The parameter-server schemes (b) and (c) of "Communication step 2" (Section 3.2, Table 1).  Both first unify the
+ * scale: with LPC_OPT_SHARED_SCALE set, lpc_quantize_pack quantizes every worker's vector with
+ * delta_t = max_i delta_t^i (per tensor segment) and writes that value to all N rows of delta_out.
+ *
+ * lpc_server_reduce is the server.  codes: the N streams that lpc_quantize_pack wrote (device, layout of
+ * lpc_packed_layout for the context's b).  codes_out: ONE stream (device, 16-byte aligned), laid out by
+ * lpc_packed_layout for the output width:
+ *   LPC_SCHEME_SERVER_SUM        scheme (b): the sums K_j = sum_i k_ij of the signed grid indices, stored like codes
+ *                                in offset binary with b + ceil(log2 N) bits (lpc_sum_bits), nothing lost;
+ *   LPC_SCHEME_SERVER_REQUANTIZE scheme (c), Eq. 4: the average K_j / N rounded back to the b-bit grid by rule (1) of
+ *                                Section 2.2 with the server's own rounding stream keyed by (seed, k); b bits.
+ * A worker then decodes the server's stream with lpc_unpack_average_prox on a context made for ONE stream of the
+ * output width, passing one row of delta_out; under scheme (b) that context has LPC_OPT_AVERAGE_DIVISOR = N, so
+ * that u~_j = (delta_t * K_j) / N (Eq. 3 with a common scale).
+ * Counts N*(64 + b*d + b_out*d) step-2 bits per segment (Table 1: N(64 + 2bd + d ceil(log N)) and N(64 + 2bd)).
+ * Errors: LPC_ERR_UNSUPPORTED for b = 1 or 32 (no integer grid to add on) and when b + ceil(log2 N) > 16.
+ * lpc_scheme_bits evaluates Table 1's three formulas for one step (host only).
+ */
+#define LPC_SCHEME_BROADCAST 0
+#define LPC_SCHEME_SERVER_SUM 1
+#define LPC_SCHEME_SERVER_REQUANTIZE 2
+int lpc_server_reduce(lpc_ctx* ctx, const uint32_t* codes, int64_t len, const int64_t* seg_offsets, int32_t nseg,
+                      int scheme, uint64_t k, uint32_t* codes_out);
+int lpc_sum_bits(int32_t b, int32_t N, int32_t* bits_out); /* b + ceil(log2 N) */
+int lpc_scheme_bits(int scheme, int64_t d, int32_t b, int32_t N, uint64_t* bits_out);
 
 /*
  * ALPC-SVRG (Algorithms 2 and 3).  lpc_alpc_begin sets y_0 = z_0 = x and clears the y sum.

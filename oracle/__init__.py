@@ -62,9 +62,10 @@ def _declare(L):
     L.orc_scheme_bits.argtypes = [C.c_int, C.c_int64, C.c_int, C.c_int]
     L.orc_scheme_bits.restype = C.c_uint64
     L.orc_quantize_pack_shared.argtypes = [_f32p, C.c_int, C.c_int64, C.c_int64, C.c_int, C.c_int, C.c_float, C.c_uint64,
-                                           C.c_uint64, _u32p, C.c_int64, _f32p, _u32p]
+                                           C.c_uint64, C.c_uint32, _u32p, C.c_int64, _f32p, _u32p]
     L.orc_quantize_pack_shared.restype = C.c_int
-    L.orc_server_reduce.argtypes = [_u32p, C.c_int64, C.c_int, C.c_int64, C.c_int, C.c_int, C.c_uint64, C.c_uint64, _u32p]
+    L.orc_server_reduce.argtypes = [_u32p, C.c_int64, C.c_int, C.c_int64, C.c_int, C.c_int, C.c_uint64, C.c_uint64, C.c_uint32,
+                                    _u32p]
     L.orc_server_reduce.restype = C.c_int
     L.orc_unpack_scaled_prox.argtypes = [_u32p, C.c_float, C.c_int64, C.c_int, C.c_int, _f32p, _f32p, C.c_float, C.c_float,
                                          _f32p, _f32p]
@@ -260,7 +261,7 @@ def scheme_bits(scheme, d, b, N):
     return int(lib().orc_scheme_bits(scheme, d, b, N))
 
 
-def quantize_pack_shared(U, b, clip_mode=CLIP_NONE, clip_value=1.0, seed=0, k=0):
+def quantize_pack_shared(U, b, clip_mode=CLIP_NONE, clip_value=1.0, seed=0, k=0, block_base=0):
     """All N worker vectors (rows of U) with the unified scale of schemes (b)/(c).
     Returns (words (N, W), delta, clipped (N,))."""
     U = np.ascontiguousarray(U, dtype=np.float32)
@@ -270,19 +271,19 @@ def quantize_pack_shared(U, b, clip_mode=CLIP_NONE, clip_value=1.0, seed=0, k=0)
     delta = np.zeros(1, dtype=np.float32)
     clipped = np.zeros(N, dtype=np.uint32)
     _check(lib().orc_quantize_pack_shared(U.ctypes.data_as(_f32p), N, length, length, b, clip_mode, clip_value, seed, k,
-                                          words.ctypes.data_as(_u32p), W, delta.ctypes.data_as(_f32p),
+                                          block_base, words.ctypes.data_as(_u32p), W, delta.ctypes.data_as(_f32p),
                                           clipped.ctypes.data_as(_u32p)))
     return words[:, : packed_words(length, b)], np.float32(delta[0]), clipped
 
 
-def server_reduce(words, length, b, requantize, seed=0, k=0):
+def server_reduce(words, length, b, requantize, seed=0, k=0, block_base=0):
     """The server of scheme (b) (requantize False: index sums, b + ceil(log2 N) bits) or (c) (True: b bits)."""
     words = np.ascontiguousarray(words, dtype=np.uint32)
     N, stride = words.shape
     bo = b if requantize else sum_bits_per_coordinate(b, N)
     out = np.zeros(max(packed_words(length, bo), 1), dtype=np.uint32)
     _check(lib().orc_server_reduce(words.ctypes.data_as(_u32p), stride, N, length, b, 1 if requantize else 0, seed, k,
-                                   out.ctypes.data_as(_u32p)))
+                                   block_base, out.ctypes.data_as(_u32p)))
     return out[: packed_words(length, bo)]
 
 

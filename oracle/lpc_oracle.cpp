@@ -399,13 +399,13 @@ float orc_soft_threshold(float w, float kappa) { return soft_threshold(w, kappa)
 // ---------------------------------------------------------------------------------------
 // Parameter-server schemes (b) and (c) of Section 3.2.
 //
-// Both unify the scale first: delta_t = max_i delta_t^i, and every worker quantizes with delta_t
-// ("delta_t^i = delta_t for each i").  delta^i = T^i / levels is monotone in the threshold T^i, so the
+// Both unify the scale first: delta_t = max_i delta_t^i, and every worker quantizes with delta_t in
+// step 7.  delta^i = T^i / levels is monotone in the threshold T^i, so the
 // shared scale is the scale of the worker with the largest threshold; a worker whose own vector is all
 // zero then simply sends zero codes on the shared grid.  If every worker is degenerate so is the result.
 //
-// (b) The server adds the signed grid indices, K_j = sum_i k_ij, which needs ceil(log2 N) more bits
-//     ("allows for an overflow of ceil(log N) bits"), and sends the sums back; a worker recovers
+// (b) The server adds the signed grid indices, K_j = sum_i k_ij, which takes the ceil(log2 N) more bits
+//     per coordinate that the scheme grants the sum, and sends the sums back; a worker recovers
 //     u~_j = (delta_t * K_j) / N  (Eq. 3 with a common delta).  The sum is stored like any other code
 //     stream, in offset binary with b' = b + ceil(log2 N) bits: K_j + 2^(b'-1).
 // (c) The server averages and quantizes again with the same grid, u~ = Q_(delta_t,b)(avg) (Eq. 4):
@@ -434,9 +434,10 @@ uint64_t orc_scheme_bits(int scheme, int64_t d, int b, int N) {
 
 // Step 7 of Algorithm 1 for all N workers with the unified scale.  U: N vectors, vector i at U + i*ld.
 // words_out: N streams, stream i at words_out + i*stride_words.  delta_out: the one shared float.
-// clipped_out (nullable): N counts of coordinates outside the shared hull.
+// clipped_out (nullable): N counts of coordinates outside the shared hull.  block_base: first block of
+// the rounding streams (a tensor segment of a longer vector continues the count of its predecessors).
 int orc_quantize_pack_shared(const float* U, int N, int64_t len, int64_t ld, int b, int clip_mode,
-                             float clip_value, uint64_t seed, uint64_t k, uint32_t* words_out,
+                             float clip_value, uint64_t seed, uint64_t k, uint32_t block_base, uint32_t* words_out,
                              int64_t stride_words, float* delta_out, uint32_t* clipped_out) {
   if (len < 0 || N < 1 || b < 2 || b > 16) return ORC_ERR_INVALID;
   Scale best;
@@ -457,7 +458,7 @@ int orc_quantize_pack_shared(const float* U, int N, int64_t len, int64_t ld, int
     for (int64_t j = 0; j < len; ++j) {
       int kq = 0;
       if (have) {
-        kq = quantize_coord(u[j], best.rdelta, b, rounding_bits(seed, (uint32_t)i, k, 0, j));
+        kq = quantize_coord(u[j], best.rdelta, b, rounding_bits(seed, (uint32_t)i, k, block_base, j));
         if (u[j] > best.T || u[j] < -(best.T + best.delta)) ++clipped;
       }
       put_code(words, j, b, code_of(kq, b));
@@ -470,7 +471,7 @@ int orc_quantize_pack_shared(const float* U, int N, int64_t len, int64_t ld, int
 // The server of schemes (b) (requantize = 0) and (c) (requantize = 1).  out: one stream of
 // b + ceil(log2 N) bits per coordinate (b), or of b bits (c).
 int orc_server_reduce(const uint32_t* words, int64_t stride_words, int N, int64_t len, int b,
-                      int requantize, uint64_t seed, uint64_t k, uint32_t* out) {
+                      int requantize, uint64_t seed, uint64_t k, uint32_t block_base, uint32_t* out) {
   if (len < 0 || N < 1 || b < 2 || b > 16) return ORC_ERR_INVALID;
   const int bo = requantize ? b : b + ceil_log2(N);
   if (bo > 16) return ORC_ERR_INVALID;
@@ -484,7 +485,7 @@ int orc_server_reduce(const uint32_t* words, int64_t stride_words, int N, int64_
     } else {
       const float s = (float)K / (float)N;  // the average in grid units
       uint32_t w4[4];
-      stream_block(seed, TAG_REQUANT, 0, k, (uint32_t)(j >> 3), w4);
+      stream_block(seed, TAG_REQUANT, 0, k, block_base + (uint32_t)(j >> 3), w4);
       const int lane = (int)(j & 7);
       const uint32_t r16 = (w4[lane >> 1] >> (16 * (lane & 1))) & 0xFFFFu;
       put_code(out, j, b, code_of(quantize_coord(s, 1.0f, b, r16), b));

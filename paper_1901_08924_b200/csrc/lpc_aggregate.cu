@@ -88,7 +88,7 @@ __global__ void __launch_bounds__(AT) unpack_average_prox_kernel(AggArgs a) {
   for (int i = tid; i < a.N; i += AT) sdelta[i] = a.delta[(int64_t)i * a.nseg + seg];
   __syncthreads();
 
-  const float invN = __fdiv_rn(1.0f, (float)a.N);
+  const float invN = __fdiv_rn(1.0f, (float)a.divisor);
   float* xs = a.x + s.off;
   const float* mus = a.mu ? a.mu + s.off : nullptr;
   float* vs = a.v_out ? a.v_out + s.off : nullptr;
@@ -167,7 +167,87 @@ __global__ void __launch_bounds__(AT) unpack_average_prox_kernel(AggArgs a) {
   if (a.k_counter && blockIdx.x == 0 && tid == 0) *a.k_counter += 1;
 }
 
+// The server of schemes (b) and (c) (Section 3.2).  A thread owns 8 consecutive coordinates per sweep: it adds the
+// codes of the N streams as integers, then either stores the index sums K_j in offset binary with b_out =
+// b + ceil(log2 N) bits (scheme (b) grants the sum that many more bits), or rounds the average K_j / N back to the
+// b-bit grid with rule (1) of Section 2.2 and the server's own rounding stream (scheme (c), Eq. 4).  The 8 * b_out
+// output bits of a thread are b_out whole bytes, staged through shared memory and written out as words.
+template <int BITS>  // input width: 2, 4, 8 fixed; 0: b in 2..16 from the arguments
+__global__ void __launch_bounds__(AT) server_reduce_kernel(ServerArgs a) {
+  const int tile = blockIdx.x;
+  const int seg = a.tile_seg ? a.tile_seg[tile] : 0;
+  const SegInfo s = a.segs[seg];
+  const SegInfo so = a.segs_out[seg];
+  const int64_t tstart = (int64_t)(tile - s.tile_first) * TILE;
+  const int tid = threadIdx.x;
+  const int b = (BITS == 0) ? a.b : BITS;
+  const int bo = a.b_out;
+  const int bias_in = a.N << (b - 1);  // sum of the offsets of N codes
+  const float fN = (float)a.N;
+  __shared__ __align__(16) uint8_t stage[AT * 16];
+  const uint32_t* w = a.codes + s.word_off;
+  uint32_t* out = a.out + so.word_off;
+#pragma unroll 1
+  for (int it = 0; it < AITER; ++it) {
+    const int64_t sweep0 = tstart + (int64_t)it * AGROUP;
+    if (sweep0 >= s.len) break;  // uniform for the block
+    const int64_t j = sweep0 + tid * 8;
+    const int nvalid = (j < s.len) ? (int)min((int64_t)8, s.len - j) : 0;
+    int K[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) K[e] = -bias_in;
+    if (nvalid > 0) {
+#pragma unroll 4
+      for (int i = 0; i < a.N; ++i) {
+        uint64_t lo, hi;
+        load_chunk<BITS>(w + (int64_t)i * a.stride_words, j >> 3, b, s.pad_words, lo, hi);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) K[e] += (int)extract(lo, hi, e * b, b);
+      }
+    }
+    uint64_t olo = 0, ohi = 0;
+    if (nvalid > 0) {
+      U4 r = U4{0, 0, 0, 0};
+      if (a.requantize) r = stream_block(a.seed, TAG_REQUANT, 0u, a.k, s.block_base + (uint32_t)(j >> 3));
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        if (e < nvalid) {
+          uint32_t code;
+          if (a.requantize) code = quantize_code_rt(__fdiv_rn((float)K[e], fN), 1.0f, lane16(r, e), b);
+          else code = (uint32_t)(K[e] + (1 << (bo - 1)));
+          const int pos = e * bo;
+          if (pos < 64) {
+            olo |= (uint64_t)code << pos;
+            if (pos + bo > 64) ohi |= (uint64_t)code >> (64 - pos);
+          } else {
+            ohi |= (uint64_t)code << (pos - 64);
+          }
+        }
+      }
+    }
+    if (it > 0) __syncthreads();
+    for (int i = 0; i < bo; ++i) stage[tid * bo + i] = (uint8_t)((i < 8) ? (olo >> (8 * i)) : (ohi >> (8 * (i - 8))));
+    __syncthreads();
+    const int64_t w0 = (sweep0 >> 5) * bo;  // sweep0 is a multiple of 2048, so this is exact
+    const uint32_t* stw = reinterpret_cast<const uint32_t*>(stage);
+    for (int q = tid; q < (AGROUP / 32) * bo; q += AT)
+      if (w0 + q < so.pad_words) out[w0 + q] = stw[q];
+  }
+}
+
 }  // namespace
+
+cudaError_t launch_server_reduce(const ServerArgs& a, cudaStream_t st) {
+  if (a.ntiles <= 0) return cudaSuccess;
+  const dim3 grid((unsigned)a.ntiles), block(AT);
+  switch (a.b) {
+    case 2: server_reduce_kernel<2><<<grid, block, 0, st>>>(a); break;
+    case 4: server_reduce_kernel<4><<<grid, block, 0, st>>>(a); break;
+    case 8: server_reduce_kernel<8><<<grid, block, 0, st>>>(a); break;
+    default: server_reduce_kernel<0><<<grid, block, 0, st>>>(a); break;
+  }
+  return cudaGetLastError();
+}
 
 cudaError_t launch_unpack_average_prox(const AggArgs& a, cudaStream_t st) {
   if (a.ntiles <= 0) return cudaSuccess;

@@ -94,6 +94,9 @@ struct lpc_ctx {
   int64_t persist_launches = 0;
   // stand-alone quantizer
   SegPlan seg;
+  SegPlan seg_out;       // layout of the server's output stream (schemes (b), (c))
+  int shared_scale = 0;  // LPC_OPT_SHARED_SCALE
+  int divisor = 0;       // LPC_OPT_AVERAGE_DIVISOR; 0: the worker count N
   uint32_t* q_pmax = nullptr;
   float *q_ps1 = nullptr, *q_ps2 = nullptr;
   size_t q_part_cap = 0;
@@ -303,6 +306,7 @@ AggArgs agg_args(lpc_ctx* c, const SegPlan& p, const uint32_t* codes, const floa
                  float eta, float lambda_l1, float* v_out) {
   AggArgs a;
   a.codes = codes; a.stride_words = p.stride_words; a.delta = delta; a.N = c->N; a.b = c->b;
+  a.divisor = c->divisor > 0 ? c->divisor : c->N;
   a.segs = p.d_segs; a.tile_seg = p.d_tile_seg; a.nseg = p.nseg; a.ntiles = p.ntiles;
   a.mu = mu; a.x = x; a.eta = eta; a.lambda_l1 = lambda_l1; a.v_out = v_out; a.k_counter = nullptr;
   a.mode = 0; a.y = nullptr; a.z = nullptr; a.ysum = nullptr; a.vhat = nullptr; a.alpha = 0.f; a.inv4L = 0.f;
@@ -568,6 +572,7 @@ int lpc_destroy(lpc_ctx* c) {
     if (p) cudaFree(p);
   free_plan(c->inner_seg);
   free_plan(c->seg);
+  free_plan(c->seg_out);
   delete c;
   return LPC_OK;
 }
@@ -592,6 +597,14 @@ int lpc_set_option(lpc_ctx* c, int option, int64_t value) {
       return LPC_OK;
     case LPC_OPT_USE_GRAPH: c->use_graph = value ? 1 : 0; return LPC_OK;
     case LPC_OPT_PERSISTENT: c->use_persist = value ? 1 : 0; return LPC_OK;
+    case LPC_OPT_SHARED_SCALE:
+      if (value && (c->b < 2 || c->b > 16)) return fail(c, LPC_ERR_UNSUPPORTED, "a unified scale needs an integer grid: b in 2..16");
+      c->shared_scale = value ? 1 : 0;
+      return LPC_OK;
+    case LPC_OPT_AVERAGE_DIVISOR:
+      if (value < 0 || value > (1 << 20)) return fail(c, LPC_ERR_INVALID_ARG, "divisor");
+      c->divisor = (int)value;
+      return LPC_OK;
     case LPC_OPT_PROFILE:
       TRY(prof_resolve(c));
       c->profile = value ? 1 : 0;
@@ -780,8 +793,58 @@ int lpc_quantize_pack(lpc_ctx* c, const float* U, const float* U_sub, int64_t le
   a.pmax = c->q_pmax; a.ps1 = c->q_ps1; a.ps2 = c->q_ps2; a.scales = c->q_scales;
   a.codes = codes_out; a.stride_words = p.stride_words; a.delta_out = delta_out;
   a.clipped_out = clipped_out ? clipped_out : c->q_clip; a.count_clipped = clipped_out ? 1 : 0; a.dev_status = c->dev_status;
+  a.shared_scale = c->shared_scale;
   CU(c, launch_quantize_pack(a, c->stream, c->profile ? prof_hook : nullptr, c));
-  c->step2_bits += p.msg_bits * (uint64_t)c->N * (uint64_t)(c->N - 1);
+  if (!c->shared_scale) c->step2_bits += p.msg_bits * (uint64_t)c->N * (uint64_t)(c->N - 1);  // scheme (a); the server schemes count in lpc_server_reduce
+  return LPC_OK;
+}
+
+namespace {
+int ceil_log2_int(int N) {
+  int r = 0;
+  while ((1 << r) < N) ++r;
+  return r;
+}
+}  // namespace
+
+int lpc_sum_bits(int32_t b, int32_t N, int32_t* bits_out) {
+  if (!bits_out || b < 2 || b > 16 || N < 1) return LPC_ERR_INVALID_ARG;
+  *bits_out = b + ceil_log2_int(N);
+  return LPC_OK;
+}
+
+int lpc_scheme_bits(int scheme, int64_t d, int32_t b, int32_t N, uint64_t* bits_out) {
+  if (!bits_out || d < 0 || b < 1 || N < 1) return LPC_ERR_INVALID_ARG;
+  const uint64_t bd = (uint64_t)b * (uint64_t)d;
+  switch (scheme) {
+    case LPC_SCHEME_BROADCAST: *bits_out = (32u + bd) * (uint64_t)N * (uint64_t)(N - 1); return LPC_OK;
+    case LPC_SCHEME_SERVER_SUM: *bits_out = (uint64_t)N * (64u + 2u * bd + (uint64_t)d * (uint64_t)ceil_log2_int(N)); return LPC_OK;
+    case LPC_SCHEME_SERVER_REQUANTIZE: *bits_out = (uint64_t)N * (64u + 2u * bd); return LPC_OK;
+    default: return LPC_ERR_INVALID_ARG;
+  }
+}
+
+int lpc_server_reduce(lpc_ctx* c, const uint32_t* codes, int64_t len, const int64_t* seg_offsets, int32_t nseg, int scheme,
+                      uint64_t k, uint32_t* codes_out) {
+  if (!c) return LPC_ERR_INVALID_ARG;
+  if (len > 0 && (!codes || !codes_out)) return fail(c, LPC_ERR_INVALID_ARG, "null streams");
+  if (len < 0 || nseg < 1) return fail(c, LPC_ERR_INVALID_ARG, "len / nseg");
+  if (scheme != LPC_SCHEME_SERVER_SUM && scheme != LPC_SCHEME_SERVER_REQUANTIZE) return fail(c, LPC_ERR_INVALID_ARG, "scheme");
+  if (c->b < 2 || c->b > 16) return fail(c, LPC_ERR_UNSUPPORTED, "the server schemes need an integer grid: b in 2..16");
+  const int b_out = (scheme == LPC_SCHEME_SERVER_SUM) ? c->b + ceil_log2_int(c->N) : c->b;
+  if (b_out > 16) return fail(c, LPC_ERR_UNSUPPORTED, "b + ceil(log2 N) exceeds 16 bits");
+  if (!aligned16(codes) || !aligned16(codes_out)) return fail(c, LPC_ERR_INVALID_ARG, "streams must be 16-byte aligned");
+  TRY(make_plan(c, c->seg, len, c->b, seg_offsets, nseg));
+  TRY(make_plan(c, c->seg_out, len, b_out, seg_offsets, nseg));
+  ServerArgs a;
+  a.codes = codes; a.stride_words = c->seg.stride_words; a.N = c->N; a.b = c->b; a.b_out = b_out;
+  a.requantize = (scheme == LPC_SCHEME_SERVER_REQUANTIZE) ? 1 : 0; a.seed = c->seed; a.k = k;
+  a.segs = c->seg.d_segs; a.segs_out = c->seg_out.d_segs; a.tile_seg = c->seg.d_tile_seg; a.nseg = nseg; a.ntiles = c->seg.ntiles;
+  a.out = codes_out;
+  { ProfScope ps_(c, LPC_KERNEL_AGGREGATE); CU(c, launch_server_reduce(a, c->stream)); }
+  // Table 1: every worker sends its message (b bits per coordinate and the scale) and receives the server's (b_out bits
+  // per coordinate and the scale), per tensor segment
+  c->step2_bits += (uint64_t)c->N * (c->seg.msg_bits + c->seg_out.msg_bits);
   return LPC_OK;
 }
 

@@ -17,6 +17,7 @@ namespace lpc {
 constexpr uint32_t TAG_ROUND = 0;
 constexpr uint32_t TAG_BATCH = 1;
 constexpr uint32_t TAG_BATCH_J = 2;
+constexpr uint32_t TAG_REQUANT = 4;  // the server's rounding variables under scheme (c) of Section 3.2
 
 // Philox4x32-10 (Salmon et al., SC'11).  Ten rounds; each round multiplies counter words 0 and 2 by
 // two fixed constants, xors the high halves with the other two words and the key, and the key

@@ -49,6 +49,7 @@ struct QuantArgs {
   float* delta_out;       // N * nseg
   uint32_t* clipped_out;  // N * nseg, cleared by the finish kernel (never null: internal scratch when the caller gives none)
   int count_clipped;      // 0: skip counting the coordinates outside the hull (the counts stay zero)
+  int shared_scale;       // 1: every worker quantizes with delta_t = max_i delta_t^i (schemes (b), (c) of Section 3.2)
   unsigned int* dev_status;
 };
 
@@ -62,6 +63,7 @@ struct AggArgs {
   const float* delta;  // N * nseg
   int N;
   int b;
+  int divisor;      // the decoded sum is divided by this count: N for Eq. 3; the worker count behind a server's sum stream
   const SegInfo* segs;
   const int32_t* tile_seg;
   int nseg;
@@ -85,6 +87,25 @@ struct AggArgs {
 };
 
 cudaError_t launch_unpack_average_prox(const AggArgs& a, cudaStream_t st);
+
+// The server of the parameter-server schemes (Section 3.2): N code streams of b bits on one grid in, one stream out.
+struct ServerArgs {
+  const uint32_t* codes;   // N streams, stream i at codes + i * stride_words, segment layout `segs`
+  int64_t stride_words;
+  int N;
+  int b;
+  int b_out;               // scheme (b): b + ceil(log2 N), index sums; scheme (c): b, re-quantized average
+  int requantize;
+  uint64_t seed;
+  uint64_t k;
+  const SegInfo* segs;     // layout of the input streams (width b)
+  const SegInfo* segs_out; // layout of the output stream (width b_out): same segments and tiles, other word offsets
+  const int32_t* tile_seg;
+  int nseg;
+  int ntiles;
+  uint32_t* out;
+};
+cudaError_t launch_server_reduce(const ServerArgs& a, cudaStream_t st);
 
 }  // namespace lpc
 

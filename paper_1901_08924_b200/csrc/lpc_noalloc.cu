@@ -99,7 +99,7 @@ extern "C" int lpc_quantize_pack_static(const float* U, int64_t len, int64_t ld,
   a.ps2 = reinterpret_cast<float*>(base + OFF_PS2);
   a.scales = reinterpret_cast<ScaleRec*>(base + OFF_SCALES);
   a.codes = codes_out; a.stride_words = seg.pad_words;
-  a.delta_out = delta_out; a.clipped_out = clipped_out; a.count_clipped = 1;
+  a.delta_out = delta_out; a.clipped_out = clipped_out; a.count_clipped = 1; a.shared_scale = 0;
   a.dev_status = reinterpret_cast<unsigned int*>(base + OFF_STATUS);
   return launch_quantize_pack(a, st) == cudaSuccess ? LPC_OK : LPC_ERR_CUDA;
 }

@@ -148,6 +148,33 @@ __global__ void __launch_bounds__(QT) finish_kernel(QuantArgs a) {
   }
 }
 
+// ---- schemes (b), (c) of Section 3.2: delta_t = max_i delta_t^i.  delta^i = T^i / levels grows with the threshold
+// T^i, so the record of the worker with the largest threshold is the unified scale; it replaces every worker's
+// record of the segment.  Workers whose own vector is zero then send zeros on the shared grid; when every worker
+// is degenerate nothing changes.  One warp per segment.
+__global__ void __launch_bounds__(32) share_scale_kernel(QuantArgs a) {
+  const int seg = blockIdx.x, lane = threadIdx.x;
+  float bestT = -1.f;
+  int best = -1;
+  for (int i = lane; i < a.N; i += 32) {
+    const ScaleRec r = a.scales[(int64_t)i * a.nseg + seg];
+    if (!(r.flags & 1u) && r.T > bestT) { bestT = r.T; best = i; }  // the first worker among equal thresholds
+  }
+#pragma unroll
+  for (int m = 16; m >= 1; m >>= 1) {
+    const float oT = __shfl_xor_sync(0xFFFFFFFFu, bestT, m);
+    const int ob = __shfl_xor_sync(0xFFFFFFFFu, best, m);
+    if (ob >= 0 && (best < 0 || oT > bestT || (oT == bestT && ob < best))) { bestT = oT; best = ob; }
+  }
+  if (best < 0) return;
+  const ScaleRec r = a.scales[(int64_t)best * a.nseg + seg];
+  __syncwarp();
+  for (int i = lane; i < a.N; i += 32) {
+    a.scales[(int64_t)i * a.nseg + seg] = r;
+    a.delta_out[(int64_t)i * a.nseg + seg] = r.delta;
+  }
+}
+
 // ---- pass 2: quantize and pack -----------------------------------------------------------------------------
 // BITS = 1, 2, 4, 8: register/shuffle packing with direct coalesced stores.
 // BITS = 0: any b in 1..16 read from the arguments; each thread's 8*b bits are b whole bytes, staged
@@ -416,6 +443,7 @@ cudaError_t launch_quantize_pack(const QuantArgs& a, cudaStream_t st, LaunchHook
   if (hook) hook(user, 5 /* LPC_KERNEL_OTHER */, 1);
   finish_kernel<<<dim3((unsigned)a.nseg, (unsigned)a.N), block, 0, st>>>(a);  // also covers empty segments
   if (hook) hook(user, 5, 0);
+  if (a.shared_scale) share_scale_kernel<<<(unsigned)a.nseg, 32, 0, st>>>(a);
   if (a.ntiles <= 0) return cudaGetLastError();
   struct Close {  // closes the timing scope of the second pass on every return path
     LaunchHook h; void* u;

@@ -18,6 +18,8 @@ CLIP_NONE, CLIP_LAMBDA, CLIP_STD = 0, 1, 2
 (BUF_X, BUF_XTILDE, BUF_MU, BUF_MARGINS, BUF_Y, BUF_Z, BUF_YSUM, BUF_CODES, BUF_DELTA, BUF_CLIPPED, BUF_BATCH_IDX,
  BUF_COEF, BUF_U, BUF_V, BUF_VHAT) = range(15)
 OPT_SAMPLE_GLOBAL, OPT_TAP_U, OPT_CLUSTER_SIZE, OPT_USE_GRAPH, OPT_PROFILE, OPT_PERSISTENT = 0, 1, 2, 3, 4, 5
+OPT_SHARED_SCALE, OPT_AVERAGE_DIVISOR = 6, 7
+SCHEME_BROADCAST, SCHEME_SERVER_SUM, SCHEME_SERVER_REQUANTIZE = 0, 1, 2
 (INFO_STEP_CLUSTER_SIZE, INFO_LOOP_CLUSTER_SIZE, INFO_LOOP_LAUNCHES, INFO_SNAPSHOT_ROWS_PER_TILE, INFO_SNAPSHOT_STAGES,
  INFO_ALPC_LOOP_CLUSTER_SIZE, INFO_LOOP_ROW_BUFFERS, INFO_ALPC_LOOP_ROW_BUFFERS, INFO_STEP_RING_STAGES) = range(9)
 KERNEL_NAMES = ["snapshot", "worker", "aggregate", "quant_stats", "quant_pack", "other", "inner_loop"]
@@ -42,6 +44,9 @@ SYMBOLS = [
     ("lpc_packed_words", _int, [_i64, _i32, _i64p]),
     ("lpc_quantize_pack", _int, [_vp, _vp, _vp, _i64, _i64, _i64p, _i32, _u64, _vp, _vp, _vp]),
     ("lpc_unpack_average_prox", _int, [_vp, _vp, _vp, _i64, _i64p, _i32, _vp, _vp, _f32, _f32, _vp]),
+    ("lpc_server_reduce", _int, [_vp, _vp, _i64, _i64p, _i32, _int, _u64, _vp]),
+    ("lpc_sum_bits", _int, [_i32, _i32, C.POINTER(C.c_int32)]),
+    ("lpc_scheme_bits", _int, [_int, _i64, _i32, _i32, _u64p]),
     ("lpc_alpc_begin", _int, [_vp]),
     ("lpc_alpc_double_sample_step", _int, [_vp, _f32, _f32, _f32, _f32, _u64]),
     ("lpc_alpc_double_sample_steps", _int, [_vp, _f32, _f32, _f32, _f32, _u64, _i64]),
@@ -96,6 +101,22 @@ def packed_words(length, b):
     rc = lib().lpc_packed_words(length, b, C.byref(out))
     if rc != OK:
         raise LpcError(rc)
+    return out.value
+
+
+def sum_bits(b, N):
+    out = C.c_int32(0)
+    rc = lib().lpc_sum_bits(b, N, C.byref(out))
+    if rc != OK:
+        raise LpcError(rc, "lpc_sum_bits")
+    return out.value
+
+
+def scheme_bits(scheme, d, b, N):
+    out = C.c_uint64(0)
+    rc = lib().lpc_scheme_bits(scheme, d, b, N, C.byref(out))
+    if rc != OK:
+        raise LpcError(rc, "lpc_scheme_bits")
     return out.value
 
 
@@ -219,6 +240,16 @@ class Context:
         self._ck(lib().lpc_unpack_average_prox(self._h, _ptr(codes), _ptr(delta), length, arr, nseg, _ptr(mu), _ptr(x),
                                                eta, lambda_l1, _ptr(v_out)))
         return x
+
+    def server_reduce(self, codes, length, scheme, k, seg_offsets=None, codes_out=None):
+        """The server of scheme (b) or (c): N streams of b bits in, one stream out.  Returns (codes_out, bits_out)."""
+        arr, nseg = _seg(seg_offsets)
+        bo = sum_bits(self.b, self.N) if scheme == SCHEME_SERVER_SUM else self.b
+        _, stride = packed_layout(length, bo, seg_offsets)
+        if codes_out is None:
+            codes_out = torch.empty((1, stride), dtype=torch.int32, device=codes.device)
+        self._ck(lib().lpc_server_reduce(self._h, _ptr(codes), length, arr, nseg, scheme, k, _ptr(codes_out)))
+        return codes_out, bo
 
     def alpc_begin(self):
         self._ck(lib().lpc_alpc_begin(self._h))
