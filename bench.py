@@ -312,6 +312,27 @@ def quantize_aggregate_bench(dev, peak, log2_len=26, dnn=True):
                           "note": "two passes: 4 B stats read + 4 B quantize read + b/8 B written per element"},
         "unpack_average_prox": {"ms": round(ta, 4), "bytes": ba, "gbs": round(ba / ta * 1e-6, 1), "frac": round(ba / ta * 1e-6 / peak, 4)},
         "combined_gbs": round((bq + ba) / (tq + ta) * 1e-6, 1)}
+    # the parameter-server schemes (b) and (c) on the same vectors: unified scale, server, worker-side decode
+    q.set_option(lpc.OPT_SHARED_SCALE, 1)
+    tqs = _time_calls(quant, dev, 5)
+    ps = {"quantize_pack_unified_scale": {"ms": round(tqs, 4), "gbs": round(bq / tqs * 1e-6, 1), "frac": round(bq / tqs * 1e-6 / peak, 4)}}
+    for name, scheme in (("scheme_b_sum", lpc.SCHEME_SERVER_SUM), ("scheme_c_requantize", lpc.SCHEME_SERVER_REQUANTIZE)):
+        srv, bo = q.server_reduce(codes, length, scheme, 1)
+        ts = _time_calls(lambda: q.server_reduce(codes, length, scheme, 1, codes_out=srv), dev, 10)
+        w = lpc.Context(None, None, lpc.LOGISTIC, 0.0, 1, 1, bo, lpc.CLIP_NONE, 1.0, 0)
+        if scheme == lpc.SCHEME_SERVER_SUM:
+            w.set_option(lpc.OPT_AVERAGE_DIVISOR, N)
+        d1 = delta[:1].contiguous()
+        tw = _time_calls(lambda: w.unpack_average_prox(srv, d1, length, x, 1.0, 1e-3), dev, 10)
+        w.sync_status()
+        w.close()
+        bs, bw = length * (N * b / 8 + bo / 8), length * (bo / 8 + 12)
+        ps[name] = {"bits_back": bo,
+                    "server": {"ms": round(ts, 4), "bytes": bs, "gbs": round(bs / ts * 1e-6, 1), "frac": round(bs / ts * 1e-6 / peak, 4)},
+                    "worker_decode_prox": {"ms": round(tw, 4), "bytes": bw, "gbs": round(bw / tw * 1e-6, 1),
+                                           "frac": round(bw / tw * 1e-6 / peak, 4)}}
+    q.sync_status()
+    res["parameter_server_N8_len2^%d_b4" % log2_len] = ps
     q.close()
     del U, codes, x
     if not dnn:
@@ -359,6 +380,8 @@ def fused_large_batch_bench(dev, peak, n=65536, steps=30):
                                    device=dev)
     out = {"workload": "fused_step_logistic_%dx8192_N32" % n}
     for B, bits in ((256, (2, 8)), (1024, (2,))):
+        if N * B > n:  # a small matrix for profiler captures: the larger minibatch does not fit its row partitions
+            continue
         for b in bits:
             ctx = lpc.Context(X, y, lpc.LOGISTIC, 1e-5, N, B, b, lpc.CLIP_STD, 2.0, 0)
             ctx.snapshot_full_grad()

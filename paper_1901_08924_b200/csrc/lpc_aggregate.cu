@@ -172,6 +172,69 @@ __global__ void __launch_bounds__(AT) unpack_average_prox_kernel(AggArgs a) {
 // b + ceil(log2 N) bits (scheme (b) grants the sum that many more bits), or rounds the average K_j / N back to the
 // b-bit grid with rule (1) of Section 2.2 and the server's own rounding stream (scheme (c), Eq. 4).  The 8 * b_out
 // output bits of a thread are b_out whole bytes, staged through shared memory and written out as words.
+// Sums of the codes of the N streams at 8 coordinates (K[e] += sum_i code_ie).  The fixed widths add whole words of
+// codes as small integer lanes (4-bit codes in 8-bit lanes, 8-bit codes in 16-bit lanes) and spread the lanes out
+// before they could overflow.
+template <int BITS>
+__device__ __forceinline__ void sum_codes8(const uint32_t* __restrict__ w, int64_t stride_words, int N, int64_t g, int b,
+                                           int64_t pad_words, int* K) {
+  if constexpr (BITS == 4) {
+    // sixteen workers per round: all their words are requested before the first is used; 16 * 15 fits a byte
+    for (int i0 = 0; i0 < N; i0 += 16) {
+      uint32_t c[16];
+#pragma unroll
+      for (int q = 0; q < 16; ++q) c[q] = (i0 + q < N) ? __ldcs(w + (int64_t)(i0 + q) * stride_words + g) : 0u;
+      uint32_t ev = 0, od = 0;  // codes 0, 2, 4, 6 and 1, 3, 5, 7, one per byte
+#pragma unroll
+      for (int q = 0; q < 16; ++q) {
+        ev += c[q] & 0x0F0F0F0Fu;
+        od += (c[q] >> 4) & 0x0F0F0F0Fu;
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        K[2 * q] += (int)((ev >> (8 * q)) & 0xFFu);
+        K[2 * q + 1] += (int)((od >> (8 * q)) & 0xFFu);
+      }
+    }
+  } else if constexpr (BITS == 8) {
+    for (int i0 = 0; i0 < N; i0 += 8) {  // eight workers per round, loads first; 8 * 255 fits 16 bits
+      uint2 c[8];
+#pragma unroll
+      for (int q = 0; q < 8; ++q)
+        c[q] = (i0 + q < N) ? __ldcs(reinterpret_cast<const uint2*>(w + (int64_t)(i0 + q) * stride_words + g * 2)) : make_uint2(0u, 0u);
+      uint32_t a0 = 0, a1 = 0, a2 = 0, a3 = 0;  // codes (0, 2), (1, 3), (4, 6), (5, 7), one per half word
+#pragma unroll
+      for (int q = 0; q < 8; ++q) {
+        a0 += c[q].x & 0x00FF00FFu; a1 += (c[q].x >> 8) & 0x00FF00FFu;
+        a2 += c[q].y & 0x00FF00FFu; a3 += (c[q].y >> 8) & 0x00FF00FFu;
+      }
+      K[0] += (int)(a0 & 0xFFFFu); K[2] += (int)(a0 >> 16); K[1] += (int)(a1 & 0xFFFFu); K[3] += (int)(a1 >> 16);
+      K[4] += (int)(a2 & 0xFFFFu); K[6] += (int)(a2 >> 16); K[5] += (int)(a3 & 0xFFFFu); K[7] += (int)(a3 >> 16);
+    }
+  } else if constexpr (BITS == 2) {
+#pragma unroll 4
+    for (int i = 0; i < N; ++i) {
+      const uint32_t c = reinterpret_cast<const uint16_t*>(w + (int64_t)i * stride_words)[g];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) K[e] += (int)((c >> (2 * e)) & 3u);
+    }
+  } else {
+#pragma unroll 2
+    for (int i = 0; i < N; ++i) {
+      uint64_t lo, hi;
+      load_chunk<0>(w + (int64_t)i * stride_words, g, b, pad_words, lo, hi);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) K[e] += (int)extract(lo, hi, e * b, b);
+    }
+  }
+}
+
+// The server of schemes (b) and (c) (Section 3.2).  A thread owns 8 consecutive coordinates per sweep: it adds the
+// codes of the N streams as integers, then either stores the index sums K_j in offset binary with b_out =
+// b + ceil(log2 N) bits (scheme (b) grants the sum that many more bits), or rounds the average K_j / N back to the
+// b-bit grid with rule (1) of Section 2.2 and the server's own rounding stream (scheme (c), Eq. 4).  The 8 * b_out
+// output bits of a thread are b_out whole bytes: one or two words stored directly when b_out is 4 or 8, else staged
+// through shared memory and written out as words.
 template <int BITS>  // input width: 2, 4, 8 fixed; 0: b in 2..16 from the arguments
 __global__ void __launch_bounds__(AT) server_reduce_kernel(ServerArgs a) {
   const int tile = blockIdx.x;
@@ -184,6 +247,9 @@ __global__ void __launch_bounds__(AT) server_reduce_kernel(ServerArgs a) {
   const int bo = a.b_out;
   const int bias_in = a.N << (b - 1);  // sum of the offsets of N codes
   const float fN = (float)a.N;
+  const bool pow2 = (a.N & (a.N - 1)) == 0;
+  const float invN = __fdiv_rn(1.0f, fN);  // exact when N is a power of two: then K * invN is the division K / N
+  const bool direct = (bo == 4 || bo == 8);
   __shared__ __align__(16) uint8_t stage[AT * 16];
   const uint32_t* w = a.codes + s.word_off;
   uint32_t* out = a.out + so.word_off;
@@ -196,42 +262,70 @@ __global__ void __launch_bounds__(AT) server_reduce_kernel(ServerArgs a) {
     int K[8];
 #pragma unroll
     for (int e = 0; e < 8; ++e) K[e] = -bias_in;
-    if (nvalid > 0) {
-#pragma unroll 4
-      for (int i = 0; i < a.N; ++i) {
-        uint64_t lo, hi;
-        load_chunk<BITS>(w + (int64_t)i * a.stride_words, j >> 3, b, s.pad_words, lo, hi);
-#pragma unroll
-        for (int e = 0; e < 8; ++e) K[e] += (int)extract(lo, hi, e * b, b);
-      }
-    }
+    if (nvalid > 0) sum_codes8<BITS>(w, a.stride_words, a.N, j >> 3, b, s.pad_words, K);
     uint64_t olo = 0, ohi = 0;
     if (nvalid > 0) {
-      U4 r = U4{0, 0, 0, 0};
-      if (a.requantize) r = stream_block(a.seed, TAG_REQUANT, 0u, a.k, s.block_base + (uint32_t)(j >> 3));
+      if (a.requantize) {
+        const U4 r = stream_block(a.seed, TAG_REQUANT, 0u, a.k, s.block_base + (uint32_t)(j >> 3));
+        if constexpr (BITS != 0) {
+          uint32_t w0 = 0, w1 = 0;
 #pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        if (e < nvalid) {
-          uint32_t code;
-          if (a.requantize) code = quantize_code_rt(__fdiv_rn((float)K[e], fN), 1.0f, lane16(r, e), b);
-          else code = (uint32_t)(K[e] + (1 << (bo - 1)));
-          const int pos = e * bo;
-          if (pos < 64) {
-            olo |= (uint64_t)code << pos;
-            if (pos + bo > 64) ohi |= (uint64_t)code >> (64 - pos);
-          } else {
-            ohi |= (uint64_t)code << (pos - 64);
+          for (int e = 0; e < 8; ++e) {
+            const float avg = pow2 ? mul_rn((float)K[e], invN) : __fdiv_rn((float)K[e], fN);
+            const uint32_t code = quantize_code<BITS ? BITS : 2>(avg, 1.0f, lane16(r, e));
+            if (e * BITS < 32) w0 |= code << ((e * BITS) & 31);
+            else w1 |= code << ((e * BITS) & 31);
+          }
+          olo = (uint64_t)w0 | ((uint64_t)w1 << 32);
+          if (nvalid < 8) olo &= (1ull << (nvalid * BITS)) - 1ull;
+        } else {
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            if (e < nvalid) {
+              const float avg = pow2 ? mul_rn((float)K[e], invN) : __fdiv_rn((float)K[e], fN);
+              const uint32_t code = quantize_code_rt(avg, 1.0f, lane16(r, e), b);
+              const int pos = e * bo;
+              if (pos < 64) {
+                olo |= (uint64_t)code << pos;
+                if (pos + bo > 64) ohi |= (uint64_t)code >> (64 - pos);
+              } else {
+                ohi |= (uint64_t)code << (pos - 64);
+              }
+            }
+          }
+        }
+      } else {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          if (e < nvalid) {
+            const uint32_t code = (uint32_t)(K[e] + (1 << (bo - 1)));
+            const int pos = e * bo;
+            if (pos < 64) {
+              olo |= (uint64_t)code << pos;
+              if (pos + bo > 64) ohi |= (uint64_t)code >> (64 - pos);
+            } else {
+              ohi |= (uint64_t)code << (pos - 64);
+            }
           }
         }
       }
     }
-    if (it > 0) __syncthreads();
-    for (int i = 0; i < bo; ++i) stage[tid * bo + i] = (uint8_t)((i < 8) ? (olo >> (8 * i)) : (ohi >> (8 * (i - 8))));
-    __syncthreads();
-    const int64_t w0 = (sweep0 >> 5) * bo;  // sweep0 is a multiple of 2048, so this is exact
-    const uint32_t* stw = reinterpret_cast<const uint32_t*>(stage);
-    for (int q = tid; q < (AGROUP / 32) * bo; q += AT)
-      if (w0 + q < so.pad_words) out[w0 + q] = stw[q];
+    if (direct) {  // uniform for the launch
+      const int64_t g = j >> 3;
+      if (bo == 4) {
+        if (g < so.pad_words) out[g] = (uint32_t)olo;
+      } else {
+        if (2 * g < so.pad_words) *reinterpret_cast<uint2*>(out + 2 * g) = make_uint2((uint32_t)olo, (uint32_t)(olo >> 32));
+      }
+    } else {
+      if (it > 0) __syncthreads();
+      for (int i = 0; i < bo; ++i) stage[tid * bo + i] = (uint8_t)((i < 8) ? (olo >> (8 * i)) : (ohi >> (8 * (i - 8))));
+      __syncthreads();
+      const int64_t w0 = (sweep0 >> 5) * bo;  // sweep0 is a multiple of 2048, so this is exact
+      const uint32_t* stw = reinterpret_cast<const uint32_t*>(stage);
+      for (int q = tid; q < (AGROUP / 32) * bo; q += AT)
+        if (w0 + q < so.pad_words) out[w0 + q] = stw[q];
+    }
   }
 }
 
