@@ -318,7 +318,15 @@ def quantize_aggregate_bench(dev, peak, log2_len=26, dnn=True):
     ps = {"quantize_pack_unified_scale": {"ms": round(tqs, 4), "gbs": round(bq / tqs * 1e-6, 1), "frac": round(bq / tqs * 1e-6 / peak, 4)}}
     for name, scheme in (("scheme_b_sum", lpc.SCHEME_SERVER_SUM), ("scheme_c_requantize", lpc.SCHEME_SERVER_REQUANTIZE)):
         srv, bo = q.server_reduce(codes, length, scheme, 1)
-        ts = _time_calls(lambda: q.server_reduce(codes, length, scheme, 1, codes_out=srv), dev, 10)
+        # the library's own event pair around the launch: the Python wrapper costs more than this short kernel
+        q.set_option(lpc.OPT_PROFILE, 1)
+        q.get_profile(reset=True)
+        for _ in range(10):
+            q.server_reduce(codes, length, scheme, 1, codes_out=srv)
+        q.sync_status()
+        pr = q.get_profile(reset=True)
+        q.set_option(lpc.OPT_PROFILE, 0)
+        ts = pr["aggregate"][0] / pr["aggregate"][1]
         w = lpc.Context(None, None, lpc.LOGISTIC, 0.0, 1, 1, bo, lpc.CLIP_NONE, 1.0, 0)
         if scheme == lpc.SCHEME_SERVER_SUM:
             w.set_option(lpc.OPT_AVERAGE_DIVISOR, N)

@@ -172,71 +172,94 @@ __global__ void __launch_bounds__(AT) unpack_average_prox_kernel(AggArgs a) {
 // b + ceil(log2 N) bits (scheme (b) grants the sum that many more bits), or rounds the average K_j / N back to the
 // b-bit grid with rule (1) of Section 2.2 and the server's own rounding stream (scheme (c), Eq. 4).  The 8 * b_out
 // output bits of a thread are b_out whole bytes, staged through shared memory and written out as words.
-// Sums of the codes of the N streams at 8 coordinates (K[e] += sum_i code_ie).  The fixed widths add whole words of
-// codes as small integer lanes (4-bit codes in 8-bit lanes, 8-bit codes in 16-bit lanes) and spread the lanes out
-// before they could overflow.
+// One worker's 8 * BITS bits of coordinate group g (fixed widths), and their addition into packed integer lanes:
+// 2-bit codes in byte lanes of four half words, 4-bit codes in byte lanes of two words (even and odd codes), 8-bit
+// codes in half-word lanes of four words.
 template <int BITS>
-__device__ __forceinline__ void sum_codes8(const uint32_t* __restrict__ w, int64_t stride_words, int N, int64_t g, int b,
-                                           int64_t pad_words, int* K) {
-  if constexpr (BITS == 4) {
-    // sixteen workers per round: all their words are requested before the first is used; 16 * 15 fits a byte
-    for (int i0 = 0; i0 < N; i0 += 16) {
-      uint32_t c[16];
+__device__ __forceinline__ uint2 load_codes(const uint32_t* __restrict__ w, int64_t g) {
+  if constexpr (BITS == 8) return __ldcs(reinterpret_cast<const uint2*>(w + g * 2));
+  else if constexpr (BITS == 4) return make_uint2(__ldcs(w + g), 0u);
+  else return make_uint2((uint32_t)__ldcs(reinterpret_cast<const uint16_t*>(w) + g), 0u);
+}
+template <int BITS>
+__device__ __forceinline__ void add_lanes(uint32_t* acc, uint2 c) {
+  if constexpr (BITS == 8) {  // codes (0, 2), (1, 3), (4, 6), (5, 7)
+    acc[0] += c.x & 0x00FF00FFu; acc[1] += (c.x >> 8) & 0x00FF00FFu;
+    acc[2] += c.y & 0x00FF00FFu; acc[3] += (c.y >> 8) & 0x00FF00FFu;
+  } else if constexpr (BITS == 4) {  // codes 0, 2, 4, 6 and 1, 3, 5, 7, one per byte
+    acc[0] += c.x & 0x0F0F0F0Fu; acc[1] += (c.x >> 4) & 0x0F0F0F0Fu;
+  } else {  // codes 0, 4 | 1, 5 | 2, 6 | 3, 7 in the low and high byte of a half word
+    acc[0] += c.x & 0x0303u; acc[1] += (c.x >> 2) & 0x0303u; acc[2] += (c.x >> 4) & 0x0303u; acc[3] += (c.x >> 6) & 0x0303u;
+  }
+}
+template <int BITS>
+__device__ __forceinline__ void spread_lanes(const uint32_t* acc, int* K) {
+  if constexpr (BITS == 8) {
+    K[0] += (int)(acc[0] & 0xFFFFu); K[2] += (int)(acc[0] >> 16); K[1] += (int)(acc[1] & 0xFFFFu); K[3] += (int)(acc[1] >> 16);
+    K[4] += (int)(acc[2] & 0xFFFFu); K[6] += (int)(acc[2] >> 16); K[5] += (int)(acc[3] & 0xFFFFu); K[7] += (int)(acc[3] >> 16);
+  } else if constexpr (BITS == 4) {
 #pragma unroll
-      for (int q = 0; q < 16; ++q) c[q] = (i0 + q < N) ? __ldcs(w + (int64_t)(i0 + q) * stride_words + g) : 0u;
-      uint32_t ev = 0, od = 0;  // codes 0, 2, 4, 6 and 1, 3, 5, 7, one per byte
-#pragma unroll
-      for (int q = 0; q < 16; ++q) {
-        ev += c[q] & 0x0F0F0F0Fu;
-        od += (c[q] >> 4) & 0x0F0F0F0Fu;
-      }
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        K[2 * q] += (int)((ev >> (8 * q)) & 0xFFu);
-        K[2 * q + 1] += (int)((od >> (8 * q)) & 0xFFu);
-      }
+    for (int q = 0; q < 4; ++q) {
+      K[2 * q] += (int)((acc[0] >> (8 * q)) & 0xFFu);
+      K[2 * q + 1] += (int)((acc[1] >> (8 * q)) & 0xFFu);
     }
-  } else if constexpr (BITS == 8) {
-    for (int i0 = 0; i0 < N; i0 += 8) {  // eight workers per round, loads first; 8 * 255 fits 16 bits
-      uint2 c[8];
+  } else {
 #pragma unroll
-      for (int q = 0; q < 8; ++q)
-        c[q] = (i0 + q < N) ? __ldcs(reinterpret_cast<const uint2*>(w + (int64_t)(i0 + q) * stride_words + g * 2)) : make_uint2(0u, 0u);
-      uint32_t a0 = 0, a1 = 0, a2 = 0, a3 = 0;  // codes (0, 2), (1, 3), (4, 6), (5, 7), one per half word
+    for (int q = 0; q < 4; ++q) {
+      K[q] += (int)(acc[q] & 0xFFu);
+      K[q + 4] += (int)((acc[q] >> 8) & 0xFFu);
+    }
+  }
+}
+
+// Sums of the codes of the N streams at the 8 coordinates of group gA and of group gB (K += sum_i code_i).  Eight
+// workers per round, and the words of both groups are requested before the first is used: sixteen loads in flight
+// per thread.  Eight codes of at most 8 bits cannot overflow a lane.
+template <int BITS>
+__device__ __forceinline__ void sum_codes8x2(const uint32_t* __restrict__ w, int64_t stride_words, int N, int64_t gA,
+                                             int64_t gB, bool doA, bool doB, int b, int64_t pad_words, int* KA, int* KB) {
+  if constexpr (BITS != 0) {
+    for (int i0 = 0; i0 < N; i0 += 8) {
+      uint2 ca[8], cb[8];
 #pragma unroll
       for (int q = 0; q < 8; ++q) {
-        a0 += c[q].x & 0x00FF00FFu; a1 += (c[q].x >> 8) & 0x00FF00FFu;
-        a2 += c[q].y & 0x00FF00FFu; a3 += (c[q].y >> 8) & 0x00FF00FFu;
+        const bool live = i0 + q < N;
+        const uint32_t* wi = w + (int64_t)(i0 + q) * stride_words;
+        ca[q] = (live && doA) ? load_codes<BITS>(wi, gA) : make_uint2(0u, 0u);
+        cb[q] = (live && doB) ? load_codes<BITS>(wi, gB) : make_uint2(0u, 0u);
       }
-      K[0] += (int)(a0 & 0xFFFFu); K[2] += (int)(a0 >> 16); K[1] += (int)(a1 & 0xFFFFu); K[3] += (int)(a1 >> 16);
-      K[4] += (int)(a2 & 0xFFFFu); K[6] += (int)(a2 >> 16); K[5] += (int)(a3 & 0xFFFFu); K[7] += (int)(a3 >> 16);
-    }
-  } else if constexpr (BITS == 2) {
-#pragma unroll 4
-    for (int i = 0; i < N; ++i) {
-      const uint32_t c = reinterpret_cast<const uint16_t*>(w + (int64_t)i * stride_words)[g];
+      uint32_t aa[4] = {0, 0, 0, 0}, ab[4] = {0, 0, 0, 0};
 #pragma unroll
-      for (int e = 0; e < 8; ++e) K[e] += (int)((c >> (2 * e)) & 3u);
+      for (int q = 0; q < 8; ++q) { add_lanes<BITS>(aa, ca[q]); add_lanes<BITS>(ab, cb[q]); }
+      spread_lanes<BITS>(aa, KA);
+      spread_lanes<BITS>(ab, KB);
     }
   } else {
 #pragma unroll 2
     for (int i = 0; i < N; ++i) {
       uint64_t lo, hi;
-      load_chunk<0>(w + (int64_t)i * stride_words, g, b, pad_words, lo, hi);
+      if (doA) {
+        load_chunk<0>(w + (int64_t)i * stride_words, gA, b, pad_words, lo, hi);
 #pragma unroll
-      for (int e = 0; e < 8; ++e) K[e] += (int)extract(lo, hi, e * b, b);
+        for (int e = 0; e < 8; ++e) KA[e] += (int)extract(lo, hi, e * b, b);
+      }
+      if (doB) {
+        load_chunk<0>(w + (int64_t)i * stride_words, gB, b, pad_words, lo, hi);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) KB[e] += (int)extract(lo, hi, e * b, b);
+      }
     }
   }
 }
 
-// The server of schemes (b) and (c) (Section 3.2).  A thread owns 8 consecutive coordinates per sweep: it adds the
-// codes of the N streams as integers, then either stores the index sums K_j in offset binary with b_out =
-// b + ceil(log2 N) bits (scheme (b) grants the sum that many more bits), or rounds the average K_j / N back to the
-// b-bit grid with rule (1) of Section 2.2 and the server's own rounding stream (scheme (c), Eq. 4).  The 8 * b_out
-// output bits of a thread are b_out whole bytes: one or two words stored directly when b_out is 4 or 8, else staged
-// through shared memory and written out as words.
+// The server of schemes (b) and (c) (Section 3.2).  A thread owns 8 consecutive coordinates per sweep and takes two
+// sweeps at a time: it adds the codes of the N streams as integers, then either stores the index sums K_j in offset
+// binary with b_out = b + ceil(log2 N) bits (scheme (b) grants the sum that many more bits), or rounds the average
+// K_j / N back to the b-bit grid with rule (1) of Section 2.2 and the server's own rounding stream (scheme (c),
+// Eq. 4).  The 8 * b_out output bits of a thread are b_out whole bytes: one or two words stored directly when b_out
+// is 4 or 8, else staged through shared memory and written out as words.
 template <int BITS>  // input width: 2, 4, 8 fixed; 0: b in 2..16 from the arguments
-__global__ void __launch_bounds__(AT) server_reduce_kernel(ServerArgs a) {
+__global__ void __launch_bounds__(AT, 4) server_reduce_kernel(ServerArgs a) {
   const int tile = blockIdx.x;
   const int seg = a.tile_seg ? a.tile_seg[tile] : 0;
   const SegInfo s = a.segs[seg];
@@ -253,63 +276,50 @@ __global__ void __launch_bounds__(AT) server_reduce_kernel(ServerArgs a) {
   __shared__ __align__(16) uint8_t stage[AT * 16];
   const uint32_t* w = a.codes + s.word_off;
   uint32_t* out = a.out + so.word_off;
-#pragma unroll 1
-  for (int it = 0; it < AITER; ++it) {
-    const int64_t sweep0 = tstart + (int64_t)it * AGROUP;
-    if (sweep0 >= s.len) break;  // uniform for the block
-    const int64_t j = sweep0 + tid * 8;
-    const int nvalid = (j < s.len) ? (int)min((int64_t)8, s.len - j) : 0;
-    int K[8];
-#pragma unroll
-    for (int e = 0; e < 8; ++e) K[e] = -bias_in;
-    if (nvalid > 0) sum_codes8<BITS>(w, a.stride_words, a.N, j >> 3, b, s.pad_words, K);
-    uint64_t olo = 0, ohi = 0;
-    if (nvalid > 0) {
+
+  // the packed output bits of one group from its sums
+  auto encode = [&](const int* K, int64_t j, int nvalid, uint64_t& olo, uint64_t& ohi) {
+    olo = 0; ohi = 0;
+    if (nvalid <= 0) return;
+    U4 r = U4{0, 0, 0, 0};
+    if (a.requantize) r = stream_block(a.seed, TAG_REQUANT, 0u, a.k, s.block_base + (uint32_t)(j >> 3));
+    if constexpr (BITS != 0) {
       if (a.requantize) {
-        const U4 r = stream_block(a.seed, TAG_REQUANT, 0u, a.k, s.block_base + (uint32_t)(j >> 3));
-        if constexpr (BITS != 0) {
-          uint32_t w0 = 0, w1 = 0;
-#pragma unroll
-          for (int e = 0; e < 8; ++e) {
-            const float avg = pow2 ? mul_rn((float)K[e], invN) : __fdiv_rn((float)K[e], fN);
-            const uint32_t code = quantize_code<BITS ? BITS : 2>(avg, 1.0f, lane16(r, e));
-            if (e * BITS < 32) w0 |= code << ((e * BITS) & 31);
-            else w1 |= code << ((e * BITS) & 31);
-          }
-          olo = (uint64_t)w0 | ((uint64_t)w1 << 32);
-          if (nvalid < 8) olo &= (1ull << (nvalid * BITS)) - 1ull;
-        } else {
-#pragma unroll
-          for (int e = 0; e < 8; ++e) {
-            if (e < nvalid) {
-              const float avg = pow2 ? mul_rn((float)K[e], invN) : __fdiv_rn((float)K[e], fN);
-              const uint32_t code = quantize_code_rt(avg, 1.0f, lane16(r, e), b);
-              const int pos = e * bo;
-              if (pos < 64) {
-                olo |= (uint64_t)code << pos;
-                if (pos + bo > 64) ohi |= (uint64_t)code >> (64 - pos);
-              } else {
-                ohi |= (uint64_t)code << (pos - 64);
-              }
-            }
-          }
-        }
-      } else {
+        uint32_t w0 = 0, w1 = 0;
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
-          if (e < nvalid) {
-            const uint32_t code = (uint32_t)(K[e] + (1 << (bo - 1)));
-            const int pos = e * bo;
-            if (pos < 64) {
-              olo |= (uint64_t)code << pos;
-              if (pos + bo > 64) ohi |= (uint64_t)code >> (64 - pos);
-            } else {
-              ohi |= (uint64_t)code << (pos - 64);
-            }
-          }
+          const float avg = pow2 ? mul_rn((float)K[e], invN) : __fdiv_rn((float)K[e], fN);
+          const uint32_t code = quantize_code<BITS ? BITS : 2>(avg, 1.0f, lane16(r, e));
+          if (e * BITS < 32) w0 |= code << ((e * BITS) & 31);
+          else w1 |= code << ((e * BITS) & 31);
+        }
+        olo = (uint64_t)w0 | ((uint64_t)w1 << 32);
+        if (nvalid < 8) olo &= (1ull << (nvalid * BITS)) - 1ull;
+        return;
+      }
+    }
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      if (e < nvalid) {
+        uint32_t code;
+        if (a.requantize) {
+          const float avg = pow2 ? mul_rn((float)K[e], invN) : __fdiv_rn((float)K[e], fN);
+          code = quantize_code_rt(avg, 1.0f, lane16(r, e), b);
+        } else {
+          code = (uint32_t)(K[e] + (1 << (bo - 1)));
+        }
+        const int pos = e * bo;
+        if (pos < 64) {
+          olo |= (uint64_t)code << pos;
+          if (pos + bo > 64) ohi |= (uint64_t)code >> (64 - pos);
+        } else {
+          ohi |= (uint64_t)code << (pos - 64);
         }
       }
     }
+  };
+  bool staged_before = false;
+  auto emit = [&](int64_t sweep0, int64_t j, uint64_t olo, uint64_t ohi) {  // called by all threads of the block together
     if (direct) {  // uniform for the launch
       const int64_t g = j >> 3;
       if (bo == 4) {
@@ -318,13 +328,35 @@ __global__ void __launch_bounds__(AT) server_reduce_kernel(ServerArgs a) {
         if (2 * g < so.pad_words) *reinterpret_cast<uint2*>(out + 2 * g) = make_uint2((uint32_t)olo, (uint32_t)(olo >> 32));
       }
     } else {
-      if (it > 0) __syncthreads();
+      if (staged_before) __syncthreads();
+      staged_before = true;
       for (int i = 0; i < bo; ++i) stage[tid * bo + i] = (uint8_t)((i < 8) ? (olo >> (8 * i)) : (ohi >> (8 * (i - 8))));
       __syncthreads();
       const int64_t w0 = (sweep0 >> 5) * bo;  // sweep0 is a multiple of 2048, so this is exact
       const uint32_t* stw = reinterpret_cast<const uint32_t*>(stage);
       for (int q = tid; q < (AGROUP / 32) * bo; q += AT)
         if (w0 + q < so.pad_words) out[w0 + q] = stw[q];
+    }
+  };
+
+#pragma unroll 1
+  for (int it = 0; it < AITER; it += 2) {
+    const int64_t sweepA = tstart + (int64_t)it * AGROUP, sweepB = sweepA + AGROUP;
+    if (sweepA >= s.len) break;  // uniform for the block
+    const bool haveB = sweepB < s.len;  // uniform for the block
+    const int64_t jA = sweepA + tid * 8, jB = sweepB + tid * 8;
+    const int nvA = (jA < s.len) ? (int)min((int64_t)8, s.len - jA) : 0;
+    const int nvB = (jB < s.len) ? (int)min((int64_t)8, s.len - jB) : 0;
+    int KA[8], KB[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) { KA[e] = -bias_in; KB[e] = -bias_in; }
+    sum_codes8x2<BITS>(w, a.stride_words, a.N, jA >> 3, jB >> 3, nvA > 0, nvB > 0, b, s.pad_words, KA, KB);
+    uint64_t olo, ohi;
+    encode(KA, jA, nvA, olo, ohi);
+    emit(sweepA, jA, olo, ohi);
+    if (haveB) {
+      encode(KB, jB, nvB, olo, ohi);
+      emit(sweepB, jB, olo, ohi);
     }
   }
 }
