@@ -57,6 +57,13 @@ def _declare(L):
     L.orc_quantize_coord.argtypes = [C.c_float, C.c_float, C.c_int, C.c_uint32]
     L.orc_quantize_coord.restype = C.c_int
     L.orc_pack.argtypes = [_u32p, C.c_int64, C.c_int, _u32p]
+    _u64p = C.POINTER(C.c_uint64)
+    L.orc_code_histogram.argtypes = [_u32p, C.c_int64, C.c_int, _u64p]
+    L.orc_code_histogram.restype = C.c_int
+    L.orc_entropy_bits.argtypes = [_u64p, C.c_int]
+    L.orc_entropy_bits.restype = C.c_double
+    L.orc_huffman_bits.argtypes = [_u64p, C.c_int]
+    L.orc_huffman_bits.restype = C.c_uint64
     L.orc_sum_bits_per_coordinate.argtypes = [C.c_int, C.c_int]
     L.orc_sum_bits_per_coordinate.restype = C.c_int
     L.orc_scheme_bits.argtypes = [C.c_int, C.c_int64, C.c_int, C.c_int]
@@ -246,6 +253,26 @@ def unpack_average_prox(words, delta, length, b, mu, x, eta, lambda_l1, want_v=F
     if want_utilde:
         out += (ut,)
     return out if len(out) > 1 else xn
+
+
+def code_histogram(words, length, b):
+    """Counts of the 2^b code values in a packed message."""
+    words = np.ascontiguousarray(words, dtype=np.uint32)
+    hist = np.zeros(1 << b, dtype=np.uint64)
+    _check(lib().orc_code_histogram(words.ctypes.data_as(_u32p), length, b, hist.ctypes.data_as(C.POINTER(C.c_uint64))))
+    return hist
+
+
+def entropy_bits(hist):
+    """n * H: the empirical-entropy bound on the message's payload, in bits."""
+    hist = np.ascontiguousarray(hist, dtype=np.uint64)
+    return float(lib().orc_entropy_bits(hist.ctypes.data_as(C.POINTER(C.c_uint64)), hist.size))
+
+
+def huffman_bits(hist):
+    """Payload length in bits under a Huffman code built for this histogram."""
+    hist = np.ascontiguousarray(hist, dtype=np.uint64)
+    return int(lib().orc_huffman_bits(hist.ctypes.data_as(C.POINTER(C.c_uint64)), hist.size))
 
 
 SCHEME_A, SCHEME_B, SCHEME_C = 0, 1, 2

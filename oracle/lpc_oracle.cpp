@@ -494,6 +494,60 @@ int orc_server_reduce(const uint32_t* words, int64_t stride_words, int N, int64_
   return ORC_OK;
 }
 
+// ---------------------------------------------------------------------------------------
+// Entropy coding of a message (Section 5.1: the experiments pass the codes through Huffman's code
+// [huffman1952method] to cut the traffic further).  The paper gives no format; what is counted here is
+// the payload alone: from the histogram of a message's 2^b code values, (i) the empirical entropy
+// n * H = -sum_c count_c * log2(count_c / n), the bound no symbol code can beat, and (ii) the length of
+// the message under a Huffman code built for that histogram, sum_c count_c * len_c.  The code table and
+// the 32-bit scale are not included.  A message with one distinct value still spends one bit per
+// coordinate under (ii) (a code word cannot be empty).
+// ---------------------------------------------------------------------------------------
+// hist_out: 2^b counts.
+int orc_code_histogram(const uint32_t* words, int64_t len, int b, uint64_t* hist_out) {
+  if (len < 0 || b < 1 || b > 16) return ORC_ERR_INVALID;
+  for (int c = 0; c < (1 << b); ++c) hist_out[c] = 0;
+  for (int64_t j = 0; j < len; ++j) hist_out[get_code(words, j, b)] += 1;
+  return ORC_OK;
+}
+
+// n * H in bits (fp64) for a histogram of `bins` counts.
+double orc_entropy_bits(const uint64_t* hist, int bins) {
+  uint64_t n = 0;
+  for (int c = 0; c < bins; ++c) n += hist[c];
+  double bits = 0.0;
+  for (int c = 0; c < bins; ++c)
+    if (hist[c] > 0) bits -= (double)hist[c] * std::log2((double)hist[c] / (double)n);
+  return bits;
+}
+
+// Total length in bits under Huffman's construction: repeatedly merge the two lightest subtrees; every
+// merge adds the merged weight once (each symbol below it gets one bit longer).
+uint64_t orc_huffman_bits(const uint64_t* hist, int bins) {
+  uint64_t w[1 << 16];
+  int m = 0;
+  for (int c = 0; c < bins; ++c)
+    if (hist[c] > 0) w[m++] = hist[c];
+  if (m == 0) return 0;
+  if (m == 1) return w[0];
+  uint64_t total = 0;
+  while (m > 1) {
+    int a = 0, b2 = 1;  // indices of the two smallest weights, by plain search
+    if (w[b2] < w[a]) { a = 1; b2 = 0; }
+    for (int i = 2; i < m; ++i) {
+      if (w[i] < w[a]) { b2 = a; a = i; }
+      else if (w[i] < w[b2]) { b2 = i; }
+    }
+    const uint64_t merged = w[a] + w[b2];
+    total += merged;
+    const int hi = a > b2 ? a : b2, lo = a > b2 ? b2 : a;
+    w[lo] = merged;
+    w[hi] = w[m - 1];
+    --m;
+  }
+  return total;
+}
+
 // A worker's side after the server's message: u~_j = (delta * index_j) / divisor, then Algorithm 1
 // steps 9-10 as in orc_unpack_average_prox.  Scheme (b): bits = b + ceil(log2 N), divisor = N;
 // scheme (c): bits = b, divisor = 1.
