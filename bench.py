@@ -312,6 +312,22 @@ def quantize_aggregate_bench(dev, peak, log2_len=26, dnn=True):
                           "note": "two passes: 4 B stats read + 4 B quantize read + b/8 B written per element"},
         "unpack_average_prox": {"ms": round(ta, 4), "bytes": ba, "gbs": round(ba / ta * 1e-6, 1), "frac": round(ba / ta * 1e-6 / peak, 4)},
         "combined_gbs": round((bq + ba) / (tq + ta) * 1e-6, 1)}
+    # entropy-coding count of the messages just packed: histogram kernel (event-timed) and the host sums
+    hist = torch.empty((N, 1, 1 << b), dtype=torch.int64, device=dev)
+    q.set_option(lpc.OPT_PROFILE, 1)
+    q.get_profile(reset=True)
+    for _ in range(10):
+        q.message_entropy(codes, length, hist_out=hist, host_counts=False)
+    q.sync_status()
+    pr = q.get_profile(reset=True)
+    q.set_option(lpc.OPT_PROFILE, 0)
+    th = pr["other"][0] / pr["other"][1]
+    _, ent, huf = q.message_entropy(codes, length, hist_out=hist)
+    bh = N * length * b / 8
+    res["entropy_count_N8_len2^%d_b4" % log2_len] = {
+        "histogram": {"ms": round(th, 4), "bytes": bh, "gbs": round(bh / th * 1e-6, 1), "frac": round(bh / th * 1e-6 / peak, 4)},
+        "bits_per_coordinate": {"raw": b, "entropy_bound": round(float(ent.mean()) / length, 4),
+                                "huffman": round(float(huf.astype("float64").mean()) / length, 4)}}
     # the parameter-server schemes (b) and (c) on the same vectors: unified scale, server, worker-side decode
     q.set_option(lpc.OPT_SHARED_SCALE, 1)
     tqs = _time_calls(quant, dev, 5)

@@ -221,6 +221,24 @@ int lpc_sum_bits(int32_t b, int32_t N, int32_t* bits_out); /* b + ceil(log2 N) *
 int lpc_scheme_bits(int scheme, int64_t d, int32_t b, int32_t N, uint64_t* bits_out);
 
 /*
+ * Entropy-coding count (Section 5.1: the experiments pass the codes through Huffman's code before sending them; the
+ * paper gives no format, so the payload is counted and no bit stream is produced).  For every message, i.e. every
+ * (worker, tensor segment) pair of the N streams in `codes` (device, layout of lpc_packed_layout for the context's
+ * b, as written by lpc_quantize_pack):
+ *   hist_dev          device, N * nseg * 2^b 64-bit counts, cleared and filled by the call:
+ *                     hist_dev[(worker * nseg + seg) * 2^b + code] = coordinates of that message with that code;
+ *   entropy_bits_out  host, N * nseg doubles, nullable: n * H = -sum_c count_c log2(count_c / n), the bound no
+ *                     symbol code can beat;
+ *   huffman_bits_out  host, N * nseg, nullable: sum_c count_c * len_c under Huffman's code for that histogram (one
+ *                     bit per coordinate when a message holds a single value).
+ * Neither count includes the code table or the 32-bit scale; compare with the raw b * len of Section 3.2.
+ * With both host outputs NULL the call only enqueues the histogram; otherwise it waits for the stream and does the
+ * two sums on the host.  Errors: LPC_ERR_UNSUPPORTED unless 1 <= b <= 8.
+ */
+int lpc_message_entropy(lpc_ctx* ctx, const uint32_t* codes, int64_t len, const int64_t* seg_offsets, int32_t nseg,
+                        unsigned long long* hist_dev, double* entropy_bits_out, uint64_t* huffman_bits_out);
+
+/*
  * ALPC-SVRG (Algorithms 2 and 3).  lpc_alpc_begin sets y_0 = z_0 = x and clears the y sum.
  * lpc_alpc_double_sample_step is steps 5-13 of Algorithm 2 for iteration k:
  *   x = tau1*z + tau2*x~ + (1-tau1-tau2)*y;  v from quantized worker differences at x (as in

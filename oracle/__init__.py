@@ -115,6 +115,15 @@ def _declare(L):
                                 C.c_float, C.c_float, C.c_float, _f32p, _f32p, _f32p, _f32p, _f32p, _f32p,
                                 _f32p, _f32p, _u32p, C.c_int64, _f32p]
     L.orc_alpc_step.restype = C.c_int
+    L.orc_alpc_step_sc.argtypes = [_f32p, _f32p, C.c_int64, C.c_int64, C.c_int, C.c_float, C.c_int, C.c_int,
+                                   C.c_int, C.c_int, C.c_float, C.c_uint64, C.c_int, C.c_uint64, C.c_float,
+                                   C.c_float, C.c_float, C.c_float, C.c_float, C.c_float, _f32p, _f32p, _f32p, _f32p,
+                                   _f32p, _f32p, _f32p, _f32p, _u32p, C.c_int64, _f32p]
+    L.orc_alpc_step_sc.restype = C.c_int
+    L.orc_weighted_snapshot.argtypes = [_f32p, C.c_float, C.c_int64, _f32p]
+    L.orc_weighted_snapshot.restype = None
+    L.orc_ridge_term.argtypes = [_f32p, C.c_int64, C.c_float]
+    L.orc_ridge_term.restype = C.c_double
 
 
 def _f32(a):
@@ -437,8 +446,22 @@ def lpc_inner_step(P, k, eta, x, xs, mu, taps=False):
     return xn
 
 
-def alpc_step(P, k, tau1, tau2, alpha, inv4L, xs, mu, y, z, ysum, taps=False):
-    """Algorithm 2 steps 5-13.  Returns (y_new, z_new, ysum_new[, taps])."""
+def weighted_snapshot(ysum, wsum):
+    """Algorithm 2's snapshot from the weighted sum of the epoch's y iterates and the sum of the weights."""
+    ysum, p = _f32(ysum)
+    out = np.zeros_like(ysum)
+    lib().orc_weighted_snapshot(p, np.float32(wsum), ysum.size, out.ctypes.data_as(_f32p))
+    return out
+
+
+def ridge_term(x, sigma):
+    x, p = _f32(x)
+    return float(lib().orc_ridge_term(p, x.size, np.float32(sigma)))
+
+
+def alpc_step(P, k, tau1, tau2, alpha, inv4L, xs, mu, y, z, ysum, taps=False, sigma=None, weight=1.0):
+    """Algorithm 2 steps 5-13.  Returns (y_new, z_new, ysum_new[, taps]).  sigma (with weight): the strongly convex
+    case with h = lambda_l1*||.||_1 + (sigma/2)*||.||^2 and the snapshot weight of this step."""
     xs, pxs = _f32(xs)
     mu, pmu = _f32(mu)
     yn = np.array(y, dtype=np.float32, copy=True)
@@ -450,12 +473,14 @@ def alpc_step(P, k, tau1, tau2, alpha, inv4L, xs, mu, y, z, ysum, taps=False):
                  vhat=np.zeros(P.d, dtype=np.float32), words=np.zeros((P.N, max(P.W, 1)), dtype=np.uint32),
                  delta=np.zeros(P.N, dtype=np.float32))
     g = (lambda name, typ: _ptr(t[name], typ)) if taps else (lambda name, typ: None)
-    rc = lib().orc_alpc_step(P.X.ctypes.data_as(_f32p), P.y.ctypes.data_as(_f32p), P.n, P.d, P.loss,
-                             P.lambda_l1, P.N, P.B, P.b, P.clip_mode, P.clip_value, P.seed,
-                             int(P.partition_local), k, tau1, tau2, alpha, inv4L, pxs, pmu,
-                             yn.ctypes.data_as(_f32p), zn.ctypes.data_as(_f32p), sn.ctypes.data_as(_f32p),
-                             g("x", _f32p), g("v", _f32p), g("vhat", _f32p), g("words", _u32p), max(P.W, 1),
-                             g("delta", _f32p))
+    head = (P.X.ctypes.data_as(_f32p), P.y.ctypes.data_as(_f32p), P.n, P.d, P.loss, P.lambda_l1, P.N, P.B, P.b,
+            P.clip_mode, P.clip_value, P.seed, int(P.partition_local), k, tau1, tau2, alpha, inv4L)
+    tail = (pxs, pmu, yn.ctypes.data_as(_f32p), zn.ctypes.data_as(_f32p), sn.ctypes.data_as(_f32p),
+            g("x", _f32p), g("v", _f32p), g("vhat", _f32p), g("words", _u32p), max(P.W, 1), g("delta", _f32p))
+    if sigma is None:
+        rc = lib().orc_alpc_step(*head, *tail)
+    else:
+        rc = lib().orc_alpc_step_sc(*head, np.float32(sigma), np.float32(weight), *tail)
     _check(rc)
     if taps:
         t["words"] = t["words"][:, : P.W]

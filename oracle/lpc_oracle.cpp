@@ -689,12 +689,21 @@ int orc_lpc_inner_step(const float* X, const float* y, int64_t n, int64_t d, int
 //   y+ = argmin 2L||y-x||^2 + <v,y> + h(y)        = soft(x - v/(4L), lambda_l1/(4L))
 //   z+ = argmin ||z-z_k||^2/(2 alpha) + <v^,z> + h = soft(z - alpha v^, alpha*lambda_l1)
 //   ysum += y+   (Algorithm 3's snapshot is the mean of the epoch's y iterates)
-int orc_alpc_step(const float* X, const float* y, int64_t n, int64_t d, int loss, float lambda_l1, int N,
-                  int B, int b, int clip_mode, float clip_value, uint64_t seed, int partition_local,
-                  uint64_t k, float tau1, float tau2, float alpha, float inv4L, const float* xs,
-                  const float* mu, float* y_inout, float* z_inout, float* ysum_inout, float* x_out,
-                  float* v_out, float* vhat_out, uint32_t* words_out, int64_t stride_words,
-                  float* delta_out) {
+//
+// Strongly convex case (Algorithm 2 as printed): h(x) = lambda_l1*||x||_1 + (sigma/2)*||x||^2.  Completing the
+// square in the two argmins gives the plain soft-threshold results divided by (1 + sigma/(4L)) and by
+// (1 + alpha*sigma):
+//   y+ = soft(x - v/(4L), lambda_l1/(4L)) * cy,   cy = 1 / (1 + sigma*inv4L)
+//   z+ = soft(z - alpha v^, alpha*lambda_l1) * cz, cz = 1 / (1 + alpha*sigma)
+// and the snapshot of Algorithm 2's last step weighs y_{sm+t+1} by (1 + alpha*sigma)^t: the caller passes that
+// weight (1, theta, theta*theta, ... formed by repeated fp32 multiplication) and ysum += weight * y+.
+// sigma = 0, weight = 1 multiply by exactly 1 and reproduce the general convex step bit for bit.
+int orc_alpc_step_sc(const float* X, const float* y, int64_t n, int64_t d, int loss, float lambda_l1, int N,
+                     int B, int b, int clip_mode, float clip_value, uint64_t seed, int partition_local,
+                     uint64_t k, float tau1, float tau2, float alpha, float inv4L, float sigma, float weight,
+                     const float* xs, const float* mu, float* y_inout, float* z_inout, float* ysum_inout,
+                     float* x_out, float* v_out, float* vhat_out, uint32_t* words_out, int64_t stride_words,
+                     float* delta_out) {
   const float tau3 = (1.0f - tau1) - tau2;
   std::vector<float> x((size_t)d), xq((size_t)d), v((size_t)d), uj((size_t)d), coef((size_t)B);
   std::vector<int64_t> idx((size_t)B);
@@ -713,18 +722,46 @@ int orc_alpc_step(const float* X, const float* y, int64_t n, int64_t d, int loss
   orc_svrg_diff_from_coef(X, d, idx.data(), B, coef.data(), uj.data());
   const float kappa_y = inv4L * lambda_l1;
   const float kappa_z = alpha * lambda_l1;
+  const float cy = 1.0f / (1.0f + sigma * inv4L);
+  const float cz = 1.0f / (1.0f + alpha * sigma);
   for (int64_t j = 0; j < d; ++j) {
     const float vhat = uj[(size_t)j] + mu[j];
-    const float ynew = soft_threshold(x[(size_t)j] - inv4L * v[(size_t)j], kappa_y);
-    const float znew = soft_threshold(z_inout[j] - alpha * vhat, kappa_z);
+    const float ynew = soft_threshold(x[(size_t)j] - inv4L * v[(size_t)j], kappa_y) * cy;
+    const float znew = soft_threshold(z_inout[j] - alpha * vhat, kappa_z) * cz;
     y_inout[j] = ynew;
     z_inout[j] = znew;
-    if (ysum_inout) ysum_inout[j] = ysum_inout[j] + ynew;
+    if (ysum_inout) ysum_inout[j] = ysum_inout[j] + weight * ynew;
     if (x_out) x_out[j] = x[(size_t)j];
     if (v_out) v_out[j] = v[(size_t)j];
     if (vhat_out) vhat_out[j] = vhat;
   }
   return ORC_OK;
+}
+
+// The general convex step (Algorithm 3 runs it with its own tau1, alpha per epoch): h = lambda_l1*||.||_1.
+int orc_alpc_step(const float* X, const float* y, int64_t n, int64_t d, int loss, float lambda_l1, int N,
+                  int B, int b, int clip_mode, float clip_value, uint64_t seed, int partition_local,
+                  uint64_t k, float tau1, float tau2, float alpha, float inv4L, const float* xs,
+                  const float* mu, float* y_inout, float* z_inout, float* ysum_inout, float* x_out,
+                  float* v_out, float* vhat_out, uint32_t* words_out, int64_t stride_words,
+                  float* delta_out) {
+  return orc_alpc_step_sc(X, y, n, d, loss, lambda_l1, N, B, b, clip_mode, clip_value, seed, partition_local, k,
+                          tau1, tau2, alpha, inv4L, 0.0f, 1.0f, xs, mu, y_inout, z_inout, ysum_inout, x_out,
+                          v_out, vhat_out, words_out, stride_words, delta_out);
+}
+
+// Algorithm 2's snapshot: x~ = (sum_t w_t)^-1 * sum_t w_t y_{sm+t+1}, given the weighted sum and the weights'
+// sum (both accumulated in fp32 in step order): one reciprocal, one multiplication per coordinate.
+void orc_weighted_snapshot(const float* ysum, float wsum, int64_t d, float* xs_out) {
+  const float inv = 1.0f / wsum;
+  for (int64_t j = 0; j < d; ++j) xs_out[j] = ysum[j] * inv;
+}
+
+// P(x) with the elastic-net regulariser: the objective of Eq. 1 plus (sigma/2)*||x||^2 (fp64 sum).
+double orc_ridge_term(const float* x, int64_t d, float sigma) {
+  double s2 = 0.0;
+  for (int64_t j = 0; j < d; ++j) s2 += (double)x[j] * (double)x[j];
+  return 0.5 * (double)sigma * s2;
 }
 
 }  // extern "C"

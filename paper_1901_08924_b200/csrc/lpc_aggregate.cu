@@ -361,7 +361,99 @@ __global__ void __launch_bounds__(AT, 4) server_reduce_kernel(ServerArgs a) {
   }
 }
 
+// Histogram of a message's code values, the input of the entropy-coding count (Section 5.1: the experiments pass the
+// codes through Huffman's code).  One CTA per run of tiles of a worker.  Every thread counts the 32 codes it reads in counters
+// of its own -- one byte per code value, four values to a 32-bit word, word[value / 4][thread] -- so that counting
+// needs no atomic operation however skewed the codes are (near-Gaussian gradients put most of them on a few values)
+// and a warp's accesses fall on 32 different banks.  The block then adds the columns up with warp reductions and sends
+// the tile's count of every value to the message's histogram with one atomic addition each.
+constexpr int HRUN = 32;  // tiles per CTA: the tile counts are gathered in shared memory and reach the message's
+                          // histogram (a few hot addresses) once per run and segment
+
+template <int BITS>  // 1, 2, 4, 8: code width known at compile time; 0: b in 1..8 from the arguments
+__global__ void __launch_bounds__(AT) code_histogram_kernel(HistArgs a) {
+  const int worker = blockIdx.y;
+  const int tile0 = blockIdx.x * HRUN, tile1 = min(tile0 + HRUN, a.ntiles);
+  const int tid = threadIdx.x;
+  const int b = BITS ? BITS : a.b, bins = 1 << b;
+  const int rows = (bins + 3) / 4;  // words per thread
+  extern __shared__ __align__(16) uint32_t cw[];  // rows x AT words
+  uint8_t* mine = reinterpret_cast<uint8_t*>(cw + tid);  // this thread's counter of value c: mine[(c / 4) * AT * 4 + c % 4]
+  __shared__ unsigned int total[256];
+  for (int c = tid; c < bins; c += AT) total[c] = 0u;
+  int cur_seg = -1;
+  auto flush = [&]() {  // the counts gathered for segment cur_seg go to its histogram (all threads call this)
+    __syncthreads();
+    if (cur_seg >= 0)
+      for (int c = tid; c < bins; c += AT) {
+        if (total[c]) atomicAdd(&a.hist[((int64_t)worker * a.nseg + cur_seg) * bins + c], (unsigned long long)total[c]);
+        total[c] = 0u;
+      }
+    __syncthreads();
+  };
+#pragma unroll 1
+  for (int tile = tile0; tile < tile1; ++tile) {
+    const int seg = a.tile_seg ? a.tile_seg[tile] : 0;
+    if (seg != cur_seg) {
+      flush();
+      cur_seg = seg;
+    }
+    const SegInfo s = a.segs[seg];
+    const int64_t tstart = (int64_t)(tile - s.tile_first) * TILE;
+    for (int i = tid; i < rows * AT; i += AT) cw[i] = 0u;  // a thread clears and uses its own column only
+    const uint32_t* w = a.codes + (int64_t)worker * a.stride_words + s.word_off;
+#pragma unroll 1
+    for (int it = 0; it < AITER; ++it) {  // a thread sees at most AITER * 8 = 32 codes: a byte counter cannot overflow
+      const int64_t j = tstart + (int64_t)it * AGROUP + tid * 8;
+      if (j >= s.len) break;
+      const int nvalid = (int)min((int64_t)8, s.len - j);
+      uint64_t lo, hi;
+      load_chunk<BITS>(w, j >> 3, b, s.pad_words, lo, hi);  // 8 * b <= 64 bits: all in lo
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        if (e < nvalid) {
+          const uint32_t code = (uint32_t)(lo >> (e * b)) & (uint32_t)(bins - 1);
+          mine[((code >> 2) * (AT * 4)) | (code & 3u)] += 1;
+        }
+      }
+    }
+    // the tile's columns add up: a word's four byte counters (each <= 32) widen to two words of 16-bit lanes, a warp
+    // adds them with one integer reduction each (32 lanes * 32 fits 16 bits), lane 0 adds the sums to the run's totals
+    for (int r = 0; r < rows; ++r) {
+      const uint32_t v = cw[r * AT + tid];
+      const uint32_t even = __reduce_add_sync(0xFFFFFFFFu, v & 0x00FF00FFu);         // values 4r, 4r+2
+      const uint32_t odd = __reduce_add_sync(0xFFFFFFFFu, (v >> 8) & 0x00FF00FFu);   // values 4r+1, 4r+3
+      if ((tid & 31) == 0) {
+        if (even & 0xFFFFu) atomicAdd(&total[4 * r], even & 0xFFFFu);
+        if (even >> 16) atomicAdd(&total[4 * r + 2], even >> 16);
+        if (odd & 0xFFFFu) atomicAdd(&total[4 * r + 1], odd & 0xFFFFu);
+        if (odd >> 16) atomicAdd(&total[4 * r + 3], odd >> 16);
+      }
+    }
+  }
+  flush();
+}
+
 }  // namespace
+
+cudaError_t launch_code_histogram(const HistArgs& a, cudaStream_t st) {
+  if (a.ntiles <= 0 || a.N <= 0) return cudaSuccess;
+  const size_t sh = (size_t)(((1 << a.b) + 3) / 4) * AT * sizeof(uint32_t);
+  const dim3 grid((unsigned)((a.ntiles + HRUN - 1) / HRUN), (unsigned)a.N);
+  auto go = [&](auto kernel) {
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sh);
+    if (e != cudaSuccess) return e;
+    kernel<<<grid, AT, sh, st>>>(a);
+    return cudaGetLastError();
+  };
+  switch (a.b) {
+    case 1: return go(code_histogram_kernel<1>);
+    case 2: return go(code_histogram_kernel<2>);
+    case 4: return go(code_histogram_kernel<4>);
+    case 8: return go(code_histogram_kernel<8>);
+    default: return go(code_histogram_kernel<0>);
+  }
+}
 
 cudaError_t launch_server_reduce(const ServerArgs& a, cudaStream_t st) {
   if (a.ntiles <= 0) return cudaSuccess;

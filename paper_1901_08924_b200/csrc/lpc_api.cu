@@ -7,6 +7,9 @@
 #include <cstdio>
 #include <cstring>
 #include <string>
+#include <queue>
+#include <functional>
+#include <cmath>
 #include <vector>
 
 #include "../../include/lpc.h"
@@ -822,6 +825,61 @@ int lpc_scheme_bits(int scheme, int64_t d, int32_t b, int32_t N, uint64_t* bits_
     case LPC_SCHEME_SERVER_REQUANTIZE: *bits_out = (uint64_t)N * (64u + 2u * bd); return LPC_OK;
     default: return LPC_ERR_INVALID_ARG;
   }
+}
+
+namespace {
+// n * H in bits for a histogram.
+double entropy_of(const unsigned long long* h, int bins) {
+  unsigned long long n = 0;
+  for (int c = 0; c < bins; ++c) n += h[c];
+  double bits = 0.0;
+  for (int c = 0; c < bins; ++c)
+    if (h[c]) bits -= (double)h[c] * std::log2((double)h[c] / (double)n);
+  return bits;
+}
+// Length of the message under Huffman's code for its own histogram: the sum of the weights of all merged nodes.
+uint64_t huffman_of(const unsigned long long* h, int bins) {
+  std::vector<unsigned long long> w;
+  for (int c = 0; c < bins; ++c)
+    if (h[c]) w.push_back(h[c]);
+  if (w.empty()) return 0;
+  if (w.size() == 1) return w[0];  // a code word cannot be empty: one bit per coordinate
+  std::priority_queue<unsigned long long, std::vector<unsigned long long>, std::greater<unsigned long long>> q(w.begin(), w.end());
+  uint64_t total = 0;
+  while (q.size() > 1) {
+    const unsigned long long x = q.top(); q.pop();
+    const unsigned long long y = q.top(); q.pop();
+    total += x + y;
+    q.push(x + y);
+  }
+  return total;
+}
+}  // namespace
+
+int lpc_message_entropy(lpc_ctx* c, const uint32_t* codes, int64_t len, const int64_t* seg_offsets, int32_t nseg,
+                        unsigned long long* hist_dev, double* entropy_bits_out, uint64_t* huffman_bits_out) {
+  if (!c) return LPC_ERR_INVALID_ARG;
+  if (!hist_dev || (len > 0 && !codes)) return fail(c, LPC_ERR_INVALID_ARG, "null stream or histogram");
+  if (len < 0 || nseg < 1) return fail(c, LPC_ERR_INVALID_ARG, "len / nseg");
+  if (c->b < 1 || c->b > 8) return fail(c, LPC_ERR_UNSUPPORTED, "code histograms cover b in 1..8");
+  if (!aligned16(codes)) return fail(c, LPC_ERR_INVALID_ARG, "codes must be 16-byte aligned");
+  TRY(make_plan(c, c->seg, len, c->b, seg_offsets, nseg));
+  const int bins = 1 << c->b;
+  const size_t count = (size_t)c->N * (size_t)nseg * (size_t)bins;
+  CU(c, cudaMemsetAsync(hist_dev, 0, count * sizeof(unsigned long long), c->stream));
+  HistArgs a;
+  a.codes = codes; a.stride_words = c->seg.stride_words; a.N = c->N; a.b = c->b; a.segs = c->seg.d_segs;
+  a.tile_seg = c->seg.d_tile_seg; a.nseg = nseg; a.ntiles = c->seg.ntiles; a.hist = hist_dev;
+  { ProfScope ps_(c, LPC_KERNEL_OTHER); CU(c, launch_code_histogram(a, c->stream)); }
+  if (!entropy_bits_out && !huffman_bits_out) return LPC_OK;  // histogram only: stays asynchronous
+  std::vector<unsigned long long> h(count);
+  CU(c, cudaMemcpyAsync(h.data(), hist_dev, count * sizeof(unsigned long long), cudaMemcpyDeviceToHost, c->stream));
+  CU(c, cudaStreamSynchronize(c->stream));
+  for (size_t m = 0; m < (size_t)c->N * (size_t)nseg; ++m) {
+    if (entropy_bits_out) entropy_bits_out[m] = entropy_of(h.data() + m * bins, bins);
+    if (huffman_bits_out) huffman_bits_out[m] = huffman_of(h.data() + m * bins, bins);
+  }
+  return LPC_OK;
 }
 
 int lpc_server_reduce(lpc_ctx* c, const uint32_t* codes, int64_t len, const int64_t* seg_offsets, int32_t nseg, int scheme,

@@ -107,6 +107,20 @@ struct ServerArgs {
 };
 cudaError_t launch_server_reduce(const ServerArgs& a, cudaStream_t st);
 
+// Histogram of the code values of every (worker, segment) message: hist[(worker * nseg + seg) * 2^b + code].
+struct HistArgs {
+  const uint32_t* codes;
+  int64_t stride_words;
+  int N;
+  int b;                   // 1..8
+  const SegInfo* segs;
+  const int32_t* tile_seg;
+  int nseg;
+  int ntiles;
+  unsigned long long* hist;  // N * nseg * 2^b counts, added to (the caller clears them)
+};
+cudaError_t launch_code_histogram(const HistArgs& a, cudaStream_t st);
+
 }  // namespace lpc
 
 namespace lpc {

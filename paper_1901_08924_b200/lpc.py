@@ -44,6 +44,7 @@ SYMBOLS = [
     ("lpc_packed_words", _int, [_i64, _i32, _i64p]),
     ("lpc_quantize_pack", _int, [_vp, _vp, _vp, _i64, _i64, _i64p, _i32, _u64, _vp, _vp, _vp]),
     ("lpc_unpack_average_prox", _int, [_vp, _vp, _vp, _i64, _i64p, _i32, _vp, _vp, _f32, _f32, _vp]),
+    ("lpc_message_entropy", _int, [_vp, _vp, _i64, _i64p, _i32, _vp, _f64p, _u64p]),
     ("lpc_server_reduce", _int, [_vp, _vp, _i64, _i64p, _i32, _int, _u64, _vp]),
     ("lpc_sum_bits", _int, [_i32, _i32, C.POINTER(C.c_int32)]),
     ("lpc_scheme_bits", _int, [_int, _i64, _i32, _i32, _u64p]),
@@ -240,6 +241,21 @@ class Context:
         self._ck(lib().lpc_unpack_average_prox(self._h, _ptr(codes), _ptr(delta), length, arr, nseg, _ptr(mu), _ptr(x),
                                                eta, lambda_l1, _ptr(v_out)))
         return x
+
+    def message_entropy(self, codes, length, seg_offsets=None, hist_out=None, host_counts=True):
+        """Histogram of every (worker, segment) message and, on the host, its entropy bound and Huffman length in bits.
+        Returns (hist (N, nseg, 2^b) int64 CUDA tensor, entropy (N, nseg) or None, huffman (N, nseg) or None)."""
+        arr, nseg = _seg(seg_offsets)
+        if hist_out is None:
+            hist_out = torch.empty((self.N, nseg, 1 << self.b), dtype=torch.int64, device=codes.device)
+        ent = (C.c_double * (self.N * nseg))() if host_counts else None
+        huf = (C.c_uint64 * (self.N * nseg))() if host_counts else None
+        self._ck(lib().lpc_message_entropy(self._h, _ptr(codes), length, arr, nseg, _ptr(hist_out), ent, huf))
+        if not host_counts:
+            return hist_out, None, None
+        import numpy as np
+        return (hist_out, np.array(ent[:], dtype=np.float64).reshape(self.N, nseg),
+                np.array(huf[:], dtype=np.uint64).reshape(self.N, nseg))
 
     def server_reduce(self, codes, length, scheme, k, seg_offsets=None, codes_out=None):
         """The server of scheme (b) or (c): N streams of b bits in, one stream out.  Returns (codes_out, bits_out)."""
