@@ -254,6 +254,20 @@ int lpc_alpc_double_sample_steps(lpc_ctx* ctx, float tau1, float tau2, float alp
                                  uint64_t k0, int64_t count);
 int lpc_alpc_end_epoch(lpc_ctx* ctx, int64_t m);
 
+/*
+ * The strongly convex case of ALPC-SVRG (Algorithm 2 as printed, Theorem 3): h(x) = lambda_l1*||x||_1 +
+ * (sigma/2)*||x||^2 with sigma > 0.  After this call lpc_alpc_double_sample_step(s) solve the two argmins of steps
+ * 12-13 for that h -- the soft-threshold results divided by (1 + sigma/(4L)) and by (1 + alpha*sigma) -- and weigh the
+ * y iterate of step t of an epoch by (1 + alpha*sigma)^t (formed by repeated fp32 multiplication on the host);
+ * lpc_alpc_end_epoch then takes Algorithm 2's weighted mean instead of Algorithm 3's plain mean, and lpc_objective
+ * adds (sigma/2)*||x||^2.  tau1, tau2 and alpha stay the caller's (the theorem's choice: tau1 = sqrt(m sigma/(6L)),
+ * alpha = 1/(6 tau1 L)).  The weight changes from step to step, so these steps run as per-step launches, not as the
+ * one-launch loop.  sigma = 0 restores the general convex case (bit-identical to never having called this).
+ * Algorithm 1's proximal step (lpc_inner_step, lpc_unpack_average_prox) keeps h = lambda_l1*||.||_1.
+ * lpc_alpc_begin and lpc_alpc_end_epoch restart the weights.  Errors: LPC_ERR_INVALID_ARG for sigma < 0 or not finite.
+ */
+int lpc_set_strong_convexity(lpc_ctx* ctx, float sigma);
+
 /* P(x) = f(x) + lambda_l1*||x||_1 (Eq. 1) in one pass over X.  x nullable (= current iterate);
  * P_out is a HOST pointer; the call waits for the stream. */
 int lpc_objective(lpc_ctx* ctx, const float* x, double* P_out);

@@ -155,9 +155,9 @@ __global__ void __launch_bounds__(AT) unpack_average_prox_kernel(AggArgs a) {
       const float ky = mul_rn(a.inv4L, a.lambda_l1), kz = mul_rn(a.alpha, a.lambda_l1);
 #pragma unroll
       for (int e = 0; e < 8; ++e) {
-        yv[e] = soft_threshold(__fsub_rn(xv[e], mul_rn(a.inv4L, vv[e])), ky);
-        zv[e] = soft_threshold(__fsub_rn(zv[e], mul_rn(a.alpha, hv[e])), kz);
-        sv[e] = add_rn(sv[e], yv[e]);
+        yv[e] = mul_rn(soft_threshold(__fsub_rn(xv[e], mul_rn(a.inv4L, vv[e])), ky), a.cy);
+        zv[e] = mul_rn(soft_threshold(__fsub_rn(zv[e], mul_rn(a.alpha, hv[e])), kz), a.cz);
+        sv[e] = add_rn(sv[e], mul_rn(a.wy, yv[e]));
       }
       store8f(a.y + s.off, j, s.len, vec, yv);
       store8f(a.z + s.off, j, s.len, vec, zv);

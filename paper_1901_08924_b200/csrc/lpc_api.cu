@@ -72,7 +72,7 @@ struct lpc_ctx {
   float* coef_tap = nullptr;
   uint64_t* k_dev = nullptr;
   unsigned int* dev_status = nullptr;
-  double* f_dev = nullptr;  // [0] = f, [1] = ||x||_1
+  double* f_dev = nullptr;  // [0] = f, [1] = ||x||_1, [2] = ||x||^2
   // snapshot pass
   int snapR = 1, snapStages = 1, snapGrid = 1, dpad = 0;
   size_t snapSmem = 0;
@@ -99,6 +99,9 @@ struct lpc_ctx {
   SegPlan seg;
   SegPlan seg_out;       // layout of the server's output stream (schemes (b), (c))
   int shared_scale = 0;  // LPC_OPT_SHARED_SCALE
+  float sigma = 0.f;     // strong convexity of h (lpc_set_strong_convexity); 0: general convex case
+  float sc_w = 1.f;      // snapshot weight of the next ALPC step, (1 + alpha*sigma)^t in fp32
+  float sc_wsum = 0.f;   // sum of the weights used so far in this epoch
   int divisor = 0;       // LPC_OPT_AVERAGE_DIVISOR; 0: the worker count N
   uint32_t* q_pmax = nullptr;
   float *q_ps1 = nullptr, *q_ps2 = nullptr;
@@ -313,6 +316,7 @@ AggArgs agg_args(lpc_ctx* c, const SegPlan& p, const uint32_t* codes, const floa
   a.segs = p.d_segs; a.tile_seg = p.d_tile_seg; a.nseg = p.nseg; a.ntiles = p.ntiles;
   a.mu = mu; a.x = x; a.eta = eta; a.lambda_l1 = lambda_l1; a.v_out = v_out; a.k_counter = nullptr;
   a.mode = 0; a.y = nullptr; a.z = nullptr; a.ysum = nullptr; a.vhat = nullptr; a.alpha = 0.f; a.inv4L = 0.f;
+  a.cy = 1.f; a.cz = 1.f; a.wy = 1.f;
   return a;
 }
 
@@ -349,7 +353,18 @@ int enqueue_alpc_step(lpc_ctx* c, float tau1, float tau2, float alpha, float inv
   AggArgs ag = agg_args(c, c->inner_seg, c->codes, c->delta, c->mu, c->x, 0.f, c->lambda_l1, c->tap_u ? c->v_tap : nullptr);
   ag.k_counter = k_counter;
   ag.mode = 1; ag.y = c->yv; ag.z = c->zv; ag.ysum = c->ysum; ag.vhat = c->vhat; ag.alpha = alpha; ag.inv4L = inv4L;
+  if (c->sigma > 0.f) {  // each product and sum below is one fp32 operation, as on the device
+    volatile float t1 = c->sigma * inv4L, t2 = alpha * c->sigma;
+    volatile float d1 = 1.0f + t1, d2 = 1.0f + t2;
+    ag.cy = 1.0f / d1; ag.cz = 1.0f / d2; ag.wy = c->sc_w;
+  }
   { ProfScope ps_(c, LPC_KERNEL_AGGREGATE); CU(c, launch_unpack_average_prox(ag, c->stream)); }
+  if (c->sigma > 0.f) {  // the weight of the next step and the sum of those used (Algorithm 2's last step)
+    volatile float t2 = alpha * c->sigma;
+    volatile float theta = 1.0f + t2;
+    volatile float ws = c->sc_wsum + c->sc_w, wn = c->sc_w * theta;
+    c->sc_wsum = ws; c->sc_w = wn;
+  }
   return LPC_OK;
 }
 
@@ -363,7 +378,9 @@ int run_steps(lpc_ctx* c, int kind, const float* p, uint64_t k0, int64_t count) 
   };
   int64_t done = 0;
   const bool loop_ok = (kind == 0) ? c->persist_ok : c->apersist_ok;
-  if (c->use_persist && loop_ok && count >= 2 && count <= 0x7FFFFFFF) {
+  // the strongly convex ALPC step carries a weight that changes from step to step: plain per-step launches
+  const bool weighted = (kind == 1 && c->sigma > 0.f);
+  if (c->use_persist && loop_ok && !weighted && count >= 2 && count <= 0x7FFFFFFF) {
     // the whole loop in one cooperative launch; on a launch refusal fall through to the per-step kernels
     PersistArgs pa;
     pa.in = inner_args(c, k0, nullptr, 0);
@@ -397,7 +414,7 @@ int run_steps(lpc_ctx* c, int kind, const float* p, uint64_t k0, int64_t count) 
       if (kind == 0) c->persist_ok = false; else c->apersist_ok = false;
     }
   }
-  if (done < count && c->use_graph && !c->profile && count >= GRAPH_STEPS) {
+  if (done < count && c->use_graph && !c->profile && !weighted && count >= GRAPH_STEPS) {
     GraphKey key;
     key.kind = kind; key.steps = GRAPH_STEPS; key.tap = c->tap_u; key.cs = c->CS; key.sample_global = c->sample_global;
     for (int i = 0; i < 4; ++i) key.p[i] = p[i];
@@ -530,7 +547,7 @@ int lpc_init(lpc_ctx** out, const float* X, const float* y, int64_t n, int32_t d
   auto A = [&](int r) { if (rc == LPC_OK) rc = r; };
   A(dalloc(c, &c->dev_status, 1));
   A(dalloc(c, &c->k_dev, 1));
-  A(dalloc(c, &c->f_dev, 2));
+  A(dalloc(c, &c->f_dev, 3));
   if (model && rc == LPC_OK) {
     const size_t dd = (size_t)d;
     A(dalloc(c, &c->x, dd)); A(dalloc(c, &c->xt, dd)); A(dalloc(c, &c->mu, dd)); A(dalloc(c, &c->margins, (size_t)n));
@@ -692,6 +709,15 @@ int lpc_alpc_begin(lpc_ctx* c) {
   CU(c, cudaMemcpyAsync(c->yv, c->x, bytes, cudaMemcpyDeviceToDevice, c->stream));
   CU(c, cudaMemcpyAsync(c->zv, c->x, bytes, cudaMemcpyDeviceToDevice, c->stream));
   CU(c, cudaMemsetAsync(c->ysum, 0, bytes, c->stream));
+  c->sc_w = 1.f; c->sc_wsum = 0.f;
+  return LPC_OK;
+}
+
+int lpc_set_strong_convexity(lpc_ctx* c, float sigma) {
+  if (!c) return LPC_ERR_INVALID_ARG;
+  if (!(sigma >= 0.f) || !std::isfinite(sigma)) return fail(c, LPC_ERR_INVALID_ARG, "sigma must be finite and >= 0");
+  c->sigma = sigma;
+  c->sc_w = 1.f; c->sc_wsum = 0.f;
   return LPC_OK;
 }
 
@@ -714,7 +740,12 @@ int lpc_alpc_double_sample_steps(lpc_ctx* c, float tau1, float tau2, float alpha
 int lpc_alpc_end_epoch(lpc_ctx* c, int64_t m) {
   if (!c || m < 1) return LPC_ERR_INVALID_ARG;
   if (!has_model(c)) return fail(c, LPC_ERR_UNSUPPORTED, "quantizer-only context");
-  const float inv_m = 1.0f / (float)m;  // IEEE division on the host
+  float inv_m = 1.0f / (float)m;  // IEEE division on the host
+  if (c->sigma > 0.f) {  // Algorithm 2: the weighted mean; the weights start over with the next epoch
+    if (!(c->sc_wsum > 0.f)) return fail(c, LPC_ERR_INVALID_ARG, "no step since the last snapshot");
+    inv_m = 1.0f / c->sc_wsum;
+    c->sc_w = 1.f; c->sc_wsum = 0.f;
+  }
   CU(c, launch_mean_y(c->ysum, inv_m, c->d, c->x, c->stream));
   return LPC_OK;
 }
@@ -726,10 +757,10 @@ int lpc_objective(lpc_ctx* c, const float* x, double* P_out) {
   if (!aligned16(pt)) return fail(c, LPC_ERR_INVALID_ARG, "x must be 16-byte aligned");
   TRY(snapshot_pass(c, pt, false, nullptr));
   CU(c, launch_l1_norm(pt, c->d, &c->f_dev[1], c->stream));
-  double h[2] = {0, 0};
+  double h[3] = {0, 0, 0};
   CU(c, cudaMemcpyAsync(h, c->f_dev, sizeof(h), cudaMemcpyDeviceToHost, c->stream));
   CU(c, cudaStreamSynchronize(c->stream));
-  *P_out = h[0] + (double)c->lambda_l1 * h[1];
+  *P_out = h[0] + (double)c->lambda_l1 * h[1] + 0.5 * (double)c->sigma * h[2];
   return LPC_OK;
 }
 

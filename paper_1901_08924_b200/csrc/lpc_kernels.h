@@ -84,6 +84,10 @@ struct AggArgs {
   const float* vhat;
   float alpha;
   float inv4L;
+  // strongly convex case of Algorithm 2, h = lambda_l1*||.||_1 + (sigma/2)*||.||^2: the soft-threshold results are
+  // multiplied by cy = 1/(1 + sigma*inv4L) and cz = 1/(1 + alpha*sigma), and ysum += wy * y (the snapshot weight
+  // (1 + alpha*sigma)^t of the step).  All three are 1 in the general convex case, where they change no bit.
+  float cy, cz, wy;
 };
 
 cudaError_t launch_unpack_average_prox(const AggArgs& a, cudaStream_t st);

@@ -205,19 +205,27 @@ __global__ void snapshot_reduce_kernel(const float* __restrict__ partial_mu, con
   }
 }
 
-// lambda-free L1 norm partials for P(x): one CTA, fp64.
+// The regulariser's two norms for P(x), without their weights: out[0] = ||x||_1, out[1] = ||x||^2.  One CTA, fp64.
 __global__ void l1_norm_kernel(const float* __restrict__ x, int d, double* __restrict__ out) {
-  __shared__ double sh[32];
-  double s = 0.0;
-  for (int j = threadIdx.x; j < d; j += blockDim.x) s += fabs((double)x[j]);
+  __shared__ double sh[32], sh2[32];
+  double s = 0.0, q = 0.0;
+  for (int j = threadIdx.x; j < d; j += blockDim.x) {
+    const double v = (double)x[j];
+    s += fabs(v);
+    q += v * v;
+  }
 #pragma unroll
-  for (int m = 16; m >= 1; m >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, m);
-  if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = s;
+  for (int m = 16; m >= 1; m >>= 1) {
+    s += __shfl_xor_sync(0xFFFFFFFFu, s, m);
+    q += __shfl_xor_sync(0xFFFFFFFFu, q, m);
+  }
+  if ((threadIdx.x & 31) == 0) { sh[threadIdx.x >> 5] = s; sh2[threadIdx.x >> 5] = q; }
   __syncthreads();
   if (threadIdx.x == 0) {
-    double t = 0.0;
-    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) t += sh[w];
-    *out = t;
+    double t = 0.0, t2 = 0.0;
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) { t += sh[w]; t2 += sh2[w]; }
+    out[0] = t;
+    out[1] = t2;
   }
 }
 

@@ -49,6 +49,7 @@ SYMBOLS = [
     ("lpc_sum_bits", _int, [_i32, _i32, C.POINTER(C.c_int32)]),
     ("lpc_scheme_bits", _int, [_int, _i64, _i32, _i32, _u64p]),
     ("lpc_alpc_begin", _int, [_vp]),
+    ("lpc_set_strong_convexity", _int, [_vp, _f32]),
     ("lpc_alpc_double_sample_step", _int, [_vp, _f32, _f32, _f32, _f32, _u64]),
     ("lpc_alpc_double_sample_steps", _int, [_vp, _f32, _f32, _f32, _f32, _u64, _i64]),
     ("lpc_alpc_end_epoch", _int, [_vp, _i64]),
@@ -266,6 +267,9 @@ class Context:
             codes_out = torch.empty((1, stride), dtype=torch.int32, device=codes.device)
         self._ck(lib().lpc_server_reduce(self._h, _ptr(codes), length, arr, nseg, scheme, k, _ptr(codes_out)))
         return codes_out, bo
+
+    def set_strong_convexity(self, sigma):
+        self._ck(lib().lpc_set_strong_convexity(self._h, sigma))
 
     def alpc_begin(self):
         self._ck(lib().lpc_alpc_begin(self._h))
