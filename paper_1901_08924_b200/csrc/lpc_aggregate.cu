@@ -298,6 +298,15 @@ __global__ void __launch_bounds__(AT, 4) server_reduce_kernel(ServerArgs a) {
         return;
       }
     }
+    if (!a.requantize && bo <= 8) {
+      // eight sums of at most 8 bits: one 64-bit word, built from the last code down with one uniform shift each
+      const uint32_t bias_out = 1u << (bo - 1);
+      uint64_t wv = 0;
+#pragma unroll
+      for (int e = 7; e >= 0; --e) wv = (wv << bo) | (uint64_t)((e < nvalid) ? (uint32_t)K[e] + bias_out : 0u);
+      olo = wv;
+      return;
+    }
 #pragma unroll
     for (int e = 0; e < 8; ++e) {
       if (e < nvalid) {
@@ -330,7 +339,15 @@ __global__ void __launch_bounds__(AT, 4) server_reduce_kernel(ServerArgs a) {
     } else {
       if (staged_before) __syncthreads();
       staged_before = true;
-      for (int i = 0; i < bo; ++i) stage[tid * bo + i] = (uint8_t)((i < 8) ? (olo >> (8 * i)) : (ohi >> (8 * (i - 8))));
+      if (bo <= 8) {
+        const uint32_t l32 = (uint32_t)olo, h32 = (uint32_t)(olo >> 32);
+        uint8_t* dst = stage + tid * bo;
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+          if (i < bo) dst[i] = (uint8_t)(((i < 4) ? l32 : h32) >> (8 * (i & 3)));
+      } else {
+        for (int i = 0; i < bo; ++i) stage[tid * bo + i] = (uint8_t)((i < 8) ? (olo >> (8 * i)) : (ohi >> (8 * (i - 8))));
+      }
       __syncthreads();
       const int64_t w0 = (sweep0 >> 5) * bo;  // sweep0 is a multiple of 2048, so this is exact
       const uint32_t* stw = reinterpret_cast<const uint32_t*>(stage);

@@ -51,6 +51,7 @@ constexpr int SNT = (SDW + SUW + SCW + SPW + SMETAW) * 32;  // threads of the st
 
 struct Smem {
   uint64_t bar;
+  uint64_t xbar;                  // scale statistics of every CTA of the cluster have arrived (bytes of their stores)
   int64_t idx[MAXB];
   float yv[MAXB];
   float msnap[MAXB];
@@ -144,6 +145,7 @@ __global__ void __launch_bounds__(STREAM ? SNT : IT) inner_kernel(InnerArgs a) {
   }
   if (tid == 0) {
     mbar_init(&sm.bar, 1);
+    mbar_init(&sm.xbar, 1);
     if constexpr (STREAM) {
       for (int r = 0; r < SMAXR; ++r) {
         mbar_init(&sm.sbar[r], 1);
@@ -585,13 +587,16 @@ __global__ void __launch_bounds__(STREAM ? SNT : IT) inner_kernel(InnerArgs a) {
       s1 = smem_tree_sum(sm.ws1, np * 8);
       s2 = smem_tree_sum(sm.ws2, np * 8);
     }
+    // the three statistics go to every CTA of the cluster as stores that count on the receiver's barrier: the one
+    // thread that needs them waits for their bytes, and no cluster-wide barrier is paid
+    mbar_expect_tx(&sm.xbar, (uint32_t)(CS * 12));
     for (int q = 0; q < CS; ++q) {
-      cluster.map_shared_rank(sm.maxpart, q)[rank] = m;
-      cluster.map_shared_rank(sm.s1part, q)[rank] = s1;
-      cluster.map_shared_rank(sm.s2part, q)[rank] = s2;
+      st_async_cluster(&sm.maxpart[rank], &sm.xbar, (uint32_t)q, m);
+      st_async_cluster(&sm.s1part[rank], &sm.xbar, (uint32_t)q, __float_as_uint(s1));
+      st_async_cluster(&sm.s2part[rank], &sm.xbar, (uint32_t)q, __float_as_uint(s2));
     }
+    if (!mbar_wait_cluster(&sm.xbar, 0)) atomicOr(a.dev_status, DEV_TIMEOUT);
   }
-  cluster.sync();
   if (tid == 0) {
     uint32_t m = 0;
     for (int q = 0; q < CS; ++q) m = max(m, sm.maxpart[q]);
