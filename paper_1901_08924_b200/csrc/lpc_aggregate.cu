@@ -393,9 +393,13 @@ __global__ void __launch_bounds__(AT) code_histogram_kernel(HistArgs a) {
   const int tile0 = blockIdx.x * HRUN, tile1 = min(tile0 + HRUN, a.ntiles);
   const int tid = threadIdx.x;
   const int b = BITS ? BITS : a.b, bins = 1 << b;
-  const int rows = (bins + 3) / 4;  // words per thread
-  extern __shared__ __align__(16) uint32_t cw[];  // rows x AT words
-  uint8_t* mine = reinterpret_cast<uint8_t*>(cw + tid);  // this thread's counter of value c: mine[(c / 4) * AT * 4 + c % 4]
+  const int rows = (bins + 3) / 4;  // words per thread and copy
+  // Narrow codes keep NCH copies of the counters, one per coordinate position modulo NCH: the eight increments of a
+  // group then form NCH independent chains of read-modify-writes instead of one (they may hit the same counter, so
+  // the chain of one copy cannot be reordered)
+  constexpr int NCH = (BITS >= 1 && BITS <= 4) ? 4 : 1;
+  extern __shared__ __align__(16) uint32_t cw[];  // NCH x rows x AT words
+  uint8_t* mine = reinterpret_cast<uint8_t*>(cw + tid);  // this thread's counter of value c in copy q: mine[((q * rows + c / 4) * AT) * 4 + c % 4]
   __shared__ unsigned int total[256];
   for (int c = tid; c < bins; c += AT) total[c] = 0u;
   int cur_seg = -1;
@@ -417,7 +421,7 @@ __global__ void __launch_bounds__(AT) code_histogram_kernel(HistArgs a) {
     }
     const SegInfo s = a.segs[seg];
     const int64_t tstart = (int64_t)(tile - s.tile_first) * TILE;
-    for (int i = tid; i < rows * AT; i += AT) cw[i] = 0u;  // a thread clears and uses its own column only
+    for (int i = tid; i < NCH * rows * AT; i += AT) cw[i] = 0u;  // a thread clears and uses its own column only
     const uint32_t* w = a.codes + (int64_t)worker * a.stride_words + s.word_off;
 #pragma unroll 1
     for (int it = 0; it < AITER; ++it) {  // a thread sees at most AITER * 8 = 32 codes: a byte counter cannot overflow
@@ -430,14 +434,16 @@ __global__ void __launch_bounds__(AT) code_histogram_kernel(HistArgs a) {
       for (int e = 0; e < 8; ++e) {
         if (e < nvalid) {
           const uint32_t code = (uint32_t)(lo >> (e * b)) & (uint32_t)(bins - 1);
-          mine[((code >> 2) * (AT * 4)) | (code & 3u)] += 1;
+          mine[((((e % NCH) * rows + (code >> 2)) * (AT * 4))) | (code & 3u)] += 1;
         }
       }
     }
     // the tile's columns add up: a word's four byte counters (each <= 32) widen to two words of 16-bit lanes, a warp
     // adds them with one integer reduction each (32 lanes * 32 fits 16 bits), lane 0 adds the sums to the run's totals
     for (int r = 0; r < rows; ++r) {
-      const uint32_t v = cw[r * AT + tid];
+      uint32_t v = cw[r * AT + tid];
+#pragma unroll
+      for (int q = 1; q < NCH; ++q) v += cw[(q * rows + r) * AT + tid];  // byte lanes: at most 32 in all, no carry
       const uint32_t even = __reduce_add_sync(0xFFFFFFFFu, v & 0x00FF00FFu);         // values 4r, 4r+2
       const uint32_t odd = __reduce_add_sync(0xFFFFFFFFu, (v >> 8) & 0x00FF00FFu);   // values 4r+1, 4r+3
       if ((tid & 31) == 0) {
@@ -455,7 +461,7 @@ __global__ void __launch_bounds__(AT) code_histogram_kernel(HistArgs a) {
 
 cudaError_t launch_code_histogram(const HistArgs& a, cudaStream_t st) {
   if (a.ntiles <= 0 || a.N <= 0) return cudaSuccess;
-  const size_t sh = (size_t)(((1 << a.b) + 3) / 4) * AT * sizeof(uint32_t);
+  const size_t sh = (size_t)(a.b <= 4 && (a.b == 1 || a.b == 2 || a.b == 4) ? 4 : 1) * (size_t)(((1 << a.b) + 3) / 4) * AT * sizeof(uint32_t);
   const dim3 grid((unsigned)((a.ntiles + HRUN - 1) / HRUN), (unsigned)a.N);
   auto go = [&](auto kernel) {
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sh);

@@ -146,3 +146,67 @@ def test_dnn_shaped_aggregation_full_bitwise():
         assert (_bits(xh[offs[s]:offs[s + 1]]) == _bits(ref)).all(), s
         base += (ln + 7) // 8
     q.close()
+
+
+def test_server_schemes_and_entropy_count_full_length():
+    # 8 worker vectors of 2^26 Gaussian values of different magnitudes, b = 4, clip 2 std, in the launch shapes the
+    # benchmark times: unified scale from full passes, codes / server streams / updated coordinates in sampled windows;
+    # worker 0's own message (own scale) and its histogram in full
+    N, length, b, seed, k = 8, 1 << 26, 4, 13, 5
+    U = synth.gradient_vectors(N, length, "gauss", seed=6, device=DEV)
+    U *= torch.linspace(0.5, 1.5, N, device=DEV).unsqueeze(1)
+    Uh = U.cpu().numpy()
+    q = lpc.Context(None, None, lpc.LOGISTIC, 0.0, N, 1, b, lpc.CLIP_STD, 2.0, seed)
+    # -- own scales: worker 0 in full against the oracle, then its histogram and the two counts
+    codes, delta, _ = q.quantize_pack(U, k)
+    hist, ent, huf = q.message_entropy(codes, length)
+    q.sync_status()
+    w0, d0, _ = orc.quantize_pack(Uh[0], b, orc.CLIP_STD, 2.0, seed=seed, worker=0, k=k)
+    ch = codes.cpu().numpy().view(np.uint32)
+    assert (ch[0, : w0.size] == w0).all() and _bits(delta.cpu().numpy()[0, :1])[0] == _bits(np.array([d0], np.float32))[0]
+    h0 = orc.code_histogram(w0, length, b)
+    hg = hist.cpu().numpy()
+    assert (hg[0, 0].astype(np.uint64) == h0).all()
+    assert (hg.sum(axis=2) == length).all()
+    assert huf[0, 0] == orc.huffman_bits(h0) and ent[0, 0] == pytest.approx(orc.entropy_bits(h0), rel=1e-12)
+    # -- unified scale
+    q.set_option(lpc.OPT_SHARED_SCALE, 1)
+    codes, delta, clipped = q.quantize_pack(U, k)
+    srv_b, bo = q.server_reduce(codes, length, lpc.SCHEME_SERVER_SUM, k)
+    srv_c, _ = q.server_reduce(codes, length, lpc.SCHEME_SERVER_REQUANTIZE, k)
+    xb, xc = torch.zeros(length, device=DEV), torch.zeros(length, device=DEV)
+    wb = lpc.Context(None, None, lpc.LOGISTIC, 0.0, 1, 1, bo, lpc.CLIP_NONE, 1.0, seed)
+    wb.set_option(lpc.OPT_AVERAGE_DIVISOR, N)
+    wc = lpc.Context(None, None, lpc.LOGISTIC, 0.0, 1, 1, b, lpc.CLIP_NONE, 1.0, seed)
+    d1 = delta[:1].contiguous()
+    wb.unpack_average_prox(srv_b, d1, length, xb, 1.0, 1e-3)
+    wc.unpack_average_prox(srv_c, d1, length, xc, 1.0, 1e-3)
+    for c in (q, wb, wc):
+        c.sync_status()
+    sc = [orc.scale(Uh[i], b, orc.CLIP_STD, 2.0) for i in range(N)]
+    best = max(sc, key=lambda s: s["T"])
+    dl = delta.cpu().numpy()
+    assert (_bits(dl) == _bits(np.float32(best["delta"]))).all()
+    lower = -(np.float32(best["T"]) + np.float32(best["delta"]))
+    want_clip = [int(((Uh[i] > best["T"]) | (Uh[i] < lower)).sum()) for i in range(N)]
+    assert clipped.cpu().numpy()[:, 0].tolist() == want_clip
+    W = 2048
+    ch = codes.cpu().numpy().view(np.uint32)
+    sb, sc_ = srv_b.cpu().numpy().view(np.uint32).ravel(), srv_c.cpu().numpy().view(np.uint32).ravel()
+    xbh, xch = xb.cpu().numpy(), xc.cpu().numpy()
+    for s0 in [0, 8192 * 1000 + 32, (1 << 25) - 1024, length - W]:
+        words = np.zeros((N, W * b // 32), np.uint32)
+        for i in range(N):
+            c = np.array([orc.quantize_coord(Uh[i, j], best["rdelta"], b, orc.rounding_bits(seed, i, k, 0, j)) + 8
+                          for j in range(s0, s0 + W)], np.uint32)
+            words[i] = orc.pack(c, b)
+        assert (ch[:, s0 * b // 32:(s0 + W) * b // 32] == words).all(), s0
+        ref_b = orc.server_reduce(words, W, b, False)
+        ref_c = orc.server_reduce(words, W, b, True, seed=seed, k=k, block_base=s0 // 8)
+        assert (sb[s0 * bo // 32:(s0 + W) * bo // 32] == ref_b).all(), s0
+        assert (sc_[s0 * b // 32:(s0 + W) * b // 32] == ref_c).all(), s0
+        zero = np.zeros(W, np.float32)
+        assert (_bits(xbh[s0:s0 + W]) == _bits(orc.unpack_scaled_prox(ref_b, best["delta"], W, bo, N, None, zero, 1.0, 1e-3))).all()
+        assert (_bits(xch[s0:s0 + W]) == _bits(orc.unpack_scaled_prox(ref_c, best["delta"], W, b, 1, None, zero, 1.0, 1e-3))).all()
+    for c in (q, wb, wc):
+        c.close()
