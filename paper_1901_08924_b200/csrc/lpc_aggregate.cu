@@ -423,18 +423,49 @@ __global__ void __launch_bounds__(AT) code_histogram_kernel(HistArgs a) {
     const int64_t tstart = (int64_t)(tile - s.tile_first) * TILE;
     for (int i = tid; i < NCH * rows * AT; i += AT) cw[i] = 0u;  // a thread clears and uses its own column only
     const uint32_t* w = a.codes + (int64_t)worker * a.stride_words + s.word_off;
-#pragma unroll 1
-    for (int it = 0; it < AITER; ++it) {  // a thread sees at most AITER * 8 = 32 codes: a byte counter cannot overflow
-      const int64_t j = tstart + (int64_t)it * AGROUP + tid * 8;
-      if (j >= s.len) break;
-      const int nvalid = (int)min((int64_t)8, s.len - j);
-      uint64_t lo, hi;
-      load_chunk<BITS>(w, j >> 3, b, s.pad_words, lo, hi);  // 8 * b <= 64 bits: all in lo
+    if constexpr (BITS != 0) {
+      // fixed widths: which thread counts which code does not matter, so a thread takes whole words of the tile's
+      // stream, BITS of them, AT words apart (coalesced), all requested before the first is used
+      constexpr int CPW = 32 / BITS;  // codes per word
+      const int64_t nvalid_tile = min((int64_t)TILE, s.len - tstart);
+      const uint32_t* wt = w + (tstart >> 5) * BITS;
+      uint32_t cwords[BITS];
 #pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        if (e < nvalid) {
-          const uint32_t code = (uint32_t)(lo >> (e * b)) & (uint32_t)(bins - 1);
-          mine[((((e % NCH) * rows + (code >> 2)) * (AT * 4))) | (code & 3u)] += 1;
+      for (int i = 0; i < BITS; ++i) {
+        const int wi = i * AT + tid;
+        cwords[i] = ((int64_t)wi * CPW < nvalid_tile) ? __ldcs(wt + wi) : 0u;
+      }
+#pragma unroll
+      for (int i = 0; i < BITS; ++i) {
+        const int wi = i * AT + tid;
+        const int64_t left = nvalid_tile - (int64_t)wi * CPW;  // codes of this word that exist
+        if (left >= CPW) {
+#pragma unroll
+          for (int e = 0; e < CPW; ++e) {
+            const uint32_t code = (cwords[i] >> (e * BITS)) & (uint32_t)(bins - 1);
+            mine[((((e % NCH) * rows + (code >> 2)) * (AT * 4))) | (code & 3u)] += 1;
+          }
+        } else {
+          for (int e = 0; e < (int)left; ++e) {
+            const uint32_t code = (cwords[i] >> (e * BITS)) & (uint32_t)(bins - 1);
+            mine[((((e % NCH) * rows + (code >> 2)) * (AT * 4))) | (code & 3u)] += 1;
+          }
+        }
+      }
+    } else {
+#pragma unroll 1
+      for (int it = 0; it < AITER; ++it) {  // a thread sees at most AITER * 8 = 32 codes: a byte counter cannot overflow
+        const int64_t j = tstart + (int64_t)it * AGROUP + tid * 8;
+        if (j >= s.len) break;
+        const int nvalid = (int)min((int64_t)8, s.len - j);
+        uint64_t lo, hi;
+        load_chunk<0>(w, j >> 3, b, s.pad_words, lo, hi);  // 8 * b <= 64 bits: all in lo
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          if (e < nvalid) {
+            const uint32_t code = (uint32_t)(lo >> (e * b)) & (uint32_t)(bins - 1);
+            mine[((code >> 2) * (AT * 4)) | (code & 3u)] += 1;
+          }
         }
       }
     }
