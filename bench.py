@@ -461,8 +461,7 @@ def alpc_bench(dev):
                           "loop_row_buffers": ctx.query(lpc.INFO_ALPC_LOOP_ROW_BUFFERS),
                           "one_launch_loops": ctx.query(lpc.INFO_LOOP_LAUNCHES), "objective": ctx.objective()}
         ctx.close()
-    # the strongly convex case (Algorithm 2, elastic net with sigma = L/1000, Theorem 3's tau1 and alpha): per-step
-    # launches, because the snapshot weight changes from step to step
+    # the strongly convex case (Algorithm 2, elastic net with sigma = L/1000, Theorem 3's tau1 and alpha)
     b, sigma = 2, L / 1000.0
     tau1 = min(0.5, (m * sigma / (6.0 * L)) ** 0.5)
     ctx = lpc.Context(X, y, lpc.LOGISTIC, 1e-5, N, B, b, lpc.CLIP_STD, 2.0, 0)
@@ -481,7 +480,7 @@ def alpc_bench(dev):
         times.append(ev[0].elapsed_time(ev[1]))
     ctx.sync_status()
     out["strongly_convex_b2"] = {"sigma_over_L": 1e-3, "tau1": round(tau1, 4), "step_us": round(min(times[1:]) * 1e3 / m, 3),
-                                 "path": "per-step kernels", "objective": ctx.objective()}
+                                 "one_launch_loops": ctx.query(lpc.INFO_LOOP_LAUNCHES), "objective": ctx.objective()}
     ctx.close()
     return out
 

@@ -261,8 +261,9 @@ int lpc_alpc_end_epoch(lpc_ctx* ctx, int64_t m);
  * y iterate of step t of an epoch by (1 + alpha*sigma)^t (formed by repeated fp32 multiplication on the host);
  * lpc_alpc_end_epoch then takes Algorithm 2's weighted mean instead of Algorithm 3's plain mean, and lpc_objective
  * adds (sigma/2)*||x||^2.  tau1, tau2 and alpha stay the caller's (the theorem's choice: tau1 = sqrt(m sigma/(6L)),
- * alpha = 1/(6 tau1 L)).  The weight changes from step to step, so these steps run as per-step launches, not as the
- * one-launch loop.  sigma = 0 restores the general convex case (bit-identical to never having called this).
+ * alpha = 1/(6 tau1 L)).  lpc_alpc_double_sample_steps runs them in the one-launch loop like the general convex case (each
+ * CTA forms the weights of its steps itself); where that loop is not available they run as plain per-step launches,
+ * without graph replay, because the weight is a launch argument that changes from step to step.  sigma = 0 restores the general convex case (bit-identical to never having called this).
  * Algorithm 1's proximal step (lpc_inner_step, lpc_unpack_average_prox) keeps h = lambda_l1*||.||_1.
  * lpc_alpc_begin and lpc_alpc_end_epoch restart the weights.  Errors: LPC_ERR_INVALID_ARG for sigma < 0 or not finite.
  */

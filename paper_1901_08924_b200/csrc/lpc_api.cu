@@ -380,7 +380,7 @@ int run_steps(lpc_ctx* c, int kind, const float* p, uint64_t k0, int64_t count) 
   const bool loop_ok = (kind == 0) ? c->persist_ok : c->apersist_ok;
   // the strongly convex ALPC step carries a weight that changes from step to step: plain per-step launches
   const bool weighted = (kind == 1 && c->sigma > 0.f);
-  if (c->use_persist && loop_ok && !weighted && count >= 2 && count <= 0x7FFFFFFF) {
+  if (c->use_persist && loop_ok && count >= 2 && count <= 0x7FFFFFFF) {
     // the whole loop in one cooperative launch; on a launch refusal fall through to the per-step kernels
     PersistArgs pa;
     pa.in = inner_args(c, k0, nullptr, 0);
@@ -402,11 +402,23 @@ int run_steps(lpc_ctx* c, int kind, const float* p, uint64_t k0, int64_t count) 
     pa.v_tap = c->tap_u ? c->v_tap : nullptr;
     pa.alpc = kind; pa.tau1 = p[0]; pa.tau2 = p[1]; pa.alpha = p[2]; pa.inv4L = p[3];
     pa.y = c->yv; pa.z = c->zv; pa.ysum = c->ysum; pa.xt = c->xt; pa.vhat = c->vhat;
+    pa.cy = 1.f; pa.cz = 1.f; pa.w0 = 1.f; pa.theta = 1.f;
+    if (weighted) {  // each product and sum is one fp32 operation, as on the device
+      volatile float t1 = c->sigma * p[3], t2 = p[2] * c->sigma;
+      volatile float d1 = 1.0f + t1, d2 = 1.0f + t2;
+      pa.cy = 1.0f / d1; pa.cz = 1.0f / d2; pa.w0 = c->sc_w; pa.theta = d2;
+    }
     CU(c, cudaMemsetAsync(pa.abort_flag, 0, sizeof(unsigned long long), c->stream));
     cudaError_t e;
     { ProfScope ps_(c, LPC_KERNEL_INNER_LOOP); e = launch_persist(pa, kind == 0 ? c->persistSmem : c->apersistSmem, c->stream); }
     if (e == cudaSuccess) {
       done = count;
+      if (weighted) {  // the weights the loop went through, and the one the next step starts from
+        for (int64_t i = 0; i < count; ++i) {
+          volatile float ws = c->sc_wsum + c->sc_w, wn = c->sc_w * pa.theta;
+          c->sc_wsum = ws; c->sc_w = wn;
+        }
+      }
       c->persist_launches += 1;
       c->ll_tag += (uint32_t)count;
     } else {

@@ -59,6 +59,9 @@ struct PersistArgs {
   // snapshot, vhat (d floats) receives the last step's second estimator, x_out the last coupled point
   int alpc;
   float tau1, tau2, alpha, inv4L;
+  // strongly convex case (h with a (sigma/2)*||.||^2 term): factors on the two soft-threshold results, the snapshot
+  // weight of the launch's first step and its growth per step; all 1 in the general convex case
+  float cy, cz, w0, theta;
   float* y;
   float* z;
   float* ysum;

@@ -265,6 +265,7 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
   constexpr int LLCH = (BITS == 0) ? 4 : 16;
   const int wpg = (BITS == 0) ? pa.wpg : WMAX;
   const size_t groups = (size_t)(CS * SL) >> 3;
+  float wcur = pa.w0;  // snapshot weight of the step whose update comes next
   auto apply_update = [&](unsigned int target) {
     const int rpar = (pa.count - (int)target) & 1;  // parity half that holds step target-1
     const uint32_t tag = pa.tag_base + target;
@@ -355,9 +356,9 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
           const float v = add_rn(mul_rn(acc[e], invN), mur[p][e]);
           if constexpr (ALPC) {  // steps 12-13 of Algorithm 2
             const float vh = __uint_as_float((uint32_t)vw[e]);
-            yr[p][e] = soft_threshold(__fsub_rn(xr[p][e], mul_rn(pa.inv4L, v)), kappa_y);
-            zr[p][e] = soft_threshold(__fsub_rn(zr[p][e], mul_rn(pa.alpha, vh)), kappa_z);
-            sr[p][e] = add_rn(sr[p][e], yr[p][e]);
+            yr[p][e] = mul_rn(soft_threshold(__fsub_rn(xr[p][e], mul_rn(pa.inv4L, v)), kappa_y), pa.cy);
+            zr[p][e] = mul_rn(soft_threshold(__fsub_rn(zr[p][e], mul_rn(pa.alpha, vh)), kappa_z), pa.cz);
+            sr[p][e] = add_rn(sr[p][e], mul_rn(wcur, yr[p][e]));
           } else {
             xr[p][e] = soft_threshold(__fsub_rn(xr[p][e], mul_rn(pa.eta, v)), kappa);
           }
@@ -365,6 +366,7 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
         }
       }
     }
+    if constexpr (ALPC) wcur = mul_rn(wcur, pa.theta);  // the next step's snapshot weight (Algorithm 2's last step)
   };
 
 #pragma unroll 1

@@ -79,7 +79,7 @@ def test_epochs_follow_algorithm2_with_the_theorem_parameters():
         ctx.snapshot_full_grad()
         mu = ctx.get_buffer(lpc.BUF_MU).cpu().numpy()
         ctx.alpc_double_sample_steps(float(tau1), 0.5, float(alpha), float(inv4L), s * m, m)
-        assert ctx.query(lpc.INFO_LOOP_LAUNCHES) == 0  # weighted steps do not take the one-launch loop
+        assert ctx.query(lpc.INFO_LOOP_LAUNCHES) == s + 1  # the weighted steps of an epoch run as one launch
         ctx.alpc_end_epoch(m)
         ysum, w, wsum = np.zeros(P.d, np.float32), np.float32(1.0), np.float32(0.0)
         for t in range(m):
@@ -94,6 +94,34 @@ def test_epochs_follow_algorithm2_with_the_theorem_parameters():
     ref = orc.objective(P.X, P.y, P.loss, snap, P.lambda_l1) + orc.ridge_term(snap, sigma)
     assert pe == pytest.approx(ref, rel=1e-9)
     ctx.close()
+
+
+@pytest.mark.parametrize("loss", ["least_squares", "logistic"])
+def test_one_launch_loop_equals_single_steps_with_weights(loss):
+    P, ctx = _setup(512, 1024, loss, N=4, B=4, b=4)
+    ref = lpc.Context(ctx.X, ctx.y, P.loss, P.lambda_l1, P.N, P.B, P.b, P.clip_mode, P.clip_value, P.seed)
+    x0 = (np.random.default_rng(5).standard_normal(P.d) * 0.1).astype(np.float32)
+    tau1, tau2, alpha, inv4L, count = 0.4, 0.5, 0.3, 0.2, 11
+    for cx in (ctx, ref):
+        cx.set_strong_convexity(0.35)
+        cx.set_iterate(torch.from_numpy(x0).to(DEV))
+        cx.alpc_begin()
+        cx.snapshot_full_grad()
+        cx.alpc_double_sample_step(tau1, tau2, alpha, inv4L, 0)  # the loop then starts from the second weight
+    ctx.alpc_double_sample_steps(tau1, tau2, alpha, inv4L, 1, count)
+    for k in range(1, 1 + count):
+        ref.alpc_double_sample_step(tau1, tau2, alpha, inv4L, k)
+    for cx in (ctx, ref):
+        cx.sync_status()
+    assert ctx.query(lpc.INFO_LOOP_LAUNCHES) == 1 and ref.query(lpc.INFO_LOOP_LAUNCHES) == 0
+    for w in (lpc.BUF_X, lpc.BUF_Y, lpc.BUF_Z, lpc.BUF_YSUM):
+        assert _same(ctx.get_buffer(w), ref.get_buffer(w)), w
+    for cx in (ctx, ref):
+        cx.alpc_end_epoch(count + 1)
+        cx.sync_status()
+    assert _same(ctx.get_iterate(), ref.get_iterate())  # same sum of weights on both paths
+    ctx.close()
+    ref.close()
 
 
 def test_sigma_zero_is_the_general_convex_path_and_bad_values_are_rejected():
