@@ -77,7 +77,8 @@ __device__ __forceinline__ uint32_t extract(uint64_t lo, uint64_t hi, int pos, i
 
 template <int BITS>  // 1, 2, 4, 8: fixed width; 0: b in 1..16 from the arguments; 32: floats
 __global__ void __launch_bounds__(AT) unpack_average_prox_kernel(AggArgs a) {
-  const int tile = blockIdx.x;
+  // a.split CTAs share a tile (each takes AITER / split of its sweeps): short vectors still fill the machine
+  const int tile = blockIdx.x / a.split, part = blockIdx.x % a.split;
   const int seg = a.tile_seg ? a.tile_seg[tile] : 0;
   const SegInfo s = a.segs[seg];
   const int64_t tstart = (int64_t)(tile - s.tile_first) * TILE;
@@ -97,7 +98,7 @@ __global__ void __launch_bounds__(AT) unpack_average_prox_kernel(AggArgs a) {
                                     aligned16(a.vhat + s.off)));
 
 #pragma unroll 1
-  for (int it = 0; it < AITER; ++it) {
+  for (int it = part * (AITER / a.split); it < (part + 1) * (AITER / a.split); ++it) {
     const int64_t j = tstart + (int64_t)it * AGROUP + tid * 8;
     if (j >= s.len) break;
     float acc[8];
@@ -521,9 +522,11 @@ cudaError_t launch_server_reduce(const ServerArgs& a, cudaStream_t st) {
   return cudaGetLastError();
 }
 
-cudaError_t launch_unpack_average_prox(const AggArgs& a, cudaStream_t st) {
-  if (a.ntiles <= 0) return cudaSuccess;
-  const dim3 grid((unsigned)a.ntiles), block(AT);
+cudaError_t launch_unpack_average_prox(const AggArgs& a_in, cudaStream_t st) {
+  if (a_in.ntiles <= 0) return cudaSuccess;
+  AggArgs a = a_in;
+  a.split = (a.ntiles >= 4096) ? 1 : (a.ntiles >= 2048) ? 2 : AITER;  // aim at several waves of CTAs
+  const dim3 grid((unsigned)(a.ntiles * a.split)), block(AT);
   const size_t sh = (size_t)a.N * sizeof(float);
   switch (a.b) {
     case 1: unpack_average_prox_kernel<1><<<grid, block, sh, st>>>(a); break;

@@ -88,6 +88,7 @@ struct AggArgs {
   // multiplied by cy = 1/(1 + sigma*inv4L) and cz = 1/(1 + alpha*sigma), and ysum += wy * y (the snapshot weight
   // (1 + alpha*sigma)^t of the step).  All three are 1 in the general convex case, where they change no bit.
   float cy, cz, wy;
+  int split;  // CTAs per tile (1, 2 or 4), set by the launcher
 };
 
 cudaError_t launch_unpack_average_prox(const AggArgs& a, cudaStream_t st);
