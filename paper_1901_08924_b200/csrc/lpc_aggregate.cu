@@ -525,7 +525,7 @@ cudaError_t launch_server_reduce(const ServerArgs& a, cudaStream_t st) {
 cudaError_t launch_unpack_average_prox(const AggArgs& a_in, cudaStream_t st) {
   if (a_in.ntiles <= 0) return cudaSuccess;
   AggArgs a = a_in;
-  a.split = (a.ntiles >= 4096) ? 1 : (a.ntiles >= 2048) ? 2 : AITER;  // aim at several waves of CTAs
+  a.split = (a.ntiles >= 1184) ? 1 : (a.ntiles >= 592) ? 2 : AITER;  // below two waves of CTAs (148 SMs x 4) a tile is shared
   const dim3 grid((unsigned)(a.ntiles * a.split)), block(AT);
   const size_t sh = (size_t)a.N * sizeof(float);
   switch (a.b) {
