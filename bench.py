@@ -312,6 +312,24 @@ def quantize_aggregate_bench(dev, peak, log2_len=26, dnn=True):
                           "note": "two passes: 4 B stats read + 4 B quantize read + b/8 B written per element"},
         "unpack_average_prox": {"ms": round(ta, 4), "bytes": ba, "gbs": round(ba / ta * 1e-6, 1), "frac": round(ba / ta * 1e-6 / peak, 4)},
         "combined_gbs": round((bq + ba) / (tq + ta) * 1e-6, 1)}
+    # the other code widths and vector lengths of the sweep (same vectors, prefixes for the shorter lengths)
+    grid = {}
+    for bb, ll in [(1, log2_len), (2, log2_len), (8, log2_len)] + [(4, l2) for l2 in (16, 20, 24) if l2 < log2_len]:
+        ln = 1 << ll
+        qq = lpc.Context(None, None, lpc.LOGISTIC, 0.0, N, 1, bb, lpc.CLIP_STD, 2.0, 0)
+        _, st2 = lpc.packed_layout(ln, bb)
+        c2 = torch.empty((N, st2), dtype=torch.int32, device=dev)
+        Uv = U[:, :ln]
+        x2 = torch.zeros(ln, device=dev)
+        t1 = _time_calls(lambda: qq.quantize_pack(Uv, 1, codes_out=c2, delta_out=delta, clipped_out=clipped), dev, 5)
+        t2 = _time_calls(lambda: qq.unpack_average_prox(c2, delta, ln, x2, 1.0, 1e-3), dev, 10)
+        qq.sync_status()
+        qq.close()
+        b1, b2 = N * ln * (8 + bb / 8), ln * (N * bb / 8 + 12)
+        grid["b%d_len2^%d" % (bb, ll)] = {"quantize_pack_ms": round(t1, 4), "quantize_pack_frac": round(b1 / t1 * 1e-6 / peak, 4),
+                                          "unpack_average_prox_ms": round(t2, 4), "unpack_average_prox_frac": round(b2 / t2 * 1e-6 / peak, 4)}
+        del c2, x2
+    res["sweep_grid_N8"] = grid
     # entropy-coding count of the messages just packed: histogram kernel (event-timed) and the host sums
     hist = torch.empty((N, 1, 1 << b), dtype=torch.int64, device=dev)
     q.set_option(lpc.OPT_PROFILE, 1)
