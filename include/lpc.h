@@ -83,7 +83,7 @@ typedef struct lpc_ctx lpc_ctx;
 #define LPC_OPT_PROFILE 4       /* 1: record CUDA events around every kernel launch (graph replay is off meanwhile) */
 
 #define LPC_OPT_SHARED_SCALE 6  /* 1: lpc_quantize_pack gives every worker the unified scale delta_t = max_i delta_t^i of the parameter-server schemes (b), (c) of Section 3.2; needs b in 2..16 */
-#define LPC_OPT_AVERAGE_DIVISOR 7 /* lpc_unpack_average_prox divides the decoded sum by this count instead of the context's N (0 = N): the worker count behind a server's sum stream */
+#define LPC_OPT_AVERAGE_DIVISOR 7 /* lpc_unpack_average_prox (and only it: the training loops always average over N) divides the decoded sum by this count instead of the context's N (0 = N): the worker count behind a server's sum stream */
 #define LPC_OPT_PERSISTENT 5    /* 1 (default): lpc_inner_steps runs the whole loop in one cooperative launch when it fits */
 
 /* kernel classes reported by lpc_get_profile */
@@ -283,6 +283,10 @@ int lpc_objective(lpc_ctx* ctx, const float* x, double* P_out);
 #define LPC_INFO_LOOP_ROW_BUFFERS 6        /* sampled-row buffers per CTA of the one-launch loop (1 or 2; 0: not available) */
 #define LPC_INFO_ALPC_LOOP_ROW_BUFFERS 7   /* the same for the loop of Algorithm 2 */
 #define LPC_INFO_STEP_RING_STAGES 8        /* per-step kernel: 0 = minibatch rows resident on chip, else ring stages they stream through */
+#define LPC_INFO_AGGREGATE_SPLIT 9         /* last lpc_unpack_average_prox: CTAs that shared one tile of 8192 coordinates (1, 2 or 4) */
+#define LPC_INFO_QUANT_PIPELINED_RUNS 10   /* last lpc_quantize_pack: runs of 8 tiles per worker that were whole tiles of one segment of
+                                              16-byte aligned vectors and so took the second pass's software-pipelined loop (unless
+                                              that worker's scale was degenerate) */
 int lpc_query(const lpc_ctx* ctx, int what, int64_t* out);
 
 /* Per-kernel device time measured with CUDA events on the context's stream while LPC_OPT_PROFILE is
@@ -316,7 +320,8 @@ int lpc_svrg_run_host(const float* X_host, const float* y_host, int64_t n, int32
  *   U            N x len fp32, row stride ld (device)
  *   codes_out    N * stride_words words, stride_words from lpc_packed_layout(len, b, NULL, 1) (device,
  *                16-byte aligned);  delta_out N floats;  clipped_out N counts (all required)
- *   stream       cudaStream_t
+ *   stream       cudaStream_t of the device that is current when the call is made (the working memory is looked up
+ *                on the current device; with a stream of another device the launches fail with LPC_ERR_CUDA)
  * Limits: N <= LPC_STATIC_MAX_WORKERS and N * ceil(len / 8192) <= LPC_STATIC_MAX_TILES; anything larger
  * returns LPC_ERR_UNSUPPORTED and launches nothing.  Non-finite input yields a NaN delta.
  * The first call on a device looks up the array's device address; make that first call outside any
@@ -329,6 +334,17 @@ int lpc_svrg_run_host(const float* X_host, const float* y_host, int64_t n, int32
 int lpc_quantize_pack_static(const float* U, int64_t len, int64_t ld, int32_t N, int32_t b, int clip_mode,
                              float clip_value, uint64_t seed, uint64_t k, uint32_t* codes_out, float* delta_out,
                              uint32_t* clipped_out, void* stream);
+
+/*
+ * Inspection aid for the error path of the bounded device-side waits (every wait of the library on a bulk copy, on
+ * another CTA's message or on another worker's codes gives up after about two seconds, records the fact and lets the
+ * kernel finish; the next lpc_sync_status then returns LPC_ERR_TIMEOUT).  This call enqueues one tiny kernel whose
+ * waits of both kinds -- an mbarrier phase that nothing completes and, on a context with a linear model, a tagged
+ * word that nobody writes -- run out after limit_ns (1 us .. 100 ms) through the same code.  Nothing else is in
+ * flight, so the kernel ends normally and the context stays usable: lpc_sync_status returns LPC_ERR_TIMEOUT once,
+ * then LPC_OK.  The paper has no counterpart.
+ */
+int lpc_debug_wait_timeout(lpc_ctx* ctx, uint64_t limit_ns);
 
 /*
  * Inspection aid: writes `count` consecutive 4-word blocks, starting at block `block0`, of the

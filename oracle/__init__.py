@@ -486,3 +486,34 @@ def alpc_step(P, k, tau1, tau2, alpha, inv4L, xs, mu, y, z, ysum, taps=False, si
         t["words"] = t["words"][:, : P.W]
         return yn, zn, sn, t
     return yn, zn, sn
+
+
+def alpc3_epoch_params(s, L):
+    """Algorithm 3 step 3: (tau_1, alpha) of epoch s for smoothness L, as fp32 values."""
+    t, a = C.c_float(0), C.c_float(0)
+    lib().orc_alpc3_epoch_params(C.c_int64(s), C.c_double(L), C.byref(t), C.byref(a))
+    return np.float32(t.value), np.float32(a.value)
+
+
+def alpc3_mean_snapshot(ysum, m):
+    """Algorithm 3 step 5 from the running sum of the epoch's y iterates."""
+    ysum, p = _f32(ysum)
+    out = np.zeros_like(ysum)
+    lib().orc_alpc3_mean_snapshot(p, C.c_int64(m), ysum.size, out.ctypes.data_as(_f32p))
+    return out
+
+
+def alpc3_epoch(P, s, m, L, tau2, xs, mu, y, z):
+    """One epoch of Algorithm 3 after its full-gradient step.  Returns (y, z, next snapshot)."""
+    xs, pxs = _f32(xs)
+    mu, pmu = _f32(mu)
+    yn = np.array(y, dtype=np.float32, copy=True)
+    zn = np.array(z, dtype=np.float32, copy=True)
+    nxt = np.zeros(P.d, dtype=np.float32)
+    rc = lib().orc_alpc3_epoch(P.X.ctypes.data_as(_f32p), P.y.ctypes.data_as(_f32p), C.c_int64(P.n), C.c_int64(P.d),
+                               P.loss, C.c_float(P.lambda_l1), P.N, P.B, P.b, P.clip_mode, C.c_float(P.clip_value),
+                               C.c_uint64(P.seed), int(P.partition_local), C.c_int64(s), C.c_int64(m), C.c_double(L),
+                               C.c_float(tau2), pxs, pmu, yn.ctypes.data_as(_f32p), zn.ctypes.data_as(_f32p),
+                               nxt.ctypes.data_as(_f32p))
+    _check(rc)
+    return yn, zn, nxt

@@ -757,6 +757,41 @@ void orc_weighted_snapshot(const float* ysum, float wsum, int64_t d, float* xs_o
   for (int64_t j = 0; j < d; ++j) xs_out[j] = ysum[j] * inv;
 }
 
+// Algorithm 3 (general convex case), its outer rule.  Epoch s runs Algorithm 2's steps 3-14 with
+//   tau_{1,s} = 2/(s+4),   alpha_s = 1/(6 L tau_{1,s})      (step 3; evaluated in fp64, rounded to fp32 once each)
+// and tau_2 as given; its snapshot is the plain mean of the epoch's m iterates y (step 5), taken as the running
+// fp32 sum of the y's in step order times the fp32 reciprocal of m.  y and z carry over from epoch to epoch.
+void orc_alpc3_epoch_params(int64_t s, double L, float* tau1_out, float* alpha_out) {
+  const double tau1 = 2.0 / (double)(s + 4);
+  *tau1_out = (float)tau1;
+  *alpha_out = (float)(1.0 / (6.0 * L * tau1));
+}
+
+void orc_alpc3_mean_snapshot(const float* ysum, int64_t m, int64_t d, float* xs_out) {
+  const float inv_m = 1.0f / (float)m;
+  for (int64_t j = 0; j < d; ++j) xs_out[j] = ysum[j] * inv_m;
+}
+
+// One epoch of Algorithm 3 after communication step 1 (mu = grad f(xs) is given): m steps k = s*m .. s*m + m - 1 with
+// the epoch's parameters, then the mean snapshot.  inv4L = 1/(4L) rounded to fp32.
+int orc_alpc3_epoch(const float* X, const float* y, int64_t n, int64_t d, int loss, float lambda_l1, int N, int B,
+                    int b, int clip_mode, float clip_value, uint64_t seed, int partition_local, int64_t s, int64_t m,
+                    double L, float tau2, const float* xs, const float* mu, float* y_inout, float* z_inout,
+                    float* xs_next_out) {
+  float tau1, alpha;
+  orc_alpc3_epoch_params(s, L, &tau1, &alpha);
+  const float inv4L = (float)(1.0 / (4.0 * L));
+  std::vector<float> ysum((size_t)d, 0.0f);
+  for (int64_t t = 0; t < m; ++t) {
+    const int rc = orc_alpc_step(X, y, n, d, loss, lambda_l1, N, B, b, clip_mode, clip_value, seed, partition_local,
+                                 (uint64_t)(s * m + t), tau1, tau2, alpha, inv4L, xs, mu, y_inout, z_inout,
+                                 ysum.data(), nullptr, nullptr, nullptr, nullptr, 0, nullptr);
+    if (rc != ORC_OK) return rc;
+  }
+  orc_alpc3_mean_snapshot(ysum.data(), m, d, xs_next_out);
+  return ORC_OK;
+}
+
 // P(x) with the elastic-net regulariser: the objective of Eq. 1 plus (sigma/2)*||x||^2 (fp64 sum).
 double orc_ridge_term(const float* x, int64_t d, float sigma) {
   double s2 = 0.0;

@@ -522,10 +522,14 @@ cudaError_t launch_server_reduce(const ServerArgs& a, cudaStream_t st) {
   return cudaGetLastError();
 }
 
-cudaError_t launch_unpack_average_prox(const AggArgs& a_in, cudaStream_t st) {
-  if (a_in.ntiles <= 0) return cudaSuccess;
-  AggArgs a = a_in;
-  a.split = (a.ntiles >= 1184) ? 1 : (a.ntiles >= 592) ? 2 : AITER;  // below two waves of CTAs (148 SMs x 4) a tile is shared
+int aggregate_split(int ntiles, int sm_count) {
+  const int wave = 4 * (sm_count > 0 ? sm_count : 148);  // resident CTAs of this kernel
+  return (ntiles >= 2 * wave) ? 1 : (ntiles >= wave) ? 2 : AITER;
+}
+
+cudaError_t launch_unpack_average_prox(const AggArgs& a, cudaStream_t st) {
+  if (a.ntiles <= 0) return cudaSuccess;
+  if (!(a.split == 1 || a.split == 2 || a.split == AITER)) return cudaErrorInvalidValue;
   const dim3 grid((unsigned)(a.ntiles * a.split)), block(AT);
   const size_t sh = (size_t)a.N * sizeof(float);
   switch (a.b) {

@@ -103,6 +103,8 @@ struct lpc_ctx {
   float sc_w = 1.f;      // snapshot weight of the next ALPC step, (1 + alpha*sigma)^t in fp32
   float sc_wsum = 0.f;   // sum of the weights used so far in this epoch
   int divisor = 0;       // LPC_OPT_AVERAGE_DIVISOR; 0: the worker count N
+  int last_split = 0;    // CTAs per tile of the last lpc_unpack_average_prox launch
+  int64_t last_pipelined_runs = 0;  // runs of whole tiles per worker in the last lpc_quantize_pack launch
   uint32_t* q_pmax = nullptr;
   float *q_ps1 = nullptr, *q_ps2 = nullptr;
   size_t q_part_cap = 0;
@@ -308,11 +310,13 @@ InnerArgs inner_args(lpc_ctx* c, uint64_t k_base, const uint64_t* k_dev, int has
   return a;
 }
 
+// divisor: the count the decoded sum is divided by (Eq. 3: the worker count N).
 AggArgs agg_args(lpc_ctx* c, const SegPlan& p, const uint32_t* codes, const float* delta, const float* mu, float* x,
-                 float eta, float lambda_l1, float* v_out) {
+                 float eta, float lambda_l1, float* v_out, int divisor) {
   AggArgs a;
   a.codes = codes; a.stride_words = p.stride_words; a.delta = delta; a.N = c->N; a.b = c->b;
-  a.divisor = c->divisor > 0 ? c->divisor : c->N;
+  a.divisor = divisor;
+  a.split = aggregate_split(p.ntiles, c->sm_count);
   a.segs = p.d_segs; a.tile_seg = p.d_tile_seg; a.nseg = p.nseg; a.ntiles = p.ntiles;
   a.mu = mu; a.x = x; a.eta = eta; a.lambda_l1 = lambda_l1; a.v_out = v_out; a.k_counter = nullptr;
   a.mode = 0; a.y = nullptr; a.z = nullptr; a.ysum = nullptr; a.vhat = nullptr; a.alpha = 0.f; a.inv4L = 0.f;
@@ -338,7 +342,8 @@ int replan_inner(lpc_ctx* c) {
 int enqueue_lpc_step(lpc_ctx* c, float eta, uint64_t k_base, const uint64_t* k_dev, uint64_t* k_counter) {
   InnerArgs ia = inner_args(c, k_base, k_dev, 0);
   { ProfScope ps_(c, LPC_KERNEL_WORKER); CU(c, launch_inner(ia, c->innerSmem, c->stream)); }
-  AggArgs ag = agg_args(c, c->inner_seg, c->codes, c->delta, c->mu, c->x, eta, c->lambda_l1, c->tap_u ? c->v_tap : nullptr);
+  // the training loops always average over the context's N workers (Eq. 3); LPC_OPT_AVERAGE_DIVISOR does not apply
+  AggArgs ag = agg_args(c, c->inner_seg, c->codes, c->delta, c->mu, c->x, eta, c->lambda_l1, c->tap_u ? c->v_tap : nullptr, c->N);
   ag.k_counter = k_counter;
   { ProfScope ps_(c, LPC_KERNEL_AGGREGATE); CU(c, launch_unpack_average_prox(ag, c->stream)); }
   return LPC_OK;
@@ -350,7 +355,7 @@ int enqueue_alpc_step(lpc_ctx* c, float tau1, float tau2, float alpha, float inv
   { ProfScope ps_(c, LPC_KERNEL_OTHER); CU(c, launch_coupling(c->zv, c->xt, c->yv, tau1, tau2, c->d, c->x, c->stream)); }
   InnerArgs ia = inner_args(c, k_base, k_dev, 1);
   { ProfScope ps_(c, LPC_KERNEL_WORKER); CU(c, launch_inner(ia, c->innerSmem, c->stream)); }
-  AggArgs ag = agg_args(c, c->inner_seg, c->codes, c->delta, c->mu, c->x, 0.f, c->lambda_l1, c->tap_u ? c->v_tap : nullptr);
+  AggArgs ag = agg_args(c, c->inner_seg, c->codes, c->delta, c->mu, c->x, 0.f, c->lambda_l1, c->tap_u ? c->v_tap : nullptr, c->N);
   ag.k_counter = k_counter;
   ag.mode = 1; ag.y = c->yv; ag.z = c->zv; ag.ysum = c->ysum; ag.vhat = c->vhat; ag.alpha = alpha; ag.inv4L = inv4L;
   if (c->sigma > 0.f) {  // each product and sum below is one fp32 operation, as on the device
@@ -788,6 +793,8 @@ int lpc_query(const lpc_ctx* c, int what, int64_t* out) {
     case LPC_INFO_LOOP_LAUNCHES: *out = c->persist_launches; return LPC_OK;
     case LPC_INFO_SNAPSHOT_ROWS_PER_TILE: *out = c->snapR; return LPC_OK;
     case LPC_INFO_SNAPSHOT_STAGES: *out = c->snapStages; return LPC_OK;
+    case LPC_INFO_AGGREGATE_SPLIT: *out = c->last_split; return LPC_OK;
+    case LPC_INFO_QUANT_PIPELINED_RUNS: *out = c->last_pipelined_runs; return LPC_OK;
     default: return LPC_ERR_INVALID_ARG;
   }
 }
@@ -840,6 +847,18 @@ int lpc_quantize_pack(lpc_ctx* c, const float* U, const float* U_sub, int64_t le
   a.codes = codes_out; a.stride_words = p.stride_words; a.delta_out = delta_out;
   a.clipped_out = clipped_out ? clipped_out : c->q_clip; a.count_clipped = clipped_out ? 1 : 0; a.dev_status = c->dev_status;
   a.shared_scale = c->shared_scale;
+  {  // runs of the second pass that consist of whole tiles of one segment of 16-byte aligned vectors (per worker)
+    const int run = quantize_run_tiles();
+    const bool vec = aligned16(U) && (!U_sub || aligned16(U_sub)) && (ld % 4 == 0);
+    int64_t runs = 0;
+    const bool fixed_width = (c->b == 1 || c->b == 2 || c->b == 4 || c->b == 8);  // the other widths go tile by tile
+    for (int t0 = 0; vec && fixed_width && t0 < p.ntiles; t0 += run) {
+      const int t1 = std::min(t0 + run, p.ntiles) - 1;
+      const SegInfo& g = p.segs[p.tile_seg[t0]];
+      if (p.tile_seg[t0] == p.tile_seg[t1] && g.off % 4 == 0 && (int64_t)(t1 + 1 - g.tile_first) * TILE <= g.len) ++runs;
+    }
+    c->last_pipelined_runs = runs;
+  }
   CU(c, launch_quantize_pack(a, c->stream, c->profile ? prof_hook : nullptr, c));
   if (!c->shared_scale) c->step2_bits += p.msg_bits * (uint64_t)c->N * (uint64_t)(c->N - 1);  // scheme (a); the server schemes count in lpc_server_reduce
   return LPC_OK;
@@ -955,8 +974,18 @@ int lpc_unpack_average_prox(lpc_ctx* c, const uint32_t* codes, const float* delt
   if (len < 0 || nseg < 1) return fail(c, LPC_ERR_INVALID_ARG, "len / nseg");
   if (!aligned16(codes)) return fail(c, LPC_ERR_INVALID_ARG, "codes must be 16-byte aligned");
   TRY(make_plan(c, c->seg, len, c->b, seg_offsets, nseg));
-  AggArgs a = agg_args(c, c->seg, codes, delta, mu, x_inout, eta, lambda_l1, v_out);
+  AggArgs a = agg_args(c, c->seg, codes, delta, mu, x_inout, eta, lambda_l1, v_out, c->divisor > 0 ? c->divisor : c->N);
+  c->last_split = a.split;
   { ProfScope ps_(c, LPC_KERNEL_AGGREGATE); CU(c, launch_unpack_average_prox(a, c->stream)); }
+  return LPC_OK;
+}
+
+int lpc_debug_wait_timeout(lpc_ctx* c, uint64_t limit_ns) {
+  if (!c) return LPC_ERR_INVALID_ARG;
+  if (limit_ns < 1000ull || limit_ns > 100000000ull) return fail(c, LPC_ERR_INVALID_ARG, "limit must be 1 us .. 100 ms");
+  unsigned int* abort_flag = c->flags ? reinterpret_cast<unsigned int*>(c->flags + 512 * 16) : nullptr;
+  if (abort_flag) CU(c, cudaMemsetAsync(abort_flag, 0, sizeof(unsigned long long), c->stream));
+  CU(c, launch_wait_timeout(c->flags, abort_flag, c->dev_status, limit_ns, c->stream));
   return LPC_OK;
 }
 

@@ -396,6 +396,26 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint64
     }
   }
 }
+// Bounded spin on data that another CTA writes (tagged words): call once per unsuccessful look, `it` counting the looks
+// and t0 starting at 0.  Returns true when the caller must stop looking: another thread raised `abort_flag`, or no
+// progress for limit_ns, in which case this thread records DEV_TIMEOUT in `dev_status` and raises the flag itself, so
+// that every other spin of the grid ends at its next look.
+__device__ __forceinline__ bool spin_expired(uint32_t it, uint64_t& t0, unsigned int* abort_flag, unsigned int* dev_status,
+                                             uint64_t limit_ns = 2000000000ull) {
+  if ((it & 63u) != 63u) return false;
+  unsigned int raised;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(raised) : "l"(abort_flag) : "memory");
+  if (raised != 0u) return true;
+  const uint64_t now = global_ns();
+  if (t0 == 0) {
+    t0 = now;
+    return false;
+  }
+  if (now - t0 <= limit_ns) return false;
+  atomicOr(dev_status, DEV_TIMEOUT);
+  asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(abort_flag), "r"(1u) : "memory");
+  return true;
+}
 // Same bounded wait with acquire semantics at cluster scope: for phases completed by stores of other CTAs of the
 // cluster (st_async_cluster below).
 __device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity, uint64_t limit_ns = 2000000000ull) {

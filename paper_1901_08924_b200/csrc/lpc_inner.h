@@ -71,6 +71,9 @@ struct PersistArgs {
 bool persist_plan(int d, int N, int B, int b, int alpc, int want_cs, int max_smem, int* CS_out, int* SL_out,
                   size_t* smem_out, int* nbuf_out);
 cudaError_t launch_persist(const PersistArgs& pa, size_t smem, cudaStream_t st);
+// One small kernel whose bounded waits (an mbarrier phase; a tagged word when `word` is given) run out after limit_ns.
+cudaError_t launch_wait_timeout(const unsigned long long* word, unsigned int* abort_flag, unsigned int* dev_status,
+                                uint64_t limit_ns, cudaStream_t st);
 
 int inner_max_b();
 int inner_clipped_stride();

@@ -55,6 +55,9 @@ struct QuantArgs {
 
 // hook(user, kind, begin) is called around each kernel of the sequence (kind = LPC_KERNEL_* of lpc.h) when non-null.
 typedef void (*LaunchHook)(void* user, int kind, int begin);
+// Tiles per CTA of the second pass, and whether the run of tiles that starts at tile0 consists of whole tiles of one
+// segment (the condition, besides 16-byte aligned vectors and a non-degenerate scale, for its pipelined loop).
+int quantize_run_tiles();
 cudaError_t launch_quantize_pack(const QuantArgs& a, cudaStream_t st, LaunchHook hook = nullptr, void* user = nullptr);
 
 struct AggArgs {
@@ -88,9 +91,12 @@ struct AggArgs {
   // multiplied by cy = 1/(1 + sigma*inv4L) and cz = 1/(1 + alpha*sigma), and ysum += wy * y (the snapshot weight
   // (1 + alpha*sigma)^t of the step).  All three are 1 in the general convex case, where they change no bit.
   float cy, cz, wy;
-  int split;  // CTAs per tile (1, 2 or 4), set by the launcher
+  int split;  // CTAs per tile (1, 2 or 4): aggregate_split(ntiles, sm_count), set by the caller
 };
 
+// CTAs that share one tile of the aggregator: below two waves of resident CTAs (4 per SM) a tile's sweeps are spread
+// over 2 or 4 CTAs so that short vectors still fill the machine.
+int aggregate_split(int ntiles, int sm_count);
 cudaError_t launch_unpack_average_prox(const AggArgs& a, cudaStream_t st);
 
 // The server of the parameter-server schemes (Section 3.2): N code streams of b bits on one grid in, one stream out.

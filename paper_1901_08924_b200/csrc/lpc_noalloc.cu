@@ -20,7 +20,8 @@ using namespace lpc;
 
 // Layout of the fixed working memory (bytes from the start of the array):
 //   [0, 64)                      one SegInfo (the vector as a single segment)
-//   [64, 128)                    status word
+//   [64, 128)                    status word: the kernels need a place to flag non-finite input; nothing reads it back
+//                                (there is no context to report through), the caller's signal is the NaN delta
 //   [256, 256 + 32*MAX_N)        ScaleRec per worker
 //   then three arrays of MAX_PARTS 32-bit entries: tile maxima, tile sums, tile sums of squares
 constexpr int MAX_N = LPC_STATIC_MAX_WORKERS;

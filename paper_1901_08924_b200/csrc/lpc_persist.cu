@@ -90,14 +90,6 @@ __device__ __forceinline__ unsigned long long ld_shared_word(const unsigned long
   asm volatile("ld.relaxed.cluster.shared::cta.u64 %0, [%1];" : "=l"(v) : "r"(smem_u32(slot)) : "memory");
   return v;
 }
-__device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int* p) {
-  unsigned int v;
-  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-  return v;
-}
-__device__ __forceinline__ void st_release_u32(unsigned int* p, unsigned int v) {
-  asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
-}
 
 __device__ __forceinline__ uint32_t extract_bits(uint64_t lo, uint64_t hi, int pos, int b) {
   uint64_t v;
@@ -243,19 +235,7 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
 
   // Every spin in this kernel ends: after about two seconds without progress the thread records a timeout and
   // raises the abort flag, which ends all other spins at their next look at it.
-  auto wait_expired = [&](uint32_t it, uint64_t& t0) -> bool {
-    if ((it & 63u) != 63u) return false;
-    if (ld_acquire_u32(pa.abort_flag) != 0u) return true;
-    const uint64_t now = global_ns();
-    if (t0 == 0) {
-      t0 = now;
-      return false;
-    }
-    if (now - t0 <= 2000000000ull) return false;
-    atomicOr(a.dev_status, DEV_TIMEOUT);
-    st_release_u32(pa.abort_flag, 1u);
-    return true;
-  };
+  auto wait_expired = [&](uint32_t it, uint64_t& t0) -> bool { return spin_expired(it, t0, pa.abort_flag, a.dev_status); };
 
   // Applies step target-1's update to this thread's coordinates:
   //   x <- prox_{eta h}(x - eta (mean_i delta_i k_i + mu))      (Algorithm 2: the y and z updates).
@@ -834,6 +814,33 @@ bool persist_plan(int d, int N, int B, int b, int alpc, int want_cs, int max_sme
     if (SL <= 512) break;  // slices below 512 coordinates leave most of a CTA idle
   }
   return found;
+}
+
+namespace {
+// Exercises the two kinds of bounded wait of the library on things that never happen: thread 0 waits on an mbarrier
+// that nobody arrives at and no copy counts on, thread 32 polls a tagged word for a tag that is never handed out.
+// Both give up after limit_ns, record DEV_TIMEOUT and return; nothing is in flight, so the kernel simply ends.
+__global__ void __launch_bounds__(64) wait_timeout_kernel(const unsigned long long* word, unsigned int* abort_flag,
+                                                          unsigned int* dev_status, uint64_t limit_ns) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    mbar_fence_init();
+    if (!mbar_wait(&bar, 0, limit_ns)) atomicOr(dev_status, DEV_TIMEOUT);
+  } else if (threadIdx.x == 32 && word != nullptr) {
+    uint64_t t0 = 0;
+    for (uint32_t it = 0;; ++it) {
+      if (word_tag(ld_word(word)) == 0xFFFFFFFFu) break;  // tags stop short of this value
+      if (spin_expired(it, t0, abort_flag, dev_status, limit_ns)) break;
+    }
+  }
+}
+}  // namespace
+
+cudaError_t launch_wait_timeout(const unsigned long long* word, unsigned int* abort_flag, unsigned int* dev_status,
+                                uint64_t limit_ns, cudaStream_t st) {
+  wait_timeout_kernel<<<1, 64, 0, st>>>(word, abort_flag, dev_status, limit_ns);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_persist(const PersistArgs& pa, size_t smem, cudaStream_t st) {

@@ -429,6 +429,8 @@ __global__ void __launch_bounds__(QT) bypass_kernel(QuantArgs a) {
 
 }  // namespace
 
+int quantize_run_tiles() { return QRUN; }
+
 cudaError_t launch_quantize_pack(const QuantArgs& a, cudaStream_t st, LaunchHook hook, void* user) {
   if (a.N <= 0 || a.nseg <= 0) return cudaSuccess;
   const dim3 grid((unsigned)(a.ntiles > 0 ? a.ntiles : 1), (unsigned)a.N), block(QT);

@@ -21,7 +21,8 @@ OPT_SAMPLE_GLOBAL, OPT_TAP_U, OPT_CLUSTER_SIZE, OPT_USE_GRAPH, OPT_PROFILE, OPT_
 OPT_SHARED_SCALE, OPT_AVERAGE_DIVISOR = 6, 7
 SCHEME_BROADCAST, SCHEME_SERVER_SUM, SCHEME_SERVER_REQUANTIZE = 0, 1, 2
 (INFO_STEP_CLUSTER_SIZE, INFO_LOOP_CLUSTER_SIZE, INFO_LOOP_LAUNCHES, INFO_SNAPSHOT_ROWS_PER_TILE, INFO_SNAPSHOT_STAGES,
- INFO_ALPC_LOOP_CLUSTER_SIZE, INFO_LOOP_ROW_BUFFERS, INFO_ALPC_LOOP_ROW_BUFFERS, INFO_STEP_RING_STAGES) = range(9)
+ INFO_ALPC_LOOP_CLUSTER_SIZE, INFO_LOOP_ROW_BUFFERS, INFO_ALPC_LOOP_ROW_BUFFERS, INFO_STEP_RING_STAGES,
+ INFO_AGGREGATE_SPLIT, INFO_QUANT_PIPELINED_RUNS) = range(11)
 KERNEL_NAMES = ["snapshot", "worker", "aggregate", "quant_stats", "quant_pack", "other", "inner_loop"]
 
 # every symbol that include/lpc.h declares: (name, restype, argtypes)
@@ -60,6 +61,7 @@ SYMBOLS = [
     ("lpc_svrg_run_host", _int, [_vp, _vp, _i64, _i32, _int, _f32, _i32, _i32, _i32, _int, _f32, _u64, _i32, _i64,
                                  _f32, _vp, _f64p, _u64p]),
     ("lpc_quantize_pack_static", _int, [_vp, _i64, _i64, _i32, _i32, _int, _f32, _u64, _u64, _vp, _vp, _vp, _vp]),
+    ("lpc_debug_wait_timeout", _int, [_vp, _u64]),
     ("lpc_debug_stream_blocks", _int, [_u64, C.c_uint32, C.c_uint32, _u64, C.c_uint32, _i64, _vp, _vp]),
 ]
 
@@ -300,6 +302,10 @@ class Context:
         self._ck(lib().lpc_get_profile(self._h, ms, cnt, 1 if reset else 0))
         return {KERNEL_NAMES[i]: (ms[i], cnt[i]) for i in range(n)}
 
+    def debug_wait_timeout(self, limit_ns):
+        """Enqueues a kernel whose bounded waits run out after limit_ns (see lpc_debug_wait_timeout)."""
+        self._ck(lib().lpc_debug_wait_timeout(self._h, limit_ns))
+
     def comm_bits(self):
         a, b = C.c_uint64(0), C.c_uint64(0)
         self._ck(lib().lpc_comm_bits(self._h, C.byref(a), C.byref(b)))
@@ -339,5 +345,6 @@ def quantize_pack_static(U, b, clip_mode, clip_value, seed, k, codes_out, delta_
     N, length = U.shape
     ld = U.stride(0) if N > 1 else max(length, 1)
     st = torch.cuda.current_stream(U.device)
-    return lib().lpc_quantize_pack_static(_ptr(U), length, ld, N, b, clip_mode, clip_value, seed, k, _ptr(codes_out),
-                                          _ptr(delta_out), _ptr(clipped_out), C.c_void_p(st.cuda_stream))
+    with torch.cuda.device(U.device):  # the library looks its working memory up on the current device
+        return lib().lpc_quantize_pack_static(_ptr(U), length, ld, N, b, clip_mode, clip_value, seed, k, _ptr(codes_out),
+                                              _ptr(delta_out), _ptr(clipped_out), C.c_void_p(st.cuda_stream))

@@ -1,6 +1,7 @@
 """The multi-GPU leg runs independent replicas; ranks only meet for a barrier and to combine timings.
 This covers that host logic with two gloo ranks on CPU."""
 import os
+import socket
 import subprocess
 import sys
 import textwrap
@@ -26,11 +27,17 @@ WORKER = textwrap.dedent("""
 """) % ROOT
 
 
+def _free_port():
+    with socket.socket(socket.AF_INET, socket.SOCK_STREAM) as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
 def test_two_rank_timing_aggregation(tmp_path):
     script = tmp_path / "worker.py"
     script.write_text(WORKER)
     cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2", "--master-addr",
-           "127.0.0.1", "--master-port", "29613", str(script)]
+           "127.0.0.1", "--master-port", str(_free_port()), str(script)]
     env = dict(os.environ, OMP_NUM_THREADS="1")
     r = subprocess.run(cmd, capture_output=True, text=True, timeout=240, env=env)
     assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]

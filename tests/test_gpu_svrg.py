@@ -334,17 +334,13 @@ def test_alpc_epochs_follow_algorithm3():
     snap, y, z = x0.copy(), x0.copy(), x0.copy()
     p0 = ctx.objective()
     for s in range(S):
-        tau1 = np.float32(2.0 / (s + 4))
-        alpha = np.float32(1.0 / (6.0 * L * float(tau1)))
+        tau1, alpha = orc.alpc3_epoch_params(s, L)  # the oracle's outer rule (Algorithm 3 step 3)
         inv4L = np.float32(1.0 / (4.0 * L))
         ctx.snapshot_full_grad()
         mu = ctx.get_buffer(lpc.BUF_MU).cpu().numpy()
         ctx.alpc_double_sample_steps(float(tau1), 0.5, float(alpha), float(inv4L), s * m, m)
         ctx.alpc_end_epoch(m)
-        ysum = np.zeros(P.d, np.float32)
-        for t in range(m):
-            y, z, ysum = orc.alpc_step(P, s * m + t, tau1, 0.5, alpha, inv4L, snap, mu, y, z, ysum)
-        snap = (ysum * (np.float32(1.0) / np.float32(m))).astype(np.float32)
+        y, z, snap = orc.alpc3_epoch(P, s, m, L, 0.5, snap, mu, y, z)
         assert _same(ctx.get_iterate(), snap)
         assert _same(ctx.get_buffer(lpc.BUF_Y), y) and _same(ctx.get_buffer(lpc.BUF_Z), z)
     ctx.sync_status()
@@ -408,3 +404,35 @@ def test_alpc_one_launch_loop_equals_single_steps(cfg, loss):
     assert ctx.comm_bits() == ref.comm_bits()
     ctx.close()
     ref.close()
+
+
+def test_average_divisor_option_leaves_the_training_loops_alone():
+    # LPC_OPT_AVERAGE_DIVISOR belongs to lpc_unpack_average_prox; single steps, graph replay and the one-launch loop all
+    # keep averaging over the N workers (Eq. 3) and agree bit for bit
+    P, ctx = _setup(512, 256, "least_squares", N=4, B=2, b=4, seed=9)
+    count, eta = 130, 0.05
+    results = []
+    for mode in ("single", "graph", "loop"):
+        c = lpc.Context(ctx.X, ctx.y, P.loss, P.lambda_l1, P.N, P.B, P.b, P.clip_mode, P.clip_value, P.seed)
+        c.set_option(lpc.OPT_AVERAGE_DIVISOR, 3)
+        c.snapshot_full_grad()
+        if mode == "single":
+            for k in range(count):
+                c.inner_step(eta, k)
+        else:
+            c.set_option(lpc.OPT_PERSISTENT, 1 if mode == "loop" else 0)
+            c.inner_steps(eta, 0, count)
+        c.sync_status()
+        assert c.query(lpc.INFO_LOOP_LAUNCHES) == (1 if mode == "loop" else 0)
+        results.append(c.get_iterate().cpu().numpy())
+        c.close()
+    assert _same(results[0], results[1]) and _same(results[0], results[2])
+    # and they are the oracle's iterates (which know no such option)
+    ctx.snapshot_full_grad()
+    mu = ctx.get_buffer(lpc.BUF_MU).cpu().numpy()
+    x0 = np.zeros(P.d, np.float32)
+    xr = x0
+    for k in range(count):
+        xr = orc.lpc_inner_step(P, k, eta, xr, x0, mu)
+    assert _same(results[0], xr)
+    ctx.close()
