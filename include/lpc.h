@@ -284,9 +284,9 @@ int lpc_objective(lpc_ctx* ctx, const float* x, double* P_out);
 #define LPC_INFO_ALPC_LOOP_ROW_BUFFERS 7   /* the same for the loop of Algorithm 2 */
 #define LPC_INFO_STEP_RING_STAGES 8        /* per-step kernel: 0 = minibatch rows resident on chip, else ring stages they stream through */
 #define LPC_INFO_AGGREGATE_SPLIT 9         /* last lpc_unpack_average_prox: CTAs that shared one tile of 8192 coordinates (1, 2 or 4) */
-#define LPC_INFO_QUANT_PIPELINED_RUNS 10   /* last lpc_quantize_pack: runs of 8 tiles per worker that were whole tiles of one segment of
-                                              16-byte aligned vectors and so took the second pass's software-pipelined loop (unless
-                                              that worker's scale was degenerate) */
+#define LPC_INFO_QUANT_PIPELINED_RUNS 10   /* last lpc_quantize_pack: runs of 8 tiles per worker that were whole tiles of one segment and
+                                              so took the second pass's software-pipelined loop (unless that worker's scale was
+                                              degenerate); 0 unless every worker's vector starts on a 16-byte boundary (ld % 4 == 0) */
 int lpc_query(const lpc_ctx* ctx, int what, int64_t* out);
 
 /* Per-kernel device time measured with CUDA events on the context's stream while LPC_OPT_PROFILE is

@@ -1,6 +1,9 @@
 """Build paper_1901_08924_b200/liblpcsvrg.so (the C-ABI library) with nvcc for sm_100a.
 
-    python -m paper_1901_08924_b200.build [--force] [--verbose]
+    python -m paper_1901_08924_b200.build [--force] [--verbose] [--trace]
+
+--trace builds liblpcsvrg_trace.so instead: the same sources with -DLPC_TRACE, in which one CTA of the one-launch loop
+and of the streaming worker kernel stamps %globaltimer at every phase boundary (read by paper_1901_08924_b200.trace).
 
 -fmad=false: the packed codes are defined with separate round-to-nearest multiplies and adds, so
 the compiler must not contract them into fused multiply-adds anywhere in the library.
@@ -32,18 +35,24 @@ def _newest_dep():
     return max(os.path.getmtime(p) for p in deps)
 
 
-def build(force=False, verbose=False):
+TRACE_LIB = os.path.join(HERE, "liblpcsvrg_trace.so")
+
+
+def build(force=False, verbose=False, trace=False):
     sources = [s for s in SOURCES if os.path.exists(os.path.join(CSRC, s))]
-    if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= _newest_dep():
-        return LIB
-    os.makedirs(OBJ, exist_ok=True)
+    lib = TRACE_LIB if trace else LIB
+    objdir = os.path.join(OBJ, "trace") if trace else OBJ
+    flags = NVCC_FLAGS + (["-DLPC_TRACE"] if trace else [])
+    if not force and os.path.exists(lib) and os.path.getmtime(lib) >= _newest_dep():
+        return lib
+    os.makedirs(objdir, exist_ok=True)
     nvcc = _nvcc()
 
     def compile_one(src):
-        obj = os.path.join(OBJ, src.replace(".cu", ".o"))
-        cmd = [nvcc, *NVCC_FLAGS, "-c", os.path.join(CSRC, src), "-o", obj]
+        obj = os.path.join(objdir, src.replace(".cu", ".o"))
+        cmd = [nvcc, *flags, "-c", os.path.join(CSRC, src), "-o", obj]
         r = subprocess.run(cmd, capture_output=True, text=True)
-        with open(os.path.join(OBJ, src + ".ptxas.log"), "w") as f:
+        with open(os.path.join(objdir, src + ".ptxas.log"), "w") as f:
             f.write(r.stderr)
         if r.returncode != 0:
             raise RuntimeError(f"nvcc failed on {src}:\n{r.stderr[-4000:]}")
@@ -53,13 +62,13 @@ def build(force=False, verbose=False):
 
     with concurrent.futures.ThreadPoolExecutor(max_workers=8) as ex:
         objs = list(ex.map(compile_one, sources))
-    cmd = [nvcc, "-shared", "-cudart", "static", "-o", LIB + ".tmp", *objs]
+    cmd = [nvcc, "-shared", "-cudart", "static", "-o", lib + ".tmp", *objs]
     r = subprocess.run(cmd, capture_output=True, text=True)
     if r.returncode != 0:
         raise RuntimeError(f"link failed:\n{r.stderr[-4000:]}")
-    os.replace(LIB + ".tmp", LIB)
-    return LIB
+    os.replace(lib + ".tmp", lib)
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv, trace="--trace" in sys.argv))

@@ -10,7 +10,8 @@ import os
 import torch
 
 HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(HERE, "liblpcsvrg.so")
+# LPC_LIBRARY selects another build of the same library (the phase-stamping build of paper_1901_08924_b200.trace)
+LIB_PATH = os.environ.get("LPC_LIBRARY") or os.path.join(HERE, "liblpcsvrg.so")
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_NONFINITE, ERR_CUDA, ERR_TIMEOUT = 0, -1, -2, -3, -4, -5
 LOGISTIC, LEAST_SQUARES = 0, 1

@@ -36,6 +36,15 @@ def _offset(b):
     return 0 if b == 1 else 1 << (b - 1)
 
 
+def _rows_aligned(U):
+    """U on the device with a row stride that is a multiple of 4 floats, so that every worker's vector starts on a
+    16-byte boundary (the pipelined loop needs that)."""
+    N, length = U.shape
+    buf = torch.zeros((N, (length + 3) // 4 * 4), device=DEV)
+    buf[:, :length] = torch.from_numpy(U).to(DEV)
+    return buf[:, :length]
+
+
 @pytest.mark.parametrize("b", [1, 2, 4, 8])
 def test_quantize_runs_of_whole_tiles_bit_exact(b):
     # runs of 2, 5, 8 whole tiles, a full run plus one tile and a ragged tail, two full runs plus a tail
@@ -46,7 +55,7 @@ def test_quantize_runs_of_whole_tiles_bit_exact(b):
         U = rng.standard_normal((N, length)).astype(np.float32)
         U[1] *= 37.0
         ctx = _ctx(N, b, orc.CLIP_STD, 2.0, seed)
-        codes, delta, clipped = ctx.quantize_pack(torch.from_numpy(U).to(DEV), k)
+        codes, delta, clipped = ctx.quantize_pack(_rows_aligned(U), k)
         ctx.sync_status()
         assert ctx.query(lpc.INFO_QUANT_PIPELINED_RUNS) == want_runs, length
         W = orc.packed_words(length, b)
