@@ -476,7 +476,7 @@ def alpc_bench(dev):
         out["b%d" % b] = {"iters_per_s": round(m / ((snap + loop) * 1e-3), 1), "step_us": round(loop * 1e3 / m, 3),
                           "snapshot_ms": round(snap, 4), "snapshot_gbs": round(n * d * 4 / snap * 1e-6, 1),
                           "loop_cluster_size": ctx.query(lpc.INFO_ALPC_LOOP_CLUSTER_SIZE),
-                          "loop_row_buffers": ctx.query(lpc.INFO_ALPC_LOOP_ROW_BUFFERS),
+                          "loop_row_slots": ctx.query(lpc.INFO_ALPC_LOOP_ROW_SLOTS),
                           "one_launch_loops": ctx.query(lpc.INFO_LOOP_LAUNCHES), "objective": ctx.objective()}
         ctx.close()
     # the strongly convex case (Algorithm 2, elastic net with sigma = L/1000, Theorem 3's tau1 and alpha)

@@ -280,9 +280,13 @@ int lpc_objective(lpc_ctx* ctx, const float* x, double* P_out);
 #define LPC_INFO_SNAPSHOT_ROWS_PER_TILE 3  /* rows per shared-memory stage of the snapshot pass */
 #define LPC_INFO_SNAPSHOT_STAGES 4         /* shared-memory stages of the snapshot pass */
 #define LPC_INFO_ALPC_LOOP_CLUSTER_SIZE 5  /* as LOOP_CLUSTER_SIZE, for the one-launch loop of Algorithm 2 */
-#define LPC_INFO_LOOP_ROW_BUFFERS 6        /* sampled-row buffers per CTA of the one-launch loop (1 or 2; 0: not available) */
-#define LPC_INFO_ALPC_LOOP_ROW_BUFFERS 7   /* the same for the loop of Algorithm 2 */
+#define LPC_INFO_LOOP_ROW_SLOTS 6          /* shared-memory slots for sampled-row slices per CTA of the one-launch loop: between B
+                                              (a step's rows are fetched once the step before has formed its u) and 2B (all of them
+                                              are fetched a whole step ahead); 0: loop not available */
+#define LPC_INFO_ALPC_LOOP_ROW_SLOTS 7     /* the same for the loop of Algorithm 2 */
 #define LPC_INFO_STEP_RING_STAGES 8        /* per-step kernel: 0 = minibatch rows resident on chip, else ring stages they stream through */
+#define LPC_INFO_LOOP_COORDS_PER_THREAD 11  /* one-launch loop: consecutive coordinates a thread owns (8, 4 or 2; 0: not available) */
+#define LPC_INFO_ALPC_LOOP_COORDS_PER_THREAD 12
 #define LPC_INFO_AGGREGATE_SPLIT 9         /* last lpc_unpack_average_prox: CTAs that shared one tile of 8192 coordinates (1, 2 or 4) */
 #define LPC_INFO_QUANT_PIPELINED_RUNS 10   /* last lpc_quantize_pack: runs of 8 tiles per worker that were whole tiles of one segment and
                                               so took the second pass's software-pipelined loop (unless that worker's scale was

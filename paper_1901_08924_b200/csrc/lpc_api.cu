@@ -86,7 +86,7 @@ struct lpc_ctx {
   SegPlan inner_seg;  // one segment of length d for the aggregator
   // persistent inner loop
   bool persist_ok = false, apersist_ok = false;  // Algorithm 1 loop / Algorithm 2 loop
-  int pCS = 1, pSL = 0, pNbuf = 2, aCS = 1, aSL = 0, aNbuf = 2;
+  int pCS = 1, pSL = 0, pSlots = 0, aCS = 1, aSL = 0, aSlots = 0;  // cluster size, slice, row slots of the two loops
   size_t persistSmem = 0, apersistSmem = 0;
   // exchange buffers of the one-launch loops: tagged 64-bit words (payload | tag << 32), two step-parity halves
   unsigned long long* flags = nullptr;    // scale words: 2 x 256, 128 bytes apart, + 1 abort word
@@ -330,11 +330,11 @@ int replan_inner(lpc_ctx* c) {
   int stages = 0;
   c->inner_ok = inner_plan(c->d, c->B, c->want_cs, c->max_smem, &cs, &sl, &smem, &stages);
   if (c->inner_ok) { c->CS = cs; c->SL = sl; c->innerSmem = smem; c->innerStages = stages; }
-  int nbuf = 2;
-  c->persist_ok = persist_plan(c->d, c->N, c->B, c->b, 0, c->want_cs, c->max_smem, &cs, &sl, &smem, &nbuf);
-  if (c->persist_ok) { c->pCS = cs; c->pSL = sl; c->persistSmem = smem; c->pNbuf = nbuf; }
-  c->apersist_ok = persist_plan(c->d, c->N, c->B, c->b, 1, c->want_cs, c->max_smem, &cs, &sl, &smem, &nbuf);
-  if (c->apersist_ok) { c->aCS = cs; c->aSL = sl; c->apersistSmem = smem; c->aNbuf = nbuf; }
+  int slots = 0;
+  c->persist_ok = persist_plan(c->d, c->N, c->B, c->b, 0, c->want_cs, c->max_smem, &cs, &sl, &smem, &slots);
+  if (c->persist_ok) { c->pCS = cs; c->pSL = sl; c->persistSmem = smem; c->pSlots = slots; }
+  c->apersist_ok = persist_plan(c->d, c->N, c->B, c->b, 1, c->want_cs, c->max_smem, &cs, &sl, &smem, &slots);
+  if (c->apersist_ok) { c->aCS = cs; c->aSL = sl; c->apersistSmem = smem; c->aSlots = slots; }
   return LPC_OK;
 }
 
@@ -391,7 +391,7 @@ int run_steps(lpc_ctx* c, int kind, const float* p, uint64_t k0, int64_t count) 
     pa.in = inner_args(c, k0, nullptr, 0);
     pa.in.CS = kind == 0 ? c->pCS : c->aCS;
     pa.in.SL = kind == 0 ? c->pSL : c->aSL;
-    pa.nbuf = kind == 0 ? c->pNbuf : c->aNbuf;
+    pa.row_slots = kind == 0 ? c->pSlots : c->aSlots;
     pa.count = (int)count; pa.eta = kind == 0 ? p[0] : 0.f; pa.lambda_l1 = c->lambda_l1;
     pa.pub = c->flags; pa.abort_flag = reinterpret_cast<unsigned int*>(c->flags + 512 * 16); pa.x_out = c->x;
     pa.ll = c->ll; pa.ll_vhat = c->ll_vhat; pa.wpg = c->ll_wpg;
@@ -787,8 +787,10 @@ int lpc_query(const lpc_ctx* c, int what, int64_t* out) {
     case LPC_INFO_STEP_CLUSTER_SIZE: *out = c->inner_ok ? c->CS : 0; return LPC_OK;
     case LPC_INFO_LOOP_CLUSTER_SIZE: *out = c->persist_ok ? c->pCS : 0; return LPC_OK;
     case LPC_INFO_ALPC_LOOP_CLUSTER_SIZE: *out = c->apersist_ok ? c->aCS : 0; return LPC_OK;
-    case LPC_INFO_LOOP_ROW_BUFFERS: *out = c->persist_ok ? c->pNbuf : 0; return LPC_OK;
-    case LPC_INFO_ALPC_LOOP_ROW_BUFFERS: *out = c->apersist_ok ? c->aNbuf : 0; return LPC_OK;
+    case LPC_INFO_LOOP_ROW_SLOTS: *out = c->persist_ok ? c->pSlots : 0; return LPC_OK;
+    case LPC_INFO_ALPC_LOOP_ROW_SLOTS: *out = c->apersist_ok ? c->aSlots : 0; return LPC_OK;
+    case LPC_INFO_LOOP_COORDS_PER_THREAD: *out = c->persist_ok ? persist_coords_per_thread(c->b, c->pSL) : 0; return LPC_OK;
+    case LPC_INFO_ALPC_LOOP_COORDS_PER_THREAD: *out = c->apersist_ok ? persist_coords_per_thread(c->b, c->aSL) : 0; return LPC_OK;
     case LPC_INFO_STEP_RING_STAGES: *out = c->inner_ok ? c->innerStages : 0; return LPC_OK;
     case LPC_INFO_LOOP_LAUNCHES: *out = c->persist_launches; return LPC_OK;
     case LPC_INFO_SNAPSHOT_ROWS_PER_TILE: *out = c->snapR; return LPC_OK;

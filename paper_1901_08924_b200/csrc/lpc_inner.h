@@ -54,7 +54,7 @@ struct PersistArgs {
   unsigned int* abort_flag;  // zero at launch; set when a bounded wait ran out
   float* x_out;              // iterate after `count` steps (may alias in.x)
   float* v_tap;              // nullable: v of the last step
-  int nbuf;                  // shared-memory row buffers: 2 (prefetch a step ahead) or 1
+  int row_slots;             // shared-memory row slots of SL floats: B .. 2B (2B: all rows of a step are fetched a step ahead)
   // Algorithm 2 (alpc = 1): in.x is not read; y, z, ysum are read at entry and written at exit, xt is the
   // snapshot, vhat (d floats) receives the last step's second estimator, x_out the last coupled point
   int alpc;
@@ -69,7 +69,8 @@ struct PersistArgs {
   float* vhat;
 };
 bool persist_plan(int d, int N, int B, int b, int alpc, int want_cs, int max_smem, int* CS_out, int* SL_out,
-                  size_t* smem_out, int* nbuf_out);
+                  size_t* smem_out, int* row_slots_out);
+int persist_coords_per_thread(int b, int SL);
 cudaError_t launch_persist(const PersistArgs& pa, size_t smem, cudaStream_t st);
 // One small kernel whose bounded waits (an mbarrier phase; a tagged word when `word` is given) run out after limit_ns.
 cudaError_t launch_wait_timeout(const unsigned long long* word, unsigned int* abort_flag, unsigned int* dev_status,

@@ -130,24 +130,63 @@ __device__ unsigned long long g_trace[64 * 16];
 #define LPC_TRACE_MARK(i) do { } while (0)
 #endif
 
+// A thread's EPT consecutive row values of a slice from shared memory (zero outside the existing columns).
+template <int EPT>
+__device__ __forceinline__ void row_vals(const float* rowp, int off, int width, float* v) {
+#pragma unroll
+  for (int e = 0; e < EPT; ++e) v[e] = 0.f;
+  if (off < width) {  // width is a multiple of 4 and off a multiple of EPT
+    if constexpr (EPT == 2) {
+      const float2 t = *reinterpret_cast<const float2*>(rowp + off);
+      v[0] = t.x; v[1] = t.y;
+    } else {
+      const float4 t = *reinterpret_cast<const float4*>(rowp + off);
+      v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+      if constexpr (EPT == 8) {
+        if (off + 4 < width) {
+          const float4 t1 = *reinterpret_cast<const float4*>(rowp + off + 4);
+          v[4] = t1.x; v[5] = t1.y; v[6] = t1.z; v[7] = t1.w;
+        }
+      }
+    }
+  }
+}
+// Balanced-tree sum of a thread's EPT consecutive values (the lowest levels of the tree over the coordinate index).
+template <int EPT>
+__device__ __forceinline__ float tree_ept(const float* v) {
+  if constexpr (EPT == 8) return tree8(v);
+  else if constexpr (EPT == 4) return tree4(v[0], v[1], v[2], v[3]);
+  else return add_rn(v[0], v[1]);
+}
+
 // BITS: 1, 2, 4, 8 fixed width; 0: b from the arguments (1..16 or 32).
-// NP: passes of 2048 coordinates that a CTA makes over its slice (1 or 2).
+// NP: passes of PT * EPT coordinates that a CTA makes over its slice (1 or 2).
+// EPT: consecutive coordinates a thread owns per pass (8, 4 or 2): slices of 1024 or 512 coordinates still give every
+//      thread of the CTA work, which shortens each serial phase of a step; a group of 8 coordinates (one Philox block,
+//      one tagged code word for b <= 4) is then shared by 8 / EPT neighbouring lanes.  BITS = 0 and NP = 2 use EPT = 8.
 // ALPC: Algorithm 2's step (coupling, double sampling on one more cluster, y/z updates) instead of Algorithm 1's.
-template <int BITS, int NP, bool ALPC>
+template <int BITS, int NP, int EPT, bool ALPC>
 __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
+  static_assert(EPT == 8 || ((EPT == 4 || EPT == 2) && BITS != 0 && NP == 1), "narrow threads: fixed widths, one pass");
+  constexpr int PSPAN = PT * EPT;               // coordinates per pass
+  constexpr int LPG = 8 / EPT;                  // lanes that share a group of 8 coordinates
+  constexpr int TB = EPT * (BITS ? BITS : 1);   // code bits a thread produces per pass (fixed widths)
   const InnerArgs& a = pa.in;
   cg::cluster_group cluster = cg::this_cluster();
   extern __shared__ __align__(16) unsigned char smem_raw[];
   PSmem& sm = *reinterpret_cast<PSmem*>(smem_raw);
   const int CS = a.CS, SL = a.SL, B = a.B, d = a.d, N = a.N;
-  float* rows = reinterpret_cast<float*>(smem_raw + ((sizeof(PSmem) + 15) & ~(size_t)15));  // 2 x B x SL
-  const size_t buf_floats = (size_t)B * SL;
+  float* rows = reinterpret_cast<float*>(smem_raw + ((sizeof(PSmem) + 15) & ~(size_t)15));  // RS row slots of SL floats
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int rank = (int)cluster.block_rank();
   const int worker = blockIdx.y;
   const bool is_J = ALPC && (worker == N);  // the extra cluster that handles the shared batch J
-  const int nbuf = pa.nbuf;                  // 2: rows of the next step are fetched while this one computes
+  // Row slots: step t keeps its B rows in slots (t*B + a) % RS.  RS = 2B: all rows of step t+1 are fetched while step
+  // t computes.  B <= RS < 2B (the slices of two steps do not fit): the first RS - B rows of step t+1 go into the free
+  // slots at the top of step t, the others into the slots that step t gives back once its u is formed.
+  const int RS = pa.row_slots;
+  const int PA = RS - B;                    // rows of the next step fetched at the top of a step
   const int b = BITS ? BITS : a.b;
   const int c0 = rank * SL;
   const int width = max(0, min(SL, d - c0));
@@ -155,6 +194,7 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
   const float invB = __fdiv_rn(1.0f, (float)B);
   const float kappa = mul_rn(pa.eta, pa.lambda_l1);
   const uint32_t zero_code = (b == 1) ? 0u : (1u << (b - 1));
+  const uint32_t row_bytes = (uint32_t)width * 4u;
 
   if (tid == 0) {
     mbar_init(&sm.bar[0], 1);
@@ -167,20 +207,28 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
   asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   __syncthreads();
 
-  // Thread a < B owns minibatch slot a.  prefetch(t) samples step t's row for the slot, starts the bulk copy
-  // of this CTA's slice of it into buffer t&1 and loads its label and cached snapshot margin into registers
-  // (a step ahead, so these loads never stall the step that issues them).
+  // Thread a < B owns minibatch slot a.  fetch_rows(t, sb, lo, hi) samples step t's row for the slots lo <= a < hi,
+  // starts the bulk copy of this CTA's slice of it into row slot (sb + a) % RS and loads its label and cached
+  // snapshot margin into registers (a step ahead, so these loads never stall the step that issues them).  The
+  // barrier of step t (bar[t & 1]) gets its one arrival from the call that covers the last slot.
   const int64_t samp_span = (a.sample_global || is_J) ? a.n : a.n / N;  // rows this cluster samples from
   const int64_t samp_lo = (a.sample_global || is_J) ? 0 : (int64_t)worker * samp_span;
   int64_t row_next = 0, row_cur = 0;
   float y_next = 0.f, y_cur = 0.f, ms_next = 0.f, ms_cur = 0.f;
-  auto prefetch = [&](int t) {
-    const int s = (nbuf == 2) ? (t & 1) : 0;
-    if (tid == 0 && width > 0) mbar_expect_tx(&sm.bar[s], (uint32_t)width * 4u * (uint32_t)B);
-    if (tid < B) {
+  auto fetch_rows = [&](int t, int sb, int lo, int hi) {
+    if (hi <= lo) return;
+    uint64_t* bar = &sm.bar[t & 1];
+    if (tid == 0 && width > 0) {
+      const uint32_t bytes = row_bytes * (uint32_t)(hi - lo);
+      if (hi == B) mbar_expect_tx(bar, bytes);  // arrives as well: the phase can now complete
+      else asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+    }
+    if (tid >= lo && tid < hi) {
       const U4 r = stream_block(a.seed, is_J ? TAG_BATCH_J : TAG_BATCH, is_J ? 0u : (uint32_t)worker, a.k_base + (uint64_t)t, (uint32_t)tid);
       const int64_t row = samp_lo + (int64_t)(((uint64_t)r.x * (uint64_t)samp_span) >> 32);
-      if (width > 0) bulk_load(rows + s * buf_floats + (size_t)tid * SL, a.X + row * (int64_t)d + c0, (uint32_t)width * 4u, &sm.bar[s]);
+      int slot = sb + tid;
+      if (slot >= RS) slot -= RS;
+      if (width > 0) bulk_load(rows + (size_t)slot * SL, a.X + row * (int64_t)d + c0, row_bytes, bar);
       row_next = row;
       y_next = a.y[row];
       ms_next = a.margins[row];
@@ -188,25 +236,25 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
   };
 
   // this thread's slice of the iterate and of the snapshot gradient stay in registers for the whole loop
-  float xr[NP][8], mur[NP][8];
+  float xr[NP][EPT], mur[NP][EPT];
 #pragma unroll
   for (int p = 0; p < NP; ++p) {
-    const int off = p * PGROUP + tid * 8;
+    const int off = p * PSPAN + tid * EPT;
 #pragma unroll
-    for (int e = 0; e < 8; ++e) {
+    for (int e = 0; e < EPT; ++e) {
       const bool in = off + e < width;
       xr[p][e] = in ? a.x[c0 + off + e] : 0.f;
       mur[p][e] = in ? a.mu[c0 + off + e] : 0.f;
     }
   }
   // Algorithm 2 keeps y, z, the running sum of y and the snapshot in registers too; xr is then the coupled point
-  float yr[ALPC ? NP : 1][8], zr[ALPC ? NP : 1][8], sr[ALPC ? NP : 1][8], xtr[ALPC ? NP : 1][8];
+  float yr[ALPC ? NP : 1][EPT], zr[ALPC ? NP : 1][EPT], sr[ALPC ? NP : 1][EPT], xtr[ALPC ? NP : 1][EPT];
   if constexpr (ALPC) {
 #pragma unroll
     for (int p = 0; p < NP; ++p) {
-      const int off = p * PGROUP + tid * 8;
+      const int off = p * PSPAN + tid * EPT;
 #pragma unroll
-      for (int e = 0; e < 8; ++e) {
+      for (int e = 0; e < EPT; ++e) {
         const bool in = off + e < width;
         yr[p][e] = in ? pa.y[c0 + off + e] : 0.f;
         zr[p][e] = in ? pa.z[c0 + off + e] : 0.f;
@@ -217,21 +265,8 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
   }
   const float tau3 = __fsub_rn(__fsub_rn(1.0f, pa.tau1), pa.tau2);
   const float kappa_y = mul_rn(pa.inv4L, pa.lambda_l1), kappa_z = mul_rn(pa.alpha, pa.lambda_l1);
-  if (pa.count > 0) prefetch(0);
+  if (pa.count > 0) fetch_rows(0, 0, 0, B);
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-
-  auto row8 = [&](const float* base, int r, int off, float* v) {
-#pragma unroll
-    for (int e = 0; e < 8; ++e) v[e] = 0.f;
-    if (off < width) {
-      const float4 v0 = *reinterpret_cast<const float4*>(base + (size_t)r * SL + off);
-      v[0] = v0.x; v[1] = v0.y; v[2] = v0.z; v[3] = v0.w;
-      if (off + 4 < width) {
-        const float4 v1 = *reinterpret_cast<const float4*>(base + (size_t)r * SL + off + 4);
-        v[4] = v1.x; v[5] = v1.y; v[6] = v1.z; v[7] = v1.w;
-      }
-    }
-  };
 
   // Every spin in this kernel ends: after about two seconds without progress the thread records a timeout and
   // raises the abort flag, which ends all other spins at their next look at it.
@@ -239,11 +274,15 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
 
   // Applies step target-1's update to this thread's coordinates:
   //   x <- prox_{eta h}(x - eta (mean_i delta_i k_i + mu))      (Algorithm 2: the y and z updates).
-  // The words of all workers for the thread's 8 coordinates are loaded together (one L2 round trip) and
+  // The words of all workers that hold the thread's codes are loaded together (one L2 round trip) and
   // re-loaded until every tag names step target-1; LLCH workers are handled per round.
   constexpr int WMAX = (BITS == 0) ? 8 : (BITS == 8 ? 2 : 1);  // tagged words per group of 8 coordinates
+  constexpr int NW = (BITS == 0) ? 8 : (TB >= 32 ? TB / 32 : 1);  // of which a thread reads / writes this many
   constexpr int LLCH = (BITS == 0) ? 4 : 16;
   const int wpg = (BITS == 0) ? pa.wpg : WMAX;
+  const int sub = (LPG > 1) ? (tid & (LPG - 1)) : 0;          // this thread's place in its group of 8 coordinates
+  const int wfirst = (BITS == 0) ? 0 : (sub * TB) >> 5;        // first word of the group that holds its codes
+  const int wshift = (BITS == 0) ? 0 : (sub * TB) & 31;        // and their position in it
   const size_t groups = (size_t)(CS * SL) >> 3;
   float wcur = pa.w0;  // snapshot weight of the step whose update comes next
   auto apply_update = [&](unsigned int target) {
@@ -253,30 +292,30 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
     const unsigned long long* ll_in = pa.ll + (size_t)rpar * N * groups * wpg;
 #pragma unroll
     for (int p = 0; p < NP; ++p) {
-      const int off = p * PGROUP + tid * 8;
+      const int off = p * PSPAN + tid * EPT;
       const int c = c0 + off;
       if (off >= SL || c >= d) continue;
-      float acc[8];
+      float acc[EPT];
 #pragma unroll
-      for (int e = 0; e < 8; ++e) acc[e] = 0.f;
-      unsigned long long vw[ALPC ? 8 : 1];
+      for (int e = 0; e < EPT; ++e) acc[e] = 0.f;
+      unsigned long long vw[ALPC ? EPT : 1];
 #pragma unroll 1
       for (int i0 = 0; i0 < N; i0 += LLCH) {
-        unsigned long long dw[LLCH], cw[LLCH][WMAX];
+        unsigned long long dw[LLCH], cw[LLCH][NW];
         uint64_t t0 = 0;
         for (uint32_t it = 0;; ++it) {
 #pragma unroll
           for (int j = 0; j < LLCH; ++j) {
             const int i = min(i0 + j, N - 1);  // the tail repeats the last worker: harmless
             dw[j] = ld_word(dwords + (size_t)i * CS * PUB_STRIDE);
-            const unsigned long long* q = ll_in + ((size_t)i * groups + (size_t)(c >> 3)) * wpg;
+            const unsigned long long* q = ll_in + ((size_t)i * groups + (size_t)(c >> 3)) * wpg + wfirst;
 #pragma unroll
-            for (int w = 0; w < WMAX; ++w) cw[j][w] = (w < wpg) ? ld_word(q + w) : ((unsigned long long)tag << 32);
+            for (int w = 0; w < NW; ++w) cw[j][w] = (w < wpg) ? ld_word(q + w) : ((unsigned long long)tag << 32);
           }
           if constexpr (ALPC) {
             if (i0 == 0) {
 #pragma unroll
-              for (int e = 0; e < 8; ++e) vw[e] = ld_word(pa.ll_vhat + (size_t)rpar * groups * 8 + c + e);
+              for (int e = 0; e < EPT; ++e) vw[e] = ld_word(pa.ll_vhat + (size_t)rpar * groups * 8 + c + e);
             }
           }
           bool ok = true;
@@ -284,12 +323,12 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
           for (int j = 0; j < LLCH; ++j) {
             ok = ok && word_tag(dw[j]) == tag;
 #pragma unroll
-            for (int w = 0; w < WMAX; ++w) ok = ok && word_tag(cw[j][w]) == tag;
+            for (int w = 0; w < NW; ++w) ok = ok && word_tag(cw[j][w]) == tag;
           }
           if constexpr (ALPC) {
             if (i0 == 0) {
 #pragma unroll
-              for (int e = 0; e < 8; ++e) ok = ok && word_tag(vw[e]) == tag;
+              for (int e = 0; e < EPT; ++e) ok = ok && word_tag(vw[e]) == tag;
             }
           }
 #ifdef LPC_TRACE
@@ -308,30 +347,33 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
               const float di = __uint_as_float((uint32_t)dw[j]);
               if (b == 32) {
 #pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                  const float val = (c + e < d && e < WMAX) ? __uint_as_float((uint32_t)cw[j][e < WMAX ? e : 0]) : 0.f;
+                for (int e = 0; e < EPT; ++e) {
+                  const float val = (c + e < d && e < NW) ? __uint_as_float((uint32_t)cw[j][e < NW ? e : 0]) : 0.f;
                   acc[e] = add_rn(acc[e], mul_rn(di, val));
                 }
               } else {
                 uint64_t lo = (uint64_t)(uint32_t)cw[j][0], hi = 0;
-                if constexpr (WMAX >= 2) lo |= (uint64_t)(uint32_t)cw[j][1] << 32;
-                if constexpr (WMAX >= 4) hi = (uint64_t)(uint32_t)cw[j][2] | ((uint64_t)(uint32_t)cw[j][3] << 32);
+                if constexpr (NW >= 2) lo |= (uint64_t)(uint32_t)cw[j][1] << 32;
+                if constexpr (NW >= 4) hi = (uint64_t)(uint32_t)cw[j][2] | ((uint64_t)(uint32_t)cw[j][3] << 32);
                 float kf[8];
                 if constexpr (BITS == 0) {
 #pragma unroll
                   for (int e = 0; e < 8; ++e) kf[e] = index_as_float(extract_bits(lo, hi, e * b, b), b);
                 } else {
+                  // this thread's EPT codes start at bit wshift of the word: decode them as the first codes of a group
+                  // (the entries past EPT are not used and cost nothing)
+                  if constexpr (TB < 32) lo = ((uint32_t)lo >> wshift) & ((1u << TB) - 1u);
                   decode8<BITS ? BITS : 1>(lo, kf);
                 }
 #pragma unroll
-                for (int e = 0; e < 8; ++e) acc[e] = add_rn(acc[e], mul_rn(di, kf[e]));
+                for (int e = 0; e < EPT; ++e) acc[e] = add_rn(acc[e], mul_rn(di, kf[e]));
               }
             }
           }
         }
       }
 #pragma unroll
-      for (int e = 0; e < 8; ++e) {
+      for (int e = 0; e < EPT; ++e) {
         if (c + e < d) {
           const float v = add_rn(mul_rn(acc[e], invN), mur[p][e]);
           if constexpr (ALPC) {  // steps 12-13 of Algorithm 2
@@ -349,26 +391,38 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
     if constexpr (ALPC) wcur = mul_rn(wcur, pa.theta);  // the next step's snapshot weight (Algorithm 2's last step)
   };
 
+  int sb = 0;  // first row slot of the current step, (t * B) % RS
 #pragma unroll 1
   for (int t = 0; t < pa.count; ++t) {
-    const int s = (nbuf == 2) ? (t & 1) : 0;
-    const uint32_t row_parity = (nbuf == 2) ? (uint32_t)((t >> 1) & 1) : (uint32_t)(t & 1);
+    const uint32_t row_parity = (uint32_t)((t >> 1) & 1);
     const uint64_t k = a.k_base + (uint64_t)t;
-    const float* buf = rows + s * buf_floats;
     const int wpar = (pa.count - 1 - t) & 1;  // parity half of the exchange buffers this step writes
     const bool last = (t == pa.count - 1);    // the last step also leaves its messages in the documented layouts
     const uint32_t tag = pa.tag_base + (uint32_t)(t + 1);
     uint32_t* out = a.codes + (int64_t)worker * a.stride_words;
+    int sb_next = sb + B;
+    if (sb_next >= RS) sb_next -= RS;
     LPC_TRACE_MARK(0);
     row_cur = row_next; y_cur = y_next; ms_cur = ms_next;
-    if (nbuf == 2 && t + 1 < pa.count) prefetch(t + 1);
+    if (t + 1 < pa.count) fetch_rows(t + 1, sb_next, 0, PA);
     LPC_TRACE_MARK(1);
+    // a thread that fetches its row of step t+1 only after u is formed keeps this step's label and margin until then
+    const int64_t row_use = row_cur;
+    const float y_use = y_cur, ms_use = ms_cur;
 
     // rounding bits of this step: they depend on the counters only, so they are drawn before the data arrives
+    // (with fewer than 8 coordinates per thread the lanes of a group draw the same block and keep their own 16-bit lanes
+    // of it in the leading words)
     U4 rnd[NP];
 #pragma unroll
-    for (int p = 0; p < NP; ++p)
-      rnd[p] = stream_block(a.seed, TAG_ROUND, (uint32_t)worker, k, (uint32_t)((c0 + p * PGROUP + tid * 8) >> 3));
+    for (int p = 0; p < NP; ++p) {
+      rnd[p] = stream_block(a.seed, TAG_ROUND, (uint32_t)worker, k, (uint32_t)((c0 + p * PSPAN + tid * EPT) >> 3));
+      if constexpr (EPT == 4) {
+        if (sub) { rnd[p].x = rnd[p].z; rnd[p].y = rnd[p].w; }
+      } else if constexpr (EPT == 2) {
+        rnd[p].x = (sub == 0) ? rnd[p].x : (sub == 1) ? rnd[p].y : (sub == 2) ? rnd[p].z : rnd[p].w;
+      }
+    }
 
     LPC_TRACE_MARK(2);
     if (t > 0) apply_update((unsigned int)t);  // x_t = prox(x_{t-1} - eta v_{t-1})  (Algorithm 2: y_t, z_t)
@@ -376,18 +430,23 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
 #pragma unroll
       for (int p = 0; p < NP; ++p)
 #pragma unroll
-        for (int e = 0; e < 8; ++e)
+        for (int e = 0; e < EPT; ++e)
           xr[p][e] = add_rn(add_rn(mul_rn(pa.tau1, zr[p][e]), mul_rn(pa.tau2, xtr[p][e])), mul_rn(tau3, yr[p][e]));
     }
     LPC_TRACE_MARK(4);
 
     bool ok = true;
-    if (width > 0) ok = mbar_wait(&sm.bar[s], row_parity);
+    if (width > 0) ok = mbar_wait(&sm.bar[t & 1], row_parity);
     if (!ok) {
       atomicOr(a.dev_status, DEV_TIMEOUT);
-      mbar_wait(&sm.bar[s], row_parity);
+      mbar_wait(&sm.bar[t & 1], row_parity);
     }
     LPC_TRACE_MARK(5);
+    auto row_ptr = [&](int r) {  // row r of this step
+      int slot = sb + r;
+      if (slot >= RS) slot -= RS;
+      return rows + (size_t)slot * SL;
+    };
 
     // margins <X_a, x_t>: eight rows at a time; their 8*NP per-thread partial sums are reduced across the
     // warp together by recursive halving (9 or 12 shuffles instead of 5 per value)
@@ -397,13 +456,14 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
       float sv[NVAL];
 #pragma unroll
       for (int j = 0; j < RG; ++j) {
+        const float* rp = row_ptr(min(r0 + j, B - 1));
 #pragma unroll
         for (int p = 0; p < NP; ++p) {
-          float v[8], pr[8];
-          row8(buf, min(r0 + j, B - 1), p * PGROUP + tid * 8, v);
+          float v[EPT], pr[EPT];
+          row_vals<EPT>(rp, p * PSPAN + tid * EPT, width, v);
 #pragma unroll
-          for (int e = 0; e < 8; ++e) pr[e] = mul_rn(v[e], xr[p][e]);
-          sv[j * NP + p] = tree8(pr);
+          for (int e = 0; e < EPT; ++e) pr[e] = mul_rn(v[e], xr[p][e]);
+          sv[j * NP + p] = tree_ept<EPT>(pr);
         }
       }
       WarpHalving<NVAL, 0>::run(sv, lane);
@@ -441,10 +501,10 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
         m = tree_small(mp, CS);
       }
       LPC_TRACE_MARK(7);
-      const float c = coef_out_of_line(a.loss, m, ms_cur, y_cur);
+      const float c = coef_out_of_line(a.loss, m, ms_use, y_use);
       sm.coef[tid] = c;
       if (rank == 0 && t == pa.count - 1) {
-        if (a.idx_tap) a.idx_tap[(int64_t)worker * B + tid] = row_cur;
+        if (a.idx_tap) a.idx_tap[(int64_t)worker * B + tid] = row_use;
         if (a.coef_tap) a.coef_tap[(int64_t)worker * B + tid] = c;
       }
     }
@@ -452,37 +512,37 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
     LPC_TRACE_MARK(8);
 
     // u = (1/B) sum_a c_a X_a: four rows are loaded together, the adds keep batch order
-    float u[NP][8];
+    float u[NP][EPT];
 #pragma unroll
     for (int p = 0; p < NP; ++p) {
 #pragma unroll
-      for (int e = 0; e < 8; ++e) u[p][e] = 0.f;
+      for (int e = 0; e < EPT; ++e) u[p][e] = 0.f;
 #pragma unroll 1
       for (int r0 = 0; r0 < B; r0 += 4) {
-        float v[4][8], cf[4];
+        float v[4][EPT], cf[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           const int r = min(r0 + j, B - 1);
-          row8(buf, r, p * PGROUP + tid * 8, v[j]);
+          row_vals<EPT>(row_ptr(r), p * PSPAN + tid * EPT, width, v[j]);
           cf[j] = sm.coef[r];
         }
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           if (r0 + j < B) {
 #pragma unroll
-            for (int e = 0; e < 8; ++e) u[p][e] = add_rn(u[p][e], mul_rn(cf[j], v[j][e]));
+            for (int e = 0; e < EPT; ++e) u[p][e] = add_rn(u[p][e], mul_rn(cf[j], v[j][e]));
           }
         }
       }
 #pragma unroll
-      for (int e = 0; e < 8; ++e) u[p][e] = mul_rn(u[p][e], invB);
+      for (int e = 0; e < EPT; ++e) u[p][e] = mul_rn(u[p][e], invB);
     }
     if (a.u_tap && t == pa.count - 1) {
 #pragma unroll
       for (int p = 0; p < NP; ++p) {
-        const int off = p * PGROUP + tid * 8;
+        const int off = p * PSPAN + tid * EPT;
 #pragma unroll
-        for (int e = 0; e < 8; ++e)
+        for (int e = 0; e < EPT; ++e)
           if (off + e < width) a.u_tap[(int64_t)worker * d + c0 + off + e] = u[p][e];
       }
     }
@@ -492,21 +552,22 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
       // double sampling (Algorithm 2 step 11): v^ = u_J + mu in full precision, nothing is quantized or counted
 #pragma unroll
       for (int p = 0; p < NP; ++p) {
-        const int off = p * PGROUP + tid * 8;
+        const int off = p * PSPAN + tid * EPT;
         if (off < SL) {
           unsigned long long* q = pa.ll_vhat + (size_t)wpar * groups * 8 + c0 + off;
 #pragma unroll
-          for (int e = 0; e < 8; ++e) {
+          for (int e = 0; e < EPT; ++e) {
             const float vh = add_rn(u[p][e], mur[p][e]);
             st_word(q + e, __float_as_uint(vh), tag);
             if (last && off + e < width) pa.vhat[c0 + off + e] = vh;
           }
         }
       }
-      if (nbuf == 1) {
-        __syncthreads();  // nobody reads the row buffer any more
-        if (t + 1 < pa.count) prefetch(t + 1);
+      if (PA < B) {
+        __syncthreads();  // nobody reads this step's rows any more
+        if (t + 1 < pa.count) fetch_rows(t + 1, sb_next, PA, B);
       }
+      sb = sb_next;
       continue;
     }
     // scale (Eq. 2)
@@ -514,12 +575,12 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
 #pragma unroll
     for (int p = 0; p < NP; ++p) {
 #pragma unroll
-      for (int e = 0; e < 8; ++e) mx = max(mx, __float_as_uint(fabsf(u[p][e])));
+      for (int e = 0; e < EPT; ++e) mx = max(mx, __float_as_uint(fabsf(u[p][e])));
       if (a.clip_mode == CLIP_STD) {
-        float sq[8];
+        float sq[EPT];
 #pragma unroll
-        for (int e = 0; e < 8; ++e) sq[e] = mul_rn(u[p][e], u[p][e]);
-        float s1 = tree8(u[p]), s2 = tree8(sq);
+        for (int e = 0; e < EPT; ++e) sq[e] = mul_rn(u[p][e], u[p][e]);
+        float s1 = tree_ept<EPT>(u[p]), s2 = tree_ept<EPT>(sq);
 #pragma unroll
         for (int m = 1; m < 32; m <<= 1) {
           s1 = add_rn(s1, __shfl_xor_sync(0xFFFFFFFFu, s1, m));
@@ -532,7 +593,7 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
     if (lane == 0) sm.wmax[warp] = mx;
     __syncthreads();
     LPC_TRACE_MARK(10);
-    if (nbuf == 1 && t + 1 < pa.count) prefetch(t + 1);  // single row buffer: it is free once u is formed
+    if (t + 1 < pa.count) fetch_rows(t + 1, sb_next, PA, B);  // the slots this step's rows leave free (u is formed)
     if (tid == 0) {
       uint32_t m = 0;
       for (int w = 0; w < 8; ++w) m = max(m, sm.wmax[w]);
@@ -592,14 +653,14 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
     uint32_t nclip = 0;
 #pragma unroll
     for (int p = 0; p < NP; ++p) {
-      const int off = p * PGROUP + tid * 8;
+      const int off = p * PSPAN + tid * EPT;
       const int c = c0 + off;
       const bool mine = off < SL;
       unsigned long long* q = ll_out + (size_t)(c >> 3) * wpg;
       if (b == 32) {
         if (mine) {
 #pragma unroll
-          for (int e = 0; e < 8; ++e) {
+          for (int e = 0; e < EPT; ++e) {
             float v = u[p][e];
             if (a.clip_mode != CLIP_NONE && c + e < d) {
               if (v > sc.T) { v = sc.T; ++nclip; }
@@ -612,15 +673,15 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
         }
         continue;
       }
-      uint64_t lo = 0, hi = 0;
+      uint64_t lo = 0, hi = 0;  // this thread's EPT * b code bits
       if (mine && c < d) {
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
+        for (int e = 0; e < EPT; ++e) {
           if (c + e < d) {
             uint32_t code = zero_code;
             if (!degenerate) {
-              code = BITS ? quantize_code<BITS ? BITS : 2>(u[p][e], sc.rdelta, lane16(rnd[p], e))
-                          : quantize_code_rt(u[p][e], sc.rdelta, lane16(rnd[p], e), b);
+              const uint32_t r16 = lane16(rnd[p], e);
+              code = BITS ? quantize_code<BITS ? BITS : 2>(u[p][e], sc.rdelta, r16) : quantize_code_rt(u[p][e], sc.rdelta, r16, b);
               nclip += (u[p][e] > sc.T || u[p][e] < sc.lower) ? 1u : 0u;
             }
             const int pos = e * b;
@@ -633,41 +694,48 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
           }
         }
       }
-      if (mine) {
-        st_word(q, (uint32_t)lo, tag);
-        if (WMAX >= 2 && wpg >= 2) st_word(q + 1, (uint32_t)(lo >> 32), tag);
-        if (WMAX >= 4 && wpg >= 4) {
-          st_word(q + 2, (uint32_t)hi, tag);
-          st_word(q + 3, (uint32_t)(hi >> 32), tag);
+      if constexpr (BITS == 0 || TB >= 32) {
+        // whole words per thread
+        if (mine) {
+          st_word(q + wfirst, (uint32_t)lo, tag);
+          if (NW >= 2 && wpg >= 2) st_word(q + wfirst + 1, (uint32_t)(lo >> 32), tag);
+          if (NW >= 4 && wpg >= 4) {
+            st_word(q + 2, (uint32_t)hi, tag);
+            st_word(q + 3, (uint32_t)(hi >> 32), tag);
+          }
         }
+      } else {
+        // LPW neighbouring lanes hold one word of the group between them (all lanes shuffle; lanes outside the slice hold zeros)
+        constexpr int LPW = (32 / TB < LPG) ? 32 / TB : LPG;
+        uint32_t word = (uint32_t)lo;
+#pragma unroll
+        for (int i = 1; i < LPW; ++i) word |= __shfl_down_sync(0xFFFFFFFFu, (uint32_t)lo, i) << (i * TB);
+        if (mine && (lane & (LPW - 1)) == 0) st_word(q + wfirst, word, tag);
       }
       if (!last) continue;
       // the caller's copy of the last messages: the packed little-endian bit stream
-      if (BITS == 8) {
-        const int64_t w = (int64_t)(c >> 3) * 2;
-        if (mine && w < a.pad_words) *reinterpret_cast<uint2*>(out + w) = make_uint2((uint32_t)lo, (uint32_t)(lo >> 32));
-      } else if (BITS == 4) {
-        const int64_t w = c >> 3;
-        if (mine && w < a.pad_words) out[w] = (uint32_t)lo;
-      } else if (BITS == 2) {
-        const uint32_t own = (uint32_t)lo;
-        const uint32_t next = __shfl_down_sync(0xFFFFFFFFu, own, 1);
-        const int64_t w = c >> 4;
-        if (mine && (lane & 1) == 0 && w < a.pad_words) out[w] = own | (next << 16);
-      } else if (BITS == 1) {
-        const uint32_t own = (uint32_t)lo;
-        const uint32_t n1 = __shfl_down_sync(0xFFFFFFFFu, own, 1);
-        const uint32_t n2 = __shfl_down_sync(0xFFFFFFFFu, own, 2);
-        const uint32_t n3 = __shfl_down_sync(0xFFFFFFFFu, own, 3);
-        const int64_t w = c >> 5;
-        if (mine && (lane & 3) == 0 && w < a.pad_words) out[w] = own | (n1 << 8) | (n2 << 16) | (n3 << 24);
+      if constexpr (BITS != 0) {
+        if constexpr (TB >= 32) {
+          const int64_t w = ((int64_t)c * BITS) >> 5;
+          if (mine && w < a.pad_words) {
+            out[w] = (uint32_t)lo;
+            if (TB == 64) out[w + 1] = (uint32_t)(lo >> 32);  // pad_words is a multiple of 4: w + 1 is inside as well
+          }
+        } else {
+          constexpr int LPS = 32 / TB;  // lanes per word of the stream
+          uint32_t word = (uint32_t)lo;
+#pragma unroll
+          for (int i = 1; i < LPS; ++i) word |= __shfl_down_sync(0xFFFFFFFFu, (uint32_t)lo, i) << (i * TB);
+          const int64_t w = ((int64_t)c * BITS) >> 5;
+          if (mine && (lane & (LPS - 1)) == 0 && w < a.pad_words) out[w] = word;
+        }
       } else {
         if (p > 0) __syncthreads();
         for (int i = 0; i < b; ++i)
           sm.stage[tid * b + i] = (uint8_t)((i < 8) ? (lo >> (8 * i)) : (hi >> (8 * (i - 8))));
         __syncthreads();
-        const int span = min(PGROUP, SL - p * PGROUP);
-        const int64_t w0 = (int64_t)((c0 + p * PGROUP) >> 5) * b;
+        const int span = min(PSPAN, SL - p * PSPAN);
+        const int64_t w0 = (int64_t)((c0 + p * PSPAN) >> 5) * b;
         const uint32_t* st = reinterpret_cast<const uint32_t*>(sm.stage);
         for (int w = tid; w < (span / 32) * b; w += PT)
           if (w0 + w < a.pad_words) out[w0 + w] = st[w];
@@ -685,6 +753,7 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
       }
     }
     LPC_TRACE_MARK(14);
+    sb = sb_next;
   }
 
   // the last step's update, then the slices of the final state go back to memory (worker 0's cluster)
@@ -692,9 +761,9 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
   if (worker == 0) {
 #pragma unroll
     for (int p = 0; p < NP; ++p) {
-      const int off = p * PGROUP + tid * 8;
+      const int off = p * PSPAN + tid * EPT;
 #pragma unroll
-      for (int e = 0; e < 8; ++e) {
+      for (int e = 0; e < EPT; ++e) {
         if (off + e < width) {
           pa.x_out[c0 + off + e] = xr[p][e];  // Algorithm 2: the coupled point of the last step
           if constexpr (ALPC) {
@@ -709,7 +778,6 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
   cluster.sync();  // no CTA leaves while a peer could still address its shared memory
 }
 
-template <int BITS, int NP, bool ALPC>
 void fill_config(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr, int cs, int clusters, size_t smem, cudaStream_t st,
                  bool cooperative) {
   *cfg = cudaLaunchConfig_t{};
@@ -727,65 +795,68 @@ void fill_config(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr, int cs, int
   cfg->numAttrs = cooperative ? 2 : 1;
 }
 
-template <int BITS, int NP, bool ALPC>
-cudaError_t launch_p(const PersistArgs& pa, size_t smem, cudaStream_t st) {
-  cudaError_t e = cudaFuncSetAttribute(persist_kernel<BITS, NP, ALPC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) return e;
-  cudaLaunchConfig_t cfg;
-  cudaLaunchAttribute attr[2];
-  fill_config<BITS, NP, ALPC>(&cfg, attr, pa.in.CS, pa.in.N + (ALPC ? 1 : 0), smem, st, true);
-  return cudaLaunchKernelEx(&cfg, persist_kernel<BITS, NP, ALPC>, pa);
+using PersistKernel = void (*)(PersistArgs);
+
+template <int BITS, bool ALPC>
+PersistKernel pick_shape(int np, int ept) {
+  if (np == 2) return persist_kernel<BITS, 2, 8, ALPC>;
+  if constexpr (BITS != 0) {
+    if (ept == 4) return persist_kernel<BITS, 1, 4, ALPC>;
+    if (ept == 2) return persist_kernel<BITS, 1, 2, ALPC>;
+  }
+  return persist_kernel<BITS, 1, 8, ALPC>;
+}
+template <bool ALPC>
+PersistKernel pick_width(int b, int np, int ept) {
+  switch (b) {
+    case 1: return pick_shape<1, ALPC>(np, ept);
+    case 2: return pick_shape<2, ALPC>(np, ept);
+    case 4: return pick_shape<4, ALPC>(np, ept);
+    case 8: return pick_shape<8, ALPC>(np, ept);
+    default: return pick_shape<0, ALPC>(np, ept);
+  }
+}
+// The instantiation for code width b, slice SL and algorithm.
+PersistKernel pick_kernel(int b, int SL, bool alpc) {
+  const int np = (SL > PGROUP) ? 2 : 1;
+  const int ept = persist_coords_per_thread(b, SL);
+  return alpc ? pick_width<true>(b, np, ept) : pick_width<false>(b, np, ept);
 }
 
-template <int BITS, int NP, bool ALPC>
-int max_clusters_t(int cs, size_t smem) {
-  if (cudaFuncSetAttribute(persist_kernel<BITS, NP, ALPC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+int max_clusters(PersistKernel k, int cs, size_t smem) {
+  if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
     cudaGetLastError();
     return 0;
   }
   cudaLaunchConfig_t cfg;
   cudaLaunchAttribute attr[2];
-  fill_config<BITS, NP, ALPC>(&cfg, attr, cs, 1, smem, nullptr, false);
+  fill_config(&cfg, attr, cs, 1, smem, nullptr, false);
   int n = 0;
-  if (cudaOccupancyMaxActiveClusters(&n, persist_kernel<BITS, NP, ALPC>, &cfg) != cudaSuccess) {
+  if (cudaOccupancyMaxActiveClusters(&n, k, &cfg) != cudaSuccess) {
     cudaGetLastError();
     return 0;
   }
   return n;
 }
 
-template <int NP, bool ALPC>
-int max_clusters_np(int b, int cs, size_t smem) {
-  switch (b) {
-    case 1: return max_clusters_t<1, NP, ALPC>(cs, smem);
-    case 2: return max_clusters_t<2, NP, ALPC>(cs, smem);
-    case 4: return max_clusters_t<4, NP, ALPC>(cs, smem);
-    case 8: return max_clusters_t<8, NP, ALPC>(cs, smem);
-    default: return max_clusters_t<0, NP, ALPC>(cs, smem);
-  }
-}
-
-template <int NP, bool ALPC>
-cudaError_t launch_np(const PersistArgs& pa, size_t smem, cudaStream_t st) {
-  switch (pa.in.b) {
-    case 1: return launch_p<1, NP, ALPC>(pa, smem, st);
-    case 2: return launch_p<2, NP, ALPC>(pa, smem, st);
-    case 4: return launch_p<4, NP, ALPC>(pa, smem, st);
-    case 8: return launch_p<8, NP, ALPC>(pa, smem, st);
-    default: return launch_p<0, NP, ALPC>(pa, smem, st);
-  }
-}
-
 }  // namespace
+
+// Coordinates a thread owns per pass: a slice of PT * 8 or more gives every thread a whole group of 8; narrower
+// slices are spread over all threads of the CTA, 4 or 2 coordinates each (fixed code widths only).
+int persist_coords_per_thread(int b, int SL) {
+  const bool fixed = (b == 1 || b == 2 || b == 4 || b == 8);
+  if (!fixed || SL >= PT * 8) return 8;
+  return (SL >= PT * 4) ? 4 : 2;
+}
 
 // Cluster size, slice and row buffering for the persistent loop.  All clusters (N, plus one for the shared
 // batch J in Algorithm 2) must be co-resident -- the occupancy query says how many clusters of a given size the
-// device can hold -- and the row slices must fit in shared memory, double-buffered when possible (rows of the
-// next step are fetched while this one computes), single-buffered otherwise (they are fetched as soon as u is
-// formed).  Among the sizes that fit, the largest cluster whose slices still keep a CTA busy wins: more CTAs per
-// worker shorten every serial phase of a step.
+// device can hold -- and the B row slices of a step must fit in shared memory; with room for 2B slices the rows of
+// the next step are fetched while this one computes, with less the part that fits is fetched then and the rest as
+// soon as u is formed.  Among the sizes that fit, the largest cluster whose slices still keep a CTA busy wins: more
+// CTAs per worker shorten every serial phase of a step.
 bool persist_plan(int d, int N, int B, int b, int alpc, int want_cs, int max_smem, int* CS_out, int* SL_out,
-                  size_t* smem_out, int* nbuf_out) {
+                  size_t* smem_out, int* row_slots_out) {
   int P = 1;
   while (P < d) P <<= 1;
   if (P < 32) P = 32;
@@ -799,21 +870,28 @@ bool persist_plan(int d, int N, int B, int b, int alpc, int want_cs, int max_sme
     if (SL > PGROUP * PMAXP) continue;
     if (clusters * cs > PMAXFLAGS) break;
     const size_t fixed = (sizeof(PSmem) + 15) & ~(size_t)15;
-    const size_t one = (size_t)B * SL * 4;
-    int nbuf = 2;
-    if (fixed + 2 * one > (size_t)max_smem) nbuf = 1;
-    if (fixed + nbuf * one > (size_t)max_smem) continue;
-    const size_t smem = fixed + nbuf * one;
-    int fit;
-    if (alpc) fit = (SL > PGROUP) ? max_clusters_np<2, true>(b, cs, smem) : max_clusters_np<1, true>(b, cs, smem);
-    else fit = (SL > PGROUP) ? max_clusters_np<2, false>(b, cs, smem) : max_clusters_np<1, false>(b, cs, smem);
-    if (fit < clusters) continue;
-    *CS_out = cs; *SL_out = SL; *smem_out = smem; *nbuf_out = nbuf;
+    const size_t one = (size_t)SL * 4;  // one row slot
+    if (fixed + (size_t)B * one > (size_t)max_smem) continue;
+    int slots = (int)(((size_t)max_smem - fixed) / one);
+    if (slots > 2 * B) slots = 2 * B;
+    const size_t smem = fixed + (size_t)slots * one;
+    if (max_clusters(pick_kernel(b, SL, alpc != 0), cs, smem) < clusters) continue;
+    *CS_out = cs; *SL_out = SL; *smem_out = smem; *row_slots_out = slots;
     found = true;
     if (want_cs > 0) break;
     if (SL <= 512) break;  // slices below 512 coordinates leave most of a CTA idle
   }
   return found;
+}
+
+cudaError_t launch_persist(const PersistArgs& pa, size_t smem, cudaStream_t st) {
+  PersistKernel k = pick_kernel(pa.in.b, pa.in.SL, pa.alpc != 0);
+  cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  cudaLaunchConfig_t cfg;
+  cudaLaunchAttribute attr[2];
+  fill_config(&cfg, attr, pa.in.CS, pa.in.N + (pa.alpc ? 1 : 0), smem, st, true);
+  return cudaLaunchKernelEx(&cfg, k, pa);
 }
 
 namespace {
@@ -841,11 +919,6 @@ cudaError_t launch_wait_timeout(const unsigned long long* word, unsigned int* ab
                                 uint64_t limit_ns, cudaStream_t st) {
   wait_timeout_kernel<<<1, 64, 0, st>>>(word, abort_flag, dev_status, limit_ns);
   return cudaGetLastError();
-}
-
-cudaError_t launch_persist(const PersistArgs& pa, size_t smem, cudaStream_t st) {
-  if (pa.alpc) return (pa.in.SL > PGROUP) ? launch_np<2, true>(pa, smem, st) : launch_np<1, true>(pa, smem, st);
-  return (pa.in.SL > PGROUP) ? launch_np<2, false>(pa, smem, st) : launch_np<1, false>(pa, smem, st);
 }
 
 #ifdef LPC_TRACE

@@ -22,8 +22,8 @@ OPT_SAMPLE_GLOBAL, OPT_TAP_U, OPT_CLUSTER_SIZE, OPT_USE_GRAPH, OPT_PROFILE, OPT_
 OPT_SHARED_SCALE, OPT_AVERAGE_DIVISOR = 6, 7
 SCHEME_BROADCAST, SCHEME_SERVER_SUM, SCHEME_SERVER_REQUANTIZE = 0, 1, 2
 (INFO_STEP_CLUSTER_SIZE, INFO_LOOP_CLUSTER_SIZE, INFO_LOOP_LAUNCHES, INFO_SNAPSHOT_ROWS_PER_TILE, INFO_SNAPSHOT_STAGES,
- INFO_ALPC_LOOP_CLUSTER_SIZE, INFO_LOOP_ROW_BUFFERS, INFO_ALPC_LOOP_ROW_BUFFERS, INFO_STEP_RING_STAGES,
- INFO_AGGREGATE_SPLIT, INFO_QUANT_PIPELINED_RUNS) = range(11)
+ INFO_ALPC_LOOP_CLUSTER_SIZE, INFO_LOOP_ROW_SLOTS, INFO_ALPC_LOOP_ROW_SLOTS, INFO_STEP_RING_STAGES,
+ INFO_AGGREGATE_SPLIT, INFO_QUANT_PIPELINED_RUNS, INFO_LOOP_COORDS_PER_THREAD, INFO_ALPC_LOOP_COORDS_PER_THREAD) = range(13)
 KERNEL_NAMES = ["snapshot", "worker", "aggregate", "quant_stats", "quant_pack", "other", "inner_loop"]
 
 # every symbol that include/lpc.h declares: (name, restype, argtypes)
