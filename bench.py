@@ -220,12 +220,26 @@ def run_ours(args):
             pair = kernels["worker"]["avg_us"] + kernels["aggregate"]["avg_us"]
             dur_us = inner_ms * 1e3 / m * kd["avg_us"] / pair
         ach = kd["bytes_per_launch"] / dur_us * 1e-3
+        traffic, traffic_src = None, None
+        if dominant == "inner_loop":
+            # profilers cannot replay the cooperative launch; the per-step worker kernel, which moves the same rows, was
+            # captured instead: its DRAM bytes per step times the steps of one launch
+            traffic, traffic_src = traffic_of("inner_kernel<4> (per step)", m)
+            traffic_src = "taken on the per-step kernels (the one-launch loop cannot be replayed by the profiler): " + traffic_src
+        elif dominant == "snapshot":
+            traffic, traffic_src = traffic_of("snapshot_kernel", n * d)
         roofline = {"bound": "hbm", "kernel": dominant, "achieved": round(ach, 1), "peak": peak, "unit": "GB/s",
-                    "frac": round(ach / peak, 4), "traffic": None, "peak_source": f"of {peak_kind}",
+                    "frac": round(ach / peak, 4), "frac_of_nominal_8TBs": round(ach / NOMINAL_HBM_GBS, 4),
+                    "traffic": traffic, "traffic_source": traffic_src, "peak_source": f"of {peak_kind}",
                     "launch_us": round(dur_us, 3),
                     "note": "latency-bound: an inner step moves %.2f MB behind a strict step-to-step dependency; "
-                            "see kernels{} and quantize_aggregate{} for the bandwidth-bound kernels"
-                            % ((bpl["worker"] + bpl["aggregate"]) / 1e6)}
+                            "kernels[] lists the bandwidth-bound kernels of the path, each with its workload"
+                            % ((bpl["worker"] + bpl["aggregate"]) / 1e6),
+                    "kernels": []}
+        if "snapshot" in kernels:
+            ks = kernels["snapshot"]
+            roofline["kernels"].append(roofline_entry("snapshot_kernel", args.workload, ks["avg_us"], ks["bytes_per_launch"], peak,
+                                                      "snapshot_kernel", n * d))
     launches_per_epoch = 2 + sum(kernels[k]["launches_per_step"] for k in kernels if k != "snapshot")
 
     out = {
@@ -243,20 +257,29 @@ def run_ours(args):
         "inner_step_us": round(inner_ms * 1e3 / m, 3), "wall_s": round(t_wall, 4), "objective_end": P_end,
         "roofline": roofline, "kernels": kernels,
         "launch_plan": {"loop_cluster_size": ctx.query(lpc.INFO_LOOP_CLUSTER_SIZE),
+                        "loop_coords_per_thread": ctx.query(lpc.INFO_LOOP_COORDS_PER_THREAD),
+                        "loop_row_slots": ctx.query(lpc.INFO_LOOP_ROW_SLOTS),
                         "loop_launches": ctx.query(lpc.INFO_LOOP_LAUNCHES),
                         "step_cluster_size": ctx.query(lpc.INFO_STEP_CLUSTER_SIZE),
                         "snapshot_rows_per_tile": ctx.query(lpc.INFO_SNAPSHOT_ROWS_PER_TILE),
                         "snapshot_stages": ctx.query(lpc.INFO_SNAPSHOT_STAGES)},
     }
     if rank == 0 and size == 1 and not args.quick:
-        out["quantize_aggregate"] = quantize_aggregate_bench(dev, peak)
         out["e2e"] = e2e_bench(w, X, y, m, eta, dev)
         out["cpu_baseline"] = cpu_baseline(w, X, y, m, eta)
         del X, y
         ctx.close()
         torch.cuda.empty_cache()
-        out["alpc"] = alpc_bench(dev)
+        out["tiny_logistic"] = tiny_logistic_bench(dev)
+        qa = quantize_aggregate_bench(dev, peak)
+        roofline["kernels"] += qa.pop("roofline_kernels")
+        out["quantize_aggregate"] = qa
+        torch.cuda.empty_cache()
+        out["alpc"] = alpc_bench(dev, peak)
+        roofline["kernels"] += out["alpc"].pop("roofline_kernels")
+        torch.cuda.empty_cache()
         out["fused_large_batch"] = fused_large_batch_bench(dev, peak)
+        roofline["kernels"] += out["fused_large_batch"].pop("roofline_kernels")
     elif rank == 0:
         out["e2e"] = None
     ctx.close()
@@ -264,6 +287,43 @@ def run_ours(args):
     if rank == 0:
         print(json.dumps(out))
     dist_util.shutdown()
+
+
+NOMINAL_HBM_GBS = 8000.0   # the vendor's round figure for the part's HBM3e, for context beside the measured copy rate
+L2_BYTES = 126e6
+
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch, from the ncu captures summarised under
+# profiles/: (bytes, units of that capture, summary file).  The captures are of smaller cases than the bench times
+# (a few hundred MB, as profiler captures must be); traffic grows in proportion to the units a launch processes, so it
+# is scaled by them.  An entry goes away when its kernel changes.
+TRAFFIC = {
+    "snapshot_kernel": (268.56e6 + 4.02e6, 16384 * 4096, "profiles/snapshot_kernel_ls_16384x4096.md"),
+    "stats_kernel": (536.95e6 + 4.10e6, 8 * (1 << 24), "profiles/quantize_aggregate_N8_len2p24_b4.md"),
+    "quantize_kernel<4>": (536.96e6 + 14.64e6, 8 * (1 << 24), "profiles/quantize_aggregate_N8_len2p24_b4.md"),
+    "unpack_average_prox_kernel<4>": (134.25e6 + 25.62e6, 1 << 24, "profiles/quantize_aggregate_N8_len2p24_b4.md"),
+    "inner_kernel<4> (per step)": (2.218e6, 1, "profiles/inner_step_kernels_ls_16384x4096_N16_B8_b4.md"),
+    "inner_kernel<2, stream>": (234.0e6 + 4.6e6, 32 * 256, "profiles/streaming_worker_kernel_logistic_16384x8192_N32_B256_b2.md"),
+}
+
+
+def traffic_of(name, units):
+    if name not in TRAFFIC:
+        return None, None
+    bytes_, cap_units, src = TRAFFIC[name]
+    return round(bytes_ * units / cap_units), "%s, scaled by %g" % (src, units / cap_units)
+
+
+def roofline_entry(kernel, workload, avg_us, alg_bytes, peak, traffic_name=None, units=None, note=None):
+    gbs = alg_bytes / avg_us * 1e-3
+    tr, src = traffic_of(traffic_name, units) if traffic_name else (None, None)
+    e = {"kernel": kernel, "workload": workload, "avg_us": round(avg_us, 3), "algorithmic_bytes": int(alg_bytes),
+         "gbs": round(gbs, 1), "frac": round(gbs / peak, 4), "frac_of_nominal_8TBs": round(gbs / NOMINAL_HBM_GBS, 4),
+         "traffic": tr}
+    if src:
+        e["traffic_source"] = src
+    if note:
+        e["note"] = note
+    return e
 
 
 def _time_calls(fn, dev, reps):
@@ -281,123 +341,173 @@ def _time_calls(fn, dev, reps):
     return a.elapsed_time(b) / reps
 
 
-def quantize_aggregate_bench(dev, peak, log2_len=26, dnn=True):
-    """Stand-alone quantize+pack and unpack+average+prox at sizes where one call is bandwidth-bound."""
+def _kernel_ms(ctx, fn, reps, kinds):
+    """Average device time per call of `fn`, summed over the kernel classes `kinds`, from the library's own event pair
+    around every launch (the Python wrapper costs more than the short kernels)."""
+    from paper_1901_08924_b200 import lpc
+    for i in range(2):
+        fn(i)
+    ctx.sync_status()
+    ctx.set_option(lpc.OPT_PROFILE, 1)
+    ctx.get_profile(reset=True)
+    for i in range(reps):
+        fn(2 + i)
+    ctx.sync_status()
+    pr = ctx.get_profile(reset=True)
+    ctx.set_option(lpc.OPT_PROFILE, 0)
+    return {k: pr.get(k, (0.0, 0))[0] / reps for k in kinds}
+
+
+def qa_point(dev, peak, U, b, clip, reps=5):
+    """Stand-alone quantize+pack then unpack+average+prox on the N vectors U (clip c*std, lambda_l1 = 1e-3, eta = 1).
+    Output buffers rotate over enough sets to exceed L2, so that no call finds its own previous output there; inputs
+    of at most half of L2 are reported as L2-resident, with the one-read bound of 4 + b/8 bytes per element."""
+    import torch
+    from paper_1901_08924_b200 import lpc
+    N, ln = U.shape
+    q = lpc.Context(None, None, lpc.LOGISTIC, 0.0, N, 1, b, lpc.CLIP_STD, clip, 0)
+    _, stride = lpc.packed_layout(ln, b)
+    out_bytes = N * stride * 4 + ln * 4
+    nsets = int(max(1, min(8, -(-2 * L2_BYTES // out_bytes))))
+    codes = [torch.empty((N, stride), dtype=torch.int32, device=dev) for _ in range(nsets)]
+    xs = [torch.zeros(ln, device=dev) for _ in range(nsets)]
+    delta = torch.empty((N, 1), dtype=torch.float32, device=dev)
+    clipped = torch.empty((N, 1), dtype=torch.int32, device=dev)
+    resident = N * ln * 4 <= L2_BYTES / 2
+    tq = _kernel_ms(q, lambda i: q.quantize_pack(U, i, codes_out=codes[i % nsets], delta_out=delta, clipped_out=clipped),
+                    reps, ("quant_stats", "other", "quant_pack", "quant_fused"))
+    for c in codes[1:]:  # every set holds valid codes before the aggregator is timed
+        c.copy_(codes[0])
+    ta = _kernel_ms(q, lambda i: q.unpack_average_prox(codes[i % nsets], delta, ln, xs[i % nsets], 1.0, 1e-3),
+                    2 * reps, ("aggregate",))["aggregate"]
+    q.close()
+    bq = N * ln * ((4 if resident else 8) + b / 8)
+    ba = ln * (N * b / 8 + 12)
+    tq_all = sum(tq.values())
+    return {"N": N, "len": ln, "b": b, "clip_std": clip, "l2_resident_input": resident, "output_sets": nsets,
+            "quantize_pack": {"ms": round(tq_all, 5), "stats_ms": round(tq["quant_stats"], 5), "scale_ms": round(tq["other"], 5),
+                              "pack_ms": round(tq["quant_pack"], 5), "one_launch_ms": round(tq["quant_fused"], 5),
+                              "bytes": bq, "gbs": round(bq / tq_all * 1e-6, 1),
+                              "frac": round(bq / tq_all * 1e-6 / peak, 4), "frac_of_nominal_8TBs": round(bq / tq_all * 1e-6 / NOMINAL_HBM_GBS, 4)},
+            "unpack_average_prox": {"ms": round(ta, 5), "bytes": ba, "gbs": round(ba / ta * 1e-6, 1), "frac": round(ba / ta * 1e-6 / peak, 4),
+                                    "frac_of_nominal_8TBs": round(ba / ta * 1e-6 / NOMINAL_HBM_GBS, 4)},
+            "combined_gbs": round((bq + ba) / (tq_all + ta) * 1e-6, 1)}
+
+
+def quantize_aggregate_bench(dev, peak, log2_len=26, full=True):
+    """The quantizer/aggregator sweep: N = 8 worker vectors, lengths 2^16 .. 2^28, Gaussian and Student-t (3 degrees of
+    freedom) values, b in {1, 2, 3, 4, 8}, clip in {1, 2, 4} std; then the entropy count, the parameter-server schemes
+    and the 62-tensor layer-wise shape.  Kernel times are the library's own event pairs around each launch."""
     import torch
     from paper_1901_08924_b200 import lpc, synth
-    res = {}
-    # sweep point: 8 workers x 2^26 coordinates (2.1 GB of gradients), Gaussian, b = 4, clip 2 std
-    N, length, b = 8, 1 << log2_len, 4
-    U = synth.gradient_vectors(N, length, "gauss", seed=1, device=dev)
+    res, roof = {}, []
+    N = 8
+    top = 28 if full else log2_len
+    U = synth.gradient_vectors(N, 1 << top, "gauss", seed=1, device=dev)
+    grid = {}
+
+    def point(name, Uv, b, clip, reps=5):
+        r = qa_point(dev, peak, Uv, b, clip, reps)
+        grid[name] = r
+        return r
+
+    lens = [l for l in (16, 20, 24, 26, 28) if l <= top]
+    for l2 in lens:
+        r = point("gauss_len2^%d_b4_clip2" % l2, U[:, : 1 << l2], 4, 2.0, reps=10 if l2 <= 24 else 4)
+        wl = "sweep N=8, len 2^%d, N(0,1), b=4, clip 2 std" % l2
+        qp, ua = r["quantize_pack"], r["unpack_average_prox"]
+        roof.append(roofline_entry("quantize+pack (stats_kernel + finish_kernel + quantize_kernel<4>)", wl, qp["ms"] * 1e3, qp["bytes"], peak,
+                                   note="L2-resident input: bound 4 + b/8 B per element" if r["l2_resident_input"] else
+                                   "two passes: 8 + b/8 B per element"))
+        if not r["l2_resident_input"] and qp["stats_ms"] > 0:
+            roof.append(roofline_entry("stats_kernel", wl, qp["stats_ms"] * 1e3, N * (1 << l2) * 4, peak, "stats_kernel", N * (1 << l2)))
+            roof.append(roofline_entry("quantize_kernel<4>", wl, qp["pack_ms"] * 1e3, N * (1 << l2) * 4.5, peak, "quantize_kernel<4>", N * (1 << l2)))
+        roof.append(roofline_entry("unpack_average_prox_kernel<4>", wl, ua["ms"] * 1e3, ua["bytes"], peak,
+                                   "unpack_average_prox_kernel<4>", 1 << l2))
+    mid = min(26, top)
+    Um = U[:, : 1 << mid]
+    for b in (1, 2, 3, 8):
+        r = point("gauss_len2^%d_b%d_clip2" % (mid, b), Um, b, 2.0)
+        wl = "sweep N=8, len 2^%d, N(0,1), b=%d, clip 2 std" % (mid, b)
+        roof.append(roofline_entry("quantize+pack, b=%d" % b, wl, r["quantize_pack"]["ms"] * 1e3, r["quantize_pack"]["bytes"], peak))
+        roof.append(roofline_entry("unpack_average_prox_kernel, b=%d" % b, wl, r["unpack_average_prox"]["ms"] * 1e3,
+                                   r["unpack_average_prox"]["bytes"], peak))
+    if full:
+        for clip in (1.0, 4.0):
+            point("gauss_len2^%d_b4_clip%g" % (mid, clip), Um, 4, clip)
+        del Um
+        Ut = synth.gradient_vectors(N, 1 << mid, "student_t3", seed=2, device=dev)
+        for clip in (1.0, 2.0, 4.0):
+            point("student_t3_len2^%d_b4_clip%g" % (mid, clip), Ut, 4, clip)
+        del Ut
+    res["sweep_grid_N8"] = grid
+    # ---- entropy count and the parameter-server schemes on 8 x 2^mid Gaussian vectors, b = 4, clip 2 std
+    length, b = 1 << mid, 4
+    Um = U[:, :length]
     q = lpc.Context(None, None, lpc.LOGISTIC, 0.0, N, 1, b, lpc.CLIP_STD, 2.0, 0)
     _, stride = lpc.packed_layout(length, b)
     codes = torch.empty((N, stride), dtype=torch.int32, device=dev)
     delta = torch.empty((N, 1), dtype=torch.float32, device=dev)
     clipped = torch.empty((N, 1), dtype=torch.int32, device=dev)
     x = torch.zeros(length, device=dev)
-    it = [0]
-
-    def quant():
-        it[0] += 1
-        q.quantize_pack(U, it[0], codes_out=codes, delta_out=delta, clipped_out=clipped)
-
-    def agg():
-        q.unpack_average_prox(codes, delta, length, x, 1.0, 1e-3)
-
-    tq, ta = _time_calls(quant, dev, 5), _time_calls(agg, dev, 10)
-    q.sync_status()
-    bq, ba = N * length * (8 + b / 8), length * (N * b / 8 + 12)
-    res["sweep_N8_len2^%d_b4" % log2_len] = {
-        "quantize_pack": {"ms": round(tq, 4), "bytes": bq, "gbs": round(bq / tq * 1e-6, 1), "frac": round(bq / tq * 1e-6 / peak, 4),
-                          "note": "two passes: 4 B stats read + 4 B quantize read + b/8 B written per element"},
-        "unpack_average_prox": {"ms": round(ta, 4), "bytes": ba, "gbs": round(ba / ta * 1e-6, 1), "frac": round(ba / ta * 1e-6 / peak, 4)},
-        "combined_gbs": round((bq + ba) / (tq + ta) * 1e-6, 1)}
-    # the other code widths and vector lengths of the sweep (same vectors, prefixes for the shorter lengths)
-    grid = {}
-    for bb, ll in [(1, log2_len), (2, log2_len), (8, log2_len)] + [(4, l2) for l2 in (16, 20, 24) if l2 < log2_len]:
-        ln = 1 << ll
-        qq = lpc.Context(None, None, lpc.LOGISTIC, 0.0, N, 1, bb, lpc.CLIP_STD, 2.0, 0)
-        _, st2 = lpc.packed_layout(ln, bb)
-        c2 = torch.empty((N, st2), dtype=torch.int32, device=dev)
-        Uv = U[:, :ln]
-        x2 = torch.zeros(ln, device=dev)
-        t1 = _time_calls(lambda: qq.quantize_pack(Uv, 1, codes_out=c2, delta_out=delta, clipped_out=clipped), dev, 5)
-        t2 = _time_calls(lambda: qq.unpack_average_prox(c2, delta, ln, x2, 1.0, 1e-3), dev, 10)
-        qq.sync_status()
-        qq.close()
-        b1, b2 = N * ln * (8 + bb / 8), ln * (N * bb / 8 + 12)
-        grid["b%d_len2^%d" % (bb, ll)] = {"quantize_pack_ms": round(t1, 4), "quantize_pack_frac": round(b1 / t1 * 1e-6 / peak, 4),
-                                          "unpack_average_prox_ms": round(t2, 4), "unpack_average_prox_frac": round(b2 / t2 * 1e-6 / peak, 4)}
-        del c2, x2
-    res["sweep_grid_N8"] = grid
-    # entropy-coding count of the messages just packed: histogram kernel (event-timed) and the host sums
+    q.quantize_pack(Um, 1, codes_out=codes, delta_out=delta, clipped_out=clipped)
     hist = torch.empty((N, 1, 1 << b), dtype=torch.int64, device=dev)
-    q.set_option(lpc.OPT_PROFILE, 1)
-    q.get_profile(reset=True)
-    for _ in range(10):
-        q.message_entropy(codes, length, hist_out=hist, host_counts=False)
-    q.sync_status()
-    pr = q.get_profile(reset=True)
-    q.set_option(lpc.OPT_PROFILE, 0)
-    th = pr["other"][0] / pr["other"][1]
+    th = _kernel_ms(q, lambda i: q.message_entropy(codes, length, hist_out=hist, host_counts=False), 10, ("other",))["other"]
     _, ent, huf = q.message_entropy(codes, length, hist_out=hist)
     bh = N * length * b / 8
-    res["entropy_count_N8_len2^%d_b4" % log2_len] = {
+    res["entropy_count_N8_len2^%d_b4" % mid] = {
         "histogram": {"ms": round(th, 4), "bytes": bh, "gbs": round(bh / th * 1e-6, 1), "frac": round(bh / th * 1e-6 / peak, 4)},
         "bits_per_coordinate": {"raw": b, "entropy_bound": round(float(ent.mean()) / length, 4),
                                 "huffman": round(float(huf.astype("float64").mean()) / length, 4)}}
-    # the parameter-server schemes (b) and (c) on the same vectors: unified scale, server, worker-side decode
+    roof.append(roofline_entry("code_histogram_kernel<4>", "8 x 2^%d 4-bit codes" % mid, th * 1e3, bh, peak))
     q.set_option(lpc.OPT_SHARED_SCALE, 1)
-    tqs = _time_calls(quant, dev, 5)
+    tqs = _kernel_ms(q, lambda i: q.quantize_pack(Um, i, codes_out=codes, delta_out=delta, clipped_out=clipped), 4,
+                     ("quant_stats", "other", "quant_pack", "quant_fused"))
+    tqs = sum(tqs.values())
+    bq = N * length * (8 + b / 8)
     ps = {"quantize_pack_unified_scale": {"ms": round(tqs, 4), "gbs": round(bq / tqs * 1e-6, 1), "frac": round(bq / tqs * 1e-6 / peak, 4)}}
     for name, scheme in (("scheme_b_sum", lpc.SCHEME_SERVER_SUM), ("scheme_c_requantize", lpc.SCHEME_SERVER_REQUANTIZE)):
         srv, bo = q.server_reduce(codes, length, scheme, 1)
-        # the library's own event pair around the launch: the Python wrapper costs more than this short kernel
-        q.set_option(lpc.OPT_PROFILE, 1)
-        q.get_profile(reset=True)
-        for _ in range(10):
-            q.server_reduce(codes, length, scheme, 1, codes_out=srv)
-        q.sync_status()
-        pr = q.get_profile(reset=True)
-        q.set_option(lpc.OPT_PROFILE, 0)
-        ts = pr["aggregate"][0] / pr["aggregate"][1]
+        ts = _kernel_ms(q, lambda i: q.server_reduce(codes, length, scheme, 1, codes_out=srv), 10, ("aggregate",))["aggregate"]
         w = lpc.Context(None, None, lpc.LOGISTIC, 0.0, 1, 1, bo, lpc.CLIP_NONE, 1.0, 0)
         if scheme == lpc.SCHEME_SERVER_SUM:
             w.set_option(lpc.OPT_AVERAGE_DIVISOR, N)
         d1 = delta[:1].contiguous()
-        tw = _time_calls(lambda: w.unpack_average_prox(srv, d1, length, x, 1.0, 1e-3), dev, 10)
-        w.sync_status()
+        x2 = [x, torch.zeros(length, device=dev)]  # two iterates in turn: none finds its own last output in L2
+        tw = _kernel_ms(w, lambda i: w.unpack_average_prox(srv, d1, length, x2[i % 2], 1.0, 1e-3), 10, ("aggregate",))["aggregate"]
         w.close()
         bs, bw = length * (N * b / 8 + bo / 8), length * (bo / 8 + 12)
         ps[name] = {"bits_back": bo,
                     "server": {"ms": round(ts, 4), "bytes": bs, "gbs": round(bs / ts * 1e-6, 1), "frac": round(bs / ts * 1e-6 / peak, 4)},
                     "worker_decode_prox": {"ms": round(tw, 4), "bytes": bw, "gbs": round(bw / tw * 1e-6, 1),
                                            "frac": round(bw / tw * 1e-6 / peak, 4)}}
+        roof.append(roofline_entry("server_reduce_kernel<4> (%s)" % name, "8 x 2^%d 4-bit codes in, %d-bit stream out" % (mid, bo),
+                                   ts * 1e3, bs, peak))
+        del x2
     q.sync_status()
-    res["parameter_server_N8_len2^%d_b4" % log2_len] = ps
+    res["parameter_server_N8_len2^%d_b4" % mid] = ps
     q.close()
-    del U, codes, x
-    if not dnn:
+    del U, Um, codes, x
+    torch.cuda.empty_cache()
+    if not full:
+        res["roofline_kernels"] = roof
         return res
-    # layer-wise DNN-shaped aggregation: 62 tensors, 11.7M parameters, 16 workers, b = 4, clip 2.5 std per tensor
+    # ---- layer-wise DNN-shaped aggregation: 62 tensors, 11.7M parameters, 16 workers, b = 4, clip 2.5 std per tensor
     N, b = 16, 4
     cur, snap, mu, offs = synth.dnn_gradients(N, seed=2, device=dev)
     total = offs[-1]
     q = lpc.Context(None, None, lpc.LOGISTIC, 0.0, N, 1, b, lpc.CLIP_STD, 2.5, 0)
     _, stride = lpc.packed_layout(total, b, offs)
-    codes = torch.empty((N, stride), dtype=torch.int32, device=dev)
+    codes = [torch.empty((N, stride), dtype=torch.int32, device=dev) for _ in range(2)]
     delta = torch.empty((N, len(offs) - 1), dtype=torch.float32, device=dev)
     clipped = torch.empty((N, len(offs) - 1), dtype=torch.int32, device=dev)
-    x = torch.zeros(total, device=dev)
-
-    def quant2():
-        it[0] += 1
-        q.quantize_pack(cur, it[0], U_sub=snap, seg_offsets=offs, codes_out=codes, delta_out=delta, clipped_out=clipped)
-
-    def agg2():
-        q.unpack_average_prox(codes, delta, total, x, 0.1, 0.0, mu=mu, seg_offsets=offs)
-
-    tq, ta = _time_calls(quant2, dev, 10), _time_calls(agg2, dev, 20)
+    xs = [torch.zeros(total, device=dev) for _ in range(4)]
+    tq = _kernel_ms(q, lambda i: q.quantize_pack(cur, i, U_sub=snap, seg_offsets=offs, codes_out=codes[i % 2], delta_out=delta,
+                                                 clipped_out=clipped), 10, ("quant_stats", "other", "quant_pack", "quant_fused"))
+    tq = sum(tq.values())
+    codes[1].copy_(codes[0])
+    ta = _kernel_ms(q, lambda i: q.unpack_average_prox(codes[i % 2], delta, total, xs[i % 4], 0.1, 0.0, mu=mu, seg_offsets=offs), 20,
+                    ("aggregate",))["aggregate"]
     q.sync_status()
     bq, ba = N * total * (16 + b / 8), total * (N * b / 8 + 16)  # aggregate: codes + mu + x read + x write
     res["dnn_62_tensors_N16_b4"] = {
@@ -405,8 +515,42 @@ def quantize_aggregate_bench(dev, peak, log2_len=26, dnn=True):
                           "note": "u = cur - snap formed on the fly: 2 x 8 B read + b/8 B written per element"},
         "unpack_average_prox": {"ms": round(ta, 4), "bytes": ba, "gbs": round(ba / ta * 1e-6, 1), "frac": round(ba / ta * 1e-6 / peak, 4)},
         "combined_gbs": round((bq + ba) / (tq + ta) * 1e-6, 1)}
+    wl = "62 tensors of an 18-layer residual network, 11.7M parameters, N=16, b=4, clip 2.5 std per tensor"
+    roof.append(roofline_entry("quantize+pack with u = cur - snap (3 launches)", wl, tq * 1e3, bq, peak))
+    roof.append(roofline_entry("unpack_average_prox_kernel<4> (+ mu)", wl, ta * 1e3, ba, peak))
     q.close()
+    res["roofline_kernels"] = roof
     return res
+
+
+def tiny_logistic_bench(dev):
+    """The small logistic workload (4,000 x 1,000, N = 4, B = 1, b = 2, clip 2.5 std, eta = 0.1): one epoch of m = 1,000
+    inner steps after the snapshot pass, value only."""
+    import torch
+    from paper_1901_08924_b200 import lpc
+    w = WORKLOADS["lpc_svrg_logistic_4000x1000_N4_B1_b2"]
+    X, y, m, eta = make_problem(w, seed=0, device=dev)
+    ctx = lpc.Context(X, y, loss_code(w), w["lam"], w["N"], w["B"], w["b"], lpc.CLIP_STD, w["c"], 0)
+    st = torch.cuda.current_stream(dev)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    p0 = ctx.objective()
+    for s in range(3):
+        ctx.snapshot_full_grad()
+        ctx.inner_steps(eta, s * m, m)
+    ctx.sync_status()
+    ev[0].record(st)
+    for s in range(3, 8):
+        ctx.snapshot_full_grad()
+        ctx.inner_steps(eta, s * m, m)
+    ev[1].record(st)
+    ctx.sync_status()
+    ms = ev[0].elapsed_time(ev[1]) / 5
+    out = {"workload": "lpc_svrg_logistic_4000x1000_N4_B1_b2", "iters_per_s": round(m / (ms * 1e-3), 1), "epoch_ms": round(ms, 4),
+           "step_us": round(ms * 1e3 / m, 3), "objective_start": p0, "objective_after_8_epochs": ctx.objective(),
+           "loop_cluster_size": ctx.query(lpc.INFO_LOOP_CLUSTER_SIZE),
+           "loop_coords_per_thread": ctx.query(lpc.INFO_LOOP_COORDS_PER_THREAD)}
+    ctx.close()
+    return out
 
 
 def fused_large_batch_bench(dev, peak, n=65536, steps=30):
@@ -420,7 +564,7 @@ def fused_large_batch_bench(dev, peak, n=65536, steps=30):
     d, N = 8192, 32
     X, y, _ = synth.linear_problem(n, d, loss="logistic", sparsity=0.02, noise=0.1, seed=1, col_scale_range=(0.1, 10.0),
                                    device=dev)
-    out = {"workload": "fused_step_logistic_%dx8192_N32" % n}
+    out = {"workload": "fused_step_logistic_%dx8192_N32" % n, "roofline_kernels": []}
     for B, bits in ((256, (2, 8)), (1024, (2,))):
         if N * B > n:  # a small matrix for profiler captures: the larger minibatch does not fit its row partitions
             continue
@@ -439,11 +583,15 @@ def fused_large_batch_bench(dev, peak, n=65536, steps=30):
                                        "worker_gbs": round(bw / tw * 1e-6, 1), "worker_frac": round(bw / tw * 1e-6 / peak, 4),
                                        "aggregate_us": round(ta * 1e3, 2), "ring_stages": ctx.query(lpc.INFO_STEP_RING_STAGES),
                                        "cluster_size": ctx.query(lpc.INFO_STEP_CLUSTER_SIZE)}
+            out["roofline_kernels"].append(roofline_entry(
+                "inner_kernel<%d, stream> (fused sampling + SVRG difference + scale + quantize + pack)" % b,
+                "logistic %d x 8192, N=32 workers, B=%d rows per worker, b=%d" % (n, B, b), tw * 1e3, bw, peak,
+                "inner_kernel<2, stream>" if b == 2 else None, N * B))
             ctx.close()
     return out
 
 
-def alpc_bench(dev):
+def alpc_bench(dev, peak):
     """ALPC-SVRG (Algorithms 2/3) on the ill-conditioned logistic workload: 262,144 x 8,192, N = 32, B = 16,
     clip 2 std, b in {2, 8}; one epoch = snapshot pass + m = n/(B N) = 512 double-sampling steps."""
     import torch
@@ -453,7 +601,7 @@ def alpc_bench(dev):
                                    device=dev)
     L = 0.25 * float((X * X).sum(dim=1).max().item())
     m = n // (B * N)
-    out = {"workload": "alpc_svrg_logistic_262144x8192_N32_B16", "m": m}
+    out = {"workload": "alpc_svrg_logistic_262144x8192_N32_B16", "m": m, "roofline_kernels": []}
     for b in (2, 8):
         ctx = lpc.Context(X, y, lpc.LOGISTIC, 1e-5, N, B, b, lpc.CLIP_STD, 2.0, 0)
         ctx.alpc_begin()
@@ -477,7 +625,16 @@ def alpc_bench(dev):
                           "snapshot_ms": round(snap, 4), "snapshot_gbs": round(n * d * 4 / snap * 1e-6, 1),
                           "loop_cluster_size": ctx.query(lpc.INFO_ALPC_LOOP_CLUSTER_SIZE),
                           "loop_row_slots": ctx.query(lpc.INFO_ALPC_LOOP_ROW_SLOTS),
+                          "loop_coords_per_thread": ctx.query(lpc.INFO_ALPC_LOOP_COORDS_PER_THREAD),
                           "one_launch_loops": ctx.query(lpc.INFO_LOOP_LAUNCHES), "objective": ctx.objective()}
+        step_bytes = (N + 1) * B * d * 4 + (N + 1) * B * 8 + 2 * N * (d // 8) * (1 if b <= 4 else 2) * 8 + 2 * d * 8
+        out["roofline_kernels"].append(roofline_entry(
+            "persist_kernel<%d, alpc> (one launch = %d steps of Algorithm 2)" % (b, m), out["workload"] + ", b=%d" % b,
+            loop * 1e3, m * step_bytes, peak, note="latency chain per step: rows of N+1 minibatches, tagged code words "
+            "written and read, second-estimator words"))
+        if b == 2:
+            out["roofline_kernels"].append(roofline_entry("snapshot_kernel", out["workload"], snap * 1e3, n * d * 4 + 8 * n + 4 * d,
+                                                          peak, "snapshot_kernel", n * d))
         ctx.close()
     # the strongly convex case (Algorithm 2, elastic net with sigma = L/1000, Theorem 3's tau1 and alpha)
     b, sigma = 2, L / 1000.0
@@ -598,6 +755,7 @@ def main():
     ap.add_argument("--per-step-kernels", action="store_true",
                     help="run the inner loop as per-step kernels (graph replay) instead of the one-launch loop; "
                          "for profiler captures, which cannot replay the cooperative launch")
+    ap.add_argument("--alpc-only", action="store_true", help="run only the ALPC-SVRG leg (262,144 x 8,192)")
     ap.add_argument("--fused-large-batch-only", type=int, default=0, metavar="ROWS",
                     help="run only the large-minibatch leg of the fused worker kernel on a ROWS x 8192 matrix "
                          "(a small case for profiler captures)")
@@ -609,7 +767,11 @@ def main():
     elif args.quantize_aggregate_only:
         import torch
         peak, _ = read_peak()
-        print(json.dumps(quantize_aggregate_bench(torch.device("cuda", 0), peak, args.quantize_aggregate_only, dnn=False)))
+        print(json.dumps(quantize_aggregate_bench(torch.device("cuda", 0), peak, args.quantize_aggregate_only, full=False)))
+    elif args.alpc_only:
+        import torch
+        peak, _ = read_peak()
+        print(json.dumps(alpc_bench(torch.device("cuda", 0), peak)))
     elif args.impl == "reference":
         run_reference(args)
     else:

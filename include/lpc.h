@@ -85,6 +85,8 @@ typedef struct lpc_ctx lpc_ctx;
 #define LPC_OPT_SHARED_SCALE 6  /* 1: lpc_quantize_pack gives every worker the unified scale delta_t = max_i delta_t^i of the parameter-server schemes (b), (c) of Section 3.2; needs b in 2..16 */
 #define LPC_OPT_AVERAGE_DIVISOR 7 /* lpc_unpack_average_prox (and only it: the training loops always average over N) divides the decoded sum by this count instead of the context's N (0 = N): the worker count behind a server's sum stream */
 #define LPC_OPT_PERSISTENT 5    /* 1 (default): lpc_inner_steps runs the whole loop in one cooperative launch when it fits */
+#define LPC_OPT_ONE_LAUNCH_QUANTIZE 8 /* 1 (default): lpc_quantize_pack uses one cooperative launch for inputs of at most LPC_ONE_LAUNCH_BYTES */
+#define LPC_ONE_LAUNCH_BYTES (48ll << 20)
 
 /* kernel classes reported by lpc_get_profile */
 #define LPC_KERNEL_SNAPSHOT 0    /* the pass over X of lpc_snapshot_full_grad / lpc_objective */
@@ -94,7 +96,8 @@ typedef struct lpc_ctx lpc_ctx;
 #define LPC_KERNEL_QUANT_PACK 4  /* second pass of lpc_quantize_pack (quantize + pack) */
 #define LPC_KERNEL_OTHER 5       /* small helper kernels */
 #define LPC_KERNEL_INNER_LOOP 6  /* the persistent kernel that runs all steps of one lpc_inner_steps call */
-#define LPC_KERNEL_KINDS 7
+#define LPC_KERNEL_QUANT_FUSED 7 /* lpc_quantize_pack in one launch (vectors that stay in L2 between its two passes) */
+#define LPC_KERNEL_KINDS 8
 
 /*
  * Creates a context for problem (1).  Section 1 "Contribution" (Eq. 1), Section 2.1 (N workers),
@@ -176,7 +179,9 @@ int lpc_packed_words(int64_t len, int32_t b, int64_t* words_out); /* ceil(len*b/
  *   codes_out  N * stride_words words, stride from lpc_packed_layout
  *   delta_out  N * nseg floats
  *   clipped_out nullable, N * nseg counts of coordinates outside the hull
- * Vectors longer than L2 are read twice (once for ||u||_inf and the variance, once to quantize).
+ * Vectors longer than L2 are read twice (once for ||u||_inf and the variance, once to quantize) by three launches;
+ * when all N vectors together take at most LPC_ONE_LAUNCH_BYTES the call is ONE cooperative launch whose second look at
+ * the values is served by L2 (LPC_OPT_ONE_LAUNCH_QUANTIZE = 0 switches that off).  Same codes either way.
  * N, b and the clip rule come from the context.
  */
 int lpc_quantize_pack(lpc_ctx* ctx, const float* U, const float* U_sub, int64_t len, int64_t ld,
@@ -287,6 +292,7 @@ int lpc_objective(lpc_ctx* ctx, const float* x, double* P_out);
 #define LPC_INFO_STEP_RING_STAGES 8        /* per-step kernel: 0 = minibatch rows resident on chip, else ring stages they stream through */
 #define LPC_INFO_LOOP_COORDS_PER_THREAD 11  /* one-launch loop: consecutive coordinates a thread owns (8, 4 or 2; 0: not available) */
 #define LPC_INFO_ALPC_LOOP_COORDS_PER_THREAD 12
+#define LPC_INFO_QUANT_ONE_LAUNCH 13        /* last lpc_quantize_pack: 1 when it ran as one cooperative launch */
 #define LPC_INFO_AGGREGATE_SPLIT 9         /* last lpc_unpack_average_prox: CTAs that shared one tile of 8192 coordinates (1, 2 or 4) */
 #define LPC_INFO_QUANT_PIPELINED_RUNS 10   /* last lpc_quantize_pack: runs of 8 tiles per worker that were whole tiles of one segment and
                                               so took the second pass's software-pipelined loop (unless that worker's scale was

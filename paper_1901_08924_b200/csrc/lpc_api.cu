@@ -34,6 +34,7 @@ struct SegPlan {
   SegInfo* d_segs = nullptr;
   int32_t* d_tile_seg = nullptr;    // nullptr when nseg == 1
   uint64_t msg_bits = 0;            // sum over segments of 32 + b*len_s
+  uint64_t version = 0;             // changes whenever the tables are rebuilt
 };
 
 struct GraphKey {
@@ -111,6 +112,12 @@ struct lpc_ctx {
   ScaleRec* q_scales = nullptr;
   uint32_t* q_clip = nullptr;
   size_t q_scale_cap = 0;
+  // one-launch quantizer: arrival counters per (worker, segment), valid for one layout; calls made with it so far
+  int one_launch = 1;             // LPC_OPT_ONE_LAUNCH_QUANTIZE
+  unsigned int* q_done = nullptr;
+  uint64_t q_done_version = ~0ull;
+  unsigned int q_epoch = 0;
+  int last_one_launch = 0;
   // graph replay
   cudaGraphExec_t graph = nullptr;
   cudaStream_t cap_stream = nullptr;  // used only to capture the graph
@@ -212,7 +219,9 @@ int make_plan(lpc_ctx* c, SegPlan& p, int64_t len, int b, const int64_t* seg_off
   const int rc = layout(len, b, seg_offsets, nseg, segs, tile_seg, &stride, &bits);
   if (rc != LPC_OK) return fail(c, rc, "invalid segment layout");
   CU(c, cudaStreamSynchronize(c->stream));  // the old tables may still be in use
+  const uint64_t version = p.version + 1;
   free_plan(p);
+  p.version = version;
   p.len = len; p.b = b; p.nseg = nseg; p.stride_words = stride; p.msg_bits = bits;
   p.ntiles = (int)tile_seg.size();
   p.offsets.resize(nseg + 1);
@@ -604,7 +613,7 @@ int lpc_destroy(lpc_ctx* c) {
   for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
   void* ptrs[] = {c->x, c->xt, c->mu, c->margins, c->yv, c->zv, c->ysum, c->vhat, c->v_tap, c->u_tap, c->codes,
                   c->delta, c->clipped_part, c->clipped, c->idx_tap, c->coef_tap, c->k_dev, c->dev_status, c->f_dev,
-                  c->partial_mu, c->partial_f, c->flags, c->ll, c->ll_vhat, c->q_pmax, c->q_ps1, c->q_ps2, c->q_scales, c->q_clip};
+                  c->partial_mu, c->partial_f, c->flags, c->ll, c->ll_vhat, c->q_pmax, c->q_ps1, c->q_ps2, c->q_scales, c->q_clip, c->q_done};
   for (void* p : ptrs)
     if (p) cudaFree(p);
   free_plan(c->inner_seg);
@@ -634,6 +643,7 @@ int lpc_set_option(lpc_ctx* c, int option, int64_t value) {
       return LPC_OK;
     case LPC_OPT_USE_GRAPH: c->use_graph = value ? 1 : 0; return LPC_OK;
     case LPC_OPT_PERSISTENT: c->use_persist = value ? 1 : 0; return LPC_OK;
+    case LPC_OPT_ONE_LAUNCH_QUANTIZE: c->one_launch = value ? 1 : 0; return LPC_OK;
     case LPC_OPT_SHARED_SCALE:
       if (value && (c->b < 2 || c->b > 16)) return fail(c, LPC_ERR_UNSUPPORTED, "a unified scale needs an integer grid: b in 2..16");
       c->shared_scale = value ? 1 : 0;
@@ -795,6 +805,7 @@ int lpc_query(const lpc_ctx* c, int what, int64_t* out) {
     case LPC_INFO_LOOP_LAUNCHES: *out = c->persist_launches; return LPC_OK;
     case LPC_INFO_SNAPSHOT_ROWS_PER_TILE: *out = c->snapR; return LPC_OK;
     case LPC_INFO_SNAPSHOT_STAGES: *out = c->snapStages; return LPC_OK;
+    case LPC_INFO_QUANT_ONE_LAUNCH: *out = c->last_one_launch; return LPC_OK;
     case LPC_INFO_AGGREGATE_SPLIT: *out = c->last_split; return LPC_OK;
     case LPC_INFO_QUANT_PIPELINED_RUNS: *out = c->last_pipelined_runs; return LPC_OK;
     default: return LPC_ERR_INVALID_ARG;
@@ -837,10 +848,12 @@ int lpc_quantize_pack(lpc_ctx* c, const float* U, const float* U_sub, int64_t le
   const size_t recs = (size_t)c->N * (size_t)nseg;
   if (recs > c->q_scale_cap) {
     CU(c, cudaStreamSynchronize(c->stream));
-    if (c->q_scales) { cudaFree(c->q_scales); cudaFree(c->q_clip); c->q_scales = nullptr; c->q_clip = nullptr; }
+    if (c->q_scales) { cudaFree(c->q_scales); cudaFree(c->q_clip); cudaFree(c->q_done); c->q_scales = nullptr; c->q_clip = nullptr; c->q_done = nullptr; }
     c->q_scale_cap = 0;
     CU(c, cudaMalloc(&c->q_scales, recs * sizeof(ScaleRec))); CU(c, cudaMalloc(&c->q_clip, recs * 4));
+    CU(c, cudaMalloc(&c->q_done, recs * 4));
     c->q_scale_cap = recs;
+    c->q_done_version = ~0ull;
   }
   QuantArgs a;
   a.U = U; a.U_sub = U_sub; a.ld = ld; a.N = c->N; a.b = c->b; a.clip_mode = c->clip_mode; a.clip_value = c->clip_value;
@@ -861,7 +874,28 @@ int lpc_quantize_pack(lpc_ctx* c, const float* U, const float* U_sub, int64_t le
     }
     c->last_pipelined_runs = runs;
   }
-  CU(c, launch_quantize_pack(a, c->stream, c->profile ? prof_hook : nullptr, c));
+  // one cooperative launch when the vectors stay in L2 between the statistics and the codes
+  c->last_one_launch = 0;
+  if (c->one_launch && !c->shared_scale && c->b != 32 && p.ntiles > 0 &&
+      (int64_t)c->N * len * 4 * (U_sub ? 2 : 1) <= LPC_ONE_LAUNCH_BYTES) {
+    int max_tiles = 1;
+    for (const SegInfo& g : p.segs) max_tiles = std::max(max_tiles, g.tile_count);
+    if (c->q_done_version != p.version || ((uint64_t)c->q_epoch + 2) * (uint64_t)max_tiles >= 0x7FFFFFFFull) {
+      CU(c, cudaMemsetAsync(c->q_done, 0, recs * 4, c->stream));
+      c->q_done_version = p.version;
+      c->q_epoch = 0;
+    }
+    cudaError_t e;
+    { ProfScope ps_(c, LPC_KERNEL_QUANT_FUSED); e = launch_quantize_fused(a, c->q_done, c->q_epoch, c->sm_count, c->stream); }
+    if (e == cudaSuccess) {
+      c->q_epoch += 1;
+      c->last_one_launch = 1;
+    } else {
+      cudaGetLastError();  // the launch was refused: nothing ran, use the three launches
+      c->one_launch = 0;
+    }
+  }
+  if (!c->last_one_launch) CU(c, launch_quantize_pack(a, c->stream, c->profile ? prof_hook : nullptr, c));
   if (!c->shared_scale) c->step2_bits += p.msg_bits * (uint64_t)c->N * (uint64_t)(c->N - 1);  // scheme (a); the server schemes count in lpc_server_reduce
   return LPC_OK;
 }

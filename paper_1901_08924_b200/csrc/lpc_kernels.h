@@ -59,6 +59,10 @@ typedef void (*LaunchHook)(void* user, int kind, int begin);
 // segment (the condition, besides 16-byte aligned vectors and a non-degenerate scale, for its pipelined loop).
 int quantize_run_tiles();
 cudaError_t launch_quantize_pack(const QuantArgs& a, cudaStream_t st, LaunchHook hook = nullptr, void* user = nullptr);
+// The same work in one cooperative launch, for vectors short enough to stay in L2 between the statistics and the codes
+// (b in 1..16, own scales).  done: N * nseg arrival counters, zero before the first call with a layout; epoch: calls
+// made with that layout since.
+cudaError_t launch_quantize_fused(const QuantArgs& a, unsigned int* done, unsigned int epoch, int sm_count, cudaStream_t st);
 
 struct AggArgs {
   const uint32_t* codes;

@@ -59,6 +59,7 @@ struct PSmem {
   // step-parity halves: margin partial sums (slot b * PMAXCS + rank) and statistics (max, S1, S2 per rank)
   unsigned long long mx[2][PMAXB * PMAXCS];
   unsigned long long sx[2][3 * PMAXCS];
+  unsigned long long dl[2][PMAXFLAGS];  // the workers' scales of a step (delta | tag), fetched by warp 0 for the whole CTA
   float ws1[PMAXP * 8], ws2[PMAXP * 8];
   uint32_t wmax[8];
   uint32_t wclip[8];
@@ -84,6 +85,9 @@ __device__ __forceinline__ void st_cluster_word(const unsigned long long* slot, 
   uint32_t remote;
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(slot)), "r"(cta));
   asm volatile("st.relaxed.cluster.shared::cluster.u64 [%0], %1;" ::"r"(remote), "l"(v) : "memory");
+}
+__device__ __forceinline__ void st_shared_word(unsigned long long* slot, unsigned long long v) {
+  asm volatile("st.relaxed.cta.shared::cta.u64 [%0], %1;" ::"r"(smem_u32(slot)), "l"(v) : "memory");
 }
 __device__ __forceinline__ unsigned long long ld_shared_word(const unsigned long long* slot) {
   unsigned long long v;
@@ -131,23 +135,31 @@ __device__ unsigned long long g_trace[64 * 16];
 #endif
 
 // A thread's EPT consecutive row values of a slice from shared memory (zero outside the existing columns).
+// EPT = 8: a thread's two 16-byte halves are 32 bytes from its neighbour's, so a plain "lower halves, then upper halves"
+// pair of loads would hit every bank twice.  Threads with `swz` set (bit 2 of the lane) read their upper half first
+// instead: each load then covers 32 distinct banks per quarter warp.  Such a thread gets its values with the halves
+// exchanged, v[e] = value of coordinate e ^ 4, and the callers keep their operands in the same order.
 template <int EPT>
-__device__ __forceinline__ void row_vals(const float* rowp, int off, int width, float* v) {
+__device__ __forceinline__ void row_vals(const float* rowp, int off, int width, bool swz, float* v) {
 #pragma unroll
   for (int e = 0; e < EPT; ++e) v[e] = 0.f;
-  if (off < width) {  // width is a multiple of 4 and off a multiple of EPT
+  if constexpr (EPT == 8) {  // width is a multiple of 4 and off a multiple of EPT
+    const int o0 = off + (swz ? 4 : 0), o1 = off + (swz ? 0 : 4);
+    if (o0 < width) {
+      const float4 t = *reinterpret_cast<const float4*>(rowp + o0);
+      v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+    }
+    if (o1 < width) {
+      const float4 t = *reinterpret_cast<const float4*>(rowp + o1);
+      v[4] = t.x; v[5] = t.y; v[6] = t.z; v[7] = t.w;
+    }
+  } else if (off < width) {
     if constexpr (EPT == 2) {
       const float2 t = *reinterpret_cast<const float2*>(rowp + off);
       v[0] = t.x; v[1] = t.y;
     } else {
       const float4 t = *reinterpret_cast<const float4*>(rowp + off);
       v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
-      if constexpr (EPT == 8) {
-        if (off + 4 < width) {
-          const float4 t1 = *reinterpret_cast<const float4*>(rowp + off + 4);
-          v[4] = t1.x; v[5] = t1.y; v[6] = t1.z; v[7] = t1.w;
-        }
-      }
     }
   }
 }
@@ -179,6 +191,7 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
   float* rows = reinterpret_cast<float*>(smem_raw + ((sizeof(PSmem) + 15) & ~(size_t)15));  // RS row slots of SL floats
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const bool swz = (EPT == 8) && ((lane >> 2) & 1);  // this thread reads the halves of its row values exchanged (row_vals)
   const int rank = (int)cluster.block_rank();
   const int worker = blockIdx.y;
   const bool is_J = ALPC && (worker == N);  // the extra cluster that handles the shared batch J
@@ -204,6 +217,7 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
   // no exchange slot may look valid before a peer has written it: tags start at 1
   for (int i = tid; i < 2 * PMAXB * PMAXCS; i += PT) (&sm.mx[0][0])[i] = 0ull;
   for (int i = tid; i < 2 * 3 * PMAXCS; i += PT) (&sm.sx[0][0])[i] = 0ull;
+  for (int i = tid; i < 2 * PMAXFLAGS; i += PT) (&sm.dl[0][0])[i] = 0ull;
   asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   __syncthreads();
 
@@ -274,11 +288,14 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
 
   // Applies step target-1's update to this thread's coordinates:
   //   x <- prox_{eta h}(x - eta (mean_i delta_i k_i + mu))      (Algorithm 2: the y and z updates).
-  // The words of all workers that hold the thread's codes are loaded together (one L2 round trip) and
-  // re-loaded until every tag names step target-1; LLCH workers are handled per round.
+  // The tagged words that hold the thread's codes are loaded for CH workers at a time, all in flight together (one L2
+  // round trip; CH covers all N workers whenever 32 words per thread suffice), and re-loaded until every tag names
+  // step target-1.  The workers' scales are the same for every thread of the CTA: the lanes of warp 0 fetch them, one
+  // worker per lane, and pass them on through shared memory as tagged words (they are published before the codes, so
+  // they are there when a thread's codes are).
   constexpr int WMAX = (BITS == 0) ? 8 : (BITS == 8 ? 2 : 1);  // tagged words per group of 8 coordinates
   constexpr int NW = (BITS == 0) ? 8 : (TB >= 32 ? TB / 32 : 1);  // of which a thread reads / writes this many
-  constexpr int LLCH = (BITS == 0) ? 4 : 16;
+  constexpr int CH = (BITS == 0) ? 4 : 32 / (NP * NW);        // workers per round of loads
   const int wpg = (BITS == 0) ? pa.wpg : WMAX;
   const int sub = (LPG > 1) ? (tid & (LPG - 1)) : 0;          // this thread's place in its group of 8 coordinates
   const int wfirst = (BITS == 0) ? 0 : (sub * TB) >> 5;        // first word of the group that holds its codes
@@ -288,103 +305,137 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
   auto apply_update = [&](unsigned int target) {
     const int rpar = (pa.count - (int)target) & 1;  // parity half that holds step target-1
     const uint32_t tag = pa.tag_base + target;
+    const unsigned long long good = (unsigned long long)tag << 32;  // stands in for words this thread does not need
     const unsigned long long* dwords = pa.pub + ((size_t)rpar * PMAXFLAGS + rank) * PUB_STRIDE;
     const unsigned long long* ll_in = pa.ll + (size_t)rpar * N * groups * wpg;
+    int cc[NP];
+    bool act[NP];
+    float acc[NP][EPT];
 #pragma unroll
     for (int p = 0; p < NP; ++p) {
       const int off = p * PSPAN + tid * EPT;
-      const int c = c0 + off;
-      if (off >= SL || c >= d) continue;
-      float acc[EPT];
+      cc[p] = c0 + off;
+      act[p] = off < SL && cc[p] < d;
 #pragma unroll
-      for (int e = 0; e < EPT; ++e) acc[e] = 0.f;
-      unsigned long long vw[ALPC ? EPT : 1];
-#pragma unroll 1
-      for (int i0 = 0; i0 < N; i0 += LLCH) {
-        unsigned long long dw[LLCH], cw[LLCH][NW];
+      for (int e = 0; e < EPT; ++e) acc[p][e] = 0.f;
+    }
+    unsigned long long cw[CH][NP][NW], vw[ALPC ? NP * EPT : 1];
+    auto issue = [&](int i0) {
+#pragma unroll
+      for (int j = 0; j < CH; ++j) {
+        const bool live = i0 + j < N;
+#pragma unroll
+        for (int p = 0; p < NP; ++p) {
+          const unsigned long long* q = ll_in + ((size_t)(i0 + j) * groups + (size_t)(cc[p] >> 3)) * wpg + wfirst;
+#pragma unroll
+          for (int w = 0; w < NW; ++w) cw[j][p][w] = (live && act[p] && w < wpg) ? ld_word(q + w) : good;
+        }
+      }
+      if constexpr (ALPC) {
+        if (i0 == 0) {
+#pragma unroll
+          for (int p = 0; p < NP; ++p)
+#pragma unroll
+            for (int e = 0; e < EPT; ++e)
+              vw[p * EPT + e] = act[p] ? ld_word(pa.ll_vhat + (size_t)rpar * groups * 8 + cc[p] + e) : good;
+        }
+      }
+    };
+    issue(0);
+    if (warp == 0) {  // the scales: lane l takes workers l, l + 32, ...
+      for (int i = lane; i < N; i += 32) {
+        unsigned long long w;
         uint64_t t0 = 0;
         for (uint32_t it = 0;; ++it) {
+          w = ld_word(dwords + (size_t)i * CS * PUB_STRIDE);
+          if (word_tag(w) == tag || wait_expired(it, t0)) break;
+        }
+        st_shared_word(&sm.dl[rpar][i], w);
+      }
+    }
+#pragma unroll 1
+    for (int i0 = 0; i0 < N; i0 += CH) {
+      uint64_t t0 = 0;
+      for (uint32_t it = 0;; ++it) {
+        bool ok = true;
 #pragma unroll
-          for (int j = 0; j < LLCH; ++j) {
-            const int i = min(i0 + j, N - 1);  // the tail repeats the last worker: harmless
-            dw[j] = ld_word(dwords + (size_t)i * CS * PUB_STRIDE);
-            const unsigned long long* q = ll_in + ((size_t)i * groups + (size_t)(c >> 3)) * wpg + wfirst;
+        for (int j = 0; j < CH; ++j)
 #pragma unroll
-            for (int w = 0; w < NW; ++w) cw[j][w] = (w < wpg) ? ld_word(q + w) : ((unsigned long long)tag << 32);
+          for (int p = 0; p < NP; ++p)
+#pragma unroll
+            for (int w = 0; w < NW; ++w) ok = ok && word_tag(cw[j][p][w]) == tag;
+        if constexpr (ALPC) {
+          if (i0 == 0) {
+#pragma unroll
+            for (int e = 0; e < NP * EPT; ++e) ok = ok && word_tag(vw[e]) == tag;
           }
-          if constexpr (ALPC) {
-            if (i0 == 0) {
-#pragma unroll
-              for (int e = 0; e < EPT; ++e) vw[e] = ld_word(pa.ll_vhat + (size_t)rpar * groups * 8 + c + e);
-            }
-          }
-          bool ok = true;
-#pragma unroll
-          for (int j = 0; j < LLCH; ++j) {
-            ok = ok && word_tag(dw[j]) == tag;
-#pragma unroll
-            for (int w = 0; w < NW; ++w) ok = ok && word_tag(cw[j][w]) == tag;
-          }
-          if constexpr (ALPC) {
-            if (i0 == 0) {
-#pragma unroll
-              for (int e = 0; e < EPT; ++e) ok = ok && word_tag(vw[e]) == tag;
-            }
-          }
-#ifdef LPC_TRACE
-          if (i0 == 0 && p == 0 && blockIdx.x == 0 && blockIdx.y == 0 && tid == 0 && target >= 8 && target < 72)
-            g_trace[(target - 8) * 16 + 15] = it + 1;
-#endif
-          if (ok || wait_expired(it, t0)) break;
         }
 #ifdef LPC_TRACE
-        if (i0 == 0 && p == 0) { const int t = (int)target; LPC_TRACE_MARK(3); }
+        if (i0 == 0 && blockIdx.x == 0 && blockIdx.y == 0 && tid == 0 && target >= 8 && target < 72)
+          g_trace[(target - 8) * 16 + 15] = it + 1;
 #endif
-        {
+        if (ok || wait_expired(it, t0)) break;
+        issue(i0);
+      }
+#ifdef LPC_TRACE
+      if (i0 == 0) { const int t = (int)target; LPC_TRACE_MARK(3); }
+#endif
 #pragma unroll
-          for (int j = 0; j < LLCH; ++j) {
-            if (i0 + j < N) {
-              const float di = __uint_as_float((uint32_t)dw[j]);
-              if (b == 32) {
+      for (int j = 0; j < CH; ++j) {
+        if (i0 + j < N) {
+          unsigned long long dword;
+          uint64_t t1 = 0;
+          for (uint32_t it = 0;; ++it) {
+            dword = ld_shared_word(&sm.dl[rpar][i0 + j]);
+            if (word_tag(dword) == tag || wait_expired(it, t1)) break;
+          }
+          const float di = __uint_as_float((uint32_t)dword);
 #pragma unroll
-                for (int e = 0; e < EPT; ++e) {
-                  const float val = (c + e < d && e < NW) ? __uint_as_float((uint32_t)cw[j][e < NW ? e : 0]) : 0.f;
-                  acc[e] = add_rn(acc[e], mul_rn(di, val));
-                }
-              } else {
-                uint64_t lo = (uint64_t)(uint32_t)cw[j][0], hi = 0;
-                if constexpr (NW >= 2) lo |= (uint64_t)(uint32_t)cw[j][1] << 32;
-                if constexpr (NW >= 4) hi = (uint64_t)(uint32_t)cw[j][2] | ((uint64_t)(uint32_t)cw[j][3] << 32);
-                float kf[8];
-                if constexpr (BITS == 0) {
+          for (int p = 0; p < NP; ++p) {
+            if (b == 32) {
 #pragma unroll
-                  for (int e = 0; e < 8; ++e) kf[e] = index_as_float(extract_bits(lo, hi, e * b, b), b);
-                } else {
-                  // this thread's EPT codes start at bit wshift of the word: decode them as the first codes of a group
-                  // (the entries past EPT are not used and cost nothing)
-                  if constexpr (TB < 32) lo = ((uint32_t)lo >> wshift) & ((1u << TB) - 1u);
-                  decode8<BITS ? BITS : 1>(lo, kf);
-                }
-#pragma unroll
-                for (int e = 0; e < EPT; ++e) acc[e] = add_rn(acc[e], mul_rn(di, kf[e]));
+              for (int e = 0; e < EPT; ++e) {
+                const float val = (cc[p] + e < d && e < NW) ? __uint_as_float((uint32_t)cw[j][p][e < NW ? e : 0]) : 0.f;
+                acc[p][e] = add_rn(acc[p][e], mul_rn(di, val));
               }
+            } else {
+              uint64_t lo = (uint64_t)(uint32_t)cw[j][p][0], hi = 0;
+              if constexpr (NW >= 2) lo |= (uint64_t)(uint32_t)cw[j][p][1] << 32;
+              if constexpr (NW >= 4) hi = (uint64_t)(uint32_t)cw[j][p][2] | ((uint64_t)(uint32_t)cw[j][p][3] << 32);
+              float kf[8];
+              if constexpr (BITS == 0) {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) kf[e] = index_as_float(extract_bits(lo, hi, e * b, b), b);
+              } else {
+                // this thread's EPT codes start at bit wshift of the word: decode them as the first codes of a group
+                // (the entries past EPT are not used and cost nothing)
+                if constexpr (TB < 32) lo = ((uint32_t)lo >> wshift) & ((1u << TB) - 1u);
+                decode8<BITS ? BITS : 1>(lo, kf);
+              }
+#pragma unroll
+              for (int e = 0; e < EPT; ++e) acc[p][e] = add_rn(acc[p][e], mul_rn(di, kf[e]));
             }
           }
         }
       }
+      if (i0 + CH < N) issue(i0 + CH);
+    }
+#pragma unroll
+    for (int p = 0; p < NP; ++p) {
+      if (!act[p]) continue;
 #pragma unroll
       for (int e = 0; e < EPT; ++e) {
-        if (c + e < d) {
-          const float v = add_rn(mul_rn(acc[e], invN), mur[p][e]);
+        if (cc[p] + e < d) {
+          const float v = add_rn(mul_rn(acc[p][e], invN), mur[p][e]);
           if constexpr (ALPC) {  // steps 12-13 of Algorithm 2
-            const float vh = __uint_as_float((uint32_t)vw[e]);
+            const float vhat = __uint_as_float((uint32_t)vw[p * EPT + e]);
             yr[p][e] = mul_rn(soft_threshold(__fsub_rn(xr[p][e], mul_rn(pa.inv4L, v)), kappa_y), pa.cy);
-            zr[p][e] = mul_rn(soft_threshold(__fsub_rn(zr[p][e], mul_rn(pa.alpha, vh)), kappa_z), pa.cz);
+            zr[p][e] = mul_rn(soft_threshold(__fsub_rn(zr[p][e], mul_rn(pa.alpha, vhat)), kappa_z), pa.cz);
             sr[p][e] = add_rn(sr[p][e], mul_rn(wcur, yr[p][e]));
           } else {
             xr[p][e] = soft_threshold(__fsub_rn(xr[p][e], mul_rn(pa.eta, v)), kappa);
           }
-          if (pa.v_tap && worker == 0) pa.v_tap[c + e] = v;
+          if (pa.v_tap && worker == 0) pa.v_tap[cc[p] + e] = v;
         }
       }
     }
@@ -451,6 +502,11 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
     // margins <X_a, x_t>: eight rows at a time; their 8*NP per-thread partial sums are reduced across the
     // warp together by recursive halving (9 or 12 shuffles instead of 5 per value)
     constexpr int RG = 8, NVAL = RG * NP, LOGV = (NP == 2) ? 4 : 3;
+    float xw[NP][EPT];  // x in the order row_vals delivers the row values
+#pragma unroll
+    for (int p = 0; p < NP; ++p)
+#pragma unroll
+      for (int e = 0; e < EPT; ++e) xw[p][e] = (EPT == 8 && swz) ? xr[p][e ^ (EPT / 2)] : xr[p][e];
 #pragma unroll 1
     for (int r0 = 0; r0 < B; r0 += RG) {
       float sv[NVAL];
@@ -460,10 +516,10 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
 #pragma unroll
         for (int p = 0; p < NP; ++p) {
           float v[EPT], pr[EPT];
-          row_vals<EPT>(rp, p * PSPAN + tid * EPT, width, v);
+          row_vals<EPT>(rp, p * PSPAN + tid * EPT, width, swz, v);
 #pragma unroll
-          for (int e = 0; e < EPT; ++e) pr[e] = mul_rn(v[e], xr[p][e]);
-          sv[j * NP + p] = tree_ept<EPT>(pr);
+          for (int e = 0; e < EPT; ++e) pr[e] = mul_rn(v[e], xw[p][e]);
+          sv[j * NP + p] = tree_ept<EPT>(pr);  // exchanged halves only swap the operands of the tree's last addition
         }
       }
       WarpHalving<NVAL, 0>::run(sv, lane);
@@ -515,27 +571,28 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
     float u[NP][EPT];
 #pragma unroll
     for (int p = 0; p < NP; ++p) {
+      float uw[EPT];  // in the order row_vals delivers the row values
 #pragma unroll
-      for (int e = 0; e < EPT; ++e) u[p][e] = 0.f;
+      for (int e = 0; e < EPT; ++e) uw[e] = 0.f;
 #pragma unroll 1
       for (int r0 = 0; r0 < B; r0 += 4) {
         float v[4][EPT], cf[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           const int r = min(r0 + j, B - 1);
-          row_vals<EPT>(row_ptr(r), p * PSPAN + tid * EPT, width, v[j]);
+          row_vals<EPT>(row_ptr(r), p * PSPAN + tid * EPT, width, swz, v[j]);
           cf[j] = sm.coef[r];
         }
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           if (r0 + j < B) {
 #pragma unroll
-            for (int e = 0; e < EPT; ++e) u[p][e] = add_rn(u[p][e], mul_rn(cf[j], v[j][e]));
+            for (int e = 0; e < EPT; ++e) uw[e] = add_rn(uw[e], mul_rn(cf[j], v[j][e]));
           }
         }
       }
 #pragma unroll
-      for (int e = 0; e < EPT; ++e) u[p][e] = mul_rn(u[p][e], invB);
+      for (int e = 0; e < EPT; ++e) u[p][e] = mul_rn((EPT == 8 && swz) ? uw[e ^ (EPT / 2)] : uw[e], invB);
     }
     if (a.u_tap && t == pa.count - 1) {
 #pragma unroll
@@ -799,12 +856,11 @@ using PersistKernel = void (*)(PersistArgs);
 
 template <int BITS, bool ALPC>
 PersistKernel pick_shape(int np, int ept) {
-  if (np == 2) return persist_kernel<BITS, 2, 8, ALPC>;
   if constexpr (BITS != 0) {
-    if (ept == 4) return persist_kernel<BITS, 1, 4, ALPC>;
-    if (ept == 2) return persist_kernel<BITS, 1, 2, ALPC>;
+    if (np == 1 && ept == 4) return persist_kernel<BITS, 1, 4, ALPC>;
+    if (np == 1 && ept == 2) return persist_kernel<BITS, 1, 2, ALPC>;
   }
-  return persist_kernel<BITS, 1, 8, ALPC>;
+  return np == 2 ? persist_kernel<BITS, 2, 8, ALPC> : persist_kernel<BITS, 1, 8, ALPC>;
 }
 template <bool ALPC>
 PersistKernel pick_width(int b, int np, int ept) {
@@ -818,8 +874,8 @@ PersistKernel pick_width(int b, int np, int ept) {
 }
 // The instantiation for code width b, slice SL and algorithm.
 PersistKernel pick_kernel(int b, int SL, bool alpc) {
-  const int np = (SL > PGROUP) ? 2 : 1;
   const int ept = persist_coords_per_thread(b, SL);
+  const int np = (SL > PT * ept) ? 2 : 1;
   return alpc ? pick_width<true>(b, np, ept) : pick_width<false>(b, np, ept);
 }
 
@@ -841,8 +897,7 @@ int max_clusters(PersistKernel k, int cs, size_t smem) {
 
 }  // namespace
 
-// Coordinates a thread owns per pass: a slice of PT * 8 or more gives every thread a whole group of 8; narrower
-// slices are spread over all threads of the CTA, 4 or 2 coordinates each (fixed code widths only).
+// Coordinates a thread owns per pass (see the kernel's EPT).
 int persist_coords_per_thread(int b, int SL) {
   const bool fixed = (b == 1 || b == 2 || b == 4 || b == 8);
   if (!fixed || SL >= PT * 8) return 8;

@@ -43,8 +43,7 @@ __device__ __forceinline__ bool aligned16(const void* p) { return (reinterpret_c
 
 // ---- pass 1: per-tile partial (max |u| as bit pattern, tree sums of u and u^2) ---------------------------
 template <bool NEED_SUMS>
-__global__ void __launch_bounds__(QT) stats_kernel(QuantArgs a) {
-  const int tile = blockIdx.x, worker = blockIdx.y;
+__device__ __forceinline__ void stats_tile(const QuantArgs& a, int tile, int worker, float* sh1, float* sh2, uint32_t* shm) {
   const int seg = a.tile_seg ? a.tile_seg[tile] : 0;
   const SegInfo s = a.segs[seg];
   const int64_t tstart = (int64_t)(tile - s.tile_first) * TILE;
@@ -52,9 +51,6 @@ __global__ void __launch_bounds__(QT) stats_kernel(QuantArgs a) {
   const float* q = a.U_sub ? a.U_sub + (int64_t)worker * a.ld + s.off : nullptr;
   const bool vec = aligned16(p) && (!q || aligned16(q));
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-
-  __shared__ float sh1[QITER * 8], sh2[QITER * 8];
-  __shared__ uint32_t shm[8];
 
   uint32_t mx = 0;
 #pragma unroll
@@ -94,6 +90,13 @@ __global__ void __launch_bounds__(QT) stats_kernel(QuantArgs a) {
   }
 }
 
+template <bool NEED_SUMS>
+__global__ void __launch_bounds__(QT) stats_kernel(QuantArgs a) {
+  __shared__ float sh1[QITER * 8], sh2[QITER * 8];
+  __shared__ uint32_t shm[8];
+  stats_tile<NEED_SUMS>(a, blockIdx.x, blockIdx.y, sh1, sh2, shm);
+}
+
 // Tree sum over `count` tile partials by one CTA of QT threads (leaf order = tile order).
 __device__ float block_tree_sum(const float* __restrict__ v, int count, float* sh8) {
   int64_t P = 1;
@@ -103,7 +106,7 @@ __device__ float block_tree_sum(const float* __restrict__ v, int count, float* s
   float stack[32];
   int top = 0;
   for (int i = 0; i < chunk; ++i) {
-    float cur = (lo + i < count) ? v[lo + i] : 0.f;
+    float cur = (lo + i < count) ? __ldcg(v + lo + i) : 0.f;  // written by other CTAs: read where they wrote it
     int idx = i;
     while (idx & 1) { cur = add_rn(stack[--top], cur); idx >>= 1; }
     stack[top++] = cur;
@@ -116,14 +119,12 @@ __device__ float block_tree_sum(const float* __restrict__ v, int count, float* s
 }
 
 // ---- between the passes: one CTA per (segment, worker) finishes the reductions and applies Eq. 2 -------
-__global__ void __launch_bounds__(QT) finish_kernel(QuantArgs a) {
-  const int seg = blockIdx.x, worker = blockIdx.y;
+// The scale record of (segment, worker) from its tile partials, by all threads of the CTA; valid in thread 0.
+__device__ __forceinline__ ScaleRec finish_segment(const QuantArgs& a, int seg, int worker, float* sh8, uint32_t* shm) {
   const SegInfo s = a.segs[seg];
   const int64_t base = (int64_t)worker * a.ntiles + s.tile_first;
-  __shared__ float sh8[8];
-  __shared__ uint32_t shm[8];
   uint32_t mx = 0;
-  for (int t = threadIdx.x; t < s.tile_count; t += QT) mx = max(mx, a.pmax[base + t]);
+  for (int t = threadIdx.x; t < s.tile_count; t += QT) mx = max(mx, __ldcg(a.pmax + base + t));
   mx = warp_max_u32(mx);
   if ((threadIdx.x & 31) == 0) shm[threadIdx.x >> 5] = mx;
   float S1 = 0.f, S2 = 0.f;
@@ -132,19 +133,30 @@ __global__ void __launch_bounds__(QT) finish_kernel(QuantArgs a) {
     S2 = block_tree_sum(a.ps2 + base, s.tile_count, sh8);
   }
   __syncthreads();
+  ScaleRec r;
+  r.delta = r.rdelta = r.T = r.lower = 0.f;
+  r.flags = r.pad0 = r.pad1 = r.pad2 = 0;
   if (threadIdx.x == 0) {
     uint32_t m = 0;
 #pragma unroll
     for (int w = 0; w < 8; ++w) m = max(m, shm[w]);
     const Scale sc = make_scale(m, S1, S2, s.len, a.b, a.clip_mode, a.clip_value);
-    const int64_t o = (int64_t)worker * a.nseg + seg;
-    ScaleRec r;
     r.delta = sc.delta; r.rdelta = sc.rdelta; r.T = sc.T; r.lower = sc.lower; r.flags = sc.flags;
-    r.pad0 = r.pad1 = r.pad2 = 0;
+  }
+  return r;
+}
+
+__global__ void __launch_bounds__(QT) finish_kernel(QuantArgs a) {
+  const int seg = blockIdx.x, worker = blockIdx.y;
+  __shared__ float sh8[8];
+  __shared__ uint32_t shm[8];
+  const ScaleRec r = finish_segment(a, seg, worker, sh8, shm);
+  if (threadIdx.x == 0) {
+    const int64_t o = (int64_t)worker * a.nseg + seg;
     a.scales[o] = r;
-    a.delta_out[o] = sc.delta;
+    a.delta_out[o] = r.delta;
     a.clipped_out[o] = 0;
-    if (sc.flags & 2u) atomicOr(a.dev_status, DEV_NONFINITE);
+    if (r.flags & 2u) atomicOr(a.dev_status, DEV_NONFINITE);
   }
 }
 
@@ -252,7 +264,7 @@ __device__ __forceinline__ void quantize_run(const QuantArgs& a, const ScaleRec&
 }
 
 template <int BITS, bool COUNT>
-__device__ __forceinline__ void quantize_tile(const QuantArgs& a, int tile, int worker, uint8_t* stage) {
+__device__ __forceinline__ void quantize_tile(const QuantArgs& a, int tile, int worker, uint8_t* stage, const ScaleRec& sc) {
   const int seg = a.tile_seg ? a.tile_seg[tile] : 0;
   const SegInfo s = a.segs[seg];
   const int64_t tstart = (int64_t)(tile - s.tile_first) * TILE;
@@ -261,7 +273,6 @@ __device__ __forceinline__ void quantize_tile(const QuantArgs& a, int tile, int 
   const bool vec = aligned16(p) && (!q || aligned16(q));
   const int tid = threadIdx.x, lane = tid & 31;
   const int b = BITS ? BITS : a.b;
-  const ScaleRec sc = a.scales[(int64_t)worker * a.nseg + seg];
   const bool degenerate = (sc.flags & 1u) != 0;
   const uint32_t zero_code = (b == 1) ? 0u : (1u << (b - 1));
   uint32_t* out = a.codes + (int64_t)worker * a.stride_words + s.word_off;
@@ -381,14 +392,89 @@ __global__ void __launch_bounds__(QT, 4) quantize_kernel(QuantArgs a) {
   }
   for (int t = 0; t < ntl; ++t) {
     if (BITS == 0 && t > 0) __syncthreads();  // the staging buffer is reused from tile to tile
-    quantize_tile<BITS, COUNT>(a, tile0 + t, worker, stage);
+    const int seg = a.tile_seg ? a.tile_seg[tile0 + t] : 0;
+    quantize_tile<BITS, COUNT>(a, tile0 + t, worker, stage, a.scales[(int64_t)worker * a.nseg + seg]);
+  }
+}
+
+// ---- one launch for vectors that stay in L2 between the two passes ------------------------------------------------
+// The grid is resident as a whole (cooperative launch) and every CTA takes the (worker, tile) pairs item, item + grid,
+// ...: first their statistics, then -- once all tiles of a pair's (worker, segment) have reported, which a counter per
+// (worker, segment) says -- the scale from the tile partials (every CTA that needs it forms it itself: same partials,
+// same tree, same bits) and the codes of its tiles, whose values come from L2 this time.  Two kernel boundaries and the
+// separate scale kernel are gone, which is most of the cost of a short vector.  The counters only grow: call number
+// `epoch` waits for (epoch + 1) * tile_count arrivals.  A wait that runs out records a timeout and goes on.
+template <int BITS, bool COUNT, bool NEED_SUMS>
+__global__ void __launch_bounds__(QT, 4) quantize_fused_kernel(QuantArgs a, unsigned int* done, unsigned int epoch) {
+  __shared__ float sh1[QITER * 8], sh2[QITER * 8], sh8[8];
+  __shared__ uint32_t shm[8];
+  __shared__ ScaleRec srec;
+  __shared__ __align__(16) uint8_t stage[BITS == 0 ? QT * 16 : 16];
+  const int items = a.N * a.ntiles, tid = threadIdx.x;
+  for (int item = blockIdx.x; item < items; item += gridDim.x) {
+    const int worker = item / a.ntiles, tile = item % a.ntiles;
+    const int seg = a.tile_seg ? a.tile_seg[tile] : 0;
+    if (item != (int)blockIdx.x) __syncthreads();  // the reduction buffers are reused from tile to tile
+    stats_tile<NEED_SUMS>(a, tile, worker, sh1, sh2, shm);
+    if (tid == 0) {
+      const int64_t o = (int64_t)worker * a.nseg + seg;
+      if (tile == a.segs[seg].tile_first) a.clipped_out[o] = 0;
+      __threadfence();  // the partials (and the cleared count) before the arrival
+      atomicAdd(&done[o], 1u);
+    }
+  }
+  // segments without a single coordinate have no tile: their records are written here
+  for (int o = blockIdx.x; o < a.N * a.nseg; o += gridDim.x) {
+    const int worker = o / a.nseg, seg = o % a.nseg;
+    if (a.segs[seg].tile_count != 0) continue;
+    __syncthreads();
+    const ScaleRec r = finish_segment(a, seg, worker, sh8, shm);
+    if (tid == 0) { a.scales[o] = r; a.delta_out[o] = r.delta; a.clipped_out[o] = 0; }
+  }
+  int have = -1;
+  for (int item = blockIdx.x; item < items; item += gridDim.x) {
+    const int worker = item / a.ntiles, tile = item % a.ntiles;
+    const int seg = a.tile_seg ? a.tile_seg[tile] : 0;
+    const int o = worker * a.nseg + seg;
+    if (o != have) {
+      const SegInfo s = a.segs[seg];
+      if (tid == 0) {
+        const unsigned int want = (epoch + 1u) * (unsigned int)s.tile_count;
+        uint64_t t0 = 0;
+        for (uint32_t it = 0;; ++it) {
+          unsigned int seen;
+          asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(done + o) : "memory");
+          if (seen >= want) break;
+          if ((it & 63u) == 63u) {
+            const uint64_t now = global_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > 2000000000ull) { atomicOr(a.dev_status, DEV_TIMEOUT); break; }
+          }
+        }
+      }
+      __syncthreads();
+      const ScaleRec r = finish_segment(a, seg, worker, sh8, shm);
+      if (tid == 0) {
+        srec = r;
+        if (tile == s.tile_first) {  // one CTA leaves the record and the scale for the caller
+          a.scales[o] = r;
+          a.delta_out[o] = r.delta;
+          if (r.flags & 2u) atomicOr(a.dev_status, DEV_NONFINITE);
+        }
+      }
+      __syncthreads();
+      have = o;
+    } else if (BITS == 0) {
+      __syncthreads();  // the staging buffer is reused from tile to tile
+    }
+    const ScaleRec sc = srec;
+    quantize_tile<BITS, COUNT>(a, tile, worker, stage, sc);
   }
 }
 
 
 // b = 32: the message is the vector itself (clamped to [-T, T] when a clip rule is set).
-__global__ void __launch_bounds__(QT) bypass_kernel(QuantArgs a) {
-  const int tile = blockIdx.x, worker = blockIdx.y;
+__device__ __forceinline__ void bypass_tile(const QuantArgs& a, int tile, int worker, const ScaleRec& sc) {
   const int seg = a.tile_seg ? a.tile_seg[tile] : 0;
   const SegInfo s = a.segs[seg];
   const int64_t tstart = (int64_t)(tile - s.tile_first) * TILE;
@@ -396,7 +482,6 @@ __global__ void __launch_bounds__(QT) bypass_kernel(QuantArgs a) {
   const float* q = a.U_sub ? a.U_sub + (int64_t)worker * a.ld + s.off : nullptr;
   const bool vec = aligned16(p) && (!q || aligned16(q));
   const int tid = threadIdx.x, lane = tid & 31;
-  const ScaleRec sc = a.scales[(int64_t)worker * a.nseg + seg];
   uint32_t* out = a.codes + (int64_t)worker * a.stride_words + s.word_off;
   uint32_t nclip = 0;
 #pragma unroll
@@ -427,7 +512,52 @@ __global__ void __launch_bounds__(QT) bypass_kernel(QuantArgs a) {
   if (lane == 0 && nclip) atomicAdd(&a.clipped_out[(int64_t)worker * a.nseg + seg], nclip);
 }
 
+__global__ void __launch_bounds__(QT) bypass_kernel(QuantArgs a) {
+  const int tile = blockIdx.x, worker = blockIdx.y;
+  const int seg = a.tile_seg ? a.tile_seg[tile] : 0;
+  bypass_tile(a, tile, worker, a.scales[(int64_t)worker * a.nseg + seg]);
+}
+
+using FusedKernel = void (*)(QuantArgs, unsigned int*, unsigned int);
+template <int BITS>
+FusedKernel pick_fused(bool count, bool sums) {
+  if (count) return sums ? quantize_fused_kernel<BITS, true, true> : quantize_fused_kernel<BITS, true, false>;
+  return sums ? quantize_fused_kernel<BITS, false, true> : quantize_fused_kernel<BITS, false, false>;
+}
+
 }  // namespace
+
+// The one-launch path (see quantize_fused_kernel): `done` holds N * nseg arrival counters that have seen `epoch` calls
+// with this layout.  Returns cudaErrorCooperativeLaunchTooLarge when no CTA of the kernel fits on the device.
+cudaError_t launch_quantize_fused(const QuantArgs& a, unsigned int* done, unsigned int epoch, int sm_count, cudaStream_t st) {
+  if (a.N <= 0 || a.nseg <= 0) return cudaSuccess;
+  FusedKernel k;
+  const bool sums = a.clip_mode == CLIP_STD, count = a.count_clipped != 0;
+  switch (a.b) {
+    case 1: k = pick_fused<1>(count, sums); break;
+    case 2: k = pick_fused<2>(count, sums); break;
+    case 4: k = pick_fused<4>(count, sums); break;
+    case 8: k = pick_fused<8>(count, sums); break;
+    default: k = pick_fused<0>(count, sums); break;
+  }
+  int per_sm = 0;
+  cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, QT, 0);
+  if (e != cudaSuccess) return e;
+  if (per_sm < 1) return cudaErrorCooperativeLaunchTooLarge;
+  const long long items = (long long)a.N * (a.ntiles > 0 ? a.ntiles : 1);
+  const long long resident = (long long)per_sm * sm_count;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(items < resident ? items : resident), 1, 1);
+  cfg.blockDim = dim3(QT, 1, 1);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeCooperative;  // all CTAs co-resident or the launch fails: they wait on one another
+  attr[0].val.cooperative = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, k, a, done, epoch);
+}
 
 int quantize_run_tiles() { return QRUN; }
 

@@ -19,12 +19,13 @@ CLIP_NONE, CLIP_LAMBDA, CLIP_STD = 0, 1, 2
 (BUF_X, BUF_XTILDE, BUF_MU, BUF_MARGINS, BUF_Y, BUF_Z, BUF_YSUM, BUF_CODES, BUF_DELTA, BUF_CLIPPED, BUF_BATCH_IDX,
  BUF_COEF, BUF_U, BUF_V, BUF_VHAT) = range(15)
 OPT_SAMPLE_GLOBAL, OPT_TAP_U, OPT_CLUSTER_SIZE, OPT_USE_GRAPH, OPT_PROFILE, OPT_PERSISTENT = 0, 1, 2, 3, 4, 5
-OPT_SHARED_SCALE, OPT_AVERAGE_DIVISOR = 6, 7
+OPT_SHARED_SCALE, OPT_AVERAGE_DIVISOR, OPT_ONE_LAUNCH_QUANTIZE = 6, 7, 8
 SCHEME_BROADCAST, SCHEME_SERVER_SUM, SCHEME_SERVER_REQUANTIZE = 0, 1, 2
 (INFO_STEP_CLUSTER_SIZE, INFO_LOOP_CLUSTER_SIZE, INFO_LOOP_LAUNCHES, INFO_SNAPSHOT_ROWS_PER_TILE, INFO_SNAPSHOT_STAGES,
  INFO_ALPC_LOOP_CLUSTER_SIZE, INFO_LOOP_ROW_SLOTS, INFO_ALPC_LOOP_ROW_SLOTS, INFO_STEP_RING_STAGES,
- INFO_AGGREGATE_SPLIT, INFO_QUANT_PIPELINED_RUNS, INFO_LOOP_COORDS_PER_THREAD, INFO_ALPC_LOOP_COORDS_PER_THREAD) = range(13)
-KERNEL_NAMES = ["snapshot", "worker", "aggregate", "quant_stats", "quant_pack", "other", "inner_loop"]
+ INFO_AGGREGATE_SPLIT, INFO_QUANT_PIPELINED_RUNS, INFO_LOOP_COORDS_PER_THREAD, INFO_ALPC_LOOP_COORDS_PER_THREAD,
+ INFO_QUANT_ONE_LAUNCH) = range(14)
+KERNEL_NAMES = ["snapshot", "worker", "aggregate", "quant_stats", "quant_pack", "other", "inner_loop", "quant_fused"]
 
 # every symbol that include/lpc.h declares: (name, restype, argtypes)
 _vp, _i64, _i32, _u64, _f32, _int = C.c_void_p, C.c_int64, C.c_int32, C.c_uint64, C.c_float, C.c_int
