@@ -379,15 +379,106 @@ __global__ void __launch_bounds__(AT, 4) server_reduce_kernel(ServerArgs a) {
   }
 }
 
-// Histogram of a message's code values, the input of the entropy-coding count (Section 5.1: the experiments pass the
-// codes through Huffman's code).  One CTA per run of tiles of a worker.  Every thread counts the 32 codes it reads in counters
-// of its own -- one byte per code value, four values to a 32-bit word, word[value / 4][thread] -- so that counting
-// needs no atomic operation however skewed the codes are (near-Gaussian gradients put most of them on a few values)
-// and a warp's accesses fall on 32 different banks.  The block then adds the columns up with warp reductions and sends
-// the tile's count of every value to the message's histogram with one atomic addition each.
-constexpr int HRUN = 32;  // tiles per CTA: the tile counts are gathered in shared memory and reach the message's
-                          // histogram (a few hot addresses) once per run and segment
+constexpr int HRUN = 32;  // tiles per CTA: the counts reach the message's histogram (a few hot addresses) once per run and segment
 
+// Histogram of a message's code values, the input of the entropy-coding count (Section 5.1: the experiments pass the
+// codes through Huffman's code).
+//
+// Widths 1, 2 and 4 are counted without looking at single codes.  A thread takes 16 bytes of the stream at a time and
+// keeps one counter per code value in registers:
+//   b = 4: the four words hold 32 codes.  A 4 x 4 bit transpose across the words (two rounds of masked swaps) gives
+//          R_k, whose bit 4 i + r is bit k of code i of word r; the codes equal to v are the bits of
+//          AND_k (v_k ? R_k : ~R_k), and their number is one population count -- about 2.3 instructions per code
+//          instead of an extraction, an address and a shared-memory read-modify-write for each;
+//   b = 2: two bit planes per word, four masks and population counts per 16 codes;
+//   b = 1: the population count of the word.
+// A CTA takes a run of tiles of one worker; the thread counters are added up by warp reductions when the run or
+// the tensor segment ends, and one 64-bit atomic per value, run and segment reaches the message's histogram.  Codes
+// of a ragged end (less than 16 bytes of valid codes) are counted one by one.
+template <int BITS>
+__device__ __forceinline__ void count_unit(uint4 q, uint32_t* cnt) {
+  if constexpr (BITS == 4) {
+    uint32_t a = q.x, b = q.y, c = q.z, d = q.w, t;
+    t = ((a >> 1) ^ b) & 0x55555555u; b ^= t; a ^= t << 1;
+    t = ((c >> 1) ^ d) & 0x55555555u; d ^= t; c ^= t << 1;
+    t = ((a >> 2) ^ c) & 0x33333333u; c ^= t; a ^= t << 2;
+    t = ((b >> 2) ^ d) & 0x33333333u; d ^= t; b ^= t << 2;
+#pragma unroll
+    for (int v = 0; v < 8; ++v) {  // the low three bits of the value, then both settings of the fourth
+      const uint32_t m = ((v & 1) ? a : ~a) & ((v & 2) ? b : ~b) & ((v & 4) ? c : ~c);
+      cnt[v] += __popc(m & ~d);
+      cnt[v + 8] += __popc(m & d);
+    }
+  } else if constexpr (BITS == 2) {
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const uint32_t lo = w[i] & 0x55555555u, hi = (w[i] >> 1) & 0x55555555u;
+      cnt[0] += __popc(~(lo | hi) & 0x55555555u);
+      cnt[1] += __popc(lo & ~hi);
+      cnt[2] += __popc(hi & ~lo);
+      cnt[3] += __popc(lo & hi);
+    }
+  } else {
+    const uint32_t ones = __popc(q.x) + __popc(q.y) + __popc(q.z) + __popc(q.w);
+    cnt[1] += ones;
+    cnt[0] += 128u - ones;
+  }
+}
+
+template <int BITS>  // 1, 2, 4
+__global__ void __launch_bounds__(AT) code_histogram_swar_kernel(HistArgs a) {
+  constexpr int BINS = 1 << BITS, CPU = 128 / BITS;  // codes per 16-byte unit
+  const int worker = blockIdx.y, tid = threadIdx.x, lane = tid & 31;
+  const int tile0 = blockIdx.x * HRUN, tile1 = min(tile0 + HRUN, a.ntiles);
+  __shared__ unsigned int total[BINS];
+  if (tid < BINS) total[tid] = 0u;
+  __syncthreads();
+  uint32_t cnt[BINS];
+#pragma unroll
+  for (int v = 0; v < BINS; ++v) cnt[v] = 0u;
+  int tile = tile0;
+  while (tile < tile1) {  // one pass per tensor segment that the run touches
+    const int seg = a.tile_seg ? a.tile_seg[tile] : 0;
+    const SegInfo s = a.segs[seg];
+    const int tend = min(tile1, s.tile_first + s.tile_count);  // the run's tiles of this segment: [tile, tend)
+    const int64_t j0 = (int64_t)(tile - s.tile_first) * TILE;
+    const int64_t n = min(s.len, (int64_t)(tend - s.tile_first) * TILE) - j0;  // codes to count
+    const uint32_t* w = a.codes + (int64_t)worker * a.stride_words + s.word_off + (j0 >> 5) * BITS;  // 16-byte aligned
+    const int64_t units = n / CPU;
+    const uint4* wu = reinterpret_cast<const uint4*>(w);
+    int64_t u = tid;
+    for (; u + 3 * AT < units; u += 4 * AT) {  // four loads in flight
+      const uint4 q0 = __ldcs(wu + u), q1 = __ldcs(wu + u + AT), q2 = __ldcs(wu + u + 2 * AT), q3 = __ldcs(wu + u + 3 * AT);
+      count_unit<BITS>(q0, cnt); count_unit<BITS>(q1, cnt); count_unit<BITS>(q2, cnt); count_unit<BITS>(q3, cnt);
+    }
+    for (; u < units; u += AT) count_unit<BITS>(__ldcs(wu + u), cnt);
+    for (int64_t j = units * CPU + tid; j < n; j += AT) {  // the ragged end, code by code
+      const uint32_t code = (w[(j * BITS) >> 5] >> ((j * BITS) & 31)) & (uint32_t)(BINS - 1);
+      atomicAdd(&total[code], 1u);
+    }
+    // the segment's counts of this run go to its histogram
+#pragma unroll
+    for (int v = 0; v < BINS; ++v) {
+      const uint32_t sum = __reduce_add_sync(0xFFFFFFFFu, cnt[v]);
+      if (lane == 0 && sum) atomicAdd(&total[v], sum);
+      cnt[v] = 0u;
+    }
+    __syncthreads();
+    if (tid < BINS && total[tid]) {
+      atomicAdd(&a.hist[((int64_t)worker * a.nseg + seg) * BINS + tid], (unsigned long long)total[tid]);
+      total[tid] = 0u;
+    }
+    __syncthreads();
+    tile = tend;
+  }
+}
+
+// Widths without a bit-sliced count (8 bits, and the odd widths): every thread counts the 32 codes it reads in counters
+// of its own in shared memory -- one byte per code value, four values to a 32-bit word, word[value / 4][thread] -- so
+// that counting needs no atomic operation however skewed the codes are and a warp's accesses fall on 32 different banks.
+// The block then adds the columns up with warp reductions and sends the tile's count of every value to the message's
+// histogram with one atomic addition each.
 template <int BITS>  // 1, 2, 4, 8: code width known at compile time; 0: b in 1..8 from the arguments
 __global__ void __launch_bounds__(AT) code_histogram_kernel(HistArgs a) {
   const int worker = blockIdx.y;
@@ -502,9 +593,9 @@ cudaError_t launch_code_histogram(const HistArgs& a, cudaStream_t st) {
     return cudaGetLastError();
   };
   switch (a.b) {
-    case 1: return go(code_histogram_kernel<1>);
-    case 2: return go(code_histogram_kernel<2>);
-    case 4: return go(code_histogram_kernel<4>);
+    case 1: code_histogram_swar_kernel<1><<<grid, AT, 0, st>>>(a); return cudaGetLastError();
+    case 2: code_histogram_swar_kernel<2><<<grid, AT, 0, st>>>(a); return cudaGetLastError();
+    case 4: code_histogram_swar_kernel<4><<<grid, AT, 0, st>>>(a); return cudaGetLastError();
     case 8: return go(code_histogram_kernel<8>);
     default: return go(code_histogram_kernel<0>);
   }

@@ -895,7 +895,8 @@ int lpc_quantize_pack(lpc_ctx* c, const float* U, const float* U_sub, int64_t le
       c->one_launch = 0;
     }
   }
-  if (!c->last_one_launch) CU(c, launch_quantize_pack(a, c->stream, c->profile ? prof_hook : nullptr, c));
+  if (c->last_one_launch) c->last_pipelined_runs = 0;
+  else CU(c, launch_quantize_pack(a, c->stream, c->profile ? prof_hook : nullptr, c));
   if (!c->shared_scale) c->step2_bits += p.msg_bits * (uint64_t)c->N * (uint64_t)(c->N - 1);  // scheme (a); the server schemes count in lpc_server_reduce
   return LPC_OK;
 }

@@ -49,6 +49,7 @@ constexpr int PMAXP = 2;   // passes per CTA: SL <= 4096
 constexpr int PMAXB = 64;
 constexpr int PMAXCS = 8;
 constexpr int PMAXFLAGS = 256;
+constexpr int PMAXN = 64;      // workers in the one-launch loop (a lane carries the scales of PMAXN / 32 of them)
 constexpr int PUB_STRIDE = 16;  // publication words sit 128 bytes apart: one cache line each
 
 struct PSmem {
@@ -59,7 +60,6 @@ struct PSmem {
   // step-parity halves: margin partial sums (slot b * PMAXCS + rank) and statistics (max, S1, S2 per rank)
   unsigned long long mx[2][PMAXB * PMAXCS];
   unsigned long long sx[2][3 * PMAXCS];
-  unsigned long long dl[2][PMAXFLAGS];  // the workers' scales of a step (delta | tag), fetched by warp 0 for the whole CTA
   float ws1[PMAXP * 8], ws2[PMAXP * 8];
   uint32_t wmax[8];
   uint32_t wclip[8];
@@ -85,9 +85,6 @@ __device__ __forceinline__ void st_cluster_word(const unsigned long long* slot, 
   uint32_t remote;
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(slot)), "r"(cta));
   asm volatile("st.relaxed.cluster.shared::cluster.u64 [%0], %1;" ::"r"(remote), "l"(v) : "memory");
-}
-__device__ __forceinline__ void st_shared_word(unsigned long long* slot, unsigned long long v) {
-  asm volatile("st.relaxed.cta.shared::cta.u64 [%0], %1;" ::"r"(smem_u32(slot)), "l"(v) : "memory");
 }
 __device__ __forceinline__ unsigned long long ld_shared_word(const unsigned long long* slot) {
   unsigned long long v;
@@ -217,7 +214,6 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
   // no exchange slot may look valid before a peer has written it: tags start at 1
   for (int i = tid; i < 2 * PMAXB * PMAXCS; i += PT) (&sm.mx[0][0])[i] = 0ull;
   for (int i = tid; i < 2 * 3 * PMAXCS; i += PT) (&sm.sx[0][0])[i] = 0ull;
-  for (int i = tid; i < 2 * PMAXFLAGS; i += PT) (&sm.dl[0][0])[i] = 0ull;
   asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   __syncthreads();
 
@@ -289,18 +285,18 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
   // Applies step target-1's update to this thread's coordinates:
   //   x <- prox_{eta h}(x - eta (mean_i delta_i k_i + mu))      (Algorithm 2: the y and z updates).
   // The tagged words that hold the thread's codes are loaded for CH workers at a time, all in flight together (one L2
-  // round trip; CH covers all N workers whenever 32 words per thread suffice), and re-loaded until every tag names
-  // step target-1.  The workers' scales are the same for every thread of the CTA: the lanes of warp 0 fetch them, one
-  // worker per lane, and pass them on through shared memory as tagged words (they are published before the codes, so
-  // they are there when a thread's codes are).
+  // round trip), and re-loaded until every tag names step target-1.  The workers' scales are the same for every
+  // thread: lane l of a warp loads those of workers l, l + 32, ... and the warp hands them round by shuffles.
   constexpr int WMAX = (BITS == 0) ? 8 : (BITS == 8 ? 2 : 1);  // tagged words per group of 8 coordinates
   constexpr int NW = (BITS == 0) ? 8 : (TB >= 32 ? TB / 32 : 1);  // of which a thread reads / writes this many
-  constexpr int CH = (BITS == 0) ? 4 : 32 / (NP * NW);        // workers per round of loads
+  constexpr int CH = (BITS == 0) ? 4 : 32 / (NP * NW);         // workers per round of loads: 32 words in flight per thread
+  constexpr int DMAX = PMAXN / 32;                            // scale words per lane at most
   const int wpg = (BITS == 0) ? pa.wpg : WMAX;
   const int sub = (LPG > 1) ? (tid & (LPG - 1)) : 0;          // this thread's place in its group of 8 coordinates
   const int wfirst = (BITS == 0) ? 0 : (sub * TB) >> 5;        // first word of the group that holds its codes
   const int wshift = (BITS == 0) ? 0 : (sub * TB) & 31;        // and their position in it
   const size_t groups = (size_t)(CS * SL) >> 3;
+  const int nd = (N + 31) >> 5;                               // scale words this lane fetches
   float wcur = pa.w0;  // snapshot weight of the step whose update comes next
   auto apply_update = [&](unsigned int target) {
     const int rpar = (pa.count - (int)target) & 1;  // parity half that holds step target-1
@@ -319,8 +315,15 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
 #pragma unroll
       for (int e = 0; e < EPT; ++e) acc[p][e] = 0.f;
     }
-    unsigned long long cw[CH][NP][NW], vw[ALPC ? NP * EPT : 1];
+    unsigned long long cw[CH][NP][NW], vw[ALPC ? NP * EPT : 1], dw[DMAX];
     auto issue = [&](int i0) {
+      if (i0 == 0) {
+#pragma unroll
+        for (int q = 0; q < DMAX; ++q) {
+          const int i = lane + 32 * q;
+          dw[q] = (q < nd && i < N) ? ld_word(dwords + (size_t)i * CS * PUB_STRIDE) : good;
+        }
+      }
 #pragma unroll
       for (int j = 0; j < CH; ++j) {
         const bool live = i0 + j < N;
@@ -342,17 +345,6 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
       }
     };
     issue(0);
-    if (warp == 0) {  // the scales: lane l takes workers l, l + 32, ...
-      for (int i = lane; i < N; i += 32) {
-        unsigned long long w;
-        uint64_t t0 = 0;
-        for (uint32_t it = 0;; ++it) {
-          w = ld_word(dwords + (size_t)i * CS * PUB_STRIDE);
-          if (word_tag(w) == tag || wait_expired(it, t0)) break;
-        }
-        st_shared_word(&sm.dl[rpar][i], w);
-      }
-    }
 #pragma unroll 1
     for (int i0 = 0; i0 < N; i0 += CH) {
       uint64_t t0 = 0;
@@ -364,17 +356,22 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
           for (int p = 0; p < NP; ++p)
 #pragma unroll
             for (int w = 0; w < NW; ++w) ok = ok && word_tag(cw[j][p][w]) == tag;
-        if constexpr (ALPC) {
-          if (i0 == 0) {
+        if (i0 == 0) {
+#pragma unroll
+          for (int q = 0; q < DMAX; ++q) ok = ok && word_tag(dw[q]) == tag;
+          if constexpr (ALPC) {
 #pragma unroll
             for (int e = 0; e < NP * EPT; ++e) ok = ok && word_tag(vw[e]) == tag;
           }
+          ok = __all_sync(0xFFFFFFFFu, ok);  // the scales are shared by the warp: all lanes go on together
         }
 #ifdef LPC_TRACE
         if (i0 == 0 && blockIdx.x == 0 && blockIdx.y == 0 && tid == 0 && target >= 8 && target < 72)
           g_trace[(target - 8) * 16 + 15] = it + 1;
 #endif
-        if (ok || wait_expired(it, t0)) break;
+        bool stop = ok || wait_expired(it, t0);
+        if (i0 == 0) stop = __any_sync(0xFFFFFFFFu, stop);
+        if (stop) break;
         issue(i0);
       }
 #ifdef LPC_TRACE
@@ -382,14 +379,18 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
 #endif
 #pragma unroll
       for (int j = 0; j < CH; ++j) {
-        if (i0 + j < N) {
-          unsigned long long dword;
-          uint64_t t1 = 0;
-          for (uint32_t it = 0;; ++it) {
-            dword = ld_shared_word(&sm.dl[rpar][i0 + j]);
-            if (word_tag(dword) == tag || wait_expired(it, t1)) break;
+        // worker i0 + j's scale sits in lane (i0 + j) % 32, word (i0 + j) / 32 (every lane takes part in the shuffle)
+        const int i = i0 + j;
+        float di = __uint_as_float(__shfl_sync(0xFFFFFFFFu, (uint32_t)dw[0], i & 31));
+        if (nd > 1) {  // more than 32 workers (uniform for the launch)
+          const int q = i >> 5;
+#pragma unroll
+          for (int r = 1; r < DMAX; ++r) {
+            const float dr = __uint_as_float(__shfl_sync(0xFFFFFFFFu, (uint32_t)dw[r], i & 31));
+            if (q == r) di = dr;
           }
-          const float di = __uint_as_float((uint32_t)dword);
+        }
+        if (i0 + j < N) {
 #pragma unroll
           for (int p = 0; p < NP; ++p) {
             if (b == 32) {
@@ -916,7 +917,7 @@ bool persist_plan(int d, int N, int B, int b, int alpc, int want_cs, int max_sme
   while (P < d) P <<= 1;
   if (P < 32) P = 32;
   const int clusters = N + (alpc ? 1 : 0);
-  if (B > PMAXB || clusters > PMAXFLAGS) return false;
+  if (B > PMAXB || N > PMAXN || clusters > PMAXFLAGS) return false;
   bool found = false;
   for (int cs = 1; cs <= PMAXCS; cs <<= 1) {
     if (want_cs > 0 && cs != want_cs) continue;

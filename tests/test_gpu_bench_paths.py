@@ -55,9 +55,11 @@ def test_quantize_runs_of_whole_tiles_bit_exact(b):
         U = rng.standard_normal((N, length)).astype(np.float32)
         U[1] *= 37.0
         ctx = _ctx(N, b, orc.CLIP_STD, 2.0, seed)
+        ctx.set_option(lpc.OPT_ONE_LAUNCH_QUANTIZE, 0)  # the three-launch path that long vectors take
         codes, delta, clipped = ctx.quantize_pack(_rows_aligned(U), k)
         ctx.sync_status()
         assert ctx.query(lpc.INFO_QUANT_PIPELINED_RUNS) == want_runs, length
+        assert ctx.query(lpc.INFO_QUANT_ONE_LAUNCH) == 0
         W = orc.packed_words(length, b)
         for i in range(N):
             w, dl, cl = orc.quantize_pack(U[i], b, orc.CLIP_STD, 2.0, seed, i, k)
@@ -77,6 +79,7 @@ def test_quantize_runs_with_subtrahend_bit_exact(b):
     cur = rng.standard_normal((N, length)).astype(np.float32)
     snap = rng.standard_normal((N, length)).astype(np.float32)
     ctx = _ctx(N, b, orc.CLIP_STD, 2.5, seed)
+    ctx.set_option(lpc.OPT_ONE_LAUNCH_QUANTIZE, 0)
     codes, delta, clipped = ctx.quantize_pack(torch.from_numpy(cur).to(DEV), k, U_sub=torch.from_numpy(snap).to(DEV))
     ctx.sync_status()
     assert ctx.query(lpc.INFO_QUANT_PIPELINED_RUNS) == 1
@@ -108,6 +111,7 @@ def _full_length_case(N, log2_len, b, dist, clip, seed, k, want_split):
     U = synth.gradient_vectors(N, length, dist, seed=seed + 1, device=DEV)
     q = _ctx(N, b, orc.CLIP_STD, clip, seed)
     codes, delta, clipped = q.quantize_pack(U, k)
+    assert q.query(lpc.INFO_QUANT_ONE_LAUNCH) == 0  # longer than L2 holds: statistics, scale and codes as three launches
     assert q.query(lpc.INFO_QUANT_PIPELINED_RUNS) == length // (TILE * RUN)
     x = torch.zeros(length, device=DEV)
     q.unpack_average_prox(codes, delta, length, x, 1.0, 1e-3)
@@ -162,6 +166,7 @@ def test_three_level_codes_full_length_windows(b):
     q.unpack_average_prox(codes, delta, length, x, 1.0, 1e-3)
     q.sync_status()
     assert q.query(lpc.INFO_QUANT_PIPELINED_RUNS) == 0 and q.query(lpc.INFO_AGGREGATE_SPLIT) == 4
+    assert q.query(lpc.INFO_QUANT_ONE_LAUNCH) == 0  # 8 x 2^22 values = 134 MB
     Uh = U.cpu().numpy()
     W = orc.packed_words(length, b)
     ch = codes.cpu().numpy().view(np.uint32)
@@ -174,4 +179,33 @@ def test_three_level_codes_full_length_windows(b):
     assert (_bits(delta.cpu().numpy()[:, 0]) == _bits(dl)).all()
     ref = orc.unpack_average_prox(words, dl, length, b, None, np.zeros(length, np.float32), 1.0, 1e-3)
     assert (_bits(x.cpu().numpy()) == _bits(ref)).all()
+    q.close()
+
+
+@pytest.mark.parametrize("b", [1, 2, 3, 4, 8, 16])
+@pytest.mark.parametrize("log2_len", [16, 20])
+def test_one_launch_quantizer_short_vectors_bit_exact(b, log2_len):
+    # the sweep's short vectors (8 x 2^16, 8 x 2^20) stay in L2 between the statistics and the codes: one cooperative
+    # launch; at 2^20 the 1,024 tiles exceed the resident CTAs, so a CTA takes several tiles of different workers.
+    # Twice in a row: the arrival counters carry over from call to call.
+    N, seed = 8, 71
+    length = 1 << log2_len
+    U = synth.gradient_vectors(N, length, "student_t3", seed=b + log2_len)
+    q = _ctx(N, b, orc.CLIP_STD, 2.0, seed)
+    Ud = U.to(DEV)
+    for k in (3, 4):
+        codes, delta, clipped = q.quantize_pack(Ud, k)
+        q.sync_status()
+        assert q.query(lpc.INFO_QUANT_ONE_LAUNCH) == 1
+        W = orc.packed_words(length, b)
+        for i in range(N):
+            w, dl, cl = orc.quantize_pack(U[i].numpy(), b, orc.CLIP_STD, 2.0, seed, i, k)
+            assert (_u32(codes)[i, :W] == w).all(), (k, i)
+            assert _bits(np.float32(dl).reshape(1))[0] == _u32(delta)[i, 0] and int(_u32(clipped)[i, 0]) == cl
+    # the three-launch path on the same input gives the same bits
+    q.set_option(lpc.OPT_ONE_LAUNCH_QUANTIZE, 0)
+    c2, d2, cl2 = q.quantize_pack(Ud, 4)
+    q.sync_status()
+    assert q.query(lpc.INFO_QUANT_ONE_LAUNCH) == 0
+    assert torch.equal(c2, codes) and torch.equal(d2.view(torch.int32), delta.view(torch.int32)) and torch.equal(cl2, clipped)
     q.close()

@@ -52,15 +52,19 @@ def test_philox_streams_match_oracle_bitwise():
 
 @pytest.mark.parametrize("b", [1, 2, 3, 4, 5, 7, 8, 12, 16, 32])
 @pytest.mark.parametrize("clip", [(orc.CLIP_NONE, 1.0), (orc.CLIP_LAMBDA, 0.85), (orc.CLIP_STD, 2.5)])
-def test_quantize_pack_bit_exact(b, clip):
+@pytest.mark.parametrize("one_launch", [1, 0])
+def test_quantize_pack_bit_exact(b, clip, one_launch):
+    # one_launch = 1: the single cooperative launch that short vectors take (b = 32 always takes three launches)
     N, seed, k = 3, 1234, 7
     rng = np.random.default_rng(b * 10 + clip[0])
     for length in (1, 7, 8, 9, 31, 33, 257, 2047, 8191, 8192, 8193, 3 * 8192 + 1001):
         U = rng.standard_normal((N, length)).astype(np.float32)
         U[0] *= 1e-3
         ctx = _ctx(N, b, clip[0], clip[1], seed)
+        ctx.set_option(lpc.OPT_ONE_LAUNCH_QUANTIZE, one_launch)
         codes, delta, clipped = ctx.quantize_pack(torch.from_numpy(U).to(DEV), k)
         ctx.sync_status()
+        assert ctx.query(lpc.INFO_QUANT_ONE_LAUNCH) == (1 if one_launch and b != 32 else 0)
         rc, rd, rcl = _oracle_quantize(U, b, clip[0], clip[1], seed, k)
         assert (delta.cpu().numpy() == rd).all(), (length, delta, rd)
         assert (_u32(codes) == rc).all(), length
