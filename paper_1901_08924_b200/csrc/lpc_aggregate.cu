@@ -379,6 +379,85 @@ __global__ void __launch_bounds__(AT, 4) server_reduce_kernel(ServerArgs a) {
   }
 }
 
+// The server for 4-bit codes of at most 16 workers (sums of at most 8 bits).  A thread owns 32 consecutive coordinates:
+// per worker that is one 16-byte load, and its output -- 32 sums of BO bits, or 32 re-quantized 4-bit codes -- is BO (or
+// 4) whole words, so nothing is staged or exchanged.  The codes are added in byte lanes (even and odd codes of a word
+// apart), every load of the thread in flight at once; the sums are placed in the output words by multiply-adds with
+// constant powers of two (the low part of the product is the shifted value, the high part its spill into the next word).
+template <int BO, bool REQ>
+__global__ void __launch_bounds__(AT, 4) server_reduce4_kernel(ServerArgs a) {
+  constexpr int OW = REQ ? 4 : BO;  // output words per thread
+  const int tile = blockIdx.x, tid = threadIdx.x;
+  const int seg = a.tile_seg ? a.tile_seg[tile] : 0;
+  const SegInfo s = a.segs[seg];
+  const SegInfo so = a.segs_out[seg];
+  const int64_t j = (int64_t)(tile - s.tile_first) * TILE + tid * 32;  // this thread's first coordinate (segment-local)
+  if (j >= s.len) return;
+  const int nv = (int)min((int64_t)32, s.len - j);
+  const uint32_t* w = a.codes + s.word_off + (j >> 3);  // its four words of every stream: inside the padded stream
+  uint4 c[16];
+#pragma unroll
+  for (int i = 0; i < 16; ++i)
+    c[i] = (i < a.N) ? __ldcs(reinterpret_cast<const uint4*>(w + (int64_t)i * a.stride_words)) : make_uint4(0u, 0u, 0u, 0u);
+  uint32_t ev[4] = {0, 0, 0, 0}, od[4] = {0, 0, 0, 0};  // sums of the codes 8q + 2r in byte r of ev[q], of 8q + 2r + 1 in od[q]
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {  // 16 codes of at most 15: a byte lane cannot overflow
+    const uint32_t x[4] = {c[i].x, c[i].y, c[i].z, c[i].w};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      ev[q] += x[q] & 0x0F0F0F0Fu;
+      od[q] += (x[q] >> 4) & 0x0F0F0F0Fu;
+    }
+  }
+  uint32_t out[OW];
+#pragma unroll
+  for (int i = 0; i < OW; ++i) out[i] = 0u;
+  if constexpr (REQ) {
+    // scheme (c), Eq. 4: the average K / N in grid units, rounded by rule (1) with the server's own rounding stream
+    const float fN = (float)a.N;
+    const bool pow2 = (a.N & (a.N - 1)) == 0;
+    const float invN = __fdiv_rn(1.0f, fN);
+    const float magic = 8388608.f + (float)(a.N << 3);  // 2^23 + the offsets of N codes: as_float(2^23 | sum) - magic = K exactly
+    float dummy = 0.f;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      float v[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const uint32_t sum = (((e & 1) ? od[q] : ev[q]) >> (8 * (e >> 1))) & 0xFFu;
+        const float K = __fsub_rn(__uint_as_float(0x4B000000u | sum), magic);
+        v[e] = pow2 ? mul_rn(K, invN) : __fdiv_rn(K, fN);
+      }
+      const U4 r = stream_block(a.seed, TAG_REQUANT, 0u, a.k, s.block_base + (uint32_t)(j >> 3) + (uint32_t)q);
+      out[q] = (uint32_t)quantize_group8<4, false>(v, 1.0f, r, 0.f, 0.f, dummy);
+    }
+  } else {
+    // scheme (b): the index sums in offset binary; sum of codes - 8 N + 2^(BO-1) >= 0 since 2^(BO-1) >= 8 N
+    const uint32_t shift = (1u << (BO - 1)) - ((uint32_t)a.N << 3);
+#pragma unroll
+    for (int e = 0; e < 32; ++e) {
+      const int q = e >> 3, r = (e & 7) >> 1;
+      const uint32_t val = ((((e & 1) ? od[q] : ev[q]) >> (8 * r)) & 0xFFu) + shift;
+      const int pos = e * BO, wi = pos >> 5, sh = pos & 31;
+      out[wi] += val << sh;
+      if (sh + BO > 32) out[wi + 1] += val >> (32 - sh);
+    }
+  }
+  if (nv < 32) {  // nothing but zeros past the end of the segment
+    const int bits = nv * (REQ ? 4 : BO);
+#pragma unroll
+    for (int i = 0; i < OW; ++i) {
+      const int left = bits - 32 * i;
+      if (left <= 0) out[i] = 0u;
+      else if (left < 32) out[i] &= (1u << left) - 1u;
+    }
+  }
+  uint32_t* o = a.out + so.word_off + (j >> 5) * OW;
+#pragma unroll
+  for (int i = 0; i < OW; ++i)
+    if ((j >> 5) * OW + i < so.pad_words) o[i] = out[i];
+}
+
 constexpr int HRUN = 32;  // tiles per CTA: the counts reach the message's histogram (a few hot addresses) once per run and segment
 
 // Histogram of a message's code values, the input of the entropy-coding count (Section 5.1: the experiments pass the
@@ -604,6 +683,17 @@ cudaError_t launch_code_histogram(const HistArgs& a, cudaStream_t st) {
 cudaError_t launch_server_reduce(const ServerArgs& a, cudaStream_t st) {
   if (a.ntiles <= 0) return cudaSuccess;
   const dim3 grid((unsigned)a.ntiles), block(AT);
+  if (a.b == 4 && a.N <= 16) {  // sums of at most 8 bits: whole words per thread
+    if (a.requantize) { server_reduce4_kernel<4, true><<<grid, block, 0, st>>>(a); return cudaGetLastError(); }
+    switch (a.b_out) {
+      case 4: server_reduce4_kernel<4, false><<<grid, block, 0, st>>>(a); return cudaGetLastError();
+      case 5: server_reduce4_kernel<5, false><<<grid, block, 0, st>>>(a); return cudaGetLastError();
+      case 6: server_reduce4_kernel<6, false><<<grid, block, 0, st>>>(a); return cudaGetLastError();
+      case 7: server_reduce4_kernel<7, false><<<grid, block, 0, st>>>(a); return cudaGetLastError();
+      case 8: server_reduce4_kernel<8, false><<<grid, block, 0, st>>>(a); return cudaGetLastError();
+      default: break;
+    }
+  }
   switch (a.b) {
     case 2: server_reduce_kernel<2><<<grid, block, 0, st>>>(a); break;
     case 4: server_reduce_kernel<4><<<grid, block, 0, st>>>(a); break;

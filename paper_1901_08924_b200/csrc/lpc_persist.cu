@@ -112,6 +112,14 @@ __device__ __noinline__ Scale scale_out_of_line(uint32_t max_bits, float S1, flo
 __device__ __noinline__ float coef_out_of_line(int loss, float m, float m_snap, float y) {
   return __fsub_rn(loss_deriv(loss, m, y), loss_deriv(loss, m_snap, y));
 }
+__device__ __noinline__ int64_t sample_row_out_of_line(uint64_t seed, uint32_t tag, uint32_t worker, uint64_t k, uint32_t slot,
+                                                       int64_t lo, int64_t span) {
+  const U4 r = stream_block(seed, tag, worker, k, slot);
+  return lo + (int64_t)(((uint64_t)r.x * (uint64_t)span) >> 32);
+}
+__device__ __noinline__ bool spin_expired_out_of_line(uint32_t it, uint64_t& t0, unsigned int* abort_flag, unsigned int* dev_status) {
+  return spin_expired(it, t0, abort_flag, dev_status);
+}
 __device__ __forceinline__ float tree_small(const float* v, int n) {  // n in {1, 2, 4, 8}
   if (n == 1) return v[0];
   if (n == 2) return add_rn(v[0], v[1]);
@@ -234,8 +242,8 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
       else asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
     }
     if (tid >= lo && tid < hi) {
-      const U4 r = stream_block(a.seed, is_J ? TAG_BATCH_J : TAG_BATCH, is_J ? 0u : (uint32_t)worker, a.k_base + (uint64_t)t, (uint32_t)tid);
-      const int64_t row = samp_lo + (int64_t)(((uint64_t)r.x * (uint64_t)samp_span) >> 32);
+      const int64_t row = sample_row_out_of_line(a.seed, is_J ? TAG_BATCH_J : TAG_BATCH, is_J ? 0u : (uint32_t)worker,
+                                                 a.k_base + (uint64_t)t, (uint32_t)tid, samp_lo, samp_span);
       int slot = sb + tid;
       if (slot >= RS) slot -= RS;
       if (width > 0) bulk_load(rows + (size_t)slot * SL, a.X + row * (int64_t)d + c0, row_bytes, bar);
@@ -280,7 +288,10 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
 
   // Every spin in this kernel ends: after about two seconds without progress the thread records a timeout and
   // raises the abort flag, which ends all other spins at their next look at it.
-  auto wait_expired = [&](uint32_t it, uint64_t& t0) -> bool { return spin_expired(it, t0, pa.abort_flag, a.dev_status); };
+  auto wait_expired = [&](uint32_t it, uint64_t& t0) -> bool {
+    if ((it & 63u) != 63u) return false;  // the rare path is out of line: the loop body is fetched anew every step, its size counts
+    return spin_expired_out_of_line(it, t0, pa.abort_flag, a.dev_status);
+  };
 
   // Applies step target-1's update to this thread's coordinates:
   //   x <- prox_{eta h}(x - eta (mean_i delta_i k_i + mu))      (Algorithm 2: the y and z updates).
@@ -289,7 +300,7 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
   // thread: lane l of a warp loads those of workers l, l + 32, ... and the warp hands them round by shuffles.
   constexpr int WMAX = (BITS == 0) ? 8 : (BITS == 8 ? 2 : 1);  // tagged words per group of 8 coordinates
   constexpr int NW = (BITS == 0) ? 8 : (TB >= 32 ? TB / 32 : 1);  // of which a thread reads / writes this many
-  constexpr int CH = (BITS == 0) ? 4 : 32 / (NP * NW);         // workers per round of loads: 32 words in flight per thread
+  constexpr int CH = (BITS == 0) ? 4 : 16 / (NP * NW) > 0 ? 16 / (NP * NW) : 1;  // workers per round of loads
   constexpr int DMAX = PMAXN / 32;                            // scale words per lane at most
   const int wpg = (BITS == 0) ? pa.wpg : WMAX;
   const int sub = (LPG > 1) ? (tid & (LPG - 1)) : 0;          // this thread's place in its group of 8 coordinates
@@ -316,23 +327,29 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
       for (int e = 0; e < EPT; ++e) acc[p][e] = 0.f;
     }
     unsigned long long cw[CH][NP][NW], vw[ALPC ? NP * EPT : 1], dw[DMAX];
+    // No load is predicated (a branch per load would double the size of this code, and the loop body is fetched anew every
+    // step): a thread without coordinates in a pass reads the words of coordinate 0, a round that reaches past the last
+    // worker repeats the last one, and such a worker enters the sums with the scale 0 that the lanes past N hold.
+    size_t gq[NP];
+#pragma unroll
+    for (int p = 0; p < NP; ++p) gq[p] = (act[p] ? (size_t)(cc[p] >> 3) : 0) * wpg + wfirst;
+    const size_t wstride = groups * wpg;
     auto issue = [&](int i0) {
       if (i0 == 0) {
 #pragma unroll
         for (int q = 0; q < DMAX; ++q) {
           const int i = lane + 32 * q;
-          dw[q] = (q < nd && i < N) ? ld_word(dwords + (size_t)i * CS * PUB_STRIDE) : good;
+          dw[q] = ld_word(dwords + (size_t)min(i, N - 1) * CS * PUB_STRIDE);
+          if (i >= N) dw[q] = good;  // scale 0: contributes nothing
         }
       }
 #pragma unroll
       for (int j = 0; j < CH; ++j) {
-        const bool live = i0 + j < N;
+        const unsigned long long* q = ll_in + (size_t)min(i0 + j, N - 1) * wstride;
 #pragma unroll
-        for (int p = 0; p < NP; ++p) {
-          const unsigned long long* q = ll_in + ((size_t)(i0 + j) * groups + (size_t)(cc[p] >> 3)) * wpg + wfirst;
+        for (int p = 0; p < NP; ++p)
 #pragma unroll
-          for (int w = 0; w < NW; ++w) cw[j][p][w] = (live && act[p] && w < wpg) ? ld_word(q + w) : good;
-        }
+          for (int w = 0; w < NW; ++w) cw[j][p][w] = (w < wpg) ? ld_word(q + gq[p] + w) : good;
       }
       if constexpr (ALPC) {
         if (i0 == 0) {
@@ -340,15 +357,16 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
           for (int p = 0; p < NP; ++p)
 #pragma unroll
             for (int e = 0; e < EPT; ++e)
-              vw[p * EPT + e] = act[p] ? ld_word(pa.ll_vhat + (size_t)rpar * groups * 8 + cc[p] + e) : good;
+              vw[p * EPT + e] = ld_word(pa.ll_vhat + (size_t)rpar * groups * 8 + (act[p] ? cc[p] : c0) + e);
         }
       }
     };
-    issue(0);
 #pragma unroll 1
     for (int i0 = 0; i0 < N; i0 += CH) {
       uint64_t t0 = 0;
+#pragma unroll 1
       for (uint32_t it = 0;; ++it) {
+        issue(i0);
         bool ok = true;
 #pragma unroll
         for (int j = 0; j < CH; ++j)
@@ -372,7 +390,6 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
         bool stop = ok || wait_expired(it, t0);
         if (i0 == 0) stop = __any_sync(0xFFFFFFFFu, stop);
         if (stop) break;
-        issue(i0);
       }
 #ifdef LPC_TRACE
       if (i0 == 0) { const int t = (int)target; LPC_TRACE_MARK(3); }
@@ -390,7 +407,7 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
             if (q == r) di = dr;
           }
         }
-        if (i0 + j < N) {
+        {
 #pragma unroll
           for (int p = 0; p < NP; ++p) {
             if (b == 32) {
@@ -419,7 +436,6 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
           }
         }
       }
-      if (i0 + CH < N) issue(i0 + CH);
     }
 #pragma unroll
     for (int p = 0; p < NP; ++p) {
@@ -445,7 +461,7 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
 
   int sb = 0;  // first row slot of the current step, (t * B) % RS
 #pragma unroll 1
-  for (int t = 0; t < pa.count; ++t) {
+  for (int t = 0; t <= pa.count; ++t) {  // the pass t = count only applies the last step's update (one copy of that code)
     const uint32_t row_parity = (uint32_t)((t >> 1) & 1);
     const uint64_t k = a.k_base + (uint64_t)t;
     const int wpar = (pa.count - 1 - t) & 1;  // parity half of the exchange buffers this step writes
@@ -478,6 +494,7 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
 
     LPC_TRACE_MARK(2);
     if (t > 0) apply_update((unsigned int)t);  // x_t = prox(x_{t-1} - eta v_{t-1})  (Algorithm 2: y_t, z_t)
+    if (t == pa.count) break;
     if constexpr (ALPC) {  // step 6: x = tau1 z + tau2 x~ + (1 - tau1 - tau2) y
 #pragma unroll
       for (int p = 0; p < NP; ++p)
@@ -621,37 +638,36 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
           }
         }
       }
-      if (PA < B) {
-        __syncthreads();  // nobody reads this step's rows any more
-        if (t + 1 < pa.count) fetch_rows(t + 1, sb_next, PA, B);
+    } else {
+      // scale (Eq. 2): this thread's and this warp's part of max |u| and of the tree sums
+      uint32_t mx = 0;
+#pragma unroll
+      for (int p = 0; p < NP; ++p) {
+#pragma unroll
+        for (int e = 0; e < EPT; ++e) mx = max(mx, __float_as_uint(fabsf(u[p][e])));
+        if (a.clip_mode == CLIP_STD) {
+          float sq[EPT];
+#pragma unroll
+          for (int e = 0; e < EPT; ++e) sq[e] = mul_rn(u[p][e], u[p][e]);
+          float s1 = tree_ept<EPT>(u[p]), s2 = tree_ept<EPT>(sq);
+#pragma unroll
+          for (int m = 1; m < 32; m <<= 1) {
+            s1 = add_rn(s1, __shfl_xor_sync(0xFFFFFFFFu, s1, m));
+            s2 = add_rn(s2, __shfl_xor_sync(0xFFFFFFFFu, s2, m));
+          }
+          if (lane == 0) { sm.ws1[p * 8 + warp] = s1; sm.ws2[p * 8 + warp] = s2; }
+        }
       }
+      mx = warp_max_u32(mx);
+      if (lane == 0) sm.wmax[warp] = mx;
+    }
+    __syncthreads();  // u is formed everywhere: nobody reads this step's rows any more
+    LPC_TRACE_MARK(10);
+    if (t + 1 < pa.count) fetch_rows(t + 1, sb_next, PA, B);  // into the slots this step's rows leave free
+    if (is_J) {
       sb = sb_next;
       continue;
     }
-    // scale (Eq. 2)
-    uint32_t mx = 0;
-#pragma unroll
-    for (int p = 0; p < NP; ++p) {
-#pragma unroll
-      for (int e = 0; e < EPT; ++e) mx = max(mx, __float_as_uint(fabsf(u[p][e])));
-      if (a.clip_mode == CLIP_STD) {
-        float sq[EPT];
-#pragma unroll
-        for (int e = 0; e < EPT; ++e) sq[e] = mul_rn(u[p][e], u[p][e]);
-        float s1 = tree_ept<EPT>(u[p]), s2 = tree_ept<EPT>(sq);
-#pragma unroll
-        for (int m = 1; m < 32; m <<= 1) {
-          s1 = add_rn(s1, __shfl_xor_sync(0xFFFFFFFFu, s1, m));
-          s2 = add_rn(s2, __shfl_xor_sync(0xFFFFFFFFu, s2, m));
-        }
-        if (lane == 0) { sm.ws1[p * 8 + warp] = s1; sm.ws2[p * 8 + warp] = s2; }
-      }
-    }
-    mx = warp_max_u32(mx);
-    if (lane == 0) sm.wmax[warp] = mx;
-    __syncthreads();
-    LPC_TRACE_MARK(10);
-    if (t + 1 < pa.count) fetch_rows(t + 1, sb_next, PA, B);  // the slots this step's rows leave free (u is formed)
     if (tid == 0) {
       uint32_t m = 0;
       for (int w = 0; w < 8; ++w) m = max(m, sm.wmax[w]);
@@ -814,8 +830,7 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
     sb = sb_next;
   }
 
-  // the last step's update, then the slices of the final state go back to memory (worker 0's cluster)
-  if (pa.count > 0) apply_update((unsigned int)pa.count);
+  // the slices of the final state go back to memory (worker 0's cluster)
   if (worker == 0) {
 #pragma unroll
     for (int p = 0; p < NP; ++p) {
