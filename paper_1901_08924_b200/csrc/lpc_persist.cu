@@ -301,13 +301,11 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
   constexpr int WMAX = (BITS == 0) ? 8 : (BITS == 8 ? 2 : 1);  // tagged words per group of 8 coordinates
   constexpr int NW = (BITS == 0) ? 8 : (TB >= 32 ? TB / 32 : 1);  // of which a thread reads / writes this many
   constexpr int CH = (BITS == 0) ? 4 : 16 / (NP * NW) > 0 ? 16 / (NP * NW) : 1;  // workers per round of loads
-  constexpr int DMAX = PMAXN / 32;                            // scale words per lane at most
   const int wpg = (BITS == 0) ? pa.wpg : WMAX;
   const int sub = (LPG > 1) ? (tid & (LPG - 1)) : 0;          // this thread's place in its group of 8 coordinates
   const int wfirst = (BITS == 0) ? 0 : (sub * TB) >> 5;        // first word of the group that holds its codes
   const int wshift = (BITS == 0) ? 0 : (sub * TB) & 31;        // and their position in it
   const size_t groups = (size_t)(CS * SL) >> 3;
-  const int nd = (N + 31) >> 5;                               // scale words this lane fetches
   float wcur = pa.w0;  // snapshot weight of the step whose update comes next
   auto apply_update = [&](unsigned int target) {
     const int rpar = (pa.count - (int)target) & 1;  // parity half that holds step target-1
@@ -326,115 +324,96 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
 #pragma unroll
       for (int e = 0; e < EPT; ++e) acc[p][e] = 0.f;
     }
-    unsigned long long cw[CH][NP][NW], vw[ALPC ? NP * EPT : 1], dw[DMAX];
-    // No load is predicated (a branch per load would double the size of this code, and the loop body is fetched anew every
-    // step): a thread without coordinates in a pass reads the words of coordinate 0, a round that reaches past the last
-    // worker repeats the last one, and such a worker enters the sums with the scale 0 that the lanes past N hold.
+    unsigned long long cw[CH][NP][NW], vw[ALPC ? NP * EPT : 1], dw;
+    // No load is predicated and no round is special (branches and a peeled first round would double the size of this
+    // code, and the loop body is fetched anew every step): a thread without coordinates in a pass reads the words of
+    // coordinate 0, a round that reaches past the last worker repeats the last one with the scale 0, and lane l of a
+    // warp fetches the scale of the round's worker l % CH for the whole warp.
     size_t gq[NP];
 #pragma unroll
     for (int p = 0; p < NP; ++p) gq[p] = (act[p] ? (size_t)(cc[p] >> 3) : 0) * wpg + wfirst;
     const size_t wstride = groups * wpg;
-    auto issue = [&](int i0) {
-      if (i0 == 0) {
+    auto issue_vhat = [&]() {
 #pragma unroll
-        for (int q = 0; q < DMAX; ++q) {
-          const int i = lane + 32 * q;
-          dw[q] = ld_word(dwords + (size_t)min(i, N - 1) * CS * PUB_STRIDE);
-          if (i >= N) dw[q] = good;  // scale 0: contributes nothing
-        }
-      }
+      for (int p = 0; p < NP; ++p)
 #pragma unroll
-      for (int j = 0; j < CH; ++j) {
-        const unsigned long long* q = ll_in + (size_t)min(i0 + j, N - 1) * wstride;
-#pragma unroll
-        for (int p = 0; p < NP; ++p)
-#pragma unroll
-          for (int w = 0; w < NW; ++w) cw[j][p][w] = (w < wpg) ? ld_word(q + gq[p] + w) : good;
-      }
-      if constexpr (ALPC) {
-        if (i0 == 0) {
-#pragma unroll
-          for (int p = 0; p < NP; ++p)
-#pragma unroll
-            for (int e = 0; e < EPT; ++e)
-              vw[p * EPT + e] = ld_word(pa.ll_vhat + (size_t)rpar * groups * 8 + (act[p] ? cc[p] : c0) + e);
-        }
-      }
+        for (int e = 0; e < EPT; ++e)
+          vw[p * EPT + e] = ld_word(pa.ll_vhat + (size_t)rpar * groups * 8 + (act[p] ? cc[p] : c0) + e);
     };
+    if constexpr (ALPC) issue_vhat();
 #pragma unroll 1
     for (int i0 = 0; i0 < N; i0 += CH) {
       uint64_t t0 = 0;
+      const int mine = i0 + (lane & (CH - 1));  // the worker whose scale this lane fetches
 #pragma unroll 1
       for (uint32_t it = 0;; ++it) {
-        issue(i0);
-        bool ok = true;
+        dw = ld_word(dwords + (size_t)min(mine, N - 1) * CS * PUB_STRIDE);
+#pragma unroll
+        for (int j = 0; j < CH; ++j) {
+          const unsigned long long* q = ll_in + (size_t)min(i0 + j, N - 1) * wstride;
+#pragma unroll
+          for (int p = 0; p < NP; ++p)
+#pragma unroll
+            for (int w = 0; w < NW; ++w) cw[j][p][w] = (w < wpg) ? ld_word(q + gq[p] + w) : good;
+        }
+        bool ok = word_tag(dw) == tag;
 #pragma unroll
         for (int j = 0; j < CH; ++j)
 #pragma unroll
           for (int p = 0; p < NP; ++p)
 #pragma unroll
             for (int w = 0; w < NW; ++w) ok = ok && word_tag(cw[j][p][w]) == tag;
-        if (i0 == 0) {
-#pragma unroll
-          for (int q = 0; q < DMAX; ++q) ok = ok && word_tag(dw[q]) == tag;
-          if constexpr (ALPC) {
-#pragma unroll
-            for (int e = 0; e < NP * EPT; ++e) ok = ok && word_tag(vw[e]) == tag;
-          }
-          ok = __all_sync(0xFFFFFFFFu, ok);  // the scales are shared by the warp: all lanes go on together
-        }
 #ifdef LPC_TRACE
         if (i0 == 0 && blockIdx.x == 0 && blockIdx.y == 0 && tid == 0 && target >= 8 && target < 72)
           g_trace[(target - 8) * 16 + 15] = it + 1;
 #endif
-        bool stop = ok || wait_expired(it, t0);
-        if (i0 == 0) stop = __any_sync(0xFFFFFFFFu, stop);
-        if (stop) break;
+        // the scales are shared by the warp: all lanes go on together
+        if (__all_sync(0xFFFFFFFFu, ok) || __any_sync(0xFFFFFFFFu, wait_expired(it, t0))) break;
       }
 #ifdef LPC_TRACE
       if (i0 == 0) { const int t = (int)target; LPC_TRACE_MARK(3); }
 #endif
+      const uint32_t dmine = (mine < N) ? (uint32_t)dw : 0u;
 #pragma unroll
       for (int j = 0; j < CH; ++j) {
-        // worker i0 + j's scale sits in lane (i0 + j) % 32, word (i0 + j) / 32 (every lane takes part in the shuffle)
-        const int i = i0 + j;
-        float di = __uint_as_float(__shfl_sync(0xFFFFFFFFu, (uint32_t)dw[0], i & 31));
-        if (nd > 1) {  // more than 32 workers (uniform for the launch)
-          const int q = i >> 5;
+        const float di = __uint_as_float(__shfl_sync(0xFFFFFFFFu, dmine, j));
 #pragma unroll
-          for (int r = 1; r < DMAX; ++r) {
-            const float dr = __uint_as_float(__shfl_sync(0xFFFFFFFFu, (uint32_t)dw[r], i & 31));
-            if (q == r) di = dr;
-          }
-        }
-        {
+        for (int p = 0; p < NP; ++p) {
+          if (b == 32) {
 #pragma unroll
-          for (int p = 0; p < NP; ++p) {
-            if (b == 32) {
-#pragma unroll
-              for (int e = 0; e < EPT; ++e) {
-                const float val = (cc[p] + e < d && e < NW) ? __uint_as_float((uint32_t)cw[j][p][e < NW ? e : 0]) : 0.f;
-                acc[p][e] = add_rn(acc[p][e], mul_rn(di, val));
-              }
-            } else {
-              uint64_t lo = (uint64_t)(uint32_t)cw[j][p][0], hi = 0;
-              if constexpr (NW >= 2) lo |= (uint64_t)(uint32_t)cw[j][p][1] << 32;
-              if constexpr (NW >= 4) hi = (uint64_t)(uint32_t)cw[j][p][2] | ((uint64_t)(uint32_t)cw[j][p][3] << 32);
-              float kf[8];
-              if constexpr (BITS == 0) {
-#pragma unroll
-                for (int e = 0; e < 8; ++e) kf[e] = index_as_float(extract_bits(lo, hi, e * b, b), b);
-              } else {
-                // this thread's EPT codes start at bit wshift of the word: decode them as the first codes of a group
-                // (the entries past EPT are not used and cost nothing)
-                if constexpr (TB < 32) lo = ((uint32_t)lo >> wshift) & ((1u << TB) - 1u);
-                decode8<BITS ? BITS : 1>(lo, kf);
-              }
-#pragma unroll
-              for (int e = 0; e < EPT; ++e) acc[p][e] = add_rn(acc[p][e], mul_rn(di, kf[e]));
+            for (int e = 0; e < EPT; ++e) {
+              const float val = (cc[p] + e < d && e < NW) ? __uint_as_float((uint32_t)cw[j][p][e < NW ? e : 0]) : 0.f;
+              acc[p][e] = add_rn(acc[p][e], mul_rn(di, val));
             }
+          } else {
+            uint64_t lo = (uint64_t)(uint32_t)cw[j][p][0], hi = 0;
+            if constexpr (NW >= 2) lo |= (uint64_t)(uint32_t)cw[j][p][1] << 32;
+            if constexpr (NW >= 4) hi = (uint64_t)(uint32_t)cw[j][p][2] | ((uint64_t)(uint32_t)cw[j][p][3] << 32);
+            float kf[8];
+            if constexpr (BITS == 0) {
+#pragma unroll
+              for (int e = 0; e < 8; ++e) kf[e] = index_as_float(extract_bits(lo, hi, e * b, b), b);
+            } else {
+              // this thread's EPT codes start at bit wshift of the word: decode them as the first codes of a group
+              // (the entries past EPT are not used and cost nothing)
+              if constexpr (TB < 32) lo = ((uint32_t)lo >> wshift) & ((1u << TB) - 1u);
+              decode8<BITS ? BITS : 1>(lo, kf);
+            }
+#pragma unroll
+            for (int e = 0; e < EPT; ++e) acc[p][e] = add_rn(acc[p][e], mul_rn(di, kf[e]));
           }
         }
+      }
+    }
+    if constexpr (ALPC) {  // the second estimator's words were requested first: they are here by now
+      uint64_t t0 = 0;
+#pragma unroll 1
+      for (uint32_t it = 0;; ++it) {
+        bool ok = true;
+#pragma unroll
+        for (int e = 0; e < NP * EPT; ++e) ok = ok && word_tag(vw[e]) == tag;
+        if (ok || wait_expired(it, t0)) break;
+        issue_vhat();
       }
     }
 #pragma unroll
