@@ -395,18 +395,21 @@ __global__ void __launch_bounds__(AT, 4) server_reduce4_kernel(ServerArgs a) {
   if (j >= s.len) return;
   const int nv = (int)min((int64_t)32, s.len - j);
   const uint32_t* w = a.codes + s.word_off + (j >> 3);  // its four words of every stream: inside the padded stream
-  uint4 c[16];
-#pragma unroll
-  for (int i = 0; i < 16; ++i)
-    c[i] = (i < a.N) ? __ldcs(reinterpret_cast<const uint4*>(w + (int64_t)i * a.stride_words)) : make_uint4(0u, 0u, 0u, 0u);
   uint32_t ev[4] = {0, 0, 0, 0}, od[4] = {0, 0, 0, 0};  // sums of the codes 8q + 2r in byte r of ev[q], of 8q + 2r + 1 in od[q]
+#pragma unroll 1
+  for (int i0 = 0; i0 < a.N; i0 += 8) {  // eight workers per round, their loads in flight together (uniform trip count)
+    uint4 c[8];
 #pragma unroll
-  for (int i = 0; i < 16; ++i) {  // 16 codes of at most 15: a byte lane cannot overflow
-    const uint32_t x[4] = {c[i].x, c[i].y, c[i].z, c[i].w};
+    for (int i = 0; i < 8; ++i)
+      c[i] = (i0 + i < a.N) ? __ldcs(reinterpret_cast<const uint4*>(w + (int64_t)(i0 + i) * a.stride_words)) : make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      ev[q] += x[q] & 0x0F0F0F0Fu;
-      od[q] += (x[q] >> 4) & 0x0F0F0F0Fu;
+    for (int i = 0; i < 8; ++i) {  // 16 codes of at most 15: a byte lane cannot overflow
+      const uint32_t x[4] = {c[i].x, c[i].y, c[i].z, c[i].w};
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        ev[q] += x[q] & 0x0F0F0F0Fu;
+        od[q] += (x[q] >> 4) & 0x0F0F0F0Fu;
+      }
     }
   }
   uint32_t out[OW];
@@ -419,18 +422,22 @@ __global__ void __launch_bounds__(AT, 4) server_reduce4_kernel(ServerArgs a) {
     const float invN = __fdiv_rn(1.0f, fN);
     const float magic = 8388608.f + (float)(a.N << 3);  // 2^23 + the offsets of N codes: as_float(2^23 | sum) - magic = K exactly
     float dummy = 0.f;
+    auto requantize = [&](auto average) {
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      float v[8];
+      for (int q = 0; q < 4; ++q) {
+        float v[8];
 #pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        const uint32_t sum = (((e & 1) ? od[q] : ev[q]) >> (8 * (e >> 1))) & 0xFFu;
-        const float K = __fsub_rn(__uint_as_float(0x4B000000u | sum), magic);
-        v[e] = pow2 ? mul_rn(K, invN) : __fdiv_rn(K, fN);
+        for (int e = 0; e < 8; ++e) {
+          const uint32_t sum = (((e & 1) ? od[q] : ev[q]) >> (8 * (e >> 1))) & 0xFFu;
+          v[e] = average(__fsub_rn(__uint_as_float(0x4B000000u | sum), magic));
+        }
+        const U4 r = stream_block(a.seed, TAG_REQUANT, 0u, a.k, s.block_base + (uint32_t)(j >> 3) + (uint32_t)q);
+        out[q] = (uint32_t)quantize_group8<4, false>(v, 1.0f, r, 0.f, 0.f, dummy);
       }
-      const U4 r = stream_block(a.seed, TAG_REQUANT, 0u, a.k, s.block_base + (uint32_t)(j >> 3) + (uint32_t)q);
-      out[q] = (uint32_t)quantize_group8<4, false>(v, 1.0f, r, 0.f, 0.f, dummy);
-    }
+    };
+    // K / N: a multiplication by the exact reciprocal when N is a power of two (the same value), else the division
+    if (pow2) requantize([&](float K) { return mul_rn(K, invN); });
+    else requantize([&](float K) { return __fdiv_rn(K, fN); });
   } else {
     // scheme (b): the index sums in offset binary; sum of codes - 8 N + 2^(BO-1) >= 0 since 2^(BO-1) >= 8 N
     const uint32_t shift = (1u << (BO - 1)) - ((uint32_t)a.N << 3);

@@ -543,7 +543,7 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
           bool ok = true;
 #pragma unroll
           for (int q = 0; q < PMAXCS; ++q) {
-            w[q] = (q < CS) ? ld_shared_word(&sm.mx[xpar][tid * PMAXCS + q]) : ((unsigned long long)tag << 32);
+            w[q] = ld_shared_word(&sm.mx[xpar][tid * PMAXCS + min(q, CS - 1)]);  // past the cluster: the last rank again, unused
             ok = ok && word_tag(w[q]) == tag;
           }
           if (ok || wait_expired(it, t0)) break;
@@ -672,7 +672,7 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
           for (int j = 0; j < 3; ++j) {
 #pragma unroll
             for (int q = 0; q < PMAXCS; ++q) {
-              w[j][q] = (q < CS) ? ld_shared_word(&sm.sx[xpar][j * PMAXCS + q]) : ((unsigned long long)tag << 32);
+              w[j][q] = ld_shared_word(&sm.sx[xpar][j * PMAXCS + min(q, CS - 1)]);  // past the cluster: the last rank again
               ok = ok && word_tag(w[j][q]) == tag;
             }
           }
