@@ -53,6 +53,12 @@ __device__ __forceinline__ void load_chunk(const uint32_t* __restrict__ w, int64
     lo = reinterpret_cast<const uint16_t*>(w)[g];
   } else if (BITS == 1) {
     lo = reinterpret_cast<const uint8_t*>(w)[g];
+  } else if (BITS == 3) {
+    // three bytes at byte 3 g: from the aligned word that holds the first and, where they run over, the next one
+    const int64_t idx = (3 * g) >> 2;
+    const int sh = (int)((3 * g) & 3) * 8;
+    const uint32_t w0 = w[idx], w1 = (sh > 8 && idx + 1 < pad_words) ? w[idx + 1] : 0u;
+    lo = __funnelshift_r(w0, w1, sh) & 0xFFFFFFu;
   } else {
     const uint8_t* bytes = reinterpret_cast<const uint8_t*>(w);
     const int64_t b0 = g * b, limit = pad_words * 4;
@@ -75,7 +81,7 @@ __device__ __forceinline__ uint32_t extract(uint64_t lo, uint64_t hi, int pos, i
   return (uint32_t)v & ((1u << b) - 1u);
 }
 
-template <int BITS>  // 1, 2, 4, 8: fixed width; 0: b in 1..16 from the arguments; 32: floats
+template <int BITS>  // 1, 2, 3, 4, 8: fixed width; 0: b in 1..16 from the arguments; 32: floats
 __global__ void __launch_bounds__(AT) unpack_average_prox_kernel(AggArgs a) {
   // a.split CTAs share a tile (each takes AITER / split of its sweeps): short vectors still fill the machine
   const int tile = blockIdx.x / a.split, part = blockIdx.x % a.split;
@@ -723,6 +729,7 @@ cudaError_t launch_unpack_average_prox(const AggArgs& a, cudaStream_t st) {
   switch (a.b) {
     case 1: unpack_average_prox_kernel<1><<<grid, block, sh, st>>>(a); break;
     case 2: unpack_average_prox_kernel<2><<<grid, block, sh, st>>>(a); break;
+    case 3: unpack_average_prox_kernel<3><<<grid, block, sh, st>>>(a); break;
     case 4: unpack_average_prox_kernel<4><<<grid, block, sh, st>>>(a); break;
     case 8: unpack_average_prox_kernel<8><<<grid, block, sh, st>>>(a); break;
     case 32: unpack_average_prox_kernel<32><<<grid, block, sh, st>>>(a); break;

@@ -866,7 +866,7 @@ int lpc_quantize_pack(lpc_ctx* c, const float* U, const float* U_sub, int64_t le
     const int run = quantize_run_tiles();
     const bool vec = aligned16(U) && (!U_sub || aligned16(U_sub)) && (ld % 4 == 0);
     int64_t runs = 0;
-    const bool fixed_width = (c->b == 1 || c->b == 2 || c->b == 4 || c->b == 8);  // the other widths go tile by tile
+    const bool fixed_width = (c->b == 1 || c->b == 2 || c->b == 3 || c->b == 4 || c->b == 8);  // the other widths go tile by tile
     for (int t0 = 0; vec && fixed_width && t0 < p.ntiles; t0 += run) {
       const int t1 = std::min(t0 + run, p.ntiles) - 1;
       const SegInfo& g = p.segs[p.tile_seg[t0]];

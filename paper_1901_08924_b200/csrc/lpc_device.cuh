@@ -261,9 +261,13 @@ __device__ __forceinline__ float index_as_float(uint32_t code, int b) {
 // instruction per code after a few shared masks), then one exact subtraction removes 2^23 and the offset.
 template <int BITS>
 __device__ __forceinline__ void decode8(uint64_t lo, float* k) {
-  static_assert(BITS == 1 || BITS == 2 || BITS == 4 || BITS == 8, "fixed widths only");
+  static_assert(BITS == 1 || BITS == 2 || BITS == 3 || BITS == 4 || BITS == 8, "fixed widths only");
   constexpr uint32_t MAGIC = 0x4B000000u;  // 2^23
-  if constexpr (BITS == 1) {
+  if constexpr (BITS == 3) {  // the paper's three-level setting: 3-bit fields do not line up with bytes, one shift and mask each
+    const uint32_t w = (uint32_t)lo;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) k[e] = __fsub_rn(__uint_as_float(MAGIC | ((w >> (3 * e)) & 7u)), 8388608.f + 4.f);
+  } else if constexpr (BITS == 1) {
 #pragma unroll
     for (int e = 0; e < 8; ++e) k[e] = ((uint32_t)lo >> e) & 1u ? 1.0f : -1.0f;
   } else {
@@ -318,7 +322,7 @@ __device__ __forceinline__ void count_outside(float& cnt, float u, float T, floa
 template <int BITS, bool COUNT>
 __device__ __forceinline__ uint64_t quantize_group8(const float* v, float rdelta, const U4& r, float T, float lower,
                                                     float& cnt) {
-  static_assert(BITS == 1 || BITS == 2 || BITS == 4 || BITS == 8, "fixed widths only");
+  static_assert(BITS == 1 || BITS == 2 || BITS == 3 || BITS == 4 || BITS == 8, "fixed widths only");
   uint32_t w0 = 0, w1 = 0;
 #pragma unroll
   for (int e = 0; e < 8; ++e) {

@@ -188,7 +188,7 @@ __global__ void __launch_bounds__(32) share_scale_kernel(QuantArgs a) {
 }
 
 // ---- pass 2: quantize and pack -----------------------------------------------------------------------------
-// BITS = 1, 2, 4, 8: register/shuffle packing with direct coalesced stores.
+// BITS = 1, 2, 3, 4, 8: register/shuffle packing with direct coalesced stores.
 // BITS = 0: any b in 1..16 read from the arguments; each thread's 8*b bits are b whole bytes, staged
 //           through shared memory and written out as words.
 // A CTA takes a run of QRUN consecutive tiles of one worker.  Runs that consist of whole tiles of one segment of
@@ -206,6 +206,12 @@ __device__ __forceinline__ void store_group(uint32_t* __restrict__ ot, int g, in
   } else if (BITS == 2) {
     const uint32_t next = __shfl_down_sync(0xFFFFFFFFu, (uint32_t)lo, 1);
     if ((lane & 1) == 0) ot[g >> 1] = (uint32_t)lo | (next << 16);
+  } else if (BITS == 3) {
+    // 24 bits per thread: four neighbouring lanes hold three words; lane i < 3 of them builds word i from its own bits
+    // and its neighbour's
+    const uint32_t mine = (uint32_t)lo, next = __shfl_down_sync(0xFFFFFFFFu, mine, 1);
+    const int i = lane & 3;
+    if (i < 3) ot[3 * (g >> 2) + i] = (mine >> (8 * i)) | (next << (24 - 8 * i));
   } else {
     const uint32_t mine = (uint32_t)lo;
     const uint32_t n1 = __shfl_down_sync(0xFFFFFFFFu, mine, 1);
@@ -342,6 +348,11 @@ __device__ __forceinline__ void quantize_tile(const QuantArgs& a, int tile, int 
       const uint32_t n3 = __shfl_down_sync(0xFFFFFFFFu, mine, 3);
       const int64_t w = j >> 5;
       if ((lane & 3) == 0 && w < s.pad_words) out[w] = mine | (n1 << 8) | (n2 << 16) | (n3 << 24);
+    } else if (BITS == 3) {
+      const uint32_t mine = (uint32_t)lo, next = __shfl_down_sync(0xFFFFFFFFu, mine, 1);  // 24 bits each
+      const int i = lane & 3;
+      const int64_t w = 3 * (j >> 5) + i;
+      if (i < 3 && w < s.pad_words) out[w] = (mine >> (8 * i)) | (next << (24 - 8 * i));
     } else {
       // generic: b bytes per thread at byte tid*b of the sweep's 256*b-byte block
       if (it > 0) __syncthreads();
@@ -536,6 +547,7 @@ cudaError_t launch_quantize_fused(const QuantArgs& a, unsigned int* done, unsign
   switch (a.b) {
     case 1: k = pick_fused<1>(count, sums); break;
     case 2: k = pick_fused<2>(count, sums); break;
+    case 3: k = pick_fused<3>(count, sums); break;
     case 4: k = pick_fused<4>(count, sums); break;
     case 8: k = pick_fused<8>(count, sums); break;
     default: k = pick_fused<0>(count, sums); break;
@@ -588,6 +600,7 @@ cudaError_t launch_quantize_pack(const QuantArgs& a, cudaStream_t st, LaunchHook
     switch (a.b) {
       case 1: quantize_kernel<1, true><<<grid_runs, block, 0, st>>>(a); break;
       case 2: quantize_kernel<2, true><<<grid_runs, block, 0, st>>>(a); break;
+      case 3: quantize_kernel<3, true><<<grid_runs, block, 0, st>>>(a); break;
       case 4: quantize_kernel<4, true><<<grid_runs, block, 0, st>>>(a); break;
       case 8: quantize_kernel<8, true><<<grid_runs, block, 0, st>>>(a); break;
       case 32: bypass_kernel<<<grid_tiles, block, 0, st>>>(a); break;
@@ -597,6 +610,7 @@ cudaError_t launch_quantize_pack(const QuantArgs& a, cudaStream_t st, LaunchHook
     switch (a.b) {
       case 1: quantize_kernel<1, false><<<grid_runs, block, 0, st>>>(a); break;
       case 2: quantize_kernel<2, false><<<grid_runs, block, 0, st>>>(a); break;
+      case 3: quantize_kernel<3, false><<<grid_runs, block, 0, st>>>(a); break;
       case 4: quantize_kernel<4, false><<<grid_runs, block, 0, st>>>(a); break;
       case 8: quantize_kernel<8, false><<<grid_runs, block, 0, st>>>(a); break;
       case 32: bypass_kernel<<<grid_tiles, block, 0, st>>>(a); break;

@@ -19,9 +19,9 @@ import statistics
 import sys
 
 PHASES = [
-    (0, 1, "fetch issue for the next step (sampling, bulk copies, label and margin loads)"),
-    (1, 2, "rounding bits (Philox)"),
-    (2, 3, "wait for the words of all workers"),
+    (0, 1, "rounding bits (Philox)"),
+    (1, 2, "sampling of the next step's rows"),
+    (2, 3, "loads of all workers' words issued -> all tags valid (the next step's row copies are issued meanwhile)"),
     (3, 4, "decode + average + proximal step (Algorithm 2: y, z updates and coupling)"),
     (4, 5, "wait for this step's rows"),
     (5, 6, "margins (partial sums, warp reduction, block barrier)"),

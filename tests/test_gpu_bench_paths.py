@@ -45,7 +45,7 @@ def _rows_aligned(U):
     return buf[:, :length]
 
 
-@pytest.mark.parametrize("b", [1, 2, 4, 8])
+@pytest.mark.parametrize("b", [1, 2, 3, 4, 8])
 def test_quantize_runs_of_whole_tiles_bit_exact(b):
     # runs of 2, 5, 8 whole tiles, a full run plus one tile and a ragged tail, two full runs plus a tail
     N, seed, k = 3, 77, 5
@@ -70,7 +70,7 @@ def test_quantize_runs_of_whole_tiles_bit_exact(b):
         ctx.close()
 
 
-@pytest.mark.parametrize("b", [2, 8])
+@pytest.mark.parametrize("b", [2, 3, 8])
 def test_quantize_runs_with_subtrahend_bit_exact(b):
     # u = cur - snap formed on the fly inside the pipelined loop (one sweep per step instead of two)
     N, seed, k = 2, 9, 1
@@ -157,7 +157,7 @@ def test_sweep_2p28_sampled_windows():
 
 @pytest.mark.parametrize("b", [3])
 def test_three_level_codes_full_length_windows(b):
-    # the paper's own setting (three positive levels, b = 3) goes through the byte-staged generic paths
+    # the paper's own setting (three positive levels, b = 3): 24 bits per thread, three words per four lanes
     N, length, seed, k = 8, 1 << 22, 61, 8
     U = synth.gradient_vectors(N, length, "gauss", seed=seed, device=DEV)
     q = _ctx(N, b, orc.CLIP_STD, 2.0, seed)
@@ -165,7 +165,7 @@ def test_three_level_codes_full_length_windows(b):
     x = torch.zeros(length, device=DEV)
     q.unpack_average_prox(codes, delta, length, x, 1.0, 1e-3)
     q.sync_status()
-    assert q.query(lpc.INFO_QUANT_PIPELINED_RUNS) == 0 and q.query(lpc.INFO_AGGREGATE_SPLIT) == 4
+    assert q.query(lpc.INFO_QUANT_PIPELINED_RUNS) == length // (TILE * RUN) and q.query(lpc.INFO_AGGREGATE_SPLIT) == 4
     assert q.query(lpc.INFO_QUANT_ONE_LAUNCH) == 0  # 8 x 2^22 values = 134 MB
     Uh = U.cpu().numpy()
     W = orc.packed_words(length, b)
