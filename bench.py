@@ -527,6 +527,41 @@ def quantize_aggregate_bench(dev, peak, log2_len=26, full=True):
     return res
 
 
+def kernel_pass(dev, log2_len):
+    """Every stand-alone kernel of the library twice, on 8 x 2^log2_len Gaussian values, in a fixed order and with no
+    warm-up: the command that profiler captures of these kernels run (a few launches, a few hundred MB)."""
+    import torch
+    from paper_1901_08924_b200 import lpc, synth
+    N, length = 8, 1 << log2_len
+    U = synth.gradient_vectors(N, length, "gauss", seed=1, device=dev)
+    x = torch.zeros(length, device=dev)
+    done = []
+    for b in (4, 3):
+        q = lpc.Context(None, None, lpc.LOGISTIC, 0.0, N, 1, b, lpc.CLIP_STD, 2.0, 0)
+        for k in range(2):
+            codes, delta, _ = q.quantize_pack(U, k)                 # stats_kernel, finish_kernel, quantize_kernel<b>
+            q.unpack_average_prox(codes, delta, length, x, 1.0, 1e-3)  # unpack_average_prox_kernel<b>
+        if b == 4:
+            for k in range(2):
+                q.message_entropy(codes, length, host_counts=False)  # code_histogram_swar_kernel<4>
+            q.set_option(lpc.OPT_SHARED_SCALE, 1)
+            codes, delta, _ = q.quantize_pack(U, 2)                  # + share_scale_kernel
+            for k in range(2):
+                q.server_reduce(codes, length, lpc.SCHEME_SERVER_SUM, k)         # server_reduce4_kernel<7, false>
+                q.server_reduce(codes, length, lpc.SCHEME_SERVER_REQUANTIZE, k)  # server_reduce4_kernel<4, true>
+        q.sync_status()
+        q.close()
+        done.append(b)
+    short = min(length, 1 << 20)
+    q = lpc.Context(None, None, lpc.LOGISTIC, 0.0, N, 1, 4, lpc.CLIP_STD, 2.0, 0)
+    for k in range(2):
+        q.quantize_pack(U[:, :short], k)                             # quantize_fused_kernel<4> (one cooperative launch)
+    q.sync_status()
+    one = q.query(lpc.INFO_QUANT_ONE_LAUNCH)
+    q.close()
+    return {"kernel_pass": "8 x 2^%d" % log2_len, "widths": done, "one_launch_on_2^20": one}
+
+
 def tiny_logistic_bench(dev):
     """The small logistic workload (4,000 x 1,000, N = 4, B = 1, b = 2, clip 2.5 std, eta = 0.1): one epoch of m = 1,000
     inner steps after the snapshot pass, value only."""
@@ -759,12 +794,17 @@ def main():
     ap.add_argument("--per-step-kernels", action="store_true",
                     help="run the inner loop as per-step kernels (graph replay) instead of the one-launch loop; "
                          "for profiler captures, which cannot replay the cooperative launch")
+    ap.add_argument("--kernel-pass", type=int, default=0, metavar="LOG2LEN",
+                    help="launch every stand-alone kernel twice on 8 x 2^LOG2LEN values (for profiler captures)")
     ap.add_argument("--alpc-only", action="store_true", help="run only the ALPC-SVRG leg (262,144 x 8,192)")
     ap.add_argument("--fused-large-batch-only", type=int, default=0, metavar="ROWS",
                     help="run only the large-minibatch leg of the fused worker kernel on a ROWS x 8192 matrix "
                          "(a small case for profiler captures)")
     args = ap.parse_args()
-    if args.fused_large_batch_only:
+    if args.kernel_pass:
+        import torch
+        print(json.dumps(kernel_pass(torch.device("cuda", 0), args.kernel_pass)))
+    elif args.fused_large_batch_only:
         import torch
         peak, _ = read_peak()
         print(json.dumps(fused_large_batch_bench(torch.device("cuda", 0), peak, n=args.fused_large_batch_only, steps=4)))
