@@ -416,16 +416,18 @@ __global__ void __launch_bounds__(QT, 4) quantize_kernel(QuantArgs a) {
 // separate scale kernel are gone, which is most of the cost of a short vector.  The counters only grow: call number
 // `epoch` waits for (epoch + 1) * tile_count arrivals.  A wait that runs out records a timeout and goes on.
 template <int BITS, bool COUNT, bool NEED_SUMS>
-__global__ void __launch_bounds__(QT, 4) quantize_fused_kernel(QuantArgs a, unsigned int* done, unsigned int epoch) {
+__global__ void __launch_bounds__(QT, 4) quantize_fused_kernel(QuantArgs a, unsigned int* done, unsigned int epoch, int cpw) {
   __shared__ float sh1[QITER * 8], sh2[QITER * 8], sh8[8];
   __shared__ uint32_t shm[8];
   __shared__ ScaleRec srec;
   __shared__ __align__(16) uint8_t stage[BITS == 0 ? QT * 16 : 16];
-  const int items = a.N * a.ntiles, tid = threadIdx.x;
-  for (int item = blockIdx.x; item < items; item += gridDim.x) {
-    const int worker = item / a.ntiles, tile = item % a.ntiles;
+  const int tid = threadIdx.x, lane = tid & 31;
+  // CTA (chunk, worker) takes the tiles [t0, t1) of its worker: cpw chunks of consecutive tiles per worker
+  const int worker = blockIdx.x / cpw, chunk = blockIdx.x % cpw;
+  const int t0 = (int)((int64_t)a.ntiles * chunk / cpw), t1 = (int)((int64_t)a.ntiles * (chunk + 1) / cpw);
+  for (int tile = t0; tile < t1; ++tile) {
     const int seg = a.tile_seg ? a.tile_seg[tile] : 0;
-    if (item != (int)blockIdx.x) __syncthreads();  // the reduction buffers are reused from tile to tile
+    if (tile != t0) __syncthreads();  // the reduction buffers are reused from tile to tile
     stats_tile<NEED_SUMS>(a, tile, worker, sh1, sh2, shm);
     if (tid == 0) {
       const int64_t o = (int64_t)worker * a.nseg + seg;
@@ -436,53 +438,76 @@ __global__ void __launch_bounds__(QT, 4) quantize_fused_kernel(QuantArgs a, unsi
   }
   // segments without a single coordinate have no tile: their records are written here
   for (int o = blockIdx.x; o < a.N * a.nseg; o += gridDim.x) {
-    const int worker = o / a.nseg, seg = o % a.nseg;
+    const int w = o / a.nseg, seg = o % a.nseg;
     if (a.segs[seg].tile_count != 0) continue;
     __syncthreads();
-    const ScaleRec r = finish_segment(a, seg, worker, sh8, shm);
+    const ScaleRec r = finish_segment(a, seg, w, sh8, shm);
     if (tid == 0) { a.scales[o] = r; a.delta_out[o] = r.delta; a.clipped_out[o] = 0; }
   }
-  int have = -1;
-  for (int item = blockIdx.x; item < items; item += gridDim.x) {
-    const int worker = item / a.ntiles, tile = item % a.ntiles;
+  int tile = t0;
+  while (tile < t1) {  // one pass per tensor segment that the chunk touches
     const int seg = a.tile_seg ? a.tile_seg[tile] : 0;
+    const SegInfo s = a.segs[seg];
+    const int tend = min(t1, s.tile_first + s.tile_count);
     const int o = worker * a.nseg + seg;
-    if (o != have) {
-      const SegInfo s = a.segs[seg];
-      if (tid == 0) {
-        const unsigned int want = (epoch + 1u) * (unsigned int)s.tile_count;
-        uint64_t t0 = 0;
-        for (uint32_t it = 0;; ++it) {
-          unsigned int seen;
-          asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(done + o) : "memory");
-          if (seen >= want) break;
-          if ((it & 63u) == 63u) {
-            const uint64_t now = global_ns();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > 2000000000ull) { atomicOr(a.dev_status, DEV_TIMEOUT); break; }
-          }
+    if (tid == 0) {
+      const unsigned int want = (epoch + 1u) * (unsigned int)s.tile_count;
+      uint64_t t0ns = 0;
+      for (uint32_t it = 0;; ++it) {
+        unsigned int seen;
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(done + o) : "memory");
+        if (seen >= want) break;
+        if ((it & 63u) == 63u) {
+          const uint64_t now = global_ns();
+          if (t0ns == 0) t0ns = now;
+          else if (now - t0ns > 2000000000ull) { atomicOr(a.dev_status, DEV_TIMEOUT); break; }
         }
       }
-      __syncthreads();
-      const ScaleRec r = finish_segment(a, seg, worker, sh8, shm);
-      if (tid == 0) {
-        srec = r;
-        if (tile == s.tile_first) {  // one CTA leaves the record and the scale for the caller
-          a.scales[o] = r;
-          a.delta_out[o] = r.delta;
-          if (r.flags & 2u) atomicOr(a.dev_status, DEV_NONFINITE);
-        }
-      }
-      __syncthreads();
-      have = o;
-    } else if (BITS == 0) {
-      __syncthreads();  // the staging buffer is reused from tile to tile
     }
+    __syncthreads();
+    const ScaleRec r = finish_segment(a, seg, worker, sh8, shm);
+    if (tid == 0) {
+      srec = r;
+      if (tile == s.tile_first) {  // one CTA leaves the record and the scale for the caller
+        a.scales[o] = r;
+        a.delta_out[o] = r.delta;
+        if (r.flags & 2u) atomicOr(a.dev_status, DEV_NONFINITE);
+      }
+    }
+    __syncthreads();
     const ScaleRec sc = srec;
-    quantize_tile<BITS, COUNT>(a, tile, worker, stage, sc);
+    // whole tiles of aligned vectors go through the pipelined loop, the rest tile by tile
+    const float* p = a.U + (int64_t)worker * a.ld + s.off;
+    const float* q = a.U_sub ? a.U_sub + (int64_t)worker * a.ld + s.off : nullptr;
+    int whole = 0;
+    if constexpr (BITS != 0) {
+      if (aligned16(p) && (!q || aligned16(q)) && !(sc.flags & 1u)) {
+        const int64_t full_tiles = s.len / TILE;  // tiles of the segment without a ragged end
+        whole = (int)max((int64_t)0, min((int64_t)(tend - s.tile_first), full_tiles) - (tile - s.tile_first));
+      }
+      if (whole > 0) {
+        const int64_t tstart = (int64_t)(tile - s.tile_first) * TILE;
+        const uint32_t block0 = s.block_base + (uint32_t)(tstart >> 3);
+        uint32_t* ot = a.codes + (int64_t)worker * a.stride_words + s.word_off + (tstart >> 5) * BITS;
+        float fclip = 0.f;
+        if (q)
+          quantize_run<BITS ? BITS : 1, COUNT, true>(a, sc, p + tstart + tid * 8, q + tstart + tid * 8, block0, ot, whole * QITER,
+                                                     worker, tid, lane, fclip);
+        else
+          quantize_run<BITS ? BITS : 1, COUNT, false>(a, sc, p + tstart + tid * 8, nullptr, block0, ot, whole * QITER, worker,
+                                                      tid, lane, fclip);
+        const uint32_t nclip = __reduce_add_sync(0xFFFFFFFFu, (uint32_t)fclip);
+        if (COUNT && lane == 0 && nclip) atomicAdd(&a.clipped_out[o], nclip);
+      }
+    }
+    for (int t = tile + whole; t < tend; ++t) {
+      if (BITS == 0 && t > tile) __syncthreads();  // the staging buffer is reused from tile to tile
+      quantize_tile<BITS, COUNT>(a, t, worker, stage, sc);
+    }
+    tile = tend;
+    if (tile < t1) __syncthreads();  // srec and the reduction buffers are reused for the next segment
   }
 }
-
 
 // b = 32: the message is the vector itself (clamped to [-T, T] when a clip rule is set).
 __device__ __forceinline__ void bypass_tile(const QuantArgs& a, int tile, int worker, const ScaleRec& sc) {
@@ -529,7 +554,7 @@ __global__ void __launch_bounds__(QT) bypass_kernel(QuantArgs a) {
   bypass_tile(a, tile, worker, a.scales[(int64_t)worker * a.nseg + seg]);
 }
 
-using FusedKernel = void (*)(QuantArgs, unsigned int*, unsigned int);
+using FusedKernel = void (*)(QuantArgs, unsigned int*, unsigned int, int);
 template <int BITS>
 FusedKernel pick_fused(bool count, bool sums) {
   if (count) return sums ? quantize_fused_kernel<BITS, true, true> : quantize_fused_kernel<BITS, true, false>;
@@ -556,10 +581,14 @@ cudaError_t launch_quantize_fused(const QuantArgs& a, unsigned int* done, unsign
   cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, QT, 0);
   if (e != cudaSuccess) return e;
   if (per_sm < 1) return cudaErrorCooperativeLaunchTooLarge;
-  const long long items = (long long)a.N * (a.ntiles > 0 ? a.ntiles : 1);
   const long long resident = (long long)per_sm * sm_count;
+  if (resident < a.N) return cudaErrorCooperativeLaunchTooLarge;
+  // chunks of consecutive tiles per worker: as many as fit the resident grid, at most one per tile
+  long long cpw = resident / a.N;
+  if (cpw > a.ntiles) cpw = a.ntiles;
+  if (cpw < 1) cpw = 1;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)(items < resident ? items : resident), 1, 1);
+  cfg.gridDim = dim3((unsigned)(cpw * a.N), 1, 1);
   cfg.blockDim = dim3(QT, 1, 1);
   cfg.dynamicSmemBytes = 0;
   cfg.stream = st;
@@ -568,7 +597,7 @@ cudaError_t launch_quantize_fused(const QuantArgs& a, unsigned int* done, unsign
   attr[0].val.cooperative = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, k, a, done, epoch);
+  return cudaLaunchKernelEx(&cfg, k, a, done, epoch, (int)cpw);
 }
 
 int quantize_run_tiles() { return QRUN; }
