@@ -441,9 +441,26 @@ __global__ void __launch_bounds__(AT, 4) server_reduce4_kernel(ServerArgs a) {
         out[q] = (uint32_t)quantize_group8<4, false>(v, 1.0f, r, 0.f, 0.f, dummy);
       }
     };
-    // K / N: a multiplication by the exact reciprocal when N is a power of two (the same value), else the division
-    if (pow2) requantize([&](float K) { return mul_rn(K, invN); });
-    else requantize([&](float K) { return __fdiv_rn(K, fN); });
+    if (pow2) {
+      // N a power of two: K / N is exact in fp32 and Z = ceil(s * 2^17) of the rounding rule (lpc_device.cuh) is the
+      // integer K * (2^17 / N); the average of N hull points lies in the hull, so nothing is clamped.  The code
+      // floor((Z + 131070 + 2^17 * 8 - 2 r16) / 2^17) then takes integer operations only:
+      //   (sum * c1 + c0 - 2 r16) >> 17,   c1 = 2^17 / N,   c0 = 131070 + 2^20 - 8 N c1.
+      const uint32_t c1 = 131072u / (uint32_t)a.N, c0 = 131070u + (1u << 20) - 8u * (uint32_t)a.N * c1;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const U4 r = stream_block(a.seed, TAG_REQUANT, 0u, a.k, s.block_base + (uint32_t)(j >> 3) + (uint32_t)q);
+        uint32_t word = 0;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const uint32_t sum = (((e & 1) ? od[q] : ev[q]) >> (8 * (e >> 1))) & 0xFFu;
+          word += ((sum * c1 + c0 - 2u * lane16(r, e)) >> 17) << (4 * e);
+        }
+        out[q] = word;
+      }
+    } else {
+      requantize([&](float K) { return __fdiv_rn(K, fN); });
+    }
   } else {
     // scheme (b): the index sums in offset binary; sum of codes - 8 N + 2^(BO-1) >= 0 since 2^(BO-1) >= 8 N
     const uint32_t shift = (1u << (BO - 1)) - ((uint32_t)a.N << 3);

@@ -306,9 +306,9 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
   // thread: lane l of a warp loads those of workers l, l + 32, ... and the warp hands them round by shuffles.
   constexpr int WMAX = (BITS == 0) ? 8 : (BITS == 8 ? 2 : 1);  // tagged words per group of 8 coordinates
   constexpr int NW = (BITS == 0) ? 8 : (TB >= 32 ? TB / 32 : 1);  // of which a thread reads / writes this many
-  // workers per round of loads: 16 words in flight per thread, 32 in the loop of Algorithm 2 (its workload has 32 workers:
-  // one exposed round trip instead of two is worth the registers there)
-  constexpr int CH = (BITS == 0) ? 4 : (ALPC ? 32 : 16) / (NP * NW) > 0 ? (ALPC ? 32 : 16) / (NP * NW) : 1;
+  // workers per round of loads: 16 words in flight per thread.  (32 per round for the 32 workers of the Algorithm 2
+  // workload moved the second round's time into the first: 40 loads per thread queue up on the way from L2.)
+  constexpr int CH = (BITS == 0) ? 4 : 16 / (NP * NW) > 0 ? 16 / (NP * NW) : 1;
   const int wpg = (BITS == 0) ? pa.wpg : WMAX;
   const int sub = (LPG > 1) ? (tid & (LPG - 1)) : 0;          // this thread's place in its group of 8 coordinates
   const int wfirst = (BITS == 0) ? 0 : (sub * TB) >> 5;        // first word of the group that holds its codes
