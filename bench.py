@@ -298,9 +298,13 @@ L2_BYTES = 126e6
 # is scaled by them.  An entry goes away when its kernel changes.
 TRAFFIC = {
     "snapshot_kernel": (268.56e6 + 4.02e6, 16384 * 4096, "profiles/snapshot_kernel_ls_16384x4096.md"),
-    "stats_kernel": (536.95e6 + 4.10e6, 8 * (1 << 24), "profiles/quantize_aggregate_N8_len2p24_b4.md"),
-    "quantize_kernel<4>": (536.96e6 + 14.64e6, 8 * (1 << 24), "profiles/quantize_aggregate_N8_len2p24_b4.md"),
-    "unpack_average_prox_kernel<4>": (134.25e6 + 25.62e6, 1 << 24, "profiles/quantize_aggregate_N8_len2p24_b4.md"),
+    "stats_kernel": (536.96e6 + 4.20e6, 8 * (1 << 24), "profiles/quantize_aggregate_N8_len2p24_b4_b3.md"),
+    "quantize_kernel<4>": (536.95e6 + 14.21e6, 8 * (1 << 24), "profiles/quantize_aggregate_N8_len2p24_b4_b3.md"),
+    "quantize_kernel<3>": (536.92e6 + 8.00e6, 8 * (1 << 24), "profiles/quantize_aggregate_N8_len2p24_b4_b3.md"),
+    "unpack_average_prox_kernel<4>": (134.25e6 + 25.20e6, 1 << 24, "profiles/quantize_aggregate_N8_len2p24_b4_b3.md"),
+    "unpack_average_prox_kernel<3>": (117.47e6 + 21.75e6, 1 << 24, "profiles/quantize_aggregate_N8_len2p24_b4_b3.md"),
+    "code_histogram_swar_kernel<4>": (67.13e6 + 0.26e6, 8 * (1 << 24), "profiles/server_reduce4_and_code_histogram_N8_len2p24_b4.md"),
+    "server_reduce4_kernel<7, sum>": (67.12e6 + 1.84e6, 1 << 24, "profiles/server_reduce4_and_code_histogram_N8_len2p24_b4.md"),
     "inner_kernel<4> (per step)": (2.218e6, 1, "profiles/inner_step_kernels_ls_16384x4096_N16_B8_b4.md"),
     "inner_kernel<2, stream>": (234.0e6 + 4.6e6, 32 * 256, "profiles/streaming_worker_kernel_logistic_16384x8192_N32_B256_b2.md"),
 }
@@ -420,22 +424,30 @@ def quantize_aggregate_bench(dev, peak, log2_len=26, full=True):
         r = point("gauss_len2^%d_b4_clip2" % l2, U[:, : 1 << l2], 4, 2.0, reps=10 if l2 <= 24 else 4)
         wl = "sweep N=8, len 2^%d, N(0,1), b=4, clip 2 std" % l2
         qp, ua = r["quantize_pack"], r["unpack_average_prox"]
-        roof.append(roofline_entry("quantize+pack (stats_kernel + finish_kernel + quantize_kernel<4>)", wl, qp["ms"] * 1e3, qp["bytes"], peak,
-                                   note="L2-resident input: bound 4 + b/8 B per element" if r["l2_resident_input"] else
+        resident = r["l2_resident_input"]
+        name = ("quantize_fused_kernel<4> (quantize+pack in one cooperative launch)" if qp["one_launch_ms"] > 0 else
+                "quantize+pack (stats_kernel + finish_kernel + quantize_kernel<4>)")
+        roof.append(roofline_entry(name, wl, qp["ms"] * 1e3, qp["bytes"], peak,
+                                   note="input stays in L2 between the two looks at it: bound 4 + b/8 B per element; launch-bound at "
+                                        "this size (an event pair around one launch reads about 8 us)" if resident else
                                    "two passes: 8 + b/8 B per element"))
-        if not r["l2_resident_input"] and qp["stats_ms"] > 0:
+        if not resident and qp["stats_ms"] > 0:
             roof.append(roofline_entry("stats_kernel", wl, qp["stats_ms"] * 1e3, N * (1 << l2) * 4, peak, "stats_kernel", N * (1 << l2)))
             roof.append(roofline_entry("quantize_kernel<4>", wl, qp["pack_ms"] * 1e3, N * (1 << l2) * 4.5, peak, "quantize_kernel<4>", N * (1 << l2)))
         roof.append(roofline_entry("unpack_average_prox_kernel<4>", wl, ua["ms"] * 1e3, ua["bytes"], peak,
-                                   "unpack_average_prox_kernel<4>", 1 << l2))
+                                   None if resident else "unpack_average_prox_kernel<4>", 1 << l2,
+                                   note="launch-bound at this size" if resident else None))
     mid = min(26, top)
     Um = U[:, : 1 << mid]
     for b in (1, 2, 3, 8):
         r = point("gauss_len2^%d_b%d_clip2" % (mid, b), Um, b, 2.0)
         wl = "sweep N=8, len 2^%d, N(0,1), b=%d, clip 2 std" % (mid, b)
         roof.append(roofline_entry("quantize+pack, b=%d" % b, wl, r["quantize_pack"]["ms"] * 1e3, r["quantize_pack"]["bytes"], peak))
-        roof.append(roofline_entry("unpack_average_prox_kernel, b=%d" % b, wl, r["unpack_average_prox"]["ms"] * 1e3,
-                                   r["unpack_average_prox"]["bytes"], peak))
+        if b == 3:
+            roof.append(roofline_entry("quantize_kernel<3>", wl, r["quantize_pack"]["pack_ms"] * 1e3, N * (1 << mid) * (4 + 3 / 8), peak,
+                                       "quantize_kernel<3>", N * (1 << mid)))
+        roof.append(roofline_entry("unpack_average_prox_kernel<%d>" % b, wl, r["unpack_average_prox"]["ms"] * 1e3,
+                                   r["unpack_average_prox"]["bytes"], peak, "unpack_average_prox_kernel<3>" if b == 3 else None, 1 << mid))
     if full:
         for clip in (1.0, 4.0):
             point("gauss_len2^%d_b4_clip%g" % (mid, clip), Um, 4, clip)
@@ -463,7 +475,8 @@ def quantize_aggregate_bench(dev, peak, log2_len=26, full=True):
         "histogram": {"ms": round(th, 4), "bytes": bh, "gbs": round(bh / th * 1e-6, 1), "frac": round(bh / th * 1e-6 / peak, 4)},
         "bits_per_coordinate": {"raw": b, "entropy_bound": round(float(ent.mean()) / length, 4),
                                 "huffman": round(float(huf.astype("float64").mean()) / length, 4)}}
-    roof.append(roofline_entry("code_histogram_kernel<4>", "8 x 2^%d 4-bit codes" % mid, th * 1e3, bh, peak))
+    roof.append(roofline_entry("code_histogram_swar_kernel<4>", "8 x 2^%d 4-bit codes" % mid, th * 1e3, bh, peak,
+                               "code_histogram_swar_kernel<4>", N * length))
     q.set_option(lpc.OPT_SHARED_SCALE, 1)
     tqs = _kernel_ms(q, lambda i: q.quantize_pack(Um, i, codes_out=codes, delta_out=delta, clipped_out=clipped), 4,
                      ("quant_stats", "other", "quant_pack", "quant_fused"))
@@ -485,8 +498,8 @@ def quantize_aggregate_bench(dev, peak, log2_len=26, full=True):
                     "server": {"ms": round(ts, 4), "bytes": bs, "gbs": round(bs / ts * 1e-6, 1), "frac": round(bs / ts * 1e-6 / peak, 4)},
                     "worker_decode_prox": {"ms": round(tw, 4), "bytes": bw, "gbs": round(bw / tw * 1e-6, 1),
                                            "frac": round(bw / tw * 1e-6 / peak, 4)}}
-        roof.append(roofline_entry("server_reduce_kernel<4> (%s)" % name, "8 x 2^%d 4-bit codes in, %d-bit stream out" % (mid, bo),
-                                   ts * 1e3, bs, peak))
+        roof.append(roofline_entry("server_reduce4_kernel (%s)" % name, "8 x 2^%d 4-bit codes in, %d-bit stream out" % (mid, bo),
+                                   ts * 1e3, bs, peak, "server_reduce4_kernel<7, sum>" if scheme == lpc.SCHEME_SERVER_SUM else None, length))
         del x2
     q.sync_status()
     res["parameter_server_N8_len2^%d_b4" % mid] = ps
