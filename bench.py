@@ -148,6 +148,8 @@ def run_ours(args):
     ctx = lpc.Context(X, y, loss_code(w), w["lam"], N, B, b, lpc.CLIP_STD, w["c"], seed=rank)
     if args.per_step_kernels:
         ctx.set_option(lpc.OPT_PERSISTENT, 0)
+    if args.loop_not_cooperative:
+        ctx.set_option(lpc.OPT_LOOP_COOPERATIVE, 0)
 
     def epoch(s):
         ctx.snapshot_full_grad()
@@ -807,6 +809,9 @@ def main():
     ap.add_argument("--per-step-kernels", action="store_true",
                     help="run the inner loop as per-step kernels (graph replay) instead of the one-launch loop; "
                          "for profiler captures, which cannot replay the cooperative launch")
+    ap.add_argument("--loop-not-cooperative", action="store_true",
+                    help="launch the one-launch loop without the cooperative attribute (same grid, same kernel): for profiler "
+                         "captures of it on a GPU that runs nothing else")
     ap.add_argument("--kernel-pass", type=int, default=0, metavar="LOG2LEN",
                     help="launch every stand-alone kernel twice on 8 x 2^LOG2LEN values (for profiler captures)")
     ap.add_argument("--alpc-only", action="store_true", help="run only the ALPC-SVRG leg (262,144 x 8,192)")

@@ -87,6 +87,7 @@ typedef struct lpc_ctx lpc_ctx;
 #define LPC_OPT_PERSISTENT 5    /* 1 (default): lpc_inner_steps runs the whole loop in one cooperative launch when it fits */
 #define LPC_OPT_ONE_LAUNCH_QUANTIZE 8 /* 1 (default): lpc_quantize_pack uses one cooperative launch for inputs of at most LPC_ONE_LAUNCH_BYTES */
 #define LPC_ONE_LAUNCH_BYTES (48ll << 20)
+#define LPC_OPT_LOOP_COOPERATIVE 9 /* 1 (default): the one-launch loops are cooperative launches (the driver guarantees that all their CTAs are resident together, which they rely on).  0: a plain cluster launch of the same grid, for profilers that cannot replay a cooperative cluster launch; use it only on a GPU that runs nothing else (the launch plan has checked that all clusters fit, and every wait in the kernel is bounded, so a grid that is not resident together ends with LPC_ERR_TIMEOUT instead of hanging) */
 
 /* kernel classes reported by lpc_get_profile */
 #define LPC_KERNEL_SNAPSHOT 0    /* the pass over X of lpc_snapshot_full_grad / lpc_objective */

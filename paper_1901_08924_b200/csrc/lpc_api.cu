@@ -113,6 +113,7 @@ struct lpc_ctx {
   uint32_t* q_clip = nullptr;
   size_t q_scale_cap = 0;
   // one-launch quantizer: arrival counters per (worker, segment), valid for one layout; calls made with it so far
+  int loop_cooperative = 1;       // LPC_OPT_LOOP_COOPERATIVE
   int one_launch = 1;             // LPC_OPT_ONE_LAUNCH_QUANTIZE
   unsigned int* q_done = nullptr;
   uint64_t q_done_version = ~0ull;
@@ -424,7 +425,7 @@ int run_steps(lpc_ctx* c, int kind, const float* p, uint64_t k0, int64_t count) 
     }
     CU(c, cudaMemsetAsync(pa.abort_flag, 0, sizeof(unsigned long long), c->stream));
     cudaError_t e;
-    { ProfScope ps_(c, LPC_KERNEL_INNER_LOOP); e = launch_persist(pa, kind == 0 ? c->persistSmem : c->apersistSmem, c->stream); }
+    { ProfScope ps_(c, LPC_KERNEL_INNER_LOOP); e = launch_persist(pa, kind == 0 ? c->persistSmem : c->apersistSmem, c->stream, c->loop_cooperative != 0); }
     if (e == cudaSuccess) {
       done = count;
       if (weighted) {  // the weights the loop went through, and the one the next step starts from
@@ -644,6 +645,7 @@ int lpc_set_option(lpc_ctx* c, int option, int64_t value) {
     case LPC_OPT_USE_GRAPH: c->use_graph = value ? 1 : 0; return LPC_OK;
     case LPC_OPT_PERSISTENT: c->use_persist = value ? 1 : 0; return LPC_OK;
     case LPC_OPT_ONE_LAUNCH_QUANTIZE: c->one_launch = value ? 1 : 0; return LPC_OK;
+    case LPC_OPT_LOOP_COOPERATIVE: c->loop_cooperative = value ? 1 : 0; return LPC_OK;
     case LPC_OPT_SHARED_SCALE:
       if (value && (c->b < 2 || c->b > 16)) return fail(c, LPC_ERR_UNSUPPORTED, "a unified scale needs an integer grid: b in 2..16");
       c->shared_scale = value ? 1 : 0;

@@ -71,7 +71,9 @@ struct PersistArgs {
 bool persist_plan(int d, int N, int B, int b, int alpc, int want_cs, int max_smem, int* CS_out, int* SL_out,
                   size_t* smem_out, int* row_slots_out);
 int persist_coords_per_thread(int b, int SL);
-cudaError_t launch_persist(const PersistArgs& pa, size_t smem, cudaStream_t st);
+// cooperative = false drops the launch attribute that makes the driver guarantee co-residency of the grid (the plan has
+// checked that all clusters fit; the kernel's waits are bounded): for profilers that cannot replay cooperative launches.
+cudaError_t launch_persist(const PersistArgs& pa, size_t smem, cudaStream_t st, bool cooperative = true);
 // One small kernel whose bounded waits (an mbarrier phase; a tagged word when `word` is given) run out after limit_ns.
 cudaError_t launch_wait_timeout(const unsigned long long* word, unsigned int* abort_flag, unsigned int* dev_status,
                                 uint64_t limit_ns, cudaStream_t st);

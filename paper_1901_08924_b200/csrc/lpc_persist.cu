@@ -950,13 +950,13 @@ bool persist_plan(int d, int N, int B, int b, int alpc, int want_cs, int max_sme
   return found;
 }
 
-cudaError_t launch_persist(const PersistArgs& pa, size_t smem, cudaStream_t st) {
+cudaError_t launch_persist(const PersistArgs& pa, size_t smem, cudaStream_t st, bool cooperative) {
   PersistKernel k = pick_kernel(pa.in.b, pa.in.SL, pa.alpc != 0);
   cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg;
   cudaLaunchAttribute attr[2];
-  fill_config(&cfg, attr, pa.in.CS, pa.in.N + (pa.alpc ? 1 : 0), smem, st, true);
+  fill_config(&cfg, attr, pa.in.CS, pa.in.N + (pa.alpc ? 1 : 0), smem, st, cooperative);
   return cudaLaunchKernelEx(&cfg, k, pa);
 }
 

@@ -19,7 +19,7 @@ CLIP_NONE, CLIP_LAMBDA, CLIP_STD = 0, 1, 2
 (BUF_X, BUF_XTILDE, BUF_MU, BUF_MARGINS, BUF_Y, BUF_Z, BUF_YSUM, BUF_CODES, BUF_DELTA, BUF_CLIPPED, BUF_BATCH_IDX,
  BUF_COEF, BUF_U, BUF_V, BUF_VHAT) = range(15)
 OPT_SAMPLE_GLOBAL, OPT_TAP_U, OPT_CLUSTER_SIZE, OPT_USE_GRAPH, OPT_PROFILE, OPT_PERSISTENT = 0, 1, 2, 3, 4, 5
-OPT_SHARED_SCALE, OPT_AVERAGE_DIVISOR, OPT_ONE_LAUNCH_QUANTIZE = 6, 7, 8
+OPT_SHARED_SCALE, OPT_AVERAGE_DIVISOR, OPT_ONE_LAUNCH_QUANTIZE, OPT_LOOP_COOPERATIVE = 6, 7, 8, 9
 SCHEME_BROADCAST, SCHEME_SERVER_SUM, SCHEME_SERVER_REQUANTIZE = 0, 1, 2
 (INFO_STEP_CLUSTER_SIZE, INFO_LOOP_CLUSTER_SIZE, INFO_LOOP_LAUNCHES, INFO_SNAPSHOT_ROWS_PER_TILE, INFO_SNAPSHOT_STAGES,
  INFO_ALPC_LOOP_CLUSTER_SIZE, INFO_LOOP_ROW_SLOTS, INFO_ALPC_LOOP_ROW_SLOTS, INFO_STEP_RING_STAGES,

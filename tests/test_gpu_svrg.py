@@ -436,3 +436,19 @@ def test_average_divisor_option_leaves_the_training_loops_alone():
         xr = orc.lpc_inner_step(P, k, eta, xr, x0, mu)
     assert _same(results[0], xr)
     ctx.close()
+
+
+def test_loop_without_the_cooperative_attribute_gives_the_same_bits():
+    # the profiling configuration of the one-launch loop: a plain cluster launch of the same grid
+    P, ctx = _setup(512, 1000, "least_squares", N=4, B=2, b=4, seed=13)
+    ref = lpc.Context(ctx.X, ctx.y, P.loss, P.lambda_l1, P.N, P.B, P.b, P.clip_mode, P.clip_value, P.seed)
+    ctx.set_option(lpc.OPT_LOOP_COOPERATIVE, 0)
+    for c in (ctx, ref):
+        c.snapshot_full_grad()
+        c.inner_steps(0.05, 0, 40)
+        c.sync_status()
+        assert c.query(lpc.INFO_LOOP_LAUNCHES) == 1
+    assert _same(ctx.get_iterate(), ref.get_iterate())
+    assert _same(ctx.get_buffer(lpc.BUF_CODES), ref.get_buffer(lpc.BUF_CODES))
+    ctx.close()
+    ref.close()
