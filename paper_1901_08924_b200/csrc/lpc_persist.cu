@@ -183,7 +183,7 @@ __device__ __forceinline__ float tree_ept(const float* v) {
 //      one tagged code word for b <= 4) is then shared by 8 / EPT neighbouring lanes.  BITS = 0 and NP = 2 use EPT = 8.
 // ALPC: Algorithm 2's step (coupling, double sampling on one more cluster, y/z updates) instead of Algorithm 1's.
 template <int BITS, int NP, int EPT, bool ALPC>
-__global__ void __launch_bounds__(PT, EPT <= 4 ? 2 : 1) persist_kernel(PersistArgs pa) {
+__global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
   static_assert(EPT == 8 || ((EPT == 4 || EPT == 2) && BITS != 0 && NP == 1), "narrow threads: fixed widths, one pass");
   constexpr int PSPAN = PT * EPT;               // coordinates per pass
   constexpr int LPG = 8 / EPT;                  // lanes that share a group of 8 coordinates
@@ -937,21 +937,11 @@ bool persist_plan(int d, int N, int B, int b, int alpc, int want_cs, int max_sme
     if (clusters * cs > PMAXFLAGS) break;
     const size_t fixed = (sizeof(PSmem) + 15) & ~(size_t)15;
     const size_t one = (size_t)SL * 4;  // one row slot
-    // The variants with 4 or 2 coordinates per thread are built for two CTAs per SM (128 registers): a cluster size whose
-    // CTAs do not all fit one to an SM may still fit two to an SM, with half the shared memory each.
-    size_t smem = 0;
-    int slots = 0;
-    bool fits = false;
-    const size_t budgets[2] = {(size_t)max_smem, ((size_t)max_smem - 2048) / 2};
-    for (int h = 0; h < 2 && !fits; ++h) {
-      if (h == 1 && persist_coords_per_thread(b, SL) > 4) break;
-      if (fixed + (size_t)B * one > budgets[h]) continue;
-      slots = (int)((budgets[h] - fixed) / one);
-      if (slots > 2 * B) slots = 2 * B;
-      smem = fixed + (size_t)slots * one;
-      fits = max_clusters(pick_kernel(b, SL, alpc != 0), cs, smem) >= clusters;
-    }
-    if (!fits) continue;
+    if (fixed + (size_t)B * one > (size_t)max_smem) continue;
+    int slots = (int)(((size_t)max_smem - fixed) / one);
+    if (slots > 2 * B) slots = 2 * B;
+    const size_t smem = fixed + (size_t)slots * one;
+    if (max_clusters(pick_kernel(b, SL, alpc != 0), cs, smem) < clusters) continue;
     *CS_out = cs; *SL_out = SL; *smem_out = smem; *row_slots_out = slots;
     found = true;
     if (want_cs > 0) break;
