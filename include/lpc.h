@@ -110,8 +110,8 @@ typedef struct lpc_ctx lpc_ctx;
  *   n        rows; must be a multiple of N.  Worker i owns rows [i*n/N, (i+1)*n/N).
  *   d        features, multiple of 4, at most 16384
  *   N        simulated workers, 1..1024;  B minibatch size per worker, 1..1024 (up to 64 rows per worker stay
- *            resident on chip and the one-launch loops are available; larger minibatches stream through
- *            the per-step kernel)
+ *            resident on chip; the one-launch loops are available for N <= 64 and B <= 64 when all worker
+ *            clusters fit on the device together; larger minibatches stream through the per-step kernel)
  *   b        bits per coordinate: 1..16 or 32 (32 = full precision, the codes are the floats)
  *   seed     key of every random stream (minibatches, shared batch J, stochastic rounding)
  *   stream   cudaStream_t (NULL = default stream)
