@@ -68,7 +68,7 @@ struct Smem {
   __align__(16) uint8_t stage[IT * 16];
   // streaming path: every hand-over is an mbarrier phase, so a waiting warp sleeps in hardware instead of polling
   uint64_t sbar[SMAXR];           // stage filled (bulk-copy bytes)
-  uint64_t ebar[SMAXR];           // stage consumed (one arrival per warp that adds rows into u)
+  uint64_t ebar[SMAXR];           // stage read (one arrival per warp that adds rows into u and per margin warp of the group's side)
   uint64_t pbar[SSLOTS];          // margin partial sums of a group have arrived from every CTA (bytes of their stores)
   uint64_t cbar[SSLOTS];          // coefficients of a group are in `coefs`
   uint64_t mbar_meta[SMAXB / 32]; // labels and snapshot-side derivatives of 32 sampled rows are in place (used once each)
@@ -80,14 +80,14 @@ struct Smem {
 
 // Phase timestamps of the streaming path of one CTA, for latency studies; compiled in only with -DLPC_TRACE.
 #ifdef LPC_TRACE
-__device__ unsigned long long g_stream_trace[64 * 8 + 16];  // per group: 8 marks; then 16 phase marks of the kernel
+__device__ unsigned long long g_stream_trace[64 * 16 + 16];  // per group: 16 marks; then 16 phase marks of the kernel
 #define LPC_STREAM_MARK(g, i)                                                                       \
   do {                                                                                              \
-    if (blockIdx.x == 0 && blockIdx.y == 0 && (g) < 64) g_stream_trace[(g) * 8 + (i)] = global_ns(); \
+    if (blockIdx.x == 0 && blockIdx.y == 0 && (g) < 64) g_stream_trace[(g) * 16 + (i)] = global_ns(); \
   } while (0)
 #define LPC_PHASE_MARK(i)                                                                            \
   do {                                                                                               \
-    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) g_stream_trace[64 * 8 + (i)] = global_ns(); \
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) g_stream_trace[64 * 16 + (i)] = global_ns(); \
   } while (0)
 #else
 #define LPC_STREAM_MARK(g, i) do { } while (0)
@@ -149,7 +149,7 @@ __global__ void __launch_bounds__(STREAM ? SNT : IT) inner_kernel(InnerArgs a) {
     if constexpr (STREAM) {
       for (int r = 0; r < SMAXR; ++r) {
         mbar_init(&sm.sbar[r], 1);
-        mbar_init(&sm.ebar[r], SUW);
+        mbar_init(&sm.ebar[r], SUW + SDW / 2);
       }
       for (int r = 0; r < SSLOTS; ++r) {
         mbar_init(&sm.pbar[r], 1);
@@ -319,6 +319,8 @@ __global__ void __launch_bounds__(STREAM ? SNT : IT) inner_kernel(InnerArgs a) {
           for (int q = 0; q < QB; ++q)
             sv[j * QB + q] = tree4(mul_rn(v[j][q].x, xs[q].x), mul_rn(v[j][q].y, xs[q].y), mul_rn(v[j][q].z, xs[q].z),
                                    mul_rn(v[j][q].w, xs[q].w));
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.ebar[g % R]);  // this warp has read its quarter of the stage
         WarpHalving<SG * QB, 0>::run(sv, lane);  // lane holds the 32-lane tree sum of (row, block) halving_index<4>(lane)
         float part = sv[0];
         part = add_rn(part, __shfl_xor_sync(0xFFFFFFFFu, part, 8));  // blocks 2k, 2k+1 of the row
@@ -329,18 +331,16 @@ __global__ void __launch_bounds__(STREAM ? SNT : IT) inner_kernel(InnerArgs a) {
         if (wq == 0 && lane == 0) LPC_STREAM_MARK(g, 1);
       }
     } else if (warp < SDW + SUW) {
-      // -- u: thread t of these warps owns the coordinates 4 t .. 4 t + 3 of each half of the slice
+      // -- u: thread t of these warps owns the coordinates 4 t .. 4 t + 3 of each half of the slice.  The rows of a
+      // group go from the stage into registers as soon as the stage is filled, one group ahead of the group whose
+      // coefficients are awaited, and the stage is handed back at once: a stage is then occupied for the time of
+      // its copies and two shared-memory reads, not for the round trip of the margins through the cluster.
       const int t = tid - SDW * 32;
-#pragma unroll 1
-      for (int g = 0; g < ngroups; ++g) {
-        const int cnt = min(SG, B - g * SG);
+      float4 va[SG][UC], vb[SG][UC];
+      auto take = [&](int g, float4 (&v)[SG][UC]) {  // rows past a ragged end are read and not used
         const int s = g % R;
-        wait_on(&sm.cbar[g % SSLOTS], (uint32_t)((g / SSLOTS) & 1), false);
         wait_stage(g);
-        if (t == 0) LPC_STREAM_MARK(g, 4);
-        const float4 c4 = *reinterpret_cast<const float4*>(sm.coefs[g % SSLOTS]);
-        const float cj[SG] = {c4.x, c4.y, c4.z, c4.w};
-        float4 v[SG][UC];  // all loads of the group first (rows past a ragged end are read and not used)
+        if (t == 0) LPC_STREAM_MARK(g, 8);
         if (full) {
           const float* src = rows + (size_t)(s * SG) * SL + t * 4;
 #pragma unroll
@@ -353,6 +353,16 @@ __global__ void __launch_bounds__(STREAM ? SNT : IT) inner_kernel(InnerArgs a) {
 #pragma unroll
             for (int q = 0; q < UC; ++q) v[j][q] = row4(s * SG + j, q * (IGROUP / UC) + t * 4);
         }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.ebar[s]);  // release: the loads above are performed before the arrival counts
+        if (t == 0) LPC_STREAM_MARK(g, 9);
+      };
+      auto add = [&](int g, const float4 (&v)[SG][UC]) {
+        const int cnt = min(SG, B - g * SG);
+        wait_on(&sm.cbar[g % SSLOTS], (uint32_t)((g / SSLOTS) & 1), false);
+        if (t == 0) LPC_STREAM_MARK(g, 4);
+        const float4 c4 = *reinterpret_cast<const float4*>(sm.coefs[g % SSLOTS]);
+        const float cj[SG] = {c4.x, c4.y, c4.z, c4.w};
 #pragma unroll
         for (int j = 0; j < SG; ++j) {
           if (j < cnt) {
@@ -365,11 +375,19 @@ __global__ void __launch_bounds__(STREAM ? SNT : IT) inner_kernel(InnerArgs a) {
             }
           }
         }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&sm.ebar[s]);  // this warp is done with the stage
 #ifdef LPC_TRACE
-        if (lane == 0 && blockIdx.x == 0 && blockIdx.y == 0 && g < 64) atomicMax(&g_stream_trace[g * 8 + 5], global_ns());
+        if (lane == 0 && blockIdx.x == 0 && blockIdx.y == 0 && g < 64) atomicMax(&g_stream_trace[g * 16 + 5], global_ns());
 #endif
+      };
+      take(0, va);
+#pragma unroll 1
+      for (int g = 0; g < ngroups; g += 2) {
+        if (g + 1 < ngroups) take(g + 1, vb);
+        add(g, va);
+        if (g + 1 < ngroups) {
+          if (g + 2 < ngroups) take(g + 2, va);
+          add(g + 1, vb);
+        }
       }
     } else if (warp < SDW + SUW + SCW) {
       // -- coefficients (warp c of this side takes the groups c, c + SCW, ...): lane j collects the partial sums of
@@ -808,7 +826,7 @@ cudaError_t launch_inner(const InnerArgs& a, size_t smem, cudaStream_t st) {
 
 #ifdef LPC_TRACE
 cudaError_t read_stream_trace(unsigned long long* host_out) {
-  return cudaMemcpyFromSymbol(host_out, g_stream_trace, sizeof(unsigned long long) * (64 * 8 + 16));
+  return cudaMemcpyFromSymbol(host_out, g_stream_trace, sizeof(unsigned long long) * (64 * 16 + 16));
 }
 #endif
 
