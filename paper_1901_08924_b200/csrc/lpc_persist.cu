@@ -54,7 +54,7 @@ constexpr int PUB_STRIDE = 16;  // publication words sit 128 bytes apart: one ca
 
 struct PSmem {
   uint64_t bar[2];
-  float coef[PMAXB];
+  __align__(16) float coef[PMAXB];
   float wpart[PMAXB * PMAXP * 8];
   // cluster exchange slots, written by the peers through distributed shared memory as tagged words, two
   // step-parity halves: margin partial sums (slot b * PMAXCS + rank) and statistics (max, S1, S2 per rank)
@@ -515,13 +515,38 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
     // margins <X_a, x_t>: eight rows at a time; their 8*NP per-thread partial sums are reduced across the
     // warp together by recursive halving (9 or 12 shuffles instead of 5 per value)
     constexpr int RG = 8, NVAL = RG * NP, LOGV = (NP == 2) ? 4 : 3;
+    constexpr int KB = (NP != 1) ? 0 : (EPT == 8 && (ALPC || BITS == 0)) ? 8 : 16;  // leading rows of a minibatch that a thread keeps in registers
     float xw[NP][EPT];  // x in the order row_vals delivers the row values
 #pragma unroll
     for (int p = 0; p < NP; ++p)
 #pragma unroll
       for (int e = 0; e < EPT; ++e) xw[p][e] = (EPT == 8 && swz) ? xr[p][e ^ (EPT / 2)] : xr[p][e];
+    // The first KB rows of the minibatch (one pass per CTA) stay in REGISTERS from here to the end of u: those slices
+    // are read from shared memory once per step instead of twice, and their part of u needs only the coefficients.
+    float rv[KB ? KB : 1][EPT];
+    if constexpr (KB > 0) {
+#pragma unroll
+      for (int g8 = 0; g8 < KB; g8 += RG) {
+        if (g8 < B) {
+          float sv[RG];
+#pragma unroll
+          for (int j = 0; j < RG; ++j) {
+            float pr[EPT];
+            row_vals<EPT>(row_ptr(min(g8 + j, B - 1)), tid * EPT, width, swz, rv[g8 + j]);
+#pragma unroll
+            for (int e = 0; e < EPT; ++e) pr[e] = mul_rn(rv[g8 + j][e], xw[0][e]);
+            sv[j] = tree_ept<EPT>(pr);
+          }
+          WarpHalving<RG, 0>::run(sv, lane);
+          if ((lane >> 3) == 0) {
+            const int j = halving_index<3>(lane);
+            if (g8 + j < B) sm.wpart[(g8 + j) * NP * 8 + warp] = sv[0];
+          }
+        }
+      }
+    }
 #pragma unroll 1
-    for (int r0 = 0; r0 < B; r0 += RG) {
+    for (int r0 = KB; r0 < B; r0 += RG) {
       float sv[NVAL];
 #pragma unroll
       for (int j = 0; j < RG; ++j) {
@@ -587,8 +612,24 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
       float uw[EPT];  // in the order row_vals delivers the row values
 #pragma unroll
       for (int e = 0; e < EPT; ++e) uw[e] = 0.f;
+      if constexpr (KB > 0) {  // the rows kept in registers (NP = 1)
+#pragma unroll
+        for (int g4 = 0; g4 < KB; g4 += 4) {
+          if (g4 < B) {
+            const float4 c4 = *reinterpret_cast<const float4*>(&sm.coef[g4]);
+            const float cf[4] = {c4.x, c4.y, c4.z, c4.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              if (g4 + j < B) {
+#pragma unroll
+                for (int e = 0; e < EPT; ++e) uw[e] = add_rn(uw[e], mul_rn(cf[j], rv[g4 + j][e]));
+              }
+            }
+          }
+        }
+      }
 #pragma unroll 1
-      for (int r0 = 0; r0 < B; r0 += 4) {
+      for (int r0 = KB; r0 < B; r0 += 4) {
         float v[4][EPT], cf[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
