@@ -598,7 +598,7 @@ int lpc_init(lpc_ctx** out, const float* X, const float* y, int64_t n, int32_t d
     snapshot_plan(d, c->max_smem, &c->snapR, &c->snapStages, &c->snapSmem);
     c->snapGrid = c->sm_count;
     A(dalloc(c, &c->partial_mu, (size_t)c->snapGrid * c->dpad));
-    A(dalloc(c, &c->partial_f, (size_t)c->snapGrid));
+    A(dalloc(c, &c->partial_f, 2 * (size_t)c->snapGrid));
     replan_inner(c);
   }
   if (rc != LPC_OK) { lpc_destroy(c); return rc; }

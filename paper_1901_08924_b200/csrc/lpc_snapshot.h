@@ -17,7 +17,7 @@ struct SnapArgs {
   int64_t ntiles;      // ceil(n / R)
   float* partial_mu;   // grid * dpad column sums, or NULL for the objective-only pass
   float* margins_out;  // n, nullable
-  double* partial_f;   // grid
+  double* partial_f;   // 2 * grid: one partial sum of f per row warp of every CTA
   unsigned int* dev_status;
 };
 
