@@ -109,9 +109,7 @@ __device__ __noinline__ Scale scale_out_of_line(uint32_t max_bits, float S1, flo
                                                float clip_value) {
   return make_scale(max_bits, S1, S2, len, b, clip_mode, clip_value);
 }
-__device__ __noinline__ float coef_out_of_line(int loss, float m, float m_snap, float y) {
-  return __fsub_rn(loss_deriv(loss, m, y), loss_deriv(loss, m_snap, y));
-}
+__device__ __noinline__ float deriv_out_of_line(int loss, float m, float y) { return loss_deriv(loss, m, y); }
 __device__ __noinline__ int64_t sample_row_out_of_line(uint64_t seed, uint32_t tag, uint32_t worker, uint64_t k, uint32_t slot,
                                                        int64_t lo, int64_t span) {
   const U4 r = stream_block(seed, tag, worker, k, slot);
@@ -487,8 +485,15 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
     const bool more = t + 1 < pa.count;
     if (more) sample_rows(t + 1, 0, PA);
     LPC_TRACE_MARK(2);
-    if (t > 0) apply_update((unsigned int)t, [&] { if (more) copy_rows(t + 1, sb_next, 0, PA); });
-    else if (more) copy_rows(t + 1, sb_next, 0, PA);
+    // The snapshot side of this step's coefficients, l'(m~_a), depends on nothing of this step: the owner of a minibatch
+    // slot forms it while the peers' words are on their way (for the logistic loss it is half of the fp64 work).
+    float gs_use = 0.f;
+    auto ahead = [&] {
+      if (more) copy_rows(t + 1, sb_next, 0, PA);
+      if (tid < B && t < pa.count) gs_use = deriv_out_of_line(a.loss, ms_use, y_use);
+    };
+    if (t > 0) apply_update((unsigned int)t, ahead);
+    else ahead();
     if (t == pa.count) break;
     if constexpr (ALPC) {  // step 6: x = tau1 z + tau2 x~ + (1 - tau1 - tau2) y
 #pragma unroll
@@ -515,7 +520,7 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
     // margins <X_a, x_t>: eight rows at a time; their 8*NP per-thread partial sums are reduced across the
     // warp together by recursive halving (9 or 12 shuffles instead of 5 per value)
     constexpr int RG = 8, NVAL = RG * NP, LOGV = (NP == 2) ? 4 : 3;
-    constexpr int KB = (NP != 1) ? 0 : (EPT == 8 && (ALPC || BITS == 0)) ? 8 : 16;  // leading rows of a minibatch that a thread keeps in registers
+    constexpr int KB = (NP != 1) ? 0 : (EPT == 8) ? 8 : 16;  // leading rows of a minibatch that a thread keeps in registers
     float xw[NP][EPT];  // x in the order row_vals delivers the row values
 #pragma unroll
     for (int p = 0; p < NP; ++p)
@@ -595,7 +600,7 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
         m = tree_small(mp, CS);
       }
       LPC_TRACE_MARK(7);
-      const float c = coef_out_of_line(a.loss, m, ms_use, y_use);
+      const float c = __fsub_rn(deriv_out_of_line(a.loss, m, y_use), gs_use);
       sm.coef[tid] = c;
       if (rank == 0 && t == pa.count - 1) {
         if (a.idx_tap) a.idx_tap[(int64_t)worker * B + tid] = row_use;
