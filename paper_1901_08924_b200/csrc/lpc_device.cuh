@@ -102,22 +102,23 @@ __device__ __forceinline__ int halving_index(int lane) {
   return q;
 }
 
-// Tree sum of `count` floats (count a power of two, <= 1024) stored in order in shared memory,
-// evaluated by one thread.  Small counts only (cross-warp / cross-CTA partials).
+// Tree sum of N floats (N a power of two) stored in order in memory, evaluated by one thread: the recursive definition,
+// unrolled, so the operands stay in registers and independent additions overlap.
+template <int N>
+__device__ __forceinline__ float tree_sum_n(const float* v) {
+  if constexpr (N == 1) return v[0];
+  else return add_rn(tree_sum_n<N / 2>(v), tree_sum_n<N / 2>(v + N / 2));
+}
+// The same for a count known only at run time (a power of two, <= 32: cross-warp and cross-CTA partial sums).
 __device__ __forceinline__ float smem_tree_sum(const float* v, int count) {
-  // iterative pairwise reduction with a small stack, same association as the recursive definition
-  float stack[12];
-  int top = 0;
-  for (int i = 0; i < count; ++i) {
-    float cur = v[i];
-    int idx = i;
-    while (idx & 1) {  // completed a right child: combine with the waiting left sibling
-      cur = add_rn(stack[--top], cur);
-      idx >>= 1;
-    }
-    stack[top++] = cur;
+  switch (count) {
+    case 1: return v[0];
+    case 2: return tree_sum_n<2>(v);
+    case 4: return tree_sum_n<4>(v);
+    case 8: return tree_sum_n<8>(v);
+    case 16: return tree_sum_n<16>(v);
+    default: return tree_sum_n<32>(v);
   }
-  return stack[0];
 }
 
 // ---- scale (Eq. 2) -----------------------------------------------------------------------------------

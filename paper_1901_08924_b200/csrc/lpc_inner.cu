@@ -143,22 +143,28 @@ __global__ void __launch_bounds__(STREAM ? SNT : IT) inner_kernel(InnerArgs a) {
       s_ms[slot] = a.margins[row];
     }
   }
-  if (tid == 0) {
-    mbar_init(&sm.bar, 1);
-    mbar_init(&sm.xbar, 1);
-    if constexpr (STREAM) {
-      for (int r = 0; r < SMAXR; ++r) {
-        mbar_init(&sm.sbar[r], 1);
-        mbar_init(&sm.ebar[r], SUW + SDW / 2);
-      }
-      for (int r = 0; r < SSLOTS; ++r) {
-        mbar_init(&sm.pbar[r], 1);
-        mbar_init(&sm.cbar[r], 1);
-      }
-      for (int r = 0; r < (B + 31) / 32; ++r) mbar_init(&sm.mbar_meta[r], 1);
+  if constexpr (STREAM) {
+    // the barriers of the streaming path are set up side by side, one or two per thread
+    static_assert(SMAXR + SSLOTS + SMAXB / 32 <= 64, "two warps set up the barriers");
+    if (tid < SMAXR) {
+      mbar_init(&sm.sbar[tid], 1);
+      mbar_init(&sm.ebar[tid], SUW + SDW / 2);
+    } else if (tid < SMAXR + SSLOTS) {
+      mbar_init(&sm.pbar[tid - SMAXR], 1);
+      mbar_init(&sm.cbar[tid - SMAXR], 1);
+    } else if (tid < SMAXR + SSLOTS + (B + 31) / 32) {
+      mbar_init(&sm.mbar_meta[tid - SMAXR - SSLOTS], 1);
+    }
+    if (tid == 0) {
+      mbar_init(&sm.bar, 1);
+      mbar_init(&sm.xbar, 1);
       sm.stream_fail = 0;
       sm.issued = 0;
     }
+    if (tid < 64) mbar_fence_init();
+  } else if (tid == 0) {
+    mbar_init(&sm.bar, 1);
+    mbar_init(&sm.xbar, 1);
     mbar_fence_init();
   }
   // Every CTA of the cluster announces that it is running (its barriers exist); peers wait for this before their
@@ -299,26 +305,30 @@ __global__ void __launch_bounds__(STREAM ? SNT : IT) inner_kernel(InnerArgs a) {
         const int cnt = min(SG, B - g * SG);
         wait_stage(g);
         if (warp < 2 * SMW && wq == 0 && lane == 0) LPC_STREAM_MARK(g, 0);
-        float4 v[SG][QB];  // all sixteen loads first
-        if (full) {
-          const float* src = rows + (size_t)((g % R) * SG) * SL + wq * QB * 128 + lane * 4;
-#pragma unroll
-          for (int j = 0; j < SG; ++j)
-#pragma unroll
-            for (int q = 0; q < QB; ++q) v[j][q] = *reinterpret_cast<const float4*>(src + j * SL + q * 128);
-        } else {
-#pragma unroll
-          for (int j = 0; j < SG; ++j)
-#pragma unroll
-            for (int q = 0; q < QB; ++q) v[j][q] = row4((g % R) * SG + j, (wq * QB + q) * 128 + lane * 4);
-        }
+        // two rows at a time (eight loads in flight): the sixteen partial sums of the group are all that stays
         float sv[SG * QB];
 #pragma unroll
-        for (int j = 0; j < SG; ++j)
+        for (int h = 0; h < SG; h += 2) {
+          float4 v[2][QB];
+          if (full) {
+            const float* src = rows + (size_t)((g % R) * SG + h) * SL + wq * QB * 128 + lane * 4;
 #pragma unroll
-          for (int q = 0; q < QB; ++q)
-            sv[j * QB + q] = tree4(mul_rn(v[j][q].x, xs[q].x), mul_rn(v[j][q].y, xs[q].y), mul_rn(v[j][q].z, xs[q].z),
-                                   mul_rn(v[j][q].w, xs[q].w));
+            for (int j = 0; j < 2; ++j)
+#pragma unroll
+              for (int q = 0; q < QB; ++q) v[j][q] = *reinterpret_cast<const float4*>(src + j * SL + q * 128);
+          } else {
+#pragma unroll
+            for (int j = 0; j < 2; ++j)
+#pragma unroll
+              for (int q = 0; q < QB; ++q) v[j][q] = row4((g % R) * SG + h + j, (wq * QB + q) * 128 + lane * 4);
+          }
+#pragma unroll
+          for (int j = 0; j < 2; ++j)
+#pragma unroll
+            for (int q = 0; q < QB; ++q)
+              sv[(h + j) * QB + q] = tree4(mul_rn(v[j][q].x, xs[q].x), mul_rn(v[j][q].y, xs[q].y), mul_rn(v[j][q].z, xs[q].z),
+                                           mul_rn(v[j][q].w, xs[q].w));
+        }
         __syncwarp();
         if (lane == 0) mbar_arrive(&sm.ebar[g % R]);  // this warp has read its quarter of the stage
         WarpHalving<SG * QB, 0>::run(sv, lane);  // lane holds the 32-lane tree sum of (row, block) halving_index<4>(lane)
@@ -573,6 +583,10 @@ __global__ void __launch_bounds__(STREAM ? SNT : IT) inner_kernel(InnerArgs a) {
     }
   }
 
+  // rounding bits of the first pass: they depend on the counters only, so they are drawn before the scale is known
+  U4 r_first = U4{0, 0, 0, 0};
+  if (b != 32) r_first = stream_block(a.seed, TAG_ROUND, (uint32_t)worker, k, (uint32_t)((c0 + tid * 8) >> 3));
+
   // ---- scale (Eq. 2): max |u| and, for the c*std rule, tree sums of u and u^2 ----------------------------------
   LPC_PHASE_MARK(5);
   uint32_t mx = 0;
@@ -658,7 +672,7 @@ __global__ void __launch_bounds__(STREAM ? SNT : IT) inner_kernel(InnerArgs a) {
     uint64_t lo = 0, hi = 0;
     if (mine && c < d) {
       U4 r = U4{0, 0, 0, 0};
-      if (!degenerate) r = stream_block(a.seed, TAG_ROUND, (uint32_t)worker, k, (uint32_t)(c >> 3));
+      if (!degenerate) r = (p == 0) ? r_first : stream_block(a.seed, TAG_ROUND, (uint32_t)worker, k, (uint32_t)(c >> 3));
 #pragma unroll
       for (int e = 0; e < 8; ++e) {
         if (c + e < d) {
