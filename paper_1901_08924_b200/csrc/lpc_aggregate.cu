@@ -135,7 +135,7 @@ __global__ void __launch_bounds__(AT) unpack_average_prox_kernel(AggArgs a) {
           decode8<(BITS == 0 || BITS == 32) ? 1 : BITS>(lo, kf);
         }
 #pragma unroll
-        for (int e = 0; e < 8; ++e) acc[e] = add_rn(acc[e], mul_rn(di, kf[e]));
+        for (int e = 0; e < 8; ++e) acc[e] = add_scaled_index<BITS>(acc[e], di, kf[e]);
       }
     }
     float xv[8], mv[8], vv[8];

@@ -296,6 +296,15 @@ __device__ __forceinline__ void decode8(uint64_t lo, float* k) {
   }
 }
 
+// acc + delta * k for a signed codebook index k of a BITS-wide code.  For one- and two-bit codes k is -2, -1, 0 or 1:
+// the product is exact (as long as 2 delta is finite), so one fused multiply-add rounds exactly like the separate
+// multiply and add of wider codes.
+template <int BITS>
+__device__ __forceinline__ float add_scaled_index(float acc, float delta, float k) {
+  if constexpr (BITS == 1 || BITS == 2) return __fmaf_rn(delta, k, acc);
+  else return add_rn(acc, mul_rn(delta, k));
+}
+
 __device__ __forceinline__ float soft_threshold(float w, float kappa) {
   const float a = fmaxf(__fsub_rn(fabsf(w), kappa), 0.f);
   return copysignf(a, w);

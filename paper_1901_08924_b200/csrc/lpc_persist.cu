@@ -408,7 +408,7 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
               decode8<BITS ? BITS : 1>(lo, kf);
             }
 #pragma unroll
-            for (int e = 0; e < EPT; ++e) acc[p][e] = add_rn(acc[p][e], mul_rn(di, kf[e]));
+            for (int e = 0; e < EPT; ++e) acc[p][e] = add_scaled_index<BITS>(acc[p][e], di, kf[e]);
           }
         }
       }
@@ -991,6 +991,9 @@ bool persist_plan(int d, int N, int B, int b, int alpc, int want_cs, int max_sme
     *CS_out = cs; *SL_out = SL; *smem_out = smem; *row_slots_out = slots;
     found = true;
     if (want_cs > 0) break;
+    // (512 threads per CTA with half the coordinates per thread were tried as well: 5.53 against 4.92 us per step on the
+    // least-squares workload, 11.7 against 10.15 on the Algorithm 2 workload at b = 2 -- sixteen-warp block barriers and
+    // half as many words in flight per thread cost more than the shorter per-thread phases gain)
     // (eight-CTA clusters of narrow-thread variants squeezed two to an SM were tried for the 16-worker least-squares
     // workload: 5.8 us per step against 5.06 with four-CTA clusters -- more peers per exchange, polls that come too early)
     if (SL <= 512) break;  // slices below 512 coordinates leave most of a CTA idle
