@@ -227,14 +227,27 @@ __global__ void snapshot_reduce_kernel(const float* __restrict__ partial_mu, con
   const int j = blockIdx.x * blockDim.x + threadIdx.x;
   if (partial_mu && j < d) {
     double s = 0.0;
-    for (int c = 0; c < nparts; ++c) s += (double)partial_mu[(int64_t)c * dpad + j];
+    for (int c0 = 0; c0 < nparts; c0 += 8) {  // eight loads in flight, the additions in CTA order
+      float v[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) v[i] = (c0 + i < nparts) ? partial_mu[(int64_t)(c0 + i) * dpad + j] : 0.f;
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        if (c0 + i < nparts) s += (double)v[i];
+    }
     const float v = (float)(s / (double)n);
     mu[j] = v;
     if (mu_copy) mu_copy[j] = v;
   }
   if (j == 0) {
     double s = 0.0;
-    for (int c = 0; c < 2 * nparts; ++c) s += partial_f[c];  // one partial per row warp of every CTA
+    for (int c0 = 0; c0 < 2 * nparts; c0 += 8) {  // one partial per row warp of every CTA
+      double v[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) v[i] = (c0 + i < 2 * nparts) ? partial_f[c0 + i] : 0.0;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) s += v[i];
+    }
     *f_out = s / (double)n;
   }
 }
