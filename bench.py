@@ -299,7 +299,8 @@ L2_BYTES = 126e6
 # (a few hundred MB, as profiler captures must be); traffic grows in proportion to the units a launch processes, so it
 # is scaled by them.  An entry goes away when its kernel changes.
 TRAFFIC = {
-    "snapshot_kernel": (268.56e6 + 4.02e6, 16384 * 4096, "profiles/snapshot_kernel_ls_16384x4096.md"),
+    "snapshot_kernel": (268.56e6 + 4.25e6, 16384 * 4096, "profiles/snapshot_kernel_ls_16384x4096.md"),
+    "snapshot_kernel (logistic)": (537.00e6 + 4.16e6, 16384 * 8192, "profiles/snapshot_kernel_logistic_16384x8192.md"),
     "stats_kernel": (536.96e6 + 4.20e6, 8 * (1 << 24), "profiles/quantize_aggregate_N8_len2p24_b4_b3.md"),
     "quantize_kernel<4>": (536.95e6 + 14.21e6, 8 * (1 << 24), "profiles/quantize_aggregate_N8_len2p24_b4_b3.md"),
     "quantize_kernel<3>": (536.92e6 + 8.00e6, 8 * (1 << 24), "profiles/quantize_aggregate_N8_len2p24_b4_b3.md"),
@@ -307,8 +308,8 @@ TRAFFIC = {
     "unpack_average_prox_kernel<3>": (117.47e6 + 21.75e6, 1 << 24, "profiles/quantize_aggregate_N8_len2p24_b4_b3.md"),
     "code_histogram_swar_kernel<4>": (67.13e6 + 0.26e6, 8 * (1 << 24), "profiles/server_reduce4_and_code_histogram_N8_len2p24_b4.md"),
     "server_reduce4_kernel<7, sum>": (67.12e6 + 1.84e6, 1 << 24, "profiles/server_reduce4_and_code_histogram_N8_len2p24_b4.md"),
-    "inner_kernel<4> (per step)": (2.218e6, 1, "profiles/inner_step_kernels_ls_16384x4096_N16_B8_b4.md"),
-    "inner_kernel<2, stream>": (234.0e6 + 4.6e6, 32 * 256, "profiles/streaming_worker_kernel_logistic_16384x8192_N32_B256_b2.md"),
+    "inner_kernel<4> (per step)": (2.220e6, 1, "profiles/inner_step_kernels_ls_16384x4096_N16_B8_b4.md"),
+    "inner_kernel<2, stream>": (234.3e6 + 4.8e6, 32 * 256, "profiles/streaming_worker_kernel_logistic_16384x8192_N32_B256_b2.md"),
 }
 
 
@@ -688,7 +689,7 @@ def alpc_bench(dev, peak):
             "written and read, second-estimator words"))
         if b == 2:
             out["roofline_kernels"].append(roofline_entry("snapshot_kernel", out["workload"], snap * 1e3, n * d * 4 + 8 * n + 4 * d,
-                                                          peak, "snapshot_kernel", n * d))
+                                                          peak, "snapshot_kernel (logistic)", n * d))
         ctx.close()
     # the strongly convex case (Algorithm 2, elastic net with sigma = L/1000, Theorem 3's tau1 and alpha)
     b, sigma = 2, L / 1000.0

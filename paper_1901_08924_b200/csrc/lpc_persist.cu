@@ -78,6 +78,16 @@ __device__ __forceinline__ void st_word(unsigned long long* p, uint32_t payload,
   asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
 __device__ __forceinline__ uint32_t word_tag(unsigned long long w) { return (uint32_t)(w >> 32); }
+// Two neighbouring tagged words (16-byte aligned) by one vector access: each 64-bit element is still one indivisible
+// access that carries its own tag, the pair need not be.
+__device__ __forceinline__ void ld_word2(const unsigned long long* p, unsigned long long& w0, unsigned long long& w1) {
+  asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(w0), "=l"(w1) : "l"(p) : "memory");
+}
+__device__ __forceinline__ void st_word2(unsigned long long* p, uint32_t payload0, uint32_t payload1, uint32_t tag) {
+  const unsigned long long v0 = (unsigned long long)payload0 | ((unsigned long long)tag << 32);
+  const unsigned long long v1 = (unsigned long long)payload1 | ((unsigned long long)tag << 32);
+  asm volatile("st.relaxed.gpu.global.v2.u64 [%0], {%1, %2};" ::"l"(p), "l"(v0), "l"(v1) : "memory");
+}
 // The same kind of word in shared memory: stored into CTA `cta` of the cluster at the address that `slot` has in
 // this CTA, read back from this CTA's own shared memory.
 __device__ __forceinline__ void st_cluster_word(const unsigned long long* slot, uint32_t cta, uint32_t payload, uint32_t tag) {
@@ -359,9 +369,14 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
         for (int j = 0; j < CH; ++j) {
           const unsigned long long* q = ll_in + (size_t)min(i0 + j, N - 1) * wstride;
 #pragma unroll
-          for (int p = 0; p < NP; ++p)
+          for (int p = 0; p < NP; ++p) {
+            if constexpr (BITS == 8 && NW == 2) {  // the two words of a group of eight 8-bit codes: one 16-byte load
+              ld_word2(q + gq[p], cw[j][p][0], cw[j][p][1]);
+            } else {
 #pragma unroll
-            for (int w = 0; w < NW; ++w) cw[j][p][w] = (w < wpg) ? ld_word(q + gq[p] + w) : good;
+              for (int w = 0; w < NW; ++w) cw[j][p][w] = (w < wpg) ? ld_word(q + gq[p] + w) : good;
+            }
+          }
         }
         if (i0 == 0 && it == 0) between();
         bool ok = word_tag(dw) == tag;
@@ -812,8 +827,12 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
       if constexpr (BITS == 0 || TB >= 32) {
         // whole words per thread
         if (mine) {
-          st_word(q + wfirst, (uint32_t)lo, tag);
-          if (NW >= 2 && wpg >= 2) st_word(q + wfirst + 1, (uint32_t)(lo >> 32), tag);
+          if constexpr (BITS == 8 && NW == 2) {
+            st_word2(q + wfirst, (uint32_t)lo, (uint32_t)(lo >> 32), tag);
+          } else {
+            st_word(q + wfirst, (uint32_t)lo, tag);
+            if (NW >= 2 && wpg >= 2) st_word(q + wfirst + 1, (uint32_t)(lo >> 32), tag);
+          }
           if (NW >= 4 && wpg >= 4) {
             st_word(q + 2, (uint32_t)hi, tag);
             st_word(q + 3, (uint32_t)(hi >> 32), tag);
