@@ -314,6 +314,9 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
   // thread: lane l of a warp loads those of workers l, l + 32, ... and the warp hands them round by shuffles.
   constexpr int WMAX = (BITS == 0) ? 8 : (BITS == 8 ? 2 : 1);  // tagged words per group of 8 coordinates
   constexpr int NW = (BITS == 0) ? 8 : (TB >= 32 ? TB / 32 : 1);  // of which a thread reads / writes this many
+  // (A layout with the workers' words of a coordinate group side by side, read two workers per 16-byte load, halves the
+  // loads of the update but scatters every worker's stores over lines that the other workers write too: 5.53 against
+  // 4.93 us per step on the least-squares workload, 12.5 against 9.9 on the Algorithm 2 workload; dropped.)
   // workers per round of loads: 16 words in flight per thread.  (32 per round for the 32 workers of the Algorithm 2
   // workload moved the second round's time into the first: 40 loads per thread queue up on the way from L2.)
   constexpr int CH = (BITS == 0) ? 4 : 16 / (NP * NW) > 0 ? 16 / (NP * NW) : 1;
@@ -351,11 +354,13 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
     for (int p = 0; p < NP; ++p) gq[p] = (act[p] ? (size_t)(cc[p] >> 3) : 0) * wpg + wfirst;
     const size_t wstride = groups * wpg;
     auto issue_vhat = [&]() {
+      if constexpr (ALPC) {
 #pragma unroll
-      for (int p = 0; p < NP; ++p)
+        for (int p = 0; p < NP; ++p)
 #pragma unroll
-        for (int e = 0; e < EPT; ++e)
-          vw[p * EPT + e] = ld_word(pa.ll_vhat + (size_t)rpar * groups * 8 + (act[p] ? cc[p] : c0) + e);
+          for (int e = 0; e < EPT; e += 2)  // pairs of neighbouring words by one 16-byte access
+            ld_word2(pa.ll_vhat + (size_t)rpar * groups * 8 + (act[p] ? cc[p] : c0) + e, vw[p * EPT + e], vw[p * EPT + e + 1]);
+      }
     };
     if constexpr (ALPC) issue_vhat();
 #pragma unroll 1
@@ -687,10 +692,11 @@ __global__ void __launch_bounds__(PT, 1) persist_kernel(PersistArgs pa) {
         if (off < SL) {
           unsigned long long* q = pa.ll_vhat + (size_t)wpar * groups * 8 + c0 + off;
 #pragma unroll
-          for (int e = 0; e < EPT; ++e) {
-            const float vh = add_rn(u[p][e], mur[p][e]);
-            st_word(q + e, __float_as_uint(vh), tag);
-            if (last && off + e < width) pa.vhat[c0 + off + e] = vh;
+          for (int e = 0; e < EPT; e += 2) {
+            const float vh0 = add_rn(u[p][e], mur[p][e]), vh1 = add_rn(u[p][e + 1], mur[p][e + 1]);
+            st_word2(q + e, __float_as_uint(vh0), __float_as_uint(vh1), tag);
+            if (last && off + e < width) pa.vhat[c0 + off + e] = vh0;
+            if (last && off + e + 1 < width) pa.vhat[c0 + off + e + 1] = vh1;
           }
         }
       }
