@@ -45,7 +45,10 @@ def _inject_snapshot(ctx, P, xs):
 
 
 @pytest.mark.parametrize("loss", ["least_squares", "logistic"])
-@pytest.mark.parametrize("n,d", [(64, 8), (96, 64), (200, 1000), (120, 1500), (64, 3072), (1000, 4096), (48, 8192)])
+# the last three: many tiles per CTA (the ring of stages wraps, both row warps get tiles), a ragged last tile on a deep
+# ring, and a row wider than 8,192 columns (one row per tile, 16 values per compute thread)
+@pytest.mark.parametrize("n,d", [(64, 8), (96, 64), (200, 1000), (120, 1500), (64, 3072), (1000, 4096), (48, 8192),
+                                 (20000, 1024), (5004, 2048), (36, 12288)])
 def test_snapshot_full_gradient(loss, n, d):
     P, ctx = _setup(n, d, loss, N=4, B=2, b=4)
     rng = np.random.default_rng(d)
