@@ -210,3 +210,53 @@ def test_server_schemes_and_entropy_count_full_length():
         assert (_bits(xch[s0:s0 + W]) == _bits(orc.unpack_scaled_prox(ref_c, best["delta"], W, b, 1, None, zero, 1.0, 1e-3))).all()
     for c in (q, wb, wc):
         c.close()
+
+
+@pytest.mark.parametrize("B,b", [(256, 2), (256, 8), (1024, 2)])
+def test_fused_worker_kernel_large_minibatches_bench_shape(B, b):
+    # The streaming worker kernel in the launch shape the benchmark times on it: d = 8,192, N = 32 workers, logistic
+    # loss on ill-conditioned columns, clip 2 std, clusters of 4 CTAs, a ring of 6 (B = 256) or 5 (B = 1,024) stages.
+    # The matrix has fewer rows than the benchmark's (the launch shape does not depend on n; the oracle pays per row).
+    n, d, N = 8192, 8192, 32
+    X, y, _ = synth.linear_problem(n, d, loss="logistic", sparsity=0.02, noise=0.1, seed=1, col_scale_range=(0.1, 10.0))
+    Xh, yh = X.numpy(), y.numpy()
+    P = orc.Problem(Xh, yh, orc.LOGISTIC, 1e-5, N, B, b, orc.CLIP_STD, 2.0, 3)
+    ctx = lpc.Context(X.to(DEV), y.to(DEV), lpc.LOGISTIC, 1e-5, N, B, b, lpc.CLIP_STD, 2.0, 3)
+    assert ctx.query(lpc.INFO_STEP_CLUSTER_SIZE) == 4
+    assert ctx.query(lpc.INFO_STEP_RING_STAGES) == (6 if B == 256 else 5)
+    ctx.set_option(lpc.OPT_TAP_U, 1)
+    rng = np.random.default_rng(B + b)
+    xs = (rng.standard_normal(d) * 0.02).astype(np.float32)
+    x = (xs + rng.standard_normal(d).astype(np.float32) * 0.005).astype(np.float32)
+    mu, margins, _ = orc.full_grad(Xh, yh, P.loss, xs)
+    ctx.set_buffer(lpc.BUF_XTILDE, torch.from_numpy(xs).to(DEV))
+    ctx.set_buffer(lpc.BUF_MU, torch.from_numpy(mu).to(DEV))
+    ctx.set_buffer(lpc.BUF_MARGINS, torch.from_numpy(margins).to(DEV))
+    k, eta = 7, 0.01
+    ctx.set_iterate(torch.from_numpy(x).to(DEV))
+    ctx.inner_step(eta, k)
+    ctx.sync_status()
+    _, t = orc.lpc_inner_step(P, k, eta, x, xs, mu, taps=True)
+    idx = ctx.get_buffer(lpc.BUF_BATCH_IDX).cpu().numpy()[:N]
+    coef = ctx.get_buffer(lpc.BUF_COEF).cpu().numpy()[:N]
+    assert (idx == t["idx"]).all()
+    # the logistic derivative goes through exp on both sides: coefficients within an ulp of their largest, and everything
+    # after them bit for bit once the oracle is handed the coefficients the kernel used
+    assert np.abs(coef - t["coef"]).max() <= 1.2e-7 * max(1.0, np.abs(t["coef"]).max())
+    words = np.zeros((N, P.W), np.uint32)
+    delta = np.zeros(N, np.float32)
+    clipped = np.zeros(N, np.uint32)
+    u = np.zeros((N, d), np.float32)
+    for i in range(N):
+        u[i] = orc.svrg_diff_from_coef(Xh, idx[i], coef[i])
+        w, delta[i], clipped[i] = orc.quantize_pack(u[i], b, orc.CLIP_STD, 2.0, 3, i, k)
+        words[i] = w[: P.W]
+    xn, v = orc.unpack_average_prox(words, delta, d, b, mu, x, eta, P.lambda_l1, want_v=True)
+    assert (_bits(ctx.get_buffer(lpc.BUF_U)) == _bits(u)).all()
+    assert (_bits(ctx.get_buffer(lpc.BUF_DELTA)) == _bits(delta)).all()
+    codes = ctx.get_buffer(lpc.BUF_CODES).cpu().numpy().view(np.uint32)
+    assert (codes[:, : P.W] == words).all() and (codes[:, P.W:] == 0).all()
+    assert (ctx.get_buffer(lpc.BUF_CLIPPED).cpu().numpy().view(np.uint32) == clipped).all()
+    assert (_bits(ctx.get_buffer(lpc.BUF_V)) == _bits(v)).all()
+    assert (_bits(ctx.get_iterate()) == _bits(xn)).all()
+    ctx.close()
