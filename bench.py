@@ -422,6 +422,11 @@ def quantize_aggregate_bench(dev, peak, log2_len=26, full=True):
         grid[name] = r
         return r
 
+    # the floor of a timed launch: the same calls on 8 x 2^10 values, where there is next to nothing to do
+    r0 = qa_point(dev, peak, U[:, : 1 << 10], 4, 2.0, reps=20)
+    res["launch_floor_us"] = {"workload": "N=8, len 2^10, b=4 (an event pair around a launch that has next to nothing to do)",
+                              "quantize_fused_kernel (cooperative launch, one grid-wide hand-over)": round(r0["quantize_pack"]["one_launch_ms"] * 1e3, 2),
+                              "unpack_average_prox_kernel (plain launch)": round(r0["unpack_average_prox"]["ms"] * 1e3, 2)}
     lens = [l for l in (16, 20, 24, 26, 28) if l <= top]
     for l2 in lens:
         r = point("gauss_len2^%d_b4_clip2" % l2, U[:, : 1 << l2], 4, 2.0, reps=10 if l2 <= 24 else 4)
@@ -432,7 +437,7 @@ def quantize_aggregate_bench(dev, peak, log2_len=26, full=True):
                 "quantize+pack (stats_kernel + finish_kernel + quantize_kernel<4>)")
         roof.append(roofline_entry(name, wl, qp["ms"] * 1e3, qp["bytes"], peak,
                                    note="input stays in L2 between the two looks at it: bound 4 + b/8 B per element; launch-bound at "
-                                        "this size (an event pair around one launch reads about 8 us)" if resident else
+                                        "this size (see quantize_aggregate.launch_floor_us)" if resident else
                                    "two passes: 8 + b/8 B per element"))
         if not resident and qp["stats_ms"] > 0:
             roof.append(roofline_entry("stats_kernel", wl, qp["stats_ms"] * 1e3, N * (1 << l2) * 4, peak, "stats_kernel", N * (1 << l2)))
@@ -446,7 +451,7 @@ def quantize_aggregate_bench(dev, peak, log2_len=26, full=True):
         r = point("gauss_len2^%d_b%d_clip2" % (mid, b), Um, b, 2.0)
         wl = "sweep N=8, len 2^%d, N(0,1), b=%d, clip 2 std" % (mid, b)
         roof.append(roofline_entry("quantize+pack, b=%d" % b, wl, r["quantize_pack"]["ms"] * 1e3, r["quantize_pack"]["bytes"], peak))
-        if b == 3:
+        if b == 3 and r["quantize_pack"]["pack_ms"] > 0:  # (a short vector goes through the one-launch path instead)
             roof.append(roofline_entry("quantize_kernel<3>", wl, r["quantize_pack"]["pack_ms"] * 1e3, N * (1 << mid) * (4 + 3 / 8), peak,
                                        "quantize_kernel<3>", N * (1 << mid)))
         roof.append(roofline_entry("unpack_average_prox_kernel<%d>" % b, wl, r["unpack_average_prox"]["ms"] * 1e3,

@@ -78,19 +78,17 @@ struct Smem {
   int issued;                     // groups whose bulk copies have been issued
 };
 
-// Phase timestamps of the streaming path of one CTA, for latency studies; compiled in only with -DLPC_TRACE.
+// Phase timestamps of every CTA of the kernel (thread 0: entry, first copies about to be issued, cluster started, u
+// complete, scale known, codes stored), for latency studies; compiled in only with -DLPC_TRACE.
 #ifdef LPC_TRACE
-__device__ unsigned long long g_stream_trace[64 * 16 + 16];  // per group: 16 marks; then 16 phase marks of the kernel
-#define LPC_STREAM_MARK(g, i)                                                                       \
-  do {                                                                                              \
-    if (blockIdx.x == 0 && blockIdx.y == 0 && (g) < 64) g_stream_trace[(g) * 16 + (i)] = global_ns(); \
-  } while (0)
-#define LPC_PHASE_MARK(i)                                                                            \
-  do {                                                                                               \
-    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) g_stream_trace[64 * 16 + (i)] = global_ns(); \
+constexpr int TRACE_CTAS = 1024;
+__device__ unsigned long long g_stream_cta[TRACE_CTAS * 8];
+#define LPC_PHASE_MARK(i)                                                         \
+  do {                                                                            \
+    const unsigned int cta_ = blockIdx.y * gridDim.x + blockIdx.x;                \
+    if (threadIdx.x == 0 && cta_ < TRACE_CTAS) g_stream_cta[cta_ * 8 + (i)] = global_ns(); \
   } while (0)
 #else
-#define LPC_STREAM_MARK(g, i) do { } while (0)
 #define LPC_PHASE_MARK(i) do { } while (0)
 #endif
 
@@ -243,7 +241,6 @@ __global__ void __launch_bounds__(STREAM ? SNT : IT) inner_kernel(InnerArgs a) {
       if (lane_in_group < cnt)
         bulk_load(rows + ((size_t)s * SG + lane_in_group) * SL, a.X + s_idx[g * SG + lane_in_group] * (int64_t)d + c0,
                   row_bytes, &sm.sbar[s]);
-      if (lane_in_group == 0) LPC_STREAM_MARK(g, 6);
     };
     static_assert(SMAXR * SG <= 32, "the first fills are issued by one warp, one row per lane");
     static_assert(SG * MAXCS == 32, "one lane per (row, CTA) pair when the coefficients are formed");
@@ -304,7 +301,6 @@ __global__ void __launch_bounds__(STREAM ? SNT : IT) inner_kernel(InnerArgs a) {
       for (int g = warp / SMW; g < ngroups; g += SDW / SMW) {
         const int cnt = min(SG, B - g * SG);
         wait_stage(g);
-        if (warp < 2 * SMW && wq == 0 && lane == 0) LPC_STREAM_MARK(g, 0);
         // two rows at a time (eight loads in flight): the sixteen partial sums of the group are all that stays
         float sv[SG * QB];
 #pragma unroll
@@ -338,7 +334,6 @@ __global__ void __launch_bounds__(STREAM ? SNT : IT) inner_kernel(InnerArgs a) {
         if ((lane >> 2) < CS && myrow < cnt)
           st_async_cluster(&sm.parts[g % SSLOTS][(myrow * MAXCS + rank) * SMW + wq], &sm.pbar[g % SSLOTS],
                            (uint32_t)(lane >> 2), __float_as_uint(part));
-        if (wq == 0 && lane == 0) LPC_STREAM_MARK(g, 1);
       }
     } else if (warp < SDW + SUW) {
       // -- u: thread t of these warps owns the coordinates 4 t .. 4 t + 3 of each half of the slice.  The rows of a
@@ -350,7 +345,6 @@ __global__ void __launch_bounds__(STREAM ? SNT : IT) inner_kernel(InnerArgs a) {
       auto take = [&](int g, float4 (&v)[SG][UC]) {  // rows past a ragged end are read and not used
         const int s = g % R;
         wait_stage(g);
-        if (t == 0) LPC_STREAM_MARK(g, 8);
         if (full) {
           const float* src = rows + (size_t)(s * SG) * SL + t * 4;
 #pragma unroll
@@ -365,12 +359,10 @@ __global__ void __launch_bounds__(STREAM ? SNT : IT) inner_kernel(InnerArgs a) {
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(&sm.ebar[s]);  // release: the loads above are performed before the arrival counts
-        if (t == 0) LPC_STREAM_MARK(g, 9);
       };
       auto add = [&](int g, const float4 (&v)[SG][UC]) {
         const int cnt = min(SG, B - g * SG);
         wait_on(&sm.cbar[g % SSLOTS], (uint32_t)((g / SSLOTS) & 1), false);
-        if (t == 0) LPC_STREAM_MARK(g, 4);
         const float4 c4 = *reinterpret_cast<const float4*>(sm.coefs[g % SSLOTS]);
         const float cj[SG] = {c4.x, c4.y, c4.z, c4.w};
 #pragma unroll
@@ -385,9 +377,6 @@ __global__ void __launch_bounds__(STREAM ? SNT : IT) inner_kernel(InnerArgs a) {
             }
           }
         }
-#ifdef LPC_TRACE
-        if (lane == 0 && blockIdx.x == 0 && blockIdx.y == 0 && g < 64) atomicMax(&g_stream_trace[g * 16 + 5], global_ns());
-#endif
       };
       take(0, va);
 #pragma unroll 1
@@ -411,7 +400,6 @@ __global__ void __launch_bounds__(STREAM ? SNT : IT) inner_kernel(InnerArgs a) {
         __syncwarp();
         wait_on(&sm.mbar_meta[(g * SG) / 32], 0u, false);
         wait_on(&sm.pbar[sl], (uint32_t)((g / SSLOTS) & 1), true);
-        if (lane == 0) LPC_STREAM_MARK(g, 2);
         // lane (j, q) = (lane / MAXCS, lane % MAXCS): the tree over the four quarter sums of CTA q's slice for row j, then
         // the tree over the CTAs by shuffles; lane (j, 0) ends with the margin of row j
         {
@@ -440,7 +428,6 @@ __global__ void __launch_bounds__(STREAM ? SNT : IT) inner_kernel(InnerArgs a) {
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(&sm.cbar[sl]);
-        if (lane == 0) LPC_STREAM_MARK(g, 3);
       }
     } else if (warp < SDW + SUW + SCW + SPW) {
       // -- refills: a stage goes back to the bulk copies the moment the update side has handed it over
@@ -448,7 +435,6 @@ __global__ void __launch_bounds__(STREAM ? SNT : IT) inner_kernel(InnerArgs a) {
       for (int g = R; g < ngroups; ++g) {
         const int h = g - R;
         wait_on(&sm.ebar[h % R], (uint32_t)((h / R) & 1), false);
-        if (lane == 0) LPC_STREAM_MARK(g, 7);
         if (gave_up) break;
         if (width > 0 && lane < SG) issue(g, lane);
         __syncwarp();
@@ -839,8 +825,8 @@ cudaError_t launch_inner(const InnerArgs& a, size_t smem, cudaStream_t st) {
 }
 
 #ifdef LPC_TRACE
-cudaError_t read_stream_trace(unsigned long long* host_out) {
-  return cudaMemcpyFromSymbol(host_out, g_stream_trace, sizeof(unsigned long long) * (64 * 16 + 16));
+cudaError_t read_stream_trace(unsigned long long* host_out) {  // TRACE_CTAS x 8 marks
+  return cudaMemcpyFromSymbol(host_out, g_stream_cta, sizeof(g_stream_cta));
 }
 #endif
 

@@ -1,6 +1,7 @@
-"""Phase table of the one-launch inner loop, from %globaltimer stamps.
+"""Phase tables of the one-launch inner loop and of the streaming worker kernel, from %globaltimer stamps.
 
     python -m paper_1901_08924_b200.trace [--workload ls|alpc] [--bits B] [--rows N] [--steps M]
+    python -m paper_1901_08924_b200.trace --workload stream [--batch B] [--bits B] [--rows N]
 
 Profilers cannot replay the cooperative cluster launch of the one-launch loop, so its time is accounted for with
 time stamps instead: the library is built a second time with -DLPC_TRACE (liblpcsvrg_trace.so, see build.py), in which
@@ -11,6 +12,9 @@ than the plain one and the timer has a grain of 32 ns: read the table for where 
 workloads (synthetic, shapes of the benchmark's):
   ls    least squares, d = 4,096, N = 16 workers, B = 8, b = 4, clip 3 std   (Algorithm 1)
   alpc  logistic, d = 8,192, ill-conditioned columns, N = 32, B = 16, b = 2 (or --bits 8), clip 2 std   (Algorithm 2)
+  stream  the fused worker kernel on large minibatches: logistic, 65,536 x 8,192, N = 32, B = 256 (or --batch 1024) rows per
+          worker, b = 2.  In the stamped build thread 0 of EVERY CTA stores %globaltimer at six points of the kernel; the
+          table gives the spread of each point over the 128 CTAs of one launch, next to the launch's CUDA-event time.
 """
 import argparse
 import ctypes as C
@@ -38,7 +42,8 @@ PHASES = [
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--workload", default="ls", choices=["ls", "alpc"])
+    ap.add_argument("--workload", default="ls", choices=["ls", "alpc", "stream"])
+    ap.add_argument("--batch", type=int, default=256)
     ap.add_argument("--bits", type=int, default=0)
     ap.add_argument("--rows", type=int, default=0)
     ap.add_argument("--steps", type=int, default=128)
@@ -51,6 +56,8 @@ def main():
     assert lpc.LIB_PATH == os.environ["LPC_LIBRARY"], "import this module before paper_1901_08924_b200.lpc"
 
     dev = torch.device("cuda", 0)
+    if args.workload == "stream":
+        return stream_table(args, dev, torch, lpc, synth)
     if args.workload == "ls":
         n, d, N, B, b = args.rows or 16384, 4096, 16, 8, args.bits or 4
         X, y, _ = synth.linear_problem(n, d, loss="least_squares", sparsity=0.05, noise=0.01, seed=0, device=dev)
@@ -99,6 +106,41 @@ def main():
     print("| step period | %.0f |" % statistics.median(period))
     print("| looks at the words until all tags matched (median, max) | %d, %d |"
           % (statistics.median(m[15] for m in marks), max(m[15] for m in marks)))
+    ctx.close()
+
+
+STREAM_MARKS = [(0, "kernel entry"), (1, "first bulk copies about to be issued (sampling, barrier set-up, cluster arrival done)"),
+                (3, "every CTA of the cluster has started"), (5, "last group added to u, u with the owners of its coordinates"),
+                (6, "scale known (statistics, exchange across the cluster, Eq. 2)"), (7, "codes stored")]
+
+
+def stream_table(args, dev, torch, lpc, synth):
+    n, d, N, B, b = args.rows or 65536, 8192, 32, args.batch, args.bits or 2
+    X, y, _ = synth.linear_problem(n, d, loss="logistic", sparsity=0.02, noise=0.1, seed=1, col_scale_range=(0.1, 10.0),
+                                   device=dev)
+    ctx = lpc.Context(X, y, lpc.LOGISTIC, 1e-5, N, B, b, lpc.CLIP_STD, 2.0, 0)
+    ctx.snapshot_full_grad()
+    ctx.inner_steps(1e-3, 0, 5)
+    ctx.set_option(lpc.OPT_PROFILE, 1)
+    ctx.inner_steps(1e-3, 5, 10)
+    ctx.sync_status()
+    prof = ctx.get_profile()
+    cs = ctx.query(lpc.INFO_STEP_CLUSTER_SIZE)
+    ctas = N * cs
+    buf = (C.c_ulonglong * (1024 * 8))()
+    read = lpc.lib().lpc_debug_stream_trace
+    read.restype, read.argtypes = C.c_int, [C.POINTER(C.c_ulonglong)]
+    assert read(buf) == 0
+    marks = [[buf[c * 8 + i] for i in range(8)] for c in range(ctas)]
+    t0 = min(m[0] for m in marks)
+    print("workload stream: n = %d, d = %d, N = %d, B = %d, b = %d; clusters of %d CTAs, ring of %d stages"
+          % (n, d, N, B, b, cs, ctx.query(lpc.INFO_STEP_RING_STAGES)))
+    print("CUDA events around one launch: %.2f us (stamped build, average of 10)" % (prof["worker"][0] / prof["worker"][1] * 1e3))
+    print("| mark (thread 0 of each of the %d CTAs of the last launch, ns from the first CTA's entry) | min | median | max |" % ctas)
+    print("|---|---|---|---|")
+    for i, name in STREAM_MARKS:
+        v = sorted(m[i] - t0 for m in marks)
+        print("| %s | %d | %d | %d |" % (name, v[0], v[len(v) // 2], v[-1]))
     ctx.close()
 
 
