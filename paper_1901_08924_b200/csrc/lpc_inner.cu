@@ -78,7 +78,7 @@ struct Smem {
   int issued;                     // groups whose bulk copies have been issued
 };
 
-// Phase timestamps of every CTA of the kernel (thread 0: entry, first copies about to be issued, cluster started, u
+// Phase timestamps of every CTA of the kernel (entry, first copies issued, block-wide prologue done, cluster started, u
 // complete, scale known, codes stored), for latency studies; compiled in only with -DLPC_TRACE.
 #ifdef LPC_TRACE
 constexpr int TRACE_CTAS = 1024;
@@ -88,8 +88,14 @@ __device__ unsigned long long g_stream_cta[TRACE_CTAS * 8];
     const unsigned int cta_ = blockIdx.y * gridDim.x + blockIdx.x;                \
     if (threadIdx.x == 0 && cta_ < TRACE_CTAS) g_stream_cta[cta_ * 8 + (i)] = global_ns(); \
   } while (0)
+#define LPC_WARP_MARK(i) /* by lane 0 of the calling warp */                       \
+  do {                                                                            \
+    const unsigned int cta_ = blockIdx.y * gridDim.x + blockIdx.x;                \
+    if ((threadIdx.x & 31) == 0 && cta_ < TRACE_CTAS) g_stream_cta[cta_ * 8 + (i)] = global_ns(); \
+  } while (0)
 #else
 #define LPC_PHASE_MARK(i) do { } while (0)
+#define LPC_WARP_MARK(i) do { } while (0)
 #endif
 
 // BITS: 1, 2, 4, 8 fixed-width packing; 0: b from the arguments (1..16 or 32).
@@ -127,14 +133,38 @@ __global__ void __launch_bounds__(STREAM ? SNT : IT) inner_kernel(InnerArgs a) {
   const int width = max(0, min(SL, d - c0));        // coordinates of the slice that exist
 
   // ---- sampling (Algorithm 1 step 6): slot a uses word 0 of block a of the batch stream -----------------
-  for (int slot = tid; slot < B; slot += NT) {
+  auto sample_slot = [&](int slot) -> int64_t {
     int64_t lo, span;
     uint32_t tag, wk;
     if (is_J) { lo = 0; span = a.n; tag = TAG_BATCH_J; wk = 0; }
     else if (a.sample_global) { lo = 0; span = a.n; tag = TAG_BATCH; wk = (uint32_t)worker; }
     else { span = a.n / a.N; lo = (int64_t)worker * span; tag = TAG_BATCH; wk = (uint32_t)worker; }
     const U4 r = stream_block(a.seed, tag, wk, k, (uint32_t)slot);
-    const int64_t row = lo + (int64_t)(((uint64_t)r.x * (uint64_t)span) >> 32);
+    return lo + (int64_t)(((uint64_t)r.x * (uint64_t)span) >> 32);
+  };
+  if constexpr (STREAM) {
+    // The refill warp starts the first fills of the ring before anything else of the step: it sets up the stages'
+    // barriers itself, samples the rows of the first stages (one per lane) and issues their copies; the other warps
+    // sample the whole batch and set up the remaining barriers meanwhile.
+    static_assert(SMAXR * SG <= 32 && SMAXR <= 32, "the first fills are issued by one warp, one row per lane");
+    if (warp == SDW + SUW + SCW) {
+      const int R0 = a.stream_stages, first = min(R0, (B + SG - 1) / SG);
+      if (lane < SMAXR) mbar_init(&sm.sbar[lane], 1);
+      mbar_fence_init();
+      __syncwarp();
+      const int g = lane / SG, j = lane % SG, cnt = min(SG, B - g * SG);
+      if (width > 0 && g < first) {
+        const uint32_t bytes = (uint32_t)width * 4u;
+        if (j == 0) mbar_expect_tx(&sm.sbar[g], bytes * (uint32_t)cnt);
+        if (j < cnt)
+          bulk_load(rows + ((size_t)g * SG + j) * SL, a.X + sample_slot(g * SG + j) * (int64_t)d + c0, bytes, &sm.sbar[g]);
+      }
+      if (lane == 0) sm.issued = (width > 0) ? first : 0;
+      LPC_WARP_MARK(2);
+    }
+  }
+  for (int slot = tid; slot < B; slot += NT) {
+    const int64_t row = sample_slot(slot);
     s_idx[slot] = row;
     if constexpr (!STREAM) {
       s_yv[slot] = a.y[row];
@@ -145,7 +175,6 @@ __global__ void __launch_bounds__(STREAM ? SNT : IT) inner_kernel(InnerArgs a) {
     // the barriers of the streaming path are set up side by side, one or two per thread
     static_assert(SMAXR + SSLOTS + SMAXB / 32 <= 64, "two warps set up the barriers");
     if (tid < SMAXR) {
-      mbar_init(&sm.sbar[tid], 1);
       mbar_init(&sm.ebar[tid], SUW + SDW / 2);
     } else if (tid < SMAXR + SSLOTS) {
       mbar_init(&sm.pbar[tid - SMAXR], 1);
@@ -157,7 +186,6 @@ __global__ void __launch_bounds__(STREAM ? SNT : IT) inner_kernel(InnerArgs a) {
       mbar_init(&sm.bar, 1);
       mbar_init(&sm.xbar, 1);
       sm.stream_fail = 0;
-      sm.issued = 0;
     }
     if (tid < 64) mbar_fence_init();
   } else if (tid == 0) {
@@ -242,13 +270,8 @@ __global__ void __launch_bounds__(STREAM ? SNT : IT) inner_kernel(InnerArgs a) {
         bulk_load(rows + ((size_t)s * SG + lane_in_group) * SL, a.X + s_idx[g * SG + lane_in_group] * (int64_t)d + c0,
                   row_bytes, &sm.sbar[s]);
     };
-    static_assert(SMAXR * SG <= 32, "the first fills are issued by one warp, one row per lane");
     static_assert(SG * MAXCS == 32, "one lane per (row, CTA) pair when the coefficients are formed");
     LPC_PHASE_MARK(1);
-    if (warp == SDW + SUW + SCW && width > 0) {  // the first fills start before anything else of the step
-      const int g = lane / SG;
-      if (g < min(R, ngroups)) issue(g, lane % SG);
-    }
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");  // all peers have started
     LPC_PHASE_MARK(3);
     bool gave_up = false;  // after one wait ran out this thread waits no more (the status word says so)

@@ -109,7 +109,8 @@ def main():
     ctx.close()
 
 
-STREAM_MARKS = [(0, "kernel entry"), (1, "first bulk copies about to be issued (sampling, barrier set-up, cluster arrival done)"),
+STREAM_MARKS = [(0, "kernel entry"), (2, "first bulk copies issued (by the refill warp)"),
+                (1, "block-wide prologue done (sampling of the whole batch, barrier set-up, cluster arrival)"),
                 (3, "every CTA of the cluster has started"), (5, "last group added to u, u with the owners of its coordinates"),
                 (6, "scale known (statistics, exchange across the cluster, Eq. 2)"), (7, "codes stored")]
 
